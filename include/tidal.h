@@ -1,0 +1,161 @@
+/*
+ * libtidal — decode-step attention of TidalDecode's Position Persistent Sparse
+ * Attention (arxiv 2410.05076) for NVIDIA B200 (sm_100a).
+ *
+ * The library covers the attention branch of the paper's Algorithm 1 for one
+ * decode step: full attention over the whole KV cache (full-attention layers),
+ * full attention that also ranks every cached token by its query-key inner
+ * product and keeps the top k (token selection layers), and sparse attention
+ * over only the positions kept by the last selection layer (all other
+ * layers). Projections, FFN and the KV append are the caller's.
+ *
+ * Conventions shared by every call
+ *   - All tensor pointers are DEVICE pointers unless a parameter says "host".
+ *     The caller owns every buffer; the library owns only its context and the
+ *     workspace inside it and keeps no reference to caller memory after the
+ *     work it enqueued has run.
+ *   - Calls enqueue work on the CUDA stream passed as `stream` (a cudaStream_t
+ *     cast to void*, NULL = the legacy default stream) and return without
+ *     waiting for it, except where stated.
+ *   - Return value: TIDAL_OK or a negative tidal_status_t. Argument errors are
+ *     detected on the host before anything is enqueued. Nothing throws or
+ *     aborts across this boundary. Problems only the device can see (a token
+ *     index outside the cache, a page id outside the pool) make the kernel skip
+ *     that element and set a sticky status word read by tidal_device_status().
+ *   - q is bf16 [batch, num_q_heads, head_dim] contiguous; outputs are fp32
+ *     [batch, num_q_heads, head_dim] contiguous. Arithmetic: bf16 inputs,
+ *     fp32 accumulation.
+ *   - There is no CPU path: on a machine without a usable GPU tidal_create()
+ *     fails with TIDAL_ERR_CUDA.
+ */
+#ifndef TIDAL_H
+#define TIDAL_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tidal_ctx tidal_ctx_t;     /* opaque: device, workspace, kernel attributes */
+typedef int32_t tidal_status_t;
+
+enum {
+    TIDAL_OK = 0,
+    TIDAL_ERR_INVALID = -1,       /* bad argument (NULL pointer, k <= 0, misaligned stride, ...) */
+    TIDAL_ERR_UNSUPPORTED = -2,   /* valid request outside what is built (head_dim != 128, ...) */
+    TIDAL_ERR_NOMEM = -3,         /* workspace allocation failed */
+    TIDAL_ERR_CUDA = -4,          /* a CUDA runtime call failed */
+    TIDAL_ERR_TIMEOUT = -5,       /* reserved: a bounded device-side wait expired */
+    TIDAL_ERR_INDEX = -6          /* device saw a token index or page id out of range */
+};
+
+enum { TIDAL_KV_CONTIG = 0, TIDAL_KV_PAGED = 1 };
+
+/* Granularity of the selected token set (number of index heads Hi).
+ * PER_QHEAD is the paper's definition (Eq. 1 and Section 3.1 are per attention
+ * head): Hi = num_q_heads. The other two rank by the sum of the member heads'
+ * scaled logits: PER_KVHEAD has Hi = num_kv_heads, SHARED has Hi = 1. */
+enum { TIDAL_SEL_PER_QHEAD = 0, TIDAL_SEL_PER_KVHEAD = 1, TIDAL_SEL_SHARED = 2 };
+
+/* Layer types of Algorithm 1 / Figure 2. */
+enum { TIDAL_LAYER_FULL = 0, TIDAL_LAYER_SELECT = 1, TIDAL_LAYER_SPARSE = 2 };
+
+/* KV cache of one layer. Strides count bf16 ELEMENTS and must be multiples of
+ * 8 (16 bytes); k and v must be 16-byte aligned; a row (head_dim elements of
+ * one position and KV head) is contiguous.
+ *   contiguous: K[b, pos, g, c] at k + b*stride_b + pos*stride_pos + g*stride_head + c
+ *   paged:      page = page_table[b*max_pages_per_seq + pos/page_size], slot = pos%page_size,
+ *               K[b, pos, g, c] at k + page*stride_page + slot*stride_pos + g*stride_head + c
+ * V uses the same strides from `v`. The cache already contains the token being
+ * decoded (Algorithm 1 appends before attention), so ctx_lens[b] >= 1 counts it. */
+typedef struct {
+    int32_t batch, num_q_heads, num_kv_heads, head_dim;   /* head_dim == 128; Hq % Hkv == 0; Hq/Hkv <= 8 */
+    int32_t kv_layout;                                    /* TIDAL_KV_CONTIG or TIDAL_KV_PAGED */
+    const void *k, *v;                                    /* device, bf16 */
+    int64_t stride_b, stride_pos, stride_head, stride_page;
+    const int32_t *page_table;      /* device int32 [batch, max_pages_per_seq]; paged only */
+    int32_t page_size;              /* 16 (paged only) */
+    int32_t max_pages_per_seq;
+    int32_t num_pages;              /* physical pages in the pool; page ids are checked against it */
+    const int32_t *ctx_lens;        /* device int32 [batch] */
+    int32_t max_ctx_len;            /* host upper bound of ctx_lens; 1 .. 262144 */
+    float sm_scale;                 /* 0 => 1/sqrt(head_dim), the scale of Eq. 1 */
+} tidal_kv_t;
+
+/* Create a context on CUDA device `device`. workspace_bytes = 0 lets the
+ * workspace grow on demand (a call may then allocate, so size it up front with
+ * tidal_workspace_bytes() before capturing calls into a CUDA graph). */
+tidal_status_t tidal_create(tidal_ctx_t **ctx, int device, size_t workspace_bytes);
+tidal_status_t tidal_destroy(tidal_ctx_t *ctx);
+
+/* Workspace a call with this cache shape and budget k needs (split-context
+ * partial results, the score buffer of a selection layer, top-k histograms). */
+size_t tidal_workspace_bytes(const tidal_kv_t *kv, int32_t k);
+
+/* FullAttention(q, C[:]) of Algorithm 1, Eq. 1 per head:
+ *   out[b,h,:] = softmax_j(q[b,h,:] . K[b,j,g,:] * sm_scale) V[b,j,g,:],  j < ctx_lens[b], g = h / (Hq/Hkv).
+ * The single decode query sees every cached token (no mask). */
+tidal_status_t tidal_full_attn(tidal_ctx_t *ctx, const tidal_kv_t *kv, const void *q,
+                               float *out, void *stream);
+
+/* Token selection layer of Algorithm 1 (Section 3: the inner products are
+ * stored during full attention, then the k tokens with the highest values are
+ * kept): out as tidal_full_attn, and for every (sequence, index head) the
+ * k' = min(k, ctx_lens[b]) positions with the largest scaled logit, equal
+ * logits resolved toward the lower position.
+ *   idx       int32 [batch, Hi, k]: the positions in ascending order, padded with -1.
+ *   idx_count int32 [batch] or NULL: receives k'.
+ *   scores_opt float [batch, Hq, max_ctx_len] or NULL: receives the scaled
+ *             logits q.k*sm_scale (entries at and beyond ctx_lens[b] are unspecified);
+ *             with NULL they live in the workspace. */
+tidal_status_t tidal_select_attn(tidal_ctx_t *ctx, const tidal_kv_t *kv, const void *q,
+                                 int32_t k, int32_t granularity, float *out, int32_t *idx,
+                                 int32_t *idx_count, float *scores_opt, void *stream);
+
+/* SparseAttention(q, C[rho]) of Algorithm 1: Eq. 1 restricted to the positions
+ * listed for the query head's index head hi = h * Hi / Hq, softmax renormalised
+ * over them. Entries < 0 are padding and skipped; an entry >= ctx_lens[b] is
+ * skipped and reported as TIDAL_ERR_INDEX by tidal_device_status(); a repeated
+ * entry counts once per occurrence. Only the first idx_count[b] entries are
+ * read when idx_count is given, else k. A head with no valid entry gets zeros.
+ * num_index_heads must be Hq, Hkv or 1. */
+tidal_status_t tidal_sparse_attn(tidal_ctx_t *ctx, const tidal_kv_t *kv, const void *q,
+                                 const int32_t *idx, const int32_t *idx_count, int32_t k,
+                                 int32_t num_index_heads, float *out, void *stream);
+
+/* One decode step's attention for all layers (the loop of Algorithm 1):
+ * schedule[i] (host, TIDAL_LAYER_*) picks the call for layer i; the token set
+ * rho lives in idx/idx_count, is written by every selection layer and read by
+ * the sparse layers after it. kv_per_layer (host array of descriptors),
+ * q_per_layer and out_per_layer (host arrays of device pointers) have
+ * num_layers entries. A sparse layer before the first selection layer is
+ * TIDAL_ERR_INVALID. Everything is enqueued on `stream` without host waits. */
+tidal_status_t tidal_decode_step(tidal_ctx_t *ctx, int32_t num_layers, const uint8_t *schedule,
+                                 const tidal_kv_t *kv_per_layer, const void *const *q_per_layer,
+                                 float *const *out_per_layer, int32_t k, int32_t granularity,
+                                 int32_t *idx, int32_t *idx_count, void *stream);
+
+/* The same step for a caller whose queries and outputs live in HOST memory
+ * (pinned for full speed): q_host is bf16 [num_layers, batch, Hq, head_dim],
+ * out_host fp32 of the same shape. Copies q to the device, runs
+ * tidal_decode_step with idx/idx_count in the workspace, copies the outputs
+ * back and WAITS for the stream. The KV cache stays resident on the device. */
+tidal_status_t tidal_decode_step_host(tidal_ctx_t *ctx, int32_t num_layers, const uint8_t *schedule,
+                                      const tidal_kv_t *kv_per_layer, const void *q_host,
+                                      float *out_host, int32_t k, int32_t granularity, void *stream);
+
+/* Waits for `stream`, then returns and clears the sticky device status word:
+ * TIDAL_OK, TIDAL_ERR_INDEX, or TIDAL_ERR_CUDA if the stream reports an error. */
+tidal_status_t tidal_device_status(tidal_ctx_t *ctx, void *stream);
+
+/* Kernels launched through this context since it was created. */
+int64_t tidal_launch_count(const tidal_ctx_t *ctx);
+
+const char *tidal_strerror(tidal_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,383 @@
+"""Pins of the CPU oracle against things other than itself: an independent
+evaluation of Eq. 1, closed forms, invariances, brute force, and the facts the
+paper prints (layer mix, KV-cache size). CPU only."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+D = 128
+
+
+def bf16_bits(x: np.ndarray) -> np.ndarray:
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(torch.bfloat16)
+    return t.view(torch.int16).numpy().view(np.uint16)
+
+
+def bf16_val(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def make(B, Hq, Hkv, N, seed, lens=None, scale=0.0):
+    """NHD contiguous cache K,V [B,N,Hkv,D] as bf16 bits + oracle descriptor."""
+    r = np.random.default_rng(seed)
+    q = bf16_bits(r.standard_normal((B, Hq, D)))
+    k = bf16_bits(r.standard_normal((B, N, Hkv, D)))
+    v = bf16_bits(r.standard_normal((B, N, Hkv, D)))
+    lens = np.full(B, N, np.int32) if lens is None else np.asarray(lens, np.int32)
+    kv = oracle.KV(k=k.reshape(-1), v=v.reshape(-1), batch=B, num_q_heads=Hq, num_kv_heads=Hkv,
+                   head_dim=D, ctx_lens=lens, stride_b=N * Hkv * D, stride_pos=Hkv * D,
+                   stride_head=D, sm_scale=scale)
+    return q, k, v, kv
+
+
+def eq1_numpy(q, k, v, lens, idx=None):
+    """Eq. 1 evaluated independently in float64 with numpy matmul/softmax."""
+    B, Hq, _ = q.shape
+    Hkv = k.shape[2]
+    G = Hq // Hkv
+    qf, kf, vf = bf16_val(q), bf16_val(k), bf16_val(v)
+    out = np.zeros((B, Hq, D))
+    for b in range(B):
+        for h in range(Hq):
+            rows = np.arange(lens[b]) if idx is None else idx[b][h]
+            K = kf[b, rows, h // G]
+            V = vf[b, rows, h // G]
+            a = (K @ qf[b, h]) / np.sqrt(D)
+            p = np.exp(a - a.max())
+            out[b, h] = (p / p.sum()) @ V
+    return out
+
+
+# ---- P1: softmax weights -------------------------------------------------
+def test_softmax_weights_sum_to_one():
+    q, k, v, kv = make(1, 2, 2, 777, 1)
+    for h in range(2):
+        s = oracle.logits(kv, q, 0, h)
+        w = oracle.softmax_weights(s)
+        assert abs(w.sum() - 1.0) < 1e-6
+        assert (w >= 0).all()
+        # textbook softmax of the same logits
+        e = np.exp(s.astype(np.float64) - s.max())
+        np.testing.assert_allclose(w, e / e.sum(), rtol=1e-12)
+
+
+# ---- P2: full attention vs an independent formulation ---------------------
+@pytest.mark.parametrize("B,Hq,Hkv,N", [(1, 1, 1, 1), (2, 4, 4, 33), (1, 8, 2, 300), (3, 6, 2, 65)])
+def test_full_attention_matches_eq1(B, Hq, Hkv, N):
+    lens = [max(1, N - 7 * b) for b in range(B)]
+    q, k, v, kv = make(B, Hq, Hkv, N, 10 + N, lens)
+    out, sc = oracle.full_attn(kv, q, want_scores=True)
+    ref = eq1_numpy(q, k, v, lens)
+    np.testing.assert_allclose(out, ref, rtol=0, atol=2e-7)
+    # the emitted scores are A = q K^T / sqrt(d), not the raw inner product and not transposed
+    G = Hq // Hkv
+    for b in range(B):
+        for h in range(Hq):
+            a = bf16_val(k)[b, : lens[b], h // G] @ bf16_val(q)[b, h] / np.sqrt(D)
+            np.testing.assert_allclose(sc[b, h, : lens[b]], a, rtol=0, atol=1e-6)
+
+
+def test_full_attention_matches_torch_sdpa():
+    q, k, v, kv = make(2, 4, 4, 97, 5)
+    out = oracle.full_attn(kv, q)
+    qt = torch.from_numpy(bf16_val(q))[:, :, None, :]
+    kt = torch.from_numpy(bf16_val(k)).permute(0, 2, 1, 3)
+    vt = torch.from_numpy(bf16_val(v)).permute(0, 2, 1, 3)
+    ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt)[:, :, 0, :].numpy()
+    np.testing.assert_allclose(out, ref, rtol=0, atol=2e-7)
+
+
+def test_explicit_scale_is_used():
+    q, k, v, kv = make(1, 2, 2, 50, 6, scale=0.25)
+    _, sc = oracle.full_attn(kv, q, want_scores=True)
+    a = bf16_val(k)[0, :, 0] @ bf16_val(q)[0, 0] * 0.25
+    np.testing.assert_allclose(sc[0, 0], a, atol=1e-5)
+
+
+# ---- P3: k >= N makes sparse attention equal to full attention ------------
+@pytest.mark.parametrize("k", [40, 41, 64])
+def test_sparse_with_full_budget_equals_full(k):
+    q, k_, v, kv = make(2, 4, 2, 40, 3, lens=[40, 29])
+    full = oracle.full_attn(kv, q)
+    out, idx, cnt = oracle.select_attn(kv, q, k)
+    assert cnt.tolist() == [min(k, 40), min(k, 29)]
+    for b, n in enumerate([40, 29]):
+        assert (idx[b, :, : min(k, n)] == np.arange(min(k, n))).all()
+        assert (idx[b, :, min(k, n):] == -1).all()
+    sp = oracle.sparse_attn(kv, q, idx, cnt)
+    assert np.array_equal(out, full)
+    if k >= 40:
+        assert np.array_equal(sp, full)          # bit for bit
+    else:
+        assert np.array_equal(sp[1], full[1])    # the shorter sequence is fully covered
+
+
+# ---- P4: top-k vs brute force and vs ranking by probability ---------------
+def brute_topk(s, k):
+    s = s.astype(np.float64).copy()
+    picked = []
+    for _ in range(min(k, len(s))):
+        j = int(np.argmax(s))           # numpy argmax returns the lowest index among equals
+        picked.append(j)
+        s[j] = -np.inf
+    return sorted(picked)
+
+
+@pytest.mark.parametrize("n,k", [(1, 1), (17, 5), (256, 64), (512, 511), (100, 100), (100, 130)])
+def test_topk_matches_brute_force(n, k):
+    r = np.random.default_rng(n * 1000 + k)
+    s = r.standard_normal(n).astype(np.float32)
+    s[r.integers(0, n, n // 4)] = np.float32(0.5)      # many exact ties
+    idx = oracle.topk(s, k)
+    kk = min(n, k)
+    assert idx[:kk].tolist() == brute_topk(s, k)
+    assert (idx[kk:] == -1).all()
+
+
+def test_topk_by_logit_equals_topk_by_probability():
+    q, k, v, kv = make(1, 4, 4, 400, 8)
+    _, idx, _ = oracle.select_attn(kv, q, 37)
+    for h in range(4):
+        w = oracle.softmax_weights(oracle.logits(kv, q, 0, h))
+        by_prob = np.sort(np.argsort(-w, kind="stable")[:37])
+        assert idx[0, h].tolist() == by_prob.tolist()
+
+
+def test_topk_all_equal_takes_lowest_positions():
+    s = np.zeros(50, np.float32)
+    assert oracle.topk(s, 7).tolist() == list(range(7))
+
+
+# ---- P5: the selected set retains the most softmax mass --------------------
+def test_selected_set_maximises_retained_mass():
+    q, k, v, kv = make(1, 2, 2, 300, 9)
+    _, idx, _ = oracle.select_attn(kv, q, 30)
+    r = np.random.default_rng(0)
+    for h in range(2):
+        w = oracle.softmax_weights(oracle.logits(kv, q, 0, h))
+        mass = w[idx[0, h]].sum()
+        for _ in range(1000):
+            assert w[r.choice(300, 30, replace=False)].sum() <= mass + 1e-15
+        inside = set(idx[0, h].tolist())
+        worst_in = min(w[j] for j in inside)
+        best_out = max(w[j] for j in range(300) if j not in inside)
+        assert best_out <= worst_in                 # no single swap improves it
+
+
+# ---- P6: closed-form bound on sparse-vs-full error ------------------------
+def test_sparse_error_is_bounded_by_dropped_mass():
+    q, k, v, kv = make(1, 4, 2, 500, 11)
+    full = oracle.full_attn(kv, q)
+    _, idx, cnt = oracle.select_attn(kv, q, 100)
+    sp = oracle.sparse_attn(kv, q, idx, cnt)
+    vmax = np.abs(bf16_val(v)).max()
+    for h in range(4):
+        w = oracle.softmax_weights(oracle.logits(kv, q, 0, h))
+        dropped = 1.0 - w[idx[0, h]].sum()
+        assert np.abs(full[0, h] - sp[0, h]).max() <= 2 * dropped * vmax + 1e-6
+
+
+# ---- P7: closed-form special cases ----------------------------------------
+def test_zero_query_gives_mean_of_values_and_first_positions():
+    q, k, v, kv = make(1, 2, 1, 64, 12)
+    q[:] = 0
+    out, idx, _ = oracle.select_attn(kv, q, 9)
+    mean_v = bf16_val(v)[0, :, 0].mean(axis=0)
+    np.testing.assert_allclose(out[0, 0], mean_v, atol=1e-6)
+    np.testing.assert_allclose(out[0, 1], mean_v, atol=1e-6)
+    assert idx[0, 0].tolist() == list(range(9))
+
+
+def test_single_token_returns_its_value():
+    q, k, v, kv = make(1, 2, 2, 1, 13)
+    out = oracle.full_attn(kv, q)
+    np.testing.assert_array_equal(out[0], bf16_val(v)[0, 0].astype(np.float32))
+
+
+def test_dominant_key_returns_its_value_row():
+    q, k, v, kv = make(1, 1, 1, 128, 14)
+    kf = bf16_val(k)
+    kf[0, 77, 0] = 8.0 * bf16_val(q)[0, 0]
+    kv.k = bf16_bits(kf).reshape(-1)
+    out, idx, _ = oracle.select_attn(kv, q, 4)
+    assert 77 in idx[0, 0].tolist()
+    np.testing.assert_allclose(out[0, 0], bf16_val(v)[0, 77, 0], atol=1e-6)
+
+
+def test_sparse_uses_only_listed_rows_and_renormalises():
+    q, k, v, kv = make(1, 2, 2, 90, 15)
+    idx = np.full((1, 2, 6), -1, np.int32)
+    idx[0, 0, :4] = [3, 17, 18, 80]
+    idx[0, 1, :5] = [0, 1, 2, 88, 89]
+    sp = oracle.sparse_attn(kv, q, idx)
+    ref = eq1_numpy(q, k, v, [90], idx=[[np.array([3, 17, 18, 80]), np.array([0, 1, 2, 88, 89])]])
+    np.testing.assert_allclose(sp, ref, atol=2e-7)
+    # a repeated entry counts twice; order does not matter
+    idx2 = np.full((1, 2, 6), -1, np.int32)
+    idx2[0, 0, :5] = [80, 3, 3, 18, 17]
+    idx2[0, 1, :5] = [89, 88, 2, 1, 0]
+    sp2 = oracle.sparse_attn(kv, q, idx2)
+    ref2 = eq1_numpy(q, k, v, [90], idx=[[np.array([80, 3, 3, 18, 17]), np.array([0, 1, 2, 88, 89])]])
+    np.testing.assert_allclose(sp2, ref2, atol=2e-7)
+    # idx_count limits how many entries are read
+    sp3 = oracle.sparse_attn(kv, q, idx, np.array([2], np.int32))
+    ref3 = eq1_numpy(q, k, v, [90], idx=[[np.array([3, 17]), np.array([0, 1])]])
+    np.testing.assert_allclose(sp3, ref3, atol=2e-7)
+
+
+# ---- P8: invariances --------------------------------------------------------
+def test_permuting_positions_permutes_indices_only():
+    q, k, v, kv = make(1, 2, 2, 120, 16)
+    out, idx, _ = oracle.select_attn(kv, q, 20)
+    perm = np.random.default_rng(1).permutation(120)          # new position of old j is perm[j]
+    k2, v2 = np.empty_like(k), np.empty_like(v)
+    k2[0, perm] = k[0]
+    v2[0, perm] = v[0]
+    kv2 = oracle.KV(k=k2.reshape(-1), v=v2.reshape(-1), batch=1, num_q_heads=2, num_kv_heads=2,
+                    head_dim=D, ctx_lens=kv.ctx_lens, stride_b=kv.stride_b,
+                    stride_pos=kv.stride_pos, stride_head=kv.stride_head)
+    out2, idx2, _ = oracle.select_attn(kv2, q, 20)
+    np.testing.assert_allclose(out2, out, atol=1e-6)
+    for h in range(2):
+        assert sorted(perm[idx[0, h]].tolist()) == idx2[0, h].tolist()
+
+
+def test_constant_logit_shift_changes_nothing():
+    # adding to every key a vector u orthogonal to nothing in particular but with
+    # the same q.u for all positions shifts every logit equally
+    r = np.random.default_rng(17)
+    q, k, v, kv = make(1, 1, 1, 80, 17)
+    qf = bf16_val(q)[0, 0]
+    u = np.zeros(D)
+    u[0] = 4.0 if qf[0] != 0 else 0.0          # exactly representable shift along one axis
+    kf = bf16_val(k)
+    kf[..., 0] = np.round(kf[..., 0] * 4) / 4   # keep k + u exactly representable in bf16
+    k1 = bf16_bits(kf)
+    k2 = bf16_bits(kf + u)
+    assert np.array_equal(bf16_val(k2), kf + u)
+    outs = []
+    for kk in (k1, k2):
+        kvx = oracle.KV(k=kk.reshape(-1), v=v.reshape(-1), batch=1, num_q_heads=1, num_kv_heads=1,
+                        head_dim=D, ctx_lens=kv.ctx_lens, stride_b=kv.stride_b,
+                        stride_pos=kv.stride_pos, stride_head=kv.stride_head)
+        outs.append(oracle.select_attn(kvx, q, 10))
+    np.testing.assert_allclose(outs[0][0], outs[1][0], atol=1e-5)
+    assert outs[0][1].tolist() == outs[1][1].tolist()
+
+
+# ---- P9: GQA equals MHA on a head-repeated cache ----------------------------
+def test_gqa_equals_mha_with_repeated_kv_heads():
+    B, Hq, Hkv, N = 2, 8, 2, 70
+    q, k, v, kv = make(B, Hq, Hkv, N, 18, lens=[70, 33])
+    G = Hq // Hkv
+    k_rep = np.repeat(k, G, axis=2)
+    v_rep = np.repeat(v, G, axis=2)
+    kv_mha = oracle.KV(k=k_rep.reshape(-1), v=v_rep.reshape(-1), batch=B, num_q_heads=Hq,
+                       num_kv_heads=Hq, head_dim=D, ctx_lens=kv.ctx_lens, stride_b=N * Hq * D,
+                       stride_pos=Hq * D, stride_head=D)
+    a = oracle.select_attn(kv, q, 12)
+    b = oracle.select_attn(kv_mha, q, 12)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    assert np.array_equal(oracle.sparse_attn(kv, q, a[1], a[2]),
+                          oracle.sparse_attn(kv_mha, q, b[1], b[2]))
+
+
+# ---- P10: paged equals contiguous -------------------------------------------
+def test_paged_equals_contiguous():
+    B, Hq, Hkv, N, PS = 2, 4, 2, 75, 16
+    lens = [75, 40]
+    q, k, v, kv = make(B, Hq, Hkv, N, 19, lens=lens)
+    pages_per = [(n + PS - 1) // PS for n in lens]
+    total = sum(pages_per) + 3
+    perm = np.random.default_rng(2).permutation(total)
+    pt = np.zeros((B, max(pages_per)), np.int32)
+    pool_k = np.zeros((total, PS, Hkv, D), np.uint16)
+    pool_v = np.zeros((total, PS, Hkv, D), np.uint16)
+    at = 0
+    for b in range(B):
+        for lp in range(pages_per[b]):
+            phys = perm[at]; at += 1
+            pt[b, lp] = phys
+            lo, hi = lp * PS, min(lens[b], lp * PS + PS)
+            pool_k[phys, : hi - lo] = k[b, lo:hi]
+            pool_v[phys, : hi - lo] = v[b, lo:hi]
+    kvp = oracle.KV(k=pool_k.reshape(-1), v=pool_v.reshape(-1), batch=B, num_q_heads=Hq,
+                    num_kv_heads=Hkv, head_dim=D, ctx_lens=np.asarray(lens, np.int32),
+                    stride_pos=Hkv * D, stride_head=D, stride_page=PS * Hkv * D,
+                    page_table=pt, page_size=PS)
+    a = oracle.select_attn(kv, q, 21)
+    b = oracle.select_attn(kvp, q, 21)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    assert np.array_equal(oracle.sparse_attn(kv, q, a[1], a[2]),
+                          oracle.sparse_attn(kvp, q, b[1], b[2]))
+
+
+# ---- index-head granularities (aggregated ranking) ---------------------------
+def test_aggregated_granularity_ranks_by_summed_logits():
+    q, k, v, kv = make(1, 8, 2, 200, 20)
+    _, _, _, sc = oracle.select_attn(kv, q, 16, want_scores=True)
+    _, idx_kv, _ = oracle.select_attn(kv, q, 16, num_index_heads=2)
+    _, idx_sh, _ = oracle.select_attn(kv, q, 16, num_index_heads=1)
+    for g in range(2):
+        agg = sc[0, 4 * g: 4 * g + 4].astype(np.float64).sum(axis=0)
+        assert idx_kv[0, g].tolist() == brute_topk(agg.astype(np.float32), 16)
+    agg = sc[0].astype(np.float64).sum(axis=0)
+    assert idx_sh[0, 0].tolist() == brute_topk(agg.astype(np.float32), 16)
+    # sparse attention maps query head h to index head h*Hi/Hq
+    sp = oracle.sparse_attn(kv, q, idx_kv)
+    ref = eq1_numpy(q, k, v, [200], idx=[[idx_kv[0, h // 4] for h in range(8)]])
+    np.testing.assert_allclose(sp, ref, atol=2e-7)
+
+
+# ---- P11: schedule and rho persistence ---------------------------------------
+def _golden(name):
+    rows = {}
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                key, val = line.split("=")
+                rows[key.strip()] = val.strip()
+    return rows
+
+
+def test_layer_mix_matches_the_paper():
+    g = _golden("layer_mix.txt")
+    for L in (32, 64):
+        s = oracle.schedule(L, 13).tolist()
+        full, sel, sparse = (int(x) for x in g[f"layers_{L}"].split("+"))
+        assert (s.count(0), s.count(1), s.count(2)) == (full, sel, sparse)
+        assert s[0] == s[1] == oracle.LAYER_FULL
+        assert s[2] == oracle.LAYER_SELECT and s[13] == oracle.LAYER_SELECT
+
+
+def test_kv_cache_size_formula_matches_the_paper():
+    g = _golden("kv_cache_size.txt")
+    layers, heads, dim, seq = (int(g[x]) for x in ("layers", "kv_heads", "head_dim", "seq_len"))
+    total = layers * heads * dim * seq * 2 * 2            # K and V, 2 bytes each
+    assert total == int(g["gib"]) * 2 ** 30
+
+
+def test_decode_step_keeps_rho_until_the_next_selection_layer():
+    L, B, Hq, Hkv, N, k = 7, 1, 4, 2, 60, 9
+    sched = [0, 0, 1, 2, 1, 2, 2]
+    caches = [make(B, Hq, Hkv, N, 100 + i) for i in range(L)]
+    qs = [c[0] for c in caches]
+    kvs = [c[3] for c in caches]
+    outs, idx, cnt = oracle.decode_step(sched, kvs, qs, k)
+    _, rho2, c2 = oracle.select_attn(kvs[2], qs[2], k)
+    _, rho4, c4 = oracle.select_attn(kvs[4], qs[4], k)
+    assert not np.array_equal(rho2, rho4)
+    assert np.array_equal(idx, rho4)
+    assert np.array_equal(outs[0], oracle.full_attn(kvs[0], qs[0]))
+    assert np.array_equal(outs[2], oracle.full_attn(kvs[2], qs[2]))     # selection layer output is full attention
+    assert np.array_equal(outs[3], oracle.sparse_attn(kvs[3], qs[3], rho2, c2))
+    assert np.array_equal(outs[5], oracle.sparse_attn(kvs[5], qs[5], rho4, c4))
+    assert np.array_equal(outs[6], oracle.sparse_attn(kvs[6], qs[6], rho4, c4))
+    with pytest.raises(ValueError):
+        oracle.decode_step([0, 2], kvs[:2], qs[:2], k)
