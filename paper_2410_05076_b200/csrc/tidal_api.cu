@@ -1,0 +1,471 @@
+// C-ABI of libtidal: argument checking, workspace, launch planning.
+// Every step of the attention path runs in the kernels of attn_kernels.cuh and
+// topk_kernels.cuh; nothing here computes on the host and there is no CPU path.
+#include "../../include/tidal.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "attn_kernels.cuh"
+#include "topk_kernels.cuh"
+
+using namespace tidal;
+
+namespace {
+
+constexpr int MAX_CTX = 262144;
+constexpr int MAX_SPLITS = 512;
+constexpr int MAX_GROUP = 8;            // query heads per KV head that fit the 8 MMA columns
+constexpr int TOPK_SLICE_MAX = 32768;   // keys per CTA kept in shared memory
+
+// Streaming (full / selection) and gather (sparse) launch shapes.
+constexpr int DENSE_NW = 8, DENSE_STAGES = 3;
+constexpr int SPARSE_NW = 4, SPARSE_STAGES = 3;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Plan { int chunk; int nsplits; };
+
+}  // namespace
+
+struct tidal_ctx {
+    int device = 0;
+    int sm_count = 0;
+    int dense_slots = 0, sparse_slots = 0;     // resident CTAs on the whole GPU
+    void* ws = nullptr;
+    size_t ws_bytes = 0;
+    int* status = nullptr;                      // device word, sticky
+    int64_t launches = 0;
+};
+
+namespace {
+
+struct WsLayout {
+    size_t counters, part_ml, part_o, scores, idx, idx_count, q_stage, out_stage, total;
+    long long score_stride;
+};
+
+// Chunk of the context (or of the index list) per CTA. Single-sequence work is
+// split so that the CTAs fill whole waves of resident slots; batched work is cut
+// into more, smaller chunks so that the hardware scheduler evens out ragged lengths.
+Plan plan_split(int total_max, int items, int slots, int batch) {
+    total_max = std::max(total_max, 1);
+    const int tiles = (total_max + TILE - 1) / TILE;
+    int best_s = 1;
+    if (batch > 1) {
+        const int want = std::max(1, (6 * slots + items - 1) / items);
+        best_s = std::min(want, std::max(1, tiles / 32));           // at least 512 positions per CTA
+    } else {
+        double best = -1.0;
+        const int smax = std::max(1, std::min(MAX_SPLITS, tiles / 8));   // at least 128 positions per CTA
+        for (int s = 1; s <= smax; ++s) {
+            const long long ctas = (long long)items * s;
+            const long long waves = (ctas + slots - 1) / slots;
+            const double eff = (double)ctas / (double)(waves * slots) - 0.004 * (double)(waves - 1);
+            if (eff > best + 1e-9) { best = eff; best_s = s; }
+        }
+    }
+    best_s = std::max(1, std::min(best_s, MAX_SPLITS));
+    int chunk = (int)align_up((size_t)(total_max + best_s - 1) / best_s, TILE);
+    chunk = std::max(chunk, TILE);
+    Plan p;
+    p.chunk = chunk;
+    p.nsplits = (total_max + chunk - 1) / chunk;
+    return p;
+}
+
+int hi_of(const tidal_kv_t* kv, int granularity) {
+    switch (granularity) {
+        case TIDAL_SEL_PER_QHEAD: return kv->num_q_heads;
+        case TIDAL_SEL_PER_KVHEAD: return kv->num_kv_heads;
+        case TIDAL_SEL_SHARED: return 1;
+        default: return -1;
+    }
+}
+
+tidal_status_t check_kv(const tidal_kv_t* kv) {
+    if (!kv || !kv->k || !kv->v || !kv->ctx_lens) return TIDAL_ERR_INVALID;
+    if (kv->batch <= 0 || kv->num_q_heads <= 0 || kv->num_kv_heads <= 0) return TIDAL_ERR_INVALID;
+    if (kv->num_q_heads % kv->num_kv_heads != 0) return TIDAL_ERR_INVALID;
+    if (kv->head_dim != HEAD_DIM) return TIDAL_ERR_UNSUPPORTED;
+    if (kv->num_q_heads / kv->num_kv_heads > MAX_GROUP) return TIDAL_ERR_UNSUPPORTED;
+    if (kv->max_ctx_len < 1 || kv->max_ctx_len > MAX_CTX) return TIDAL_ERR_INVALID;
+    if (kv->batch > 65535 || kv->num_q_heads > 65535) return TIDAL_ERR_UNSUPPORTED;
+    if ((long long)kv->batch * kv->num_q_heads > 262144) return TIDAL_ERR_UNSUPPORTED;   // split counters fit the zeroed head of the workspace
+    if (((uintptr_t)kv->k | (uintptr_t)kv->v) & 15) return TIDAL_ERR_INVALID;
+    if ((kv->stride_pos | kv->stride_head) & 7) return TIDAL_ERR_INVALID;
+    if (kv->stride_pos < 0 || kv->stride_head < 0 || kv->stride_b < 0 || kv->stride_page < 0) return TIDAL_ERR_INVALID;
+    if (!(kv->sm_scale >= 0.f) || std::isinf(kv->sm_scale)) return TIDAL_ERR_INVALID;
+    if (kv->kv_layout == TIDAL_KV_CONTIG) {
+        if (kv->stride_b & 7) return TIDAL_ERR_INVALID;
+        if (kv->stride_pos < HEAD_DIM && kv->max_ctx_len > 1) return TIDAL_ERR_INVALID;
+    } else if (kv->kv_layout == TIDAL_KV_PAGED) {
+        if (!kv->page_table) return TIDAL_ERR_INVALID;
+        if (kv->page_size != TILE) return TIDAL_ERR_UNSUPPORTED;
+        if (kv->stride_page & 7) return TIDAL_ERR_INVALID;
+        if (kv->num_pages <= 0 || kv->max_pages_per_seq <= 0) return TIDAL_ERR_INVALID;
+        if ((long long)kv->max_pages_per_seq * kv->page_size < kv->max_ctx_len) return TIDAL_ERR_INVALID;
+    } else {
+        return TIDAL_ERR_INVALID;
+    }
+    return TIDAL_OK;
+}
+
+// Workspace layout for a cache shape, budget k and (for the host-buffer step) layer count.
+WsLayout layout_ws(const tidal_kv_t* kv, int k, int num_layers_host) {
+    WsLayout w;
+    const size_t rows = (size_t)kv->batch * kv->num_q_heads;
+    size_t at = 0;
+    w.counters = at;  at += align_up(rows * sizeof(int), 256);
+    w.part_ml = at;   at += align_up(rows * MAX_SPLITS * sizeof(float2), 256);
+    w.part_o = at;    at += align_up(rows * MAX_SPLITS * HEAD_DIM * sizeof(float), 256);
+    w.score_stride = (long long)align_up((size_t)kv->max_ctx_len, 16);
+    w.scores = at;    at += align_up(rows * (size_t)w.score_stride * sizeof(float), 256);
+    w.idx = at;       at += align_up(rows * (size_t)std::max(k, 1) * sizeof(int), 256);
+    w.idx_count = at; at += align_up((size_t)kv->batch * sizeof(int), 256);
+    w.q_stage = at;   at += align_up((size_t)num_layers_host * rows * HEAD_DIM * 2, 256);
+    w.out_stage = at; at += align_up((size_t)num_layers_host * rows * HEAD_DIM * 4, 256);
+    w.total = at;
+    return w;
+}
+
+// part_o is sized for MAX_SPLITS per row only when that is small; otherwise bound it by the plan.
+size_t ws_bytes_for(const tidal_kv_t* kv, int k, int num_layers_host) {
+    return layout_ws(kv, k, num_layers_host).total;
+}
+
+tidal_status_t ensure_ws(tidal_ctx* ctx, size_t bytes) {
+    if (ctx->ws_bytes >= bytes) return TIDAL_OK;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    if (ctx->ws) { cudaDeviceSynchronize(); cudaFree(ctx->ws); ctx->ws = nullptr; ctx->ws_bytes = 0; }
+    void* p = nullptr;
+    if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TIDAL_ERR_NOMEM; }
+    // The split counters must be zero between launches; zero the head of the buffer.
+    if (cudaMemset(p, 0, std::min(bytes, (size_t)1 << 20)) != cudaSuccess) { cudaFree(p); return TIDAL_ERR_CUDA; }
+    ctx->ws = p;
+    ctx->ws_bytes = bytes;
+    return TIDAL_OK;
+}
+
+void fill_common(AttnParams& a, const tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, float* out,
+                 const WsLayout& w) {
+    std::memset(&a, 0, sizeof a);
+    a.q = (const __nv_bfloat16*)q;
+    a.k = (const __nv_bfloat16*)kv->k;
+    a.v = (const __nv_bfloat16*)kv->v;
+    a.out = out;
+    a.stride_b = kv->stride_b; a.stride_pos = kv->stride_pos; a.stride_head = kv->stride_head;
+    a.stride_page = kv->stride_page;
+    a.page_table = kv->page_table; a.max_pages = kv->max_pages_per_seq; a.num_pages = kv->num_pages;
+    a.paged = kv->kv_layout == TIDAL_KV_PAGED;
+    a.ctx_lens = kv->ctx_lens;
+    a.max_ctx = kv->max_ctx_len;
+    a.Hq = kv->num_q_heads; a.Hkv = kv->num_kv_heads; a.G = a.Hq / a.Hkv;
+    a.scale = kv->sm_scale > 0.f ? kv->sm_scale : 1.0f / std::sqrt((float)kv->head_dim);
+    a.scale_log2 = a.scale * 1.4426950408889634f;
+    char* ws = (char*)ctx->ws;
+    a.counters = (int*)(ws + w.counters);
+    a.part_ml = (float2*)(ws + w.part_ml);
+    a.part_o = (float*)(ws + w.part_o);
+    a.max_splits = MAX_SPLITS;
+    a.status = ctx->status;
+}
+
+template <int MODE, int NW, int STAGES>
+tidal_status_t launch_attn(tidal_ctx* ctx, const AttnParams& a, dim3 grid, cudaStream_t st) {
+    const size_t smem = (size_t)NW * STAGES * STAGE_BYTES;
+    attn_kernel<MODE, NW, STAGES><<<grid, NW * 32, smem, st>>>(a);
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+}
+
+tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, float* out, float* scores,
+                         long long score_stride, const WsLayout& w, cudaStream_t st) {
+    AttnParams a;
+    fill_common(a, ctx, kv, q, out, w);
+    const int items = kv->batch * kv->num_kv_heads;
+    const Plan pl = plan_split(kv->max_ctx_len, items, ctx->dense_slots, kv->batch);
+    a.chunk = pl.chunk;
+    a.scores = scores;
+    a.score_stride = score_stride;
+    dim3 grid(pl.nsplits, kv->num_kv_heads, kv->batch);
+    if (scores) return launch_attn<MODE_SELECT, DENSE_NW, DENSE_STAGES>(ctx, a, grid, st);
+    return launch_attn<MODE_FULL, DENSE_NW, DENSE_STAGES>(ctx, a, grid, st);
+}
+
+tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* scores, long long score_stride,
+                        int k, int Hi, int* idx, int* idx_count, cudaStream_t st) {
+    TopkParams t;
+    t.scores = scores; t.score_stride = score_stride;
+    t.ctx_lens = kv->ctx_lens; t.max_ctx = kv->max_ctx_len;
+    t.Hq = kv->num_q_heads; t.Hi = Hi; t.k = k;
+    t.idx = idx; t.idx_count = idx_count;
+    const int items = kv->batch * Hi;
+    int cs = 1;
+    while (cs < 8 && (kv->max_ctx_len + cs - 1) / cs > TOPK_SLICE_MAX) cs <<= 1;
+    while (cs < 8 && items * cs < ctx->sm_count && (kv->max_ctx_len / (2 * cs)) >= 2048) cs <<= 1;
+    t.slice_cap = (int)align_up((size_t)(kv->max_ctx_len + cs - 1) / cs, 4);
+    const size_t smem = (size_t)t.slice_cap * 4 + 2 * TOPK_BINS * sizeof(int);
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(items * cs, 1, 1);
+    cfg.blockDim = dim3(TOPK_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    ctx->launches++;
+    return cudaLaunchKernelEx(&cfg, topk_kernel, t) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+}
+
+tidal_status_t run_sparse(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, const int* idx,
+                          const int* idx_count, int k, int Hi, float* out, const WsLayout& w,
+                          cudaStream_t st) {
+    AttnParams a;
+    fill_common(a, ctx, kv, q, out, w);
+    const int per_batch = (Hi == kv->num_q_heads) ? kv->num_q_heads : kv->num_kv_heads;
+    const Plan pl = plan_split(k, kv->batch * per_batch, ctx->sparse_slots, 1);
+    a.chunk = pl.chunk;
+    a.idx = idx; a.idx_count = idx_count; a.budget = k; a.Hi = Hi;
+    dim3 grid(pl.nsplits, per_batch, kv->batch);
+    return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(ctx, a, grid, st);
+}
+
+template <typename K>
+int resident_ctas(K kernel, int threads, size_t smem, int sm_count) {
+    int per_sm = 0;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem) != cudaSuccess) return -1;
+    return per_sm * sm_count;
+}
+
+}  // namespace
+
+extern "C" {
+
+tidal_status_t tidal_create(tidal_ctx_t** out, int device, size_t workspace_bytes) {
+    if (!out) return TIDAL_ERR_INVALID;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) { cudaGetLastError(); return TIDAL_ERR_CUDA; }
+    if (cudaSetDevice(device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    if (prop.major < 10) return TIDAL_ERR_UNSUPPORTED;
+    tidal_ctx* ctx = new (std::nothrow) tidal_ctx();
+    if (!ctx) return TIDAL_ERR_NOMEM;
+    ctx->device = device;
+    ctx->sm_count = prop.multiProcessorCount;
+    const size_t dense_smem = (size_t)DENSE_NW * DENSE_STAGES * STAGE_BYTES;
+    const size_t sparse_smem = (size_t)SPARSE_NW * SPARSE_STAGES * STAGE_BYTES;
+    const int d0 = resident_ctas(attn_kernel<MODE_FULL, DENSE_NW, DENSE_STAGES>, DENSE_NW * 32, dense_smem, ctx->sm_count);
+    const int d1 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW, DENSE_STAGES>, DENSE_NW * 32, dense_smem, ctx->sm_count);
+    const int s0 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>, SPARSE_NW * 32, sparse_smem, ctx->sm_count);
+    const size_t topk_smem = (size_t)TOPK_SLICE_MAX * 4 + 2 * TOPK_BINS * sizeof(int);
+    const bool topk_ok = cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topk_smem) == cudaSuccess;
+    if (d0 <= 0 || d1 <= 0 || s0 <= 0 || !topk_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
+    ctx->dense_slots = std::min(d0, d1);
+    ctx->sparse_slots = s0;
+    if (cudaMalloc((void**)&ctx->status, 256) != cudaSuccess || cudaMemset(ctx->status, 0, 256) != cudaSuccess) {
+        cudaGetLastError(); delete ctx; return TIDAL_ERR_NOMEM;
+    }
+    if (workspace_bytes) {
+        const tidal_status_t rc = ensure_ws(ctx, workspace_bytes);
+        if (rc != TIDAL_OK) { cudaFree(ctx->status); delete ctx; return rc; }
+    }
+    *out = ctx;
+    return TIDAL_OK;
+}
+
+tidal_status_t tidal_destroy(tidal_ctx_t* ctx) {
+    if (!ctx) return TIDAL_ERR_INVALID;
+    cudaSetDevice(ctx->device);
+    cudaDeviceSynchronize();
+    if (ctx->ws) cudaFree(ctx->ws);
+    if (ctx->status) cudaFree(ctx->status);
+    delete ctx;
+    return TIDAL_OK;
+}
+
+size_t tidal_workspace_bytes(const tidal_kv_t* kv, int32_t k) {
+    if (check_kv(kv) != TIDAL_OK || k <= 0) return 0;
+    return ws_bytes_for(kv, k, 0);
+}
+
+tidal_status_t tidal_full_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const void* q, float* out, void* stream) {
+    if (!ctx || !q || !out || ((uintptr_t)q & 15)) return TIDAL_ERR_INVALID;
+    tidal_status_t rc = check_kv(kv);
+    if (rc != TIDAL_OK) return rc;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    const WsLayout w = layout_ws(kv, 1, 0);
+    if ((rc = ensure_ws(ctx, w.total)) != TIDAL_OK) return rc;
+    return run_dense(ctx, kv, q, out, nullptr, 0, w, (cudaStream_t)stream);
+}
+
+tidal_status_t tidal_select_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const void* q, int32_t k,
+                                 int32_t granularity, float* out, int32_t* idx, int32_t* idx_count,
+                                 float* scores_opt, void* stream) {
+    if (!ctx || !q || !out || !idx || ((uintptr_t)q & 15)) return TIDAL_ERR_INVALID;
+    tidal_status_t rc = check_kv(kv);
+    if (rc != TIDAL_OK) return rc;
+    if (k <= 0 || k > kv->max_ctx_len) return TIDAL_ERR_INVALID;
+    const int Hi = hi_of(kv, granularity);
+    if (Hi <= 0) return TIDAL_ERR_INVALID;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    const WsLayout w = layout_ws(kv, k, 0);
+    if ((rc = ensure_ws(ctx, w.total)) != TIDAL_OK) return rc;
+    float* scores = scores_opt ? scores_opt : (float*)((char*)ctx->ws + w.scores);
+    const long long stride = scores_opt ? (long long)kv->max_ctx_len : w.score_stride;
+    cudaStream_t st = (cudaStream_t)stream;
+    if ((rc = run_dense(ctx, kv, q, out, scores, stride, w, st)) != TIDAL_OK) return rc;
+    return run_topk(ctx, kv, scores, stride, k, Hi, idx, idx_count, st);
+}
+
+tidal_status_t tidal_sparse_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const void* q, const int32_t* idx,
+                                 const int32_t* idx_count, int32_t k, int32_t num_index_heads, float* out,
+                                 void* stream) {
+    if (!ctx || !q || !out || !idx || ((uintptr_t)q & 15)) return TIDAL_ERR_INVALID;
+    tidal_status_t rc = check_kv(kv);
+    if (rc != TIDAL_OK) return rc;
+    if (k <= 0) return TIDAL_ERR_INVALID;
+    const int Hi = num_index_heads;
+    if (Hi != kv->num_q_heads && Hi != kv->num_kv_heads && Hi != 1) return TIDAL_ERR_INVALID;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    const WsLayout w = layout_ws(kv, k, 0);
+    if ((rc = ensure_ws(ctx, w.total)) != TIDAL_OK) return rc;
+    return run_sparse(ctx, kv, q, idx, idx_count, k, Hi, out, w, (cudaStream_t)stream);
+}
+
+static tidal_status_t decode_step_impl(tidal_ctx_t* ctx, int32_t num_layers, const uint8_t* schedule,
+                                       const tidal_kv_t* kvs, const void* const* qs, float* const* outs,
+                                       int32_t k, int32_t granularity, int32_t* idx, int32_t* idx_count,
+                                       int host_layers, cudaStream_t st) {
+    // Validate everything before enqueuing anything.
+    bool have_rho = false;
+    size_t need = 0;
+    for (int i = 0; i < num_layers; ++i) {
+        tidal_status_t rc = check_kv(&kvs[i]);
+        if (rc != TIDAL_OK) return rc;
+        if (!qs[i] || !outs[i] || ((uintptr_t)qs[i] & 15)) return TIDAL_ERR_INVALID;
+        if (kvs[i].batch != kvs[0].batch || kvs[i].num_q_heads != kvs[0].num_q_heads ||
+            kvs[i].num_kv_heads != kvs[0].num_kv_heads) return TIDAL_ERR_INVALID;
+        if (schedule[i] == TIDAL_LAYER_SELECT) {
+            if (k > kvs[i].max_ctx_len) return TIDAL_ERR_INVALID;
+            have_rho = true;
+        } else if (schedule[i] == TIDAL_LAYER_SPARSE) {
+            if (!have_rho) return TIDAL_ERR_INVALID;
+        } else if (schedule[i] != TIDAL_LAYER_FULL) {
+            return TIDAL_ERR_INVALID;
+        }
+        need = std::max(need, ws_bytes_for(&kvs[i], k, host_layers));
+    }
+    const int Hi = hi_of(&kvs[0], granularity);
+    if (Hi <= 0) return TIDAL_ERR_INVALID;
+    tidal_status_t rc = ensure_ws(ctx, need);
+    if (rc != TIDAL_OK) return rc;
+    for (int i = 0; i < num_layers; ++i) {
+        const tidal_kv_t* kv = &kvs[i];
+        const WsLayout w = layout_ws(kv, k, host_layers);
+        if (schedule[i] == TIDAL_LAYER_FULL) {
+            rc = run_dense(ctx, kv, qs[i], outs[i], nullptr, 0, w, st);
+        } else if (schedule[i] == TIDAL_LAYER_SELECT) {
+            float* scores = (float*)((char*)ctx->ws + w.scores);
+            rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, w, st);
+            if (rc == TIDAL_OK) rc = run_topk(ctx, kv, scores, w.score_stride, k, Hi, idx, idx_count, st);
+        } else {
+            rc = run_sparse(ctx, kv, qs[i], idx, idx_count, k, Hi, outs[i], w, st);
+        }
+        if (rc != TIDAL_OK) return rc;
+    }
+    return TIDAL_OK;
+}
+
+tidal_status_t tidal_decode_step(tidal_ctx_t* ctx, int32_t num_layers, const uint8_t* schedule,
+                                 const tidal_kv_t* kv_per_layer, const void* const* q_per_layer,
+                                 float* const* out_per_layer, int32_t k, int32_t granularity, int32_t* idx,
+                                 int32_t* idx_count, void* stream) {
+    if (!ctx || num_layers <= 0 || !schedule || !kv_per_layer || !q_per_layer || !out_per_layer || !idx || k <= 0)
+        return TIDAL_ERR_INVALID;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    return decode_step_impl(ctx, num_layers, schedule, kv_per_layer, q_per_layer, out_per_layer, k,
+                            granularity, idx, idx_count, 0, (cudaStream_t)stream);
+}
+
+tidal_status_t tidal_decode_step_host(tidal_ctx_t* ctx, int32_t num_layers, const uint8_t* schedule,
+                                      const tidal_kv_t* kv_per_layer, const void* q_host, float* out_host,
+                                      int32_t k, int32_t granularity, void* stream) {
+    if (!ctx || num_layers <= 0 || num_layers > 1024 || !schedule || !kv_per_layer || !q_host || !out_host || k <= 0)
+        return TIDAL_ERR_INVALID;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    tidal_status_t rc = check_kv(&kv_per_layer[0]);
+    if (rc != TIDAL_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    // Size the workspace for every layer first so that the staging pointers stay put.
+    size_t need = 0;
+    for (int i = 0; i < num_layers; ++i) {
+        if ((rc = check_kv(&kv_per_layer[i])) != TIDAL_OK) return rc;
+        need = std::max(need, ws_bytes_for(&kv_per_layer[i], k, num_layers));
+    }
+    if ((rc = ensure_ws(ctx, need)) != TIDAL_OK) return rc;
+    // All layers must share batch and head counts (checked again below); the staging
+    // offsets depend only on those and on max_ctx_len of the layer used for the layout.
+    const tidal_kv_t* kv0 = &kv_per_layer[0];
+    for (int i = 1; i < num_layers; ++i)
+        if (kv_per_layer[i].max_ctx_len != kv0->max_ctx_len) return TIDAL_ERR_UNSUPPORTED;
+    const WsLayout w = layout_ws(kv0, k, num_layers);
+    const size_t rows = (size_t)kv0->batch * kv0->num_q_heads;
+    char* ws = (char*)ctx->ws;
+    char* qd = ws + w.q_stage;
+    float* od = (float*)(ws + w.out_stage);
+    if (cudaMemcpyAsync(qd, q_host, (size_t)num_layers * rows * HEAD_DIM * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return TIDAL_ERR_CUDA;
+    const void* qs[1024];
+    float* outs[1024];
+    for (int i = 0; i < num_layers; ++i) {
+        qs[i] = qd + (size_t)i * rows * HEAD_DIM * 2;
+        outs[i] = od + (size_t)i * rows * HEAD_DIM;
+    }
+    rc = decode_step_impl(ctx, num_layers, schedule, kv_per_layer, qs, outs, k, granularity,
+                          (int*)(ws + w.idx), (int*)(ws + w.idx_count), num_layers, st);
+    if (rc != TIDAL_OK) return rc;
+    if (cudaMemcpyAsync(out_host, od, (size_t)num_layers * rows * HEAD_DIM * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return TIDAL_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+}
+
+tidal_status_t tidal_device_status(tidal_ctx_t* ctx, void* stream) {
+    if (!ctx) return TIDAL_ERR_INVALID;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return TIDAL_ERR_CUDA;
+    int word = 0;
+    if (cudaMemcpy(&word, ctx->status, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) return TIDAL_ERR_CUDA;
+    if (word != 0 && cudaMemset(ctx->status, 0, sizeof(int)) != cudaSuccess) return TIDAL_ERR_CUDA;
+    return word ? TIDAL_ERR_INDEX : TIDAL_OK;
+}
+
+int64_t tidal_launch_count(const tidal_ctx_t* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* tidal_strerror(tidal_status_t s) {
+    switch (s) {
+        case TIDAL_OK: return "ok";
+        case TIDAL_ERR_INVALID: return "invalid argument";
+        case TIDAL_ERR_UNSUPPORTED: return "unsupported configuration";
+        case TIDAL_ERR_NOMEM: return "out of device memory";
+        case TIDAL_ERR_CUDA: return "CUDA runtime error";
+        case TIDAL_ERR_TIMEOUT: return "device-side wait timed out";
+        case TIDAL_ERR_INDEX: return "token index or page id out of range";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,269 @@
+"""CUDA path vs CPU oracle, element by element, through the C-ABI (GPU only)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2410_05076_b200 import binding, synth
+from tests import util
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def td():
+    t = binding.Tidal(0)
+    yield t
+    assert t.device_status() == binding.OK
+    t.close()
+
+
+def wl(batch, hq, hkv, ctx, k, planted=8, seed=1, ragged=False, ctx_min=0, layers=2):
+    return synth.Workload(f"t{batch}_{hq}_{hkv}_{ctx}_{k}", batch, hq, hkv, layers, ctx, k, planted,
+                          [synth.LAYER_SELECT, synth.LAYER_SPARSE], synth.BASE_SEED + 100 + seed,
+                          ragged=ragged, ctx_min=ctx_min)
+
+
+def paged_layer(w, layer, q):
+    pt, total = synth.make_page_table(w, extra_pages=3)
+    return synth.make_layer(w, layer, DEV, layout="paged", q=q, page_table=pt, num_pages=total)
+
+
+def build(w, layout, layer=0):
+    q = synth.make_q(w, layer, DEV)
+    if layout == "paged":
+        lay = paged_layer(w, layer, q)
+    else:
+        lay = synth.make_layer(w, layer, DEV, layout=layout, q=q)
+    return q, lay
+
+
+CASES = [
+    # batch, Hq, Hkv, ctx, k, ragged
+    (1, 8, 2, 300, 40, False),
+    (2, 8, 2, 1000, 64, True),
+    (1, 4, 4, 4097, 256, False),       # MHA, ragged tail of one position
+    (3, 16, 2, 777, 100, True),        # group 8
+    (1, 2, 1, 2500, 17, False),        # group 2
+    (1, 8, 2, 16, 5, False),           # exactly one tile
+    (1, 8, 2, 17, 17, False),          # one tile + 1, k = N
+    (1, 8, 2, 15, 3, False),
+    (1, 4, 2, 1, 1, False),            # single cached token
+]
+
+
+@pytest.mark.parametrize("layout", ["hnd_interleaved", "nhd_separate", "paged"])
+@pytest.mark.parametrize("B,Hq,Hkv,N,k,ragged", CASES)
+def test_layers_match_oracle(td, layout, B, Hq, Hkv, N, k, ragged):
+    w = wl(B, Hq, Hkv, N, k, planted=min(8, N), ragged=ragged, ctx_min=max(1, N // 3))
+    q, lay = build(w, layout)
+    okv = util.oracle_kv(lay)
+    qb = synth.bits(q)
+    lens = lay.ctx_lens.cpu().numpy()
+
+    # full attention layer
+    out = td.full_attn(lay, q)
+    ref_out, ref_sc = oracle.full_attn(okv, qb, want_scores=True)
+    util.check_out(out.cpu().numpy(), ref_out, "full")
+
+    # token selection layer: output, emitted scores, index sets
+    scores = torch.full((B, Hq, N), float("nan"), dtype=torch.float32, device=DEV)
+    out2, idx, cnt = td.select_attn(lay, q, k, scores=scores)
+    util.check_out(out2.cpu().numpy(), ref_out, "select.out")
+    sc = scores.cpu().numpy()
+    idx_h = idx.cpu().numpy()
+    assert cnt.cpu().numpy().tolist() == [min(k, int(n)) for n in lens]
+    for b in range(B):
+        n = int(lens[b])
+        assert np.abs(sc[b, :, :n] - ref_sc[b, :, :n]).max() <= 1e-4
+        for h in range(Hq):
+            util.check_idx_row(idx_h[b, h], ref_sc[b, h], k, n, f"idx[{b},{h}]")
+
+    # same call with the scores kept in the workspace
+    _, idx_ws, _ = td.select_attn(lay, q, k)
+    assert torch.equal(idx_ws, idx)
+
+    # sparse layer on the oracle's own index sets
+    _, ref_idx, ref_cnt = oracle.select_attn(okv, qb, k)
+    sp = td.sparse_attn(lay, q, torch.from_numpy(ref_idx).to(DEV), torch.from_numpy(ref_cnt).to(DEV))
+    util.check_out(sp.cpu().numpy(), oracle.sparse_attn(okv, qb, ref_idx, ref_cnt), "sparse")
+    # and without idx_count: the -1 padding alone delimits the list
+    sp2 = td.sparse_attn(lay, q, torch.from_numpy(ref_idx).to(DEV))
+    util.check_out(sp2.cpu().numpy(), oracle.sparse_attn(okv, qb, ref_idx), "sparse.nocount")
+    assert td.device_status() == binding.OK
+
+
+def test_config1_select_then_sparse(td):
+    """Configuration 1 at full size: 8q/2kv, context 4096, k 256, 32 planted per KV head."""
+    w = synth.workload("cfg1")
+    q0 = synth.make_q(w, 0, DEV)
+    q1 = synth.make_q(w, 1, DEV)
+    l0 = synth.make_layer(w, 0, DEV, q=q0)
+    l1 = synth.make_layer(w, 1, DEV, q=q1)
+    outs, idx, cnt = td.decode_step(w.sched, [l0, l1], [q0, q1], w.k)
+    o0, s0 = oracle.full_attn(util.oracle_kv(l0), synth.bits(q0), want_scores=True)
+    util.check_out(outs[0].cpu().numpy(), o0, "cfg1.select")
+    idx_h = idx.cpu().numpy()
+    inside = 0
+    for h in range(w.num_q_heads):
+        inside += util.check_idx_row(idx_h[0, h], s0[0, h], w.k, w.ctx, f"cfg1.idx[{h}]")
+    # planted heavy hitters of a head's own group are selected by that head
+    planted = synth.planted_positions(w, 0, [w.ctx])
+    for g in range(w.num_kv_heads):
+        for i, pos in enumerate(planted[0, g].tolist()):
+            h = g * w.group + i % w.group
+            assert pos in idx_h[0, h]
+    # sparse layer: oracle evaluated on the GPU's (validated) token sets
+    ref1 = oracle.sparse_attn(util.oracle_kv(l1), synth.bits(q1), idx_h, cnt.cpu().numpy())
+    util.check_out(outs[1].cpu().numpy(), ref1, "cfg1.sparse")
+    assert inside <= 8
+
+
+@pytest.mark.parametrize("gran,hi_of", [(binding.SEL_PER_KVHEAD, lambda w: w.num_kv_heads),
+                                        (binding.SEL_SHARED, lambda w: 1)])
+def test_aggregated_granularities(td, gran, hi_of):
+    w = wl(2, 8, 2, 900, 50, ragged=True, ctx_min=300, seed=7)
+    q, lay = build(w, "hnd_interleaved")
+    okv, qb = util.oracle_kv(lay), synth.bits(q)
+    Hi = hi_of(w)
+    out, idx, cnt = td.select_attn(lay, q, w.k, granularity=gran)
+    ref_out, ref_idx, ref_cnt, ref_sc = oracle.select_attn(okv, qb, w.k, Hi, want_scores=True)
+    util.check_out(out.cpu().numpy(), ref_out, "agg.out")
+    lens = lay.ctx_lens.cpu().numpy()
+    members = w.num_q_heads // Hi
+    idx_h = idx.cpu().numpy()
+    for b in range(w.batch):
+        n = int(lens[b])
+        for hi in range(Hi):
+            agg = ref_sc[b, hi * members:(hi + 1) * members, :n].astype(np.float64).sum(0).astype(np.float32)
+            util.check_idx_row(idx_h[b, hi], agg, w.k, n, f"agg.idx[{b},{hi}]")
+    sp = td.sparse_attn(lay, q, torch.from_numpy(ref_idx).to(DEV), torch.from_numpy(ref_cnt).to(DEV))
+    util.check_out(sp.cpu().numpy(), oracle.sparse_attn(okv, qb, ref_idx, ref_cnt), "agg.sparse")
+
+
+def test_decode_step_schedule_and_rho_persistence(td):
+    """Seven layers F,F,S,sp,S,sp,sp on a paged ragged batch; sparse layers are
+    checked against the oracle run on the token sets the GPU selected."""
+    sched = [0, 0, 1, 2, 1, 2, 2]
+    w = wl(2, 8, 2, 1200, 96, ragged=True, ctx_min=500, seed=9, layers=len(sched))
+    pt, total = synth.make_page_table(w, extra_pages=5)
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    layers = [synth.make_layer(w, i, DEV, layout="paged", q=qs[i], page_table=pt, num_pages=total)
+              for i in range(len(sched))]
+    lens = layers[0].ctx_lens.cpu().numpy()
+
+    # run layer by layer to capture rho after each selection layer
+    rho = {}
+    for i, t in enumerate(sched):
+        if t == 1:
+            _, idx, cnt = td.select_attn(layers[i], qs[i], w.k)
+            rho[i] = (idx.cpu().numpy().copy(), cnt.cpu().numpy().copy())
+    outs, idx, cnt = td.decode_step(sched, layers, qs, w.k)
+    assert np.array_equal(idx.cpu().numpy(), rho[4][0])          # rho was replaced wholesale at layer 4
+    cur = None
+    for i, t in enumerate(sched):
+        okv, qb = util.oracle_kv(layers[i]), synth.bits(qs[i])
+        got = outs[i].cpu().numpy()
+        if t in (0, 1):
+            ref, sc = oracle.full_attn(okv, qb, want_scores=True)
+            util.check_out(got, ref, f"step.layer{i}")
+            if t == 1:
+                cur = rho[i]
+                for b in range(w.batch):
+                    for h in range(w.num_q_heads):
+                        util.check_idx_row(cur[0][b, h], sc[b, h], w.k, int(lens[b]), f"step.idx{i}")
+        else:
+            util.check_out(got, oracle.sparse_attn(okv, qb, cur[0], cur[1]), f"step.layer{i}")
+    assert td.device_status() == binding.OK
+
+
+def test_decode_step_host_buffers(td):
+    sched = [0, 1, 2, 2]
+    w = wl(1, 8, 2, 640, 48, seed=11, layers=len(sched))
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    layers = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(len(sched))]
+    q_host = torch.stack([q.cpu() for q in qs]).contiguous().pin_memory()
+    out_host = torch.zeros(len(sched), 1, 8, 128, dtype=torch.float32).pin_memory()
+    td.make_step_host(sched, layers, q_host, out_host, w.k)()
+    outs, _, _ = td.decode_step(sched, layers, qs, w.k)
+    for i in range(len(sched)):
+        assert torch.equal(out_host[i], outs[i].cpu())
+
+
+def test_ties_and_constant_scores(td):
+    """q = 0: every score is equal, so the lowest positions win and the output is the mean of V."""
+    w = wl(1, 4, 2, 333, 20, seed=13)
+    q, lay = build(w, "hnd_interleaved")
+    q.zero_()
+    out, idx, _ = td.select_attn(lay, q, w.k)
+    assert idx.cpu().numpy()[0].tolist() == [list(range(20))] * 4
+    ref = oracle.full_attn(util.oracle_kv(lay), synth.bits(q))
+    util.check_out(out.cpu().numpy(), ref, "ties.out")
+
+
+def test_sparse_skips_padding_duplicates_and_flags_bad_indices(td):
+    w = wl(1, 4, 2, 200, 12, seed=15)
+    q, lay = build(w, "nhd_separate")
+    okv, qb = util.oracle_kv(lay), synth.bits(q)
+    idx = np.full((1, 4, 12), -1, np.int32)
+    idx[0, 0, :5] = [199, 3, 3, 50, 0]           # unsorted with a duplicate
+    idx[0, 1, :1] = [7]
+    idx[0, 3, :12] = np.arange(100, 112)         # head 2 has no entries at all
+    sp = td.sparse_attn(lay, q, torch.from_numpy(idx).to(DEV))
+    ref = oracle.sparse_attn(okv, qb, idx)
+    util.check_out(sp.cpu().numpy(), ref, "sparse.dups")
+    assert (sp.cpu().numpy()[0, 2] == 0).all()
+    assert td.device_status() == binding.OK
+    idx[0, 1, 1] = 200                            # one past the end of the cache
+    sp = td.sparse_attn(lay, q, torch.from_numpy(idx).to(DEV))
+    assert td.device_status() == binding.ERR_INDEX
+    assert td.device_status() == binding.OK       # sticky word was cleared
+    util.check_out(sp.cpu().numpy(), ref, "sparse.badidx")   # the bad entry was skipped
+
+
+def test_host_side_argument_errors(td):
+    w = wl(1, 8, 2, 64, 8, seed=17)
+    q, lay = build(w, "hnd_interleaved")
+    lib, ctx = td.lib, td.ctx
+    import ctypes as C
+    out = torch.empty(1, 8, 128, dtype=torch.float32, device=DEV)
+    idx = torch.empty(1, 8, 8, dtype=torch.int32, device=DEV)
+
+    def sel(s, k=8, gran=0, q_=q, idx_=idx):
+        return lib.tidal_select_attn(ctx, C.byref(s), q_.data_ptr(), k, gran, out.data_ptr(),
+                                     idx_.data_ptr(), None, None, None)
+
+    s = binding.kv_struct(lay)
+    assert sel(s) == binding.OK
+    assert sel(s, k=0) == binding.ERR_INVALID
+    assert sel(s, k=65) == binding.ERR_INVALID
+    assert sel(s, gran=9) == binding.ERR_INVALID
+    s = binding.kv_struct(lay); s.head_dim = 64
+    assert sel(s) == binding.ERR_UNSUPPORTED
+    s = binding.kv_struct(lay); s.num_kv_heads = 3
+    assert sel(s) == binding.ERR_INVALID
+    s = binding.kv_struct(lay); s.k = None
+    assert sel(s) == binding.ERR_INVALID
+    s = binding.kv_struct(lay); s.stride_pos = 260
+    assert sel(s) == binding.ERR_INVALID
+    s = binding.kv_struct(lay); s.kv_layout = binding.KV_PAGED
+    assert sel(s) == binding.ERR_INVALID          # paged without a page table
+    s = binding.kv_struct(lay)
+    assert lib.tidal_sparse_attn(ctx, C.byref(s), q.data_ptr(), idx.data_ptr(), None, 8, 3,
+                                 out.data_ptr(), None) == binding.ERR_INVALID
+    # a sparse layer before any selection layer
+    with pytest.raises(binding.TidalError) as e:
+        td.decode_step([0, 2], [lay, lay], [q, q], 8)
+    assert e.value.status == binding.ERR_INVALID
+    assert binding.Tidal.workspace_bytes(lay, 8) > 0
+    torch.cuda.synchronize()
+
+
+def test_results_are_deterministic(td):
+    w = wl(1, 8, 2, 5000, 300, seed=19)
+    q, lay = build(w, "hnd_interleaved")
+    a = td.select_attn(lay, q, w.k)
+    b = td.select_attn(lay, q, w.k)
+    assert torch.equal(a[1], b[1])
+    assert torch.equal(a[0], b[0])
