@@ -239,7 +239,7 @@ def make_page_table(w: Workload, extra_pages: int = 0):
     need = [(n + PAGE_SIZE - 1) // PAGE_SIZE for n in lens]
     total = sum(need) + extra_pages
     perm = torch.randperm(total, generator=_gen("cpu", w.seed + 99))
-    maxp = max(need)
+    maxp = (w.ctx + PAGE_SIZE - 1) // PAGE_SIZE      # table width covers the declared maximum length
     pt = torch.zeros(w.batch, maxp, dtype=torch.int32)
     at = 0
     for b, nb in enumerate(need):

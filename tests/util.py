@@ -6,6 +6,7 @@ import numpy as np
 import torch
 
 import oracle
+from oracle import adapter
 from paper_2410_05076_b200 import synth
 
 MAX_ABS_TOL = 2e-2      # attention output, max |gpu - oracle|
@@ -13,31 +14,8 @@ MEAN_ABS_TOL = 2e-3     # attention output, mean |gpu - oracle|
 TIE_BAND = 1e-3         # index sets must agree outside this band around the k-th score
 
 
-def _host_bits(t: torch.Tensor, keep):
-    """(uint16 array of the whole owning buffer, element offset of t in it)."""
-    for buf in keep:
-        if buf.untyped_storage().data_ptr() == t.untyped_storage().data_ptr():
-            flat = buf.detach().reshape(-1)
-            return synth.bits(flat), t.storage_offset() - buf.storage_offset()
-    flat = t.detach().contiguous().reshape(-1)
-    return synth.bits(flat), 0
-
-
 def oracle_kv(layer: synth.LayerKV) -> oracle.KV:
-    kb, koff = _host_bits(layer.k, layer.keep)
-    if layer.v.untyped_storage().data_ptr() == layer.k.untyped_storage().data_ptr():
-        vb, voff = kb, layer.v.storage_offset() - layer.keep[0].storage_offset()
-    else:
-        vb, voff = _host_bits(layer.v, layer.keep)
-    return oracle.KV(
-        k=kb, v=vb, k_offset=koff, v_offset=voff, batch=layer.batch,
-        num_q_heads=layer.num_q_heads, num_kv_heads=layer.num_kv_heads, head_dim=layer.head_dim,
-        ctx_lens=layer.ctx_lens.cpu().numpy().astype(np.int32),
-        stride_b=layer.stride_b, stride_pos=layer.stride_pos, stride_head=layer.stride_head,
-        stride_page=layer.stride_page,
-        page_table=None if layer.page_table is None else layer.page_table.cpu().numpy(),
-        page_size=layer.page_size, max_pages_per_seq=layer.max_pages_per_seq,
-        sm_scale=layer.sm_scale)
+    return adapter.kv_from_layer(layer)
 
 
 def check_out(got, ref, what=""):
