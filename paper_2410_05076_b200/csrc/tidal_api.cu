@@ -22,7 +22,6 @@ namespace {
 constexpr int MAX_CTX = 262144;
 constexpr int MAX_SPLITS = 512;
 constexpr int MAX_GROUP = 8;            // query heads per KV head that fit the 8 MMA columns
-constexpr int TOPK_SLICE_MAX = 32768;   // keys per CTA kept in shared memory
 
 // Streaming (full / selection) and gather (sparse) launch shapes.
 constexpr int DENSE_NW = 8, DENSE_STAGES = 3;
@@ -38,8 +37,13 @@ struct tidal_ctx {
     int device = 0;
     int sm_count = 0;
     int dense_slots = 0, sparse_slots = 0;     // resident CTAs on the whole GPU
-    void* ws = nullptr;
+    void* ws = nullptr;                         // scratch: contents are garbage between calls
     size_t ws_bytes = 0;
+    // Words that must read zero when a kernel starts (split counters, top-k cursors, arrival
+    // counters and histograms). The kernels restore the zeros themselves, so this lives apart
+    // from the scratch workspace, whose layout changes with the problem shape.
+    void* state = nullptr;
+    int state_rows = 0;                         // capacity in (sequence, head) rows
     int* status = nullptr;                      // device word, sticky
     int64_t launches = 0;
 };
@@ -47,7 +51,8 @@ struct tidal_ctx {
 namespace {
 
 struct WsLayout {
-    size_t counters, part_ml, part_o, scores, idx, idx_count, q_stage, out_stage, total;
+    size_t part_ml, part_o, scores, cand, idx, idx_count, q_stage, out_stage, total;
+    long long cand_stride;
     long long score_stride;
 };
 
@@ -122,11 +127,12 @@ WsLayout layout_ws(const tidal_kv_t* kv, int k, int num_layers_host) {
     WsLayout w;
     const size_t rows = (size_t)kv->batch * kv->num_q_heads;
     size_t at = 0;
-    w.counters = at;  at += align_up(rows * sizeof(int), 256);
     w.part_ml = at;   at += align_up(rows * MAX_SPLITS * sizeof(float2), 256);
     w.part_o = at;    at += align_up(rows * MAX_SPLITS * HEAD_DIM * sizeof(float), 256);
     w.score_stride = (long long)align_up((size_t)kv->max_ctx_len, 16);
     w.scores = at;    at += align_up(rows * (size_t)w.score_stride * sizeof(float), 256);
+    w.cand_stride = w.score_stride;
+    w.cand = at;      at += align_up(rows * (size_t)w.cand_stride * sizeof(uint2), 256);
     w.idx = at;       at += align_up(rows * (size_t)std::max(k, 1) * sizeof(int), 256);
     w.idx_count = at; at += align_up((size_t)kv->batch * sizeof(int), 256);
     w.q_stage = at;   at += align_up((size_t)num_layers_host * rows * HEAD_DIM * 2, 256);
@@ -146,11 +152,34 @@ tidal_status_t ensure_ws(tidal_ctx* ctx, size_t bytes) {
     if (ctx->ws) { cudaDeviceSynchronize(); cudaFree(ctx->ws); ctx->ws = nullptr; ctx->ws_bytes = 0; }
     void* p = nullptr;
     if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TIDAL_ERR_NOMEM; }
-    // The split counters must be zero between launches; zero the head of the buffer.
-    if (cudaMemset(p, 0, std::min(bytes, (size_t)1 << 20)) != cudaSuccess) { cudaFree(p); return TIDAL_ERR_CUDA; }
     ctx->ws = p;
     ctx->ws_bytes = bytes;
     return TIDAL_OK;
+}
+
+// State layout for a capacity of R rows: counters[R] | cursor[R] | done[R] | hist[R][TK_BINS].
+inline int* state_counters(const tidal_ctx* c) { return (int*)c->state; }
+inline int* state_cursor(const tidal_ctx* c) { return (int*)c->state + c->state_rows; }
+inline int* state_done(const tidal_ctx* c) { return (int*)c->state + 2 * (size_t)c->state_rows; }
+inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + 3 * (size_t)c->state_rows; }
+
+tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
+    if (ctx->state_rows >= rows) return TIDAL_OK;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    if (ctx->state) { cudaDeviceSynchronize(); cudaFree(ctx->state); ctx->state = nullptr; ctx->state_rows = 0; }
+    const int cap = (int)align_up((size_t)rows, 64);
+    const size_t bytes = (size_t)cap * (3 + TK_BINS) * sizeof(int);
+    void* p = nullptr;
+    if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TIDAL_ERR_NOMEM; }
+    if (cudaMemset(p, 0, bytes) != cudaSuccess) { cudaFree(p); return TIDAL_ERR_CUDA; }
+    ctx->state = p;
+    ctx->state_rows = cap;
+    return TIDAL_OK;
+}
+
+tidal_status_t ensure_all(tidal_ctx* ctx, const tidal_kv_t* kv, size_t ws_bytes) {
+    const tidal_status_t rc = ensure_state(ctx, kv->batch * kv->num_q_heads);
+    return rc != TIDAL_OK ? rc : ensure_ws(ctx, ws_bytes);
 }
 
 void fill_common(AttnParams& a, const tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, float* out,
@@ -170,7 +199,7 @@ void fill_common(AttnParams& a, const tidal_ctx* ctx, const tidal_kv_t* kv, cons
     a.scale = kv->sm_scale > 0.f ? kv->sm_scale : 1.0f / std::sqrt((float)kv->head_dim);
     a.scale_log2 = a.scale * 1.4426950408889634f;
     char* ws = (char*)ctx->ws;
-    a.counters = (int*)(ws + w.counters);
+    a.counters = state_counters(ctx);
     a.part_ml = (float2*)(ws + w.part_ml);
     a.part_o = (float*)(ws + w.part_o);
     a.max_splits = MAX_SPLITS;
@@ -200,31 +229,31 @@ tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, fl
 }
 
 tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* scores, long long score_stride,
-                        int k, int Hi, int* idx, int* idx_count, cudaStream_t st) {
+                        int k, int Hi, int* idx, int* idx_count, const WsLayout& w, cudaStream_t st) {
     TopkParams t;
+    std::memset(&t, 0, sizeof t);
     t.scores = scores; t.score_stride = score_stride;
     t.ctx_lens = kv->ctx_lens; t.max_ctx = kv->max_ctx_len;
     t.Hq = kv->num_q_heads; t.Hi = Hi; t.k = k;
     t.idx = idx; t.idx_count = idx_count;
+    char* ws = (char*)ctx->ws;
+    t.hist = state_hist(ctx);
+    t.cursor = state_cursor(ctx);
+    t.done = state_done(ctx);
+    t.cand = (uint2*)(ws + w.cand);
+    t.cand_stride = w.cand_stride;
     const int items = kv->batch * Hi;
-    int cs = 1;
-    while (cs < 8 && (kv->max_ctx_len + cs - 1) / cs > TOPK_SLICE_MAX) cs <<= 1;
-    while (cs < 8 && items * cs < ctx->sm_count && (kv->max_ctx_len / (2 * cs)) >= 2048) cs <<= 1;
-    t.slice_cap = (int)align_up((size_t)(kv->max_ctx_len + cs - 1) / cs, 4);
-    const size_t smem = (size_t)t.slice_cap * 4 + 2 * TOPK_BINS * sizeof(int);
-    cudaLaunchConfig_t cfg;
-    std::memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3(items * cs, 1, 1);
-    cfg.blockDim = dim3(TOPK_THREADS, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    ctx->launches++;
-    return cudaLaunchKernelEx(&cfg, topk_kernel, t) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+    if (items > 65535) return TIDAL_ERR_UNSUPPORTED;
+    const int parts = (kv->max_ctx_len + TK_SLICE - 1) / TK_SLICE;
+    t.vec_ok = (((uintptr_t)scores & 15) == 0 && (score_stride & 3) == 0) ? 1 : 0;
+    t.cand_smem = std::min(16384, std::max(4096, (int)align_up((size_t)k + 4096, 1024)));
+    const size_t words = (size_t)(kv->max_ctx_len + 31) / 32;
+    const size_t smem = 2 * words * sizeof(unsigned) + (size_t)t.cand_smem * sizeof(uint2);
+    dim3 grid(parts, items, 1);
+    topk_hist_kernel<<<grid, TK_THREADS, 0, st>>>(t);
+    topk_select_kernel<<<grid, TK_THREADS, smem, st>>>(t);
+    ctx->launches += 2;
+    return cudaGetLastError() == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }
 
 tidal_status_t run_sparse(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, const int* idx,
@@ -270,8 +299,8 @@ tidal_status_t tidal_create(tidal_ctx_t** out, int device, size_t workspace_byte
     const int d0 = resident_ctas(attn_kernel<MODE_FULL, DENSE_NW, DENSE_STAGES>, DENSE_NW * 32, dense_smem, ctx->sm_count);
     const int d1 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW, DENSE_STAGES>, DENSE_NW * 32, dense_smem, ctx->sm_count);
     const int s0 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>, SPARSE_NW * 32, sparse_smem, ctx->sm_count);
-    const size_t topk_smem = (size_t)TOPK_SLICE_MAX * 4 + 2 * TOPK_BINS * sizeof(int);
-    const bool topk_ok = cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topk_smem) == cudaSuccess;
+    const size_t topk_smem = 2 * (size_t)(MAX_CTX / 32) * sizeof(unsigned) + 16384 * sizeof(uint2);
+    const bool topk_ok = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topk_smem) == cudaSuccess;
     if (d0 <= 0 || d1 <= 0 || s0 <= 0 || !topk_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
     ctx->dense_slots = std::min(d0, d1);
     ctx->sparse_slots = s0;
@@ -291,6 +320,7 @@ tidal_status_t tidal_destroy(tidal_ctx_t* ctx) {
     cudaSetDevice(ctx->device);
     cudaDeviceSynchronize();
     if (ctx->ws) cudaFree(ctx->ws);
+    if (ctx->state) cudaFree(ctx->state);
     if (ctx->status) cudaFree(ctx->status);
     delete ctx;
     return TIDAL_OK;
@@ -307,7 +337,7 @@ tidal_status_t tidal_full_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const voi
     if (rc != TIDAL_OK) return rc;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
     const WsLayout w = layout_ws(kv, 1, 0);
-    if ((rc = ensure_ws(ctx, w.total)) != TIDAL_OK) return rc;
+    if ((rc = ensure_all(ctx, kv, w.total)) != TIDAL_OK) return rc;
     return run_dense(ctx, kv, q, out, nullptr, 0, w, (cudaStream_t)stream);
 }
 
@@ -322,12 +352,12 @@ tidal_status_t tidal_select_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const v
     if (Hi <= 0) return TIDAL_ERR_INVALID;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
     const WsLayout w = layout_ws(kv, k, 0);
-    if ((rc = ensure_ws(ctx, w.total)) != TIDAL_OK) return rc;
+    if ((rc = ensure_all(ctx, kv, w.total)) != TIDAL_OK) return rc;
     float* scores = scores_opt ? scores_opt : (float*)((char*)ctx->ws + w.scores);
     const long long stride = scores_opt ? (long long)kv->max_ctx_len : w.score_stride;
     cudaStream_t st = (cudaStream_t)stream;
     if ((rc = run_dense(ctx, kv, q, out, scores, stride, w, st)) != TIDAL_OK) return rc;
-    return run_topk(ctx, kv, scores, stride, k, Hi, idx, idx_count, st);
+    return run_topk(ctx, kv, scores, stride, k, Hi, idx, idx_count, w, st);
 }
 
 tidal_status_t tidal_sparse_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const void* q, const int32_t* idx,
@@ -341,7 +371,7 @@ tidal_status_t tidal_sparse_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const v
     if (Hi != kv->num_q_heads && Hi != kv->num_kv_heads && Hi != 1) return TIDAL_ERR_INVALID;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
     const WsLayout w = layout_ws(kv, k, 0);
-    if ((rc = ensure_ws(ctx, w.total)) != TIDAL_OK) return rc;
+    if ((rc = ensure_all(ctx, kv, w.total)) != TIDAL_OK) return rc;
     return run_sparse(ctx, kv, q, idx, idx_count, k, Hi, out, w, (cudaStream_t)stream);
 }
 
@@ -370,7 +400,7 @@ static tidal_status_t decode_step_impl(tidal_ctx_t* ctx, int32_t num_layers, con
     }
     const int Hi = hi_of(&kvs[0], granularity);
     if (Hi <= 0) return TIDAL_ERR_INVALID;
-    tidal_status_t rc = ensure_ws(ctx, need);
+    tidal_status_t rc = ensure_all(ctx, &kvs[0], need);
     if (rc != TIDAL_OK) return rc;
     for (int i = 0; i < num_layers; ++i) {
         const tidal_kv_t* kv = &kvs[i];
@@ -380,7 +410,7 @@ static tidal_status_t decode_step_impl(tidal_ctx_t* ctx, int32_t num_layers, con
         } else if (schedule[i] == TIDAL_LAYER_SELECT) {
             float* scores = (float*)((char*)ctx->ws + w.scores);
             rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, w, st);
-            if (rc == TIDAL_OK) rc = run_topk(ctx, kv, scores, w.score_stride, k, Hi, idx, idx_count, st);
+            if (rc == TIDAL_OK) rc = run_topk(ctx, kv, scores, w.score_stride, k, Hi, idx, idx_count, w, st);
         } else {
             rc = run_sparse(ctx, kv, qs[i], idx, idx_count, k, Hi, outs[i], w, st);
         }
@@ -415,7 +445,7 @@ tidal_status_t tidal_decode_step_host(tidal_ctx_t* ctx, int32_t num_layers, cons
         if ((rc = check_kv(&kv_per_layer[i])) != TIDAL_OK) return rc;
         need = std::max(need, ws_bytes_for(&kv_per_layer[i], k, num_layers));
     }
-    if ((rc = ensure_ws(ctx, need)) != TIDAL_OK) return rc;
+    if ((rc = ensure_all(ctx, &kv_per_layer[0], need)) != TIDAL_OK) return rc;
     // All layers must share batch and head counts (checked again below); the staging
     // offsets depend only on those and on max_ctx_len of the layer used for the layout.
     const tidal_kv_t* kv0 = &kv_per_layer[0];

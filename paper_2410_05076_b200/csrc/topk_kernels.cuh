@@ -2,27 +2,32 @@
 // k' = min(k, N) positions with the largest score, equal scores resolved
 // toward the lower position, and write them in ascending position order.
 //
-// One thread-block CLUSTER works on one (sequence, index head). Each CTA of the
-// cluster owns a contiguous slice of the positions, converts its scores to
-// order-preserving 32-bit keys once and keeps them in shared memory; the exact
-// k'-th largest key is then found by a most-significant-digit radix select
-// (12 + 12 + 8 bits) whose per-digit histograms are built in shared memory and
-// summed across the cluster through distributed shared memory. The final pass
-// emits positions in order using block- and cluster-wide prefix counts, taking
-// only as many keys equal to the threshold as are still needed (lowest positions
-// first), so the result is the unique set a full sort with a (score desc,
-// position asc) order would give.
+// Scores become order-preserving 32-bit keys. The exact k'-th largest key is
+// found by a most-significant-digit radix select (11 + 11 + 10 bits):
+//   1. topk_hist_kernel: all SMs histogram the top 11 key bits of every score
+//      (shared-memory histograms, flushed to a global one per index head).
+//   2. topk_select_kernel, all SMs: every CTA derives the threshold bin from the
+//      global histogram and appends the few scores at or above that bin —
+//      about k' plus the population of one bin — to a candidate list.
+//      The last CTA of an index head to finish then resolves the remaining 21
+//      bits on the candidate list alone (in shared memory), marks the winners
+//      in a position bitmap, taking only as many keys equal to the threshold as
+//      are still needed, lowest positions first, and enumerates the bitmap in
+//      order. The result is the unique set that a full sort by (score desc,
+//      position asc) gives.
+// No CTA ever waits for another one; the per-head histogram, cursor and
+// arrival counter are cleared by the CTA that used them last.
 #pragma once
 
-#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 namespace tidal {
-namespace cg = cooperative_groups;
 
-constexpr int TOPK_THREADS = 1024;
-constexpr int TOPK_BINS = 4096;
+constexpr int TK_THREADS = 512;
+constexpr int TK_BINS = 2048;          // top 11 bits of the key
+constexpr int TK_VEC = 4;              // float4 loads per thread per slice
+constexpr int TK_SLICE = TK_THREADS * TK_VEC * 4;   // positions per CTA
 
 struct TopkParams {
     const float* scores;       // [B, Hq, score_stride]
@@ -33,7 +38,13 @@ struct TopkParams {
     int k;
     int* idx;                  // [B, Hi, k]
     int* idx_count;            // [B] or null
-    int slice_cap;             // keys a CTA can hold
+    unsigned* hist;            // [items, TK_BINS], zero between calls
+    int* cursor;               // [items], zero between calls
+    int* done;                 // [items], zero between calls
+    uint2* cand;               // [items, cand_stride] (key, position)
+    long long cand_stride;
+    int cand_smem;             // candidates the last CTA can hold in shared memory
+    int vec_ok;                // score rows are 16-byte aligned: float4 loads allowed
 };
 
 // Larger float <=> larger key; -0 and +0 map to the same key.
@@ -43,8 +54,48 @@ __device__ __forceinline__ uint32_t score_key(float s) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Inclusive scan over the block of one int per thread (TOPK_THREADS threads);
-// returns this thread's inclusive prefix and the block total.
+// Keys of this thread's 16 positions of the slice starting at s0: four groups of four
+// consecutive positions, group j at s0 + 4*(j*TK_THREADS + tid). All loads are issued
+// before any is used. Positions at or beyond n get key 0 and valid bit 0.
+__device__ __forceinline__ unsigned load_slice_keys(const TopkParams& p, const float* srow, int members,
+                                                    int s0, int n, uint32_t (&key)[TK_VEC * 4]) {
+    float v[TK_VEC * 4];
+#pragma unroll
+    for (int j = 0; j < TK_VEC; ++j) {
+        const int pos = s0 + 4 * (j * TK_THREADS + (int)threadIdx.x);
+        if (p.vec_ok && pos + 3 < n) {
+            float4 t = __ldcg(reinterpret_cast<const float4*>(srow + pos));
+            for (int m = 1; m < members; ++m) {
+                const float4 u = __ldcg(reinterpret_cast<const float4*>(srow + m * p.score_stride + pos));
+                t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+            }
+            v[4 * j] = t.x; v[4 * j + 1] = t.y; v[4 * j + 2] = t.z; v[4 * j + 3] = t.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float t = 0.f;
+                if (pos + e < n) {
+                    t = __ldcg(srow + pos + e);
+                    for (int m = 1; m < members; ++m) t += __ldcg(srow + m * p.score_stride + pos + e);
+                }
+                v[4 * j + e] = t;
+            }
+        }
+    }
+    unsigned valid = 0;
+#pragma unroll
+    for (int j = 0; j < TK_VEC; ++j)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int pos = s0 + 4 * (j * TK_THREADS + (int)threadIdx.x) + e;
+            const bool ok = pos < n;
+            key[4 * j + e] = ok ? score_key(v[4 * j + e]) : 0u;
+            valid |= (ok ? 1u : 0u) << (4 * j + e);
+        }
+    return valid;
+}
+
+// Inclusive scan of one int per thread over a TK_THREADS block.
 __device__ __forceinline__ int block_scan_incl(int v, int* warp_sums, int& total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
@@ -55,167 +106,210 @@ __device__ __forceinline__ int block_scan_incl(int v, int* warp_sums, int& total
     __syncthreads();                       // warp_sums may still be read from a previous call
     if (lane == 31) warp_sums[warp] = v;
     __syncthreads();
-    if (warp == 0) {
-        int w = warp_sums[lane];
+    int before = 0, all = 0;
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, w, d);
-            if (lane >= d) w += t;
-        }
-        warp_sums[lane] = w;
+    for (int w = 0; w < TK_THREADS / 32; ++w) {
+        const int s = warp_sums[w];
+        if (w < warp) before += s;
+        all += s;
     }
-    __syncthreads();
-    total = warp_sums[31];
-    return v + (warp ? warp_sums[warp - 1] : 0);
+    total = all;
+    return v + before;
 }
 
-// Sum the CTAs' histograms (nbins bins) over the cluster into `merged`, then
-// find the digit that holds the `need`-th largest remaining key.
-// On return (identical in every thread of every CTA): digit, and `need` reduced
-// by the number of keys in higher digits.
-__device__ __forceinline__ void cluster_pick_digit(cg::cluster_group& cluster, int* hist, int* merged,
-                                                   int nbins, int* warp_sums, int* bcast, int& digit,
-                                                   int& need) {
-    const int cs = cluster.num_blocks();
-    cluster.sync();                                    // every CTA's histogram is complete
-    for (int bin = threadIdx.x; bin < nbins; bin += TOPK_THREADS) {
-        int s = 0;
-        for (int r = 0; r < cs; ++r) s += cluster.map_shared_rank(hist, r)[bin];
-        merged[bin] = s;
-    }
-    cluster.sync();                                    // remote reads done: hist may be reused
-    // Each thread owns a run of bins, highest digits first.
-    const int per = (nbins + TOPK_THREADS - 1) / TOPK_THREADS;
-    const int hi_bin = nbins - 1 - threadIdx.x * per;  // this thread's highest bin
+// Given a histogram of `nbins` digits (shared memory), find the digit holding
+// the `need`-th largest remaining key; on return `need` is reduced by the number
+// of keys in higher digits. Identical result in every thread.
+__device__ __forceinline__ int pick_digit(const unsigned* hist, int nbins, int* warp_sums, int* bcast,
+                                          int& need) {
+    const int per = (nbins + TK_THREADS - 1) / TK_THREADS;
+    const int hi_bin = nbins - 1 - (int)threadIdx.x * per;      // this thread's highest bin
     int mine = 0;
     for (int i = 0; i < per; ++i) {
         const int bin = hi_bin - i;
-        if (bin >= 0) mine += merged[bin];
+        if (bin >= 0) mine += (int)hist[bin];
     }
     int total;
     const int incl = block_scan_incl(mine, warp_sums, total);
-    const int excl = incl - mine;                      // keys in strictly higher runs
-    if (excl < need && need <= incl) {                 // the threshold digit is in this run
+    const int excl = incl - mine;
+    if (excl < need && need <= incl) {
         int above = excl;
         for (int i = 0; i < per; ++i) {
             const int bin = hi_bin - i;
-            const int c = (bin >= 0) ? merged[bin] : 0;
+            const int c = (bin >= 0) ? (int)hist[bin] : 0;
             if (above + c >= need) { bcast[0] = bin; bcast[1] = need - above; break; }
             above += c;
         }
     }
     __syncthreads();
-    digit = bcast[0];
+    const int digit = bcast[0];
     need = bcast[1];
     __syncthreads();
+    return digit;
 }
 
-__global__ void __launch_bounds__(TOPK_THREADS, 1) topk_kernel(const TopkParams p) {
-    extern __shared__ __align__(128) uint8_t smem[];
-    uint32_t* keys = reinterpret_cast<uint32_t*>(smem);                        // [slice_cap]
-    int* hist = reinterpret_cast<int*>(smem + (size_t)p.slice_cap * 4);        // [TOPK_BINS]
-    int* merged = hist + TOPK_BINS;                                            // [TOPK_BINS]
-    __shared__ int warp_sums[32];
+__global__ void __launch_bounds__(TK_THREADS) topk_hist_kernel(const TopkParams p) {
+    __shared__ unsigned sh[TK_BINS];
+    const int item = blockIdx.y, b = item / p.Hi, hi = item % p.Hi, tid = threadIdx.x;
+    const int N = max(0, min(p.ctx_lens[b], p.max_ctx));
+    if (min(p.k, N) == N) return;                      // everything is kept: no ranking needed
+    const int s0 = blockIdx.x * TK_SLICE;
+    if (s0 >= N) return;
+    for (int i = tid; i < TK_BINS; i += TK_THREADS) sh[i] = 0;
+    const int members = p.Hq / p.Hi;
+    const float* srow = p.scores + ((long long)b * p.Hq + (long long)hi * members) * p.score_stride;
+    uint32_t key[TK_VEC * 4];
+    const unsigned valid = load_slice_keys(p, srow, members, s0, N, key);
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < TK_VEC * 4; ++e)
+        if ((valid >> e) & 1u) atomicAdd(&sh[key[e] >> 21], 1u);
+    __syncthreads();
+    unsigned* gh = p.hist + (long long)item * TK_BINS;
+    for (int i = tid; i < TK_BINS; i += TK_THREADS) {
+        const unsigned c = sh[i];
+        if (c) atomicAdd(&gh[i], c);
+    }
+}
+
+__global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParams p) {
+    extern __shared__ __align__(16) uint8_t tk_smem[];
+    __shared__ __align__(16) unsigned sh_hist[TK_BINS];
+    static_assert(TK_BINS == 4 * TK_THREADS, "one uint4 of the histogram per thread");
+    __shared__ int warp_sums[TK_THREADS / 32];
     __shared__ int bcast[2];
-    __shared__ int cta_counts[2];          // (keys above the threshold, keys equal to it) in this slice
+    __shared__ int s_last;
 
-    cg::cluster_group cluster = cg::this_cluster();
-    const int cs = cluster.num_blocks();
-    const int rank = cluster.block_rank();
-    const int item = blockIdx.x / cs;      // cluster index = b * Hi + hi
-    const int b = item / p.Hi, hi = item % p.Hi;
-    const int tid = threadIdx.x;
-
+    const int item = blockIdx.y, b = item / p.Hi, hi = item % p.Hi, tid = threadIdx.x;
     const int N = max(0, min(p.ctx_lens[b], p.max_ctx));
     const int kk = min(p.k, N);
     int* out = p.idx + (long long)item * p.k;
-    if (hi == 0 && rank == 0 && tid == 0 && p.idx_count) p.idx_count[b] = kk;
+    const int s0 = blockIdx.x * TK_SLICE, s1 = min(N, s0 + TK_SLICE);
+    if (blockIdx.x == 0 && hi == 0 && tid == 0 && p.idx_count) p.idx_count[b] = kk;
 
-    // Slice of this CTA: [s0, s1), slice length a multiple of 4 except the last.
-    int slice = ((N + cs - 1) / cs + 3) & ~3;
-    slice = min(slice, p.slice_cap);
-    const int s0 = min(N, rank * slice), s1 = min(N, s0 + slice);
-    const int n_local = s1 - s0;
-
-    if (kk == N) {                         // everything is kept: identity list, then padding
-        for (int i = s0 + tid; i < s1; i += TOPK_THREADS) out[i] = i;
-        if (rank == 0)
-            for (int i = N + tid; i < p.k; i += TOPK_THREADS) out[i] = -1;
-        return;                            // uniform over the cluster: nobody waits
+    if (kk == N) {                                     // identity list, then padding
+        for (int i = s0 + tid; i < s1; i += TK_THREADS) out[i] = i;
+        if (blockIdx.x == 0)
+            for (int i = N + tid; i < p.k; i += TK_THREADS) out[i] = -1;
+        return;
     }
+    if (s0 >= s1) return;
+    const int nparts = (N + TK_SLICE - 1) / TK_SLICE;  // CTAs that reach the arrival counter
 
-    // ---- load scores, build keys and the first (top 12 bits) histogram ----------------
-    for (int i = tid; i < TOPK_BINS; i += TOPK_THREADS) hist[i] = 0;
-    __syncthreads();
+    // ---- this CTA's keys (all loads in flight at once), then the threshold bin ------------------
     const int members = p.Hq / p.Hi;
     const float* srow = p.scores + ((long long)b * p.Hq + (long long)hi * members) * p.score_stride;
-    for (int i = tid; i < n_local; i += TOPK_THREADS) {
-        float s = __ldcg(srow + s0 + i);
-        for (int m = 1; m < members; ++m) s += __ldcg(srow + m * p.score_stride + s0 + i);
-        const uint32_t key = score_key(s);
-        keys[i] = key;
-        atomicAdd(&hist[key >> 20], 1);
+    uint32_t key[TK_VEC * 4];
+    const unsigned valid = load_slice_keys(p, srow, members, s0, N, key);
+    unsigned* gh = p.hist + (long long)item * TK_BINS;
+    {
+        const uint4 h4 = __ldcg(reinterpret_cast<const uint4*>(gh) + tid);     // TK_BINS == 4 * TK_THREADS
+        reinterpret_cast<uint4*>(sh_hist)[tid] = h4;
+    }
+    __syncthreads();
+    int need = kk;
+    const int b1 = pick_digit(sh_hist, TK_BINS, warp_sums, bcast, need);
+
+    // ---- append every score at or above that bin to the candidate list: one cursor bump per CTA ----
+    unsigned take = 0;
+#pragma unroll
+    for (int e = 0; e < TK_VEC * 4; ++e)
+        if (((valid >> e) & 1u) && (int)(key[e] >> 21) >= b1) take |= 1u << e;
+    int cta_total;
+    const int mine = __popc(take);
+    int slot = block_scan_incl(mine, warp_sums, cta_total) - mine;
+    if (tid == 0) bcast[0] = cta_total ? atomicAdd(&p.cursor[item], cta_total) : 0;
+    __syncthreads();
+    slot += bcast[0];
+    uint2* cand = p.cand + (long long)item * p.cand_stride;
+#pragma unroll
+    for (int e = 0; e < TK_VEC * 4; ++e)
+        if ((take >> e) & 1u) {
+            const int pos = s0 + 4 * ((e >> 2) * TK_THREADS + tid) + (e & 3);
+            if (slot < p.cand_stride) cand[slot] = make_uint2(key[e], (unsigned)pos);
+            ++slot;
+        }
+
+    // ---- the last CTA of this index head resolves the rest ------------------------------------------
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = (atomicAdd(&p.done[item], 1) == nparts - 1);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+
+    const int M = min((long long)__ldcg(&p.cursor[item]), p.cand_stride);
+    const int words = (N + 31) >> 5;
+    unsigned* sel = reinterpret_cast<unsigned*>(tk_smem);          // [words] keys above the threshold
+    unsigned* eqm = sel + words;                                    // [words] keys equal to it
+    uint2* scand = reinterpret_cast<uint2*>(eqm + words);          // [cand_smem]; 8*words bytes in: 8-byte aligned
+    const uint2* c = cand;
+    if (M <= p.cand_smem) {
+#pragma unroll 4
+        for (int i = tid; i < M; i += TK_THREADS) scand[i] = __ldcg(&cand[i]);
+        c = scand;
+    }
+    for (int i = tid; i < words; i += TK_THREADS) { sel[i] = 0; eqm[i] = 0; }
+    for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
+    __syncthreads();
+
+    // second digit: key bits 20..10 among keys whose top 11 bits equal b1
+    for (int i = tid; i < M; i += TK_THREADS) {
+        const uint32_t key = c[i].x;
+        if ((int)(key >> 21) == b1) atomicAdd(&sh_hist[(key >> 10) & 0x7ffu], 1u);
+    }
+    __syncthreads();
+    const int d2 = pick_digit(sh_hist, TK_BINS, warp_sums, bcast, need);
+    const uint32_t prefix2 = ((uint32_t)b1 << 21) | ((uint32_t)d2 << 10);
+
+    // third digit: key bits 9..0
+    for (int i = tid; i < 1024; i += TK_THREADS) sh_hist[i] = 0;
+    __syncthreads();
+    for (int i = tid; i < M; i += TK_THREADS) {
+        const uint32_t key = c[i].x;
+        if ((key >> 10) == (prefix2 >> 10)) atomicAdd(&sh_hist[key & 0x3ffu], 1u);
+    }
+    __syncthreads();
+    const int d3 = pick_digit(sh_hist, 1024, warp_sums, bcast, need);
+    const uint32_t thr = prefix2 | (uint32_t)d3;       // the k'-th largest key; `need` keys equal to it are taken
+
+    // bitmaps of positions above / equal to the threshold
+    for (int i = tid; i < M; i += TK_THREADS) {
+        const uint2 e = c[i];
+        if (e.x > thr) atomicOr(&sel[e.y >> 5], 1u << (e.y & 31));
+        else if (e.x == thr) atomicOr(&eqm[e.y >> 5], 1u << (e.y & 31));
     }
     __syncthreads();
 
-    int need = kk, digit;
-    cluster_pick_digit(cluster, hist, merged, TOPK_BINS, warp_sums, bcast, digit, need);
-    uint32_t prefix = (uint32_t)digit << 20;           // top 12 bits of the threshold key
+    // ordered enumeration
+    const int per = (words + TK_THREADS - 1) / TK_THREADS;
+    const int w0 = min(words, tid * per), w1 = min(words, w0 + per);
+    int ngt = 0, neq = 0;
+    for (int w = w0; w < w1; ++w) { ngt += __popc(sel[w]); neq += __popc(eqm[w]); }
+    int tot_gt, tot_eq;
+    const int gt_excl = block_scan_incl(ngt, warp_sums, tot_gt) - ngt;
+    const int eq_excl = block_scan_incl(neq, warp_sums, tot_eq) - neq;
+    int eq_seen = eq_excl;
+    int at = gt_excl + min(eq_seen, need);
+    for (int w = w0; w < w1; ++w) {
+        unsigned e = eqm[w];
+        const int ne = __popc(e);
+        int keep = min(max(need - eq_seen, 0), ne);    // lowest `keep` equal-key positions of this word
+        eq_seen += ne;
+        while (__popc(e) > keep) e &= ~(0x80000000u >> __clz(e));
+        unsigned bits = sel[w] | e;
+        while (bits) {
+            const int pbit = __ffs(bits) - 1;
+            if (at < p.k) out[at] = (w << 5) + pbit;
+            ++at;
+            bits &= bits - 1;
+        }
+    }
+    for (int i = kk + tid; i < p.k; i += TK_THREADS) out[i] = -1;
 
-    // ---- second digit: bits 19..8 among keys whose top 12 bits match -------------------
-    for (int i = tid; i < TOPK_BINS; i += TOPK_THREADS) hist[i] = 0;
-    __syncthreads();
-    for (int i = tid; i < n_local; i += TOPK_THREADS) {
-        const uint32_t key = keys[i];
-        if ((key >> 20) == (prefix >> 20)) atomicAdd(&hist[(key >> 8) & 0xfffu], 1);
-    }
-    __syncthreads();
-    cluster_pick_digit(cluster, hist, merged, TOPK_BINS, warp_sums, bcast, digit, need);
-    prefix |= (uint32_t)digit << 8;
-
-    // ---- third digit: bits 7..0 ---------------------------------------------------------
-    for (int i = tid; i < 256; i += TOPK_THREADS) hist[i] = 0;
-    __syncthreads();
-    for (int i = tid; i < n_local; i += TOPK_THREADS) {
-        const uint32_t key = keys[i];
-        if ((key >> 8) == (prefix >> 8)) atomicAdd(&hist[key & 0xffu], 1);
-    }
-    __syncthreads();
-    cluster_pick_digit(cluster, hist, merged, 256, warp_sums, bcast, digit, need);
-    const uint32_t thr = prefix | (uint32_t)digit;     // the k'-th largest key
-    // `need` keys equal to thr are taken, lowest positions first.
-
-    // ---- ordered output --------------------------------------------------------------------
-    const int per = (n_local + TOPK_THREADS - 1) / TOPK_THREADS;
-    const int r0 = min(n_local, tid * per), r1 = min(n_local, r0 + per);
-    int gt = 0, eq = 0;
-    for (int i = r0; i < r1; ++i) {
-        const uint32_t key = keys[i];
-        gt += key > thr;
-        eq += key == thr;
-    }
-    int gt_total, eq_total;
-    const int gt_excl = block_scan_incl(gt, warp_sums, gt_total) - gt;
-    const int eq_excl = block_scan_incl(eq, warp_sums, eq_total) - eq;
-    if (tid == 0) { cta_counts[0] = gt_total; cta_counts[1] = eq_total; }
-    cluster.sync();
-    int gt_base = 0, eq_base = 0;
-    for (int r = 0; r < rank; ++r) {
-        const int* rc = cluster.map_shared_rank(cta_counts, r);
-        gt_base += rc[0];
-        eq_base += rc[1];
-    }
-    int eq_seen = eq_base + eq_excl;                   // equal keys at lower positions
-    int at = gt_base + gt_excl + min(eq_seen, need);   // selected entries at lower positions
-    for (int i = r0; i < r1; ++i) {
-        const uint32_t key = keys[i];
-        bool take = key > thr;
-        if (key == thr) { take = eq_seen < need; ++eq_seen; }
-        if (take) { if (at < p.k) out[at] = s0 + i; ++at; }
-    }
-    if (rank == 0)
-        for (int i = kk + tid; i < p.k; i += TOPK_THREADS) out[i] = -1;
-    cluster.sync();                                    // keep shared memory alive until peers have read it
+    // leave the shared state clean for the next call
+    for (int i = tid; i < TK_BINS; i += TK_THREADS) gh[i] = 0;
+    if (tid == 0) { p.cursor[item] = 0; p.done[item] = 0; }
 }
 
 }  // namespace tidal
