@@ -40,6 +40,9 @@ constexpr int HEAD_DIM = 128;
 constexpr int TILE = 16;                 // positions per tile == page size
 constexpr int TILE_BYTES = TILE * HEAD_DIM * 2;   // 4 KB of K, same of V
 constexpr int STAGE_BYTES = 2 * TILE_BYTES;
+constexpr int HIST_BINS = 2048;          // global histogram row: up to 11 top bits of the score key
+constexpr int HIST_SMEM_WORDS = 8192;    // shared histogram: columns x bins <= 8192 counters (32 KB)
+constexpr int GRAB_TILES = 4;            // tiles a warp takes from its item's pool at a time
 
 struct AttnParams {
     const __nv_bfloat16* q;
@@ -53,7 +56,8 @@ struct AttnParams {
     int max_ctx;               // host bound of ctx_lens; larger device values are clamped to it
     int Hq, Hkv, G;
     float scale, scale_log2;
-    int chunk;                 // context positions (or index entries) per CTA, multiple of 16
+    int batch;
+    int splits_per_item;       // S > 0: CTAs c*S..c*S+S-1 share item c's tiles through a pool cursor; 0: static flat split
     float* scores;             // MODE_SELECT: [B, Hq, score_stride]
     long long score_stride;
     const int* idx;            // MODE_SPARSE: [B, Hi, k]
@@ -61,8 +65,11 @@ struct AttnParams {
     int budget, Hi;            // MODE_SPARSE: entries per index row, index heads
     float* part_o;             // [B*Hq, max_splits, 128] un-normalised partial outputs
     float2* part_ml;           // [B*Hq, max_splits] (running max in base 2, sum)
-    int* counters;             // [B * gridDim.y], zero between launches
-    int max_splits;
+    int* counters;             // one per (sequence, item), zero between launches
+    int max_splits;            // partial slots per (sequence, head) row
+    unsigned* hist;            // MODE_SELECT, optional: [B*Hq][HIST_BINS] += histogram of the top key bits
+    int hist_shift;            // bin = key >> hist_shift (21: 2048 bins, 22: 1024 bins for groups above 4)
+    int* tile_ctr;             // splits_per_item > 0: per-item pool cursor, zero between launches
     int* status;
 };
 
@@ -75,6 +82,9 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int sr
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes)
                  : "memory");
 }
+__device__ __forceinline__ void cp_async16_full(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
@@ -83,6 +93,14 @@ __device__ __forceinline__ void cp_async_wait() {
 
 __device__ __forceinline__ void lds128(uint32_t addr, uint32_t (&r)[4]) {
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+
+// Four 8x8 b16 matrices, transposed on the way in: register j of lane (gid, tig) holds
+// elements (row 2*tig, col gid) and (row 2*tig+1, col gid) of matrix j.
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                  : "r"(addr));
 }
@@ -115,12 +133,19 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+// Order-preserving key of a score: larger float <=> larger key, -0 counted as +0.
+__device__ __forceinline__ uint32_t score_key_bits(float s) {
+    uint32_t u = __float_as_uint(s);
+    if (u == 0x80000000u) u = 0u;
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
 // Per-warp running softmax state. Columns of the MMA tiles are query heads:
 // this lane owns heads 2*tig and 2*tig+1 of the group.
 struct WarpAcc {
     float m[2];        // running max of logit*log2(e), identical in all lanes that share tig
     float l[2];        // this lane's share of the running sum
-    float o[8][4];     // O^T fragments: o[t][0..1] d = 8*gid+t, o[t][2..3] d = 64+8*gid+t
+    float o[8][4];     // O^T fragments: o[t][0..1] d = 16*t+gid, o[t][2..3] d = 16*t+8+gid
 };
 
 // Consume one staged tile: 16 K rows at ks, 16 V rows at vs (swizzled, see
@@ -130,30 +155,52 @@ template <int MODE>
 __device__ __forceinline__ void consume_tile(const AttnParams& p, uint32_t ks, uint32_t vs,
                                              const uint32_t (&qf)[4][4], WarpAcc& acc, uint32_t vmask,
                                              int gid, int tig, float* score_row0, float* score_row1,
-                                             int pos_base) {
+                                             int pos_base, uint32_t* hist) {
     // ---- S^T = K . Q^T ------------------------------------------------------
+    // Two independent accumulator chains (even / odd 32-element blocks of the head dimension).
     float s[4] = {0.f, 0.f, 0.f, 0.f};
+    float s2[4] = {0.f, 0.f, 0.f, 0.f};
     const uint32_t krow = ks + gid * 256;
     const uint32_t kswz = (gid & 1) << 2;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        uint32_t ka[4], kb[4];
-        const uint32_t off = (((4 * j + tig) ^ kswz) << 4);
-        lds128(krow + off, ka);                 // row gid
-        lds128(krow + 8 * 256 + off, kb);       // row gid + 8
+    for (int j = 0; j < 4; j += 2) {
+        uint32_t ka[4], kb[4], kc[4], kd[4];
+        const uint32_t off0 = (((4 * j + tig) ^ kswz) << 4), off1 = (((4 * j + 4 + tig) ^ kswz) << 4);
+        lds128(krow + off0, ka);                // row gid
+        lds128(krow + 8 * 256 + off0, kb);      // row gid + 8
+        lds128(krow + off1, kc);
+        lds128(krow + 8 * 256 + off1, kd);
         mma_bf16_16816(s, ka[0], kb[0], ka[1], kb[1], qf[j][0], qf[j][1]);
+        mma_bf16_16816(s2, kc[0], kd[0], kc[1], kd[1], qf[j + 1][0], qf[j + 1][1]);
         mma_bf16_16816(s, ka[2], kb[2], ka[3], kb[3], qf[j][2], qf[j][3]);
+        mma_bf16_16816(s2, kc[2], kd[2], kc[3], kd[3], qf[j + 1][2], qf[j + 1][3]);
     }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) s[i] += s2[i];
     const bool v0 = (vmask >> gid) & 1u, v1 = (vmask >> (gid + 8)) & 1u;
     if (MODE == MODE_SELECT) {
         // s[0],s[1]: (pos gid; heads 2tig, 2tig+1)   s[2],s[3]: (pos gid+8; same heads)
+        const float f0 = s[0] * p.scale, f1 = s[1] * p.scale, f2 = s[2] * p.scale, f3 = s[3] * p.scale;
         if (score_row0) {
-            if (v0) score_row0[pos_base + gid] = s[0] * p.scale;
-            if (v1) score_row0[pos_base + gid + 8] = s[2] * p.scale;
+            if (v0) score_row0[pos_base + gid] = f0;
+            if (v1) score_row0[pos_base + gid + 8] = f2;
         }
         if (score_row1) {
-            if (v0) score_row1[pos_base + gid] = s[1] * p.scale;
-            if (v1) score_row1[pos_base + gid + 8] = s[3] * p.scale;
+            if (v0) score_row1[pos_base + gid] = f1;
+            if (v1) score_row1[pos_base + gid + 8] = f3;
+        }
+        if (hist) {      // histogram of the top key bits of every stored score, per head
+            const int nb = 1 << (32 - p.hist_shift);
+            uint32_t* h0 = hist + (2 * tig) * nb;
+            uint32_t* h1 = h0 + nb;
+            if (score_row0) {
+                if (v0) atomicAdd(h0 + (score_key_bits(f0) >> p.hist_shift), 1u);
+                if (v1) atomicAdd(h0 + (score_key_bits(f2) >> p.hist_shift), 1u);
+            }
+            if (score_row1) {
+                if (v0) atomicAdd(h1 + (score_key_bits(f1) >> p.hist_shift), 1u);
+                if (v1) atomicAdd(h1 + (score_key_bits(f3) >> p.hist_shift), 1u);
+            }
         }
     }
     // ---- running softmax (base 2) ---------------------------------------------
@@ -161,26 +208,28 @@ __device__ __forceinline__ void consume_tile(const AttnParams& p, uint32_t ks, u
     float t0 = v0 ? s[0] * p.scale_log2 : NEG_INF, t1 = v0 ? s[1] * p.scale_log2 : NEG_INF;
     float t2 = v1 ? s[2] * p.scale_log2 : NEG_INF, t3 = v1 ? s[3] * p.scale_log2 : NEG_INF;
     float mx0 = fmaxf(t0, t2), mx1 = fmaxf(t1, t3);
+    // The running max rarely grows after the first tiles: one vote decides whether the
+    // cross-lane max and the rescale of the accumulators are needed at all.
+    if (__any_sync(0xffffffffu, (mx0 > acc.m[0]) || (mx1 > acc.m[1]))) {
 #pragma unroll
-    for (int sh = 4; sh <= 16; sh <<= 1) {
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, sh));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
-    }
-    const float mn0 = fmaxf(acc.m[0], mx0), mn1 = fmaxf(acc.m[1], mx1);
-    const bool grew = (mn0 > acc.m[0]) || (mn1 > acc.m[1]);
-    if (__any_sync(0xffffffffu, grew)) {
+        for (int sh = 4; sh <= 16; sh <<= 1) {
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, sh));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
+        }
+        const float g0 = fmaxf(acc.m[0], mx0), g1 = fmaxf(acc.m[1], mx1);
         // exp2(-inf - finite) = 0; when both are -inf the accumulators are still 0.
-        const float a0 = (mn0 == NEG_INF) ? 1.f : fast_exp2(acc.m[0] - mn0);
-        const float a1 = (mn1 == NEG_INF) ? 1.f : fast_exp2(acc.m[1] - mn1);
+        const float a0 = (g0 == NEG_INF) ? 1.f : fast_exp2(acc.m[0] - g0);
+        const float a1 = (g1 == NEG_INF) ? 1.f : fast_exp2(acc.m[1] - g1);
         acc.l[0] *= a0;
         acc.l[1] *= a1;
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
             acc.o[t][0] *= a0; acc.o[t][1] *= a1; acc.o[t][2] *= a0; acc.o[t][3] *= a1;
         }
-        acc.m[0] = mn0;
-        acc.m[1] = mn1;
+        acc.m[0] = g0;
+        acc.m[1] = g1;
     }
+    const float mn0 = acc.m[0], mn1 = acc.m[1];
     const float ms0 = (mn0 == NEG_INF) ? 0.f : mn0, ms1 = (mn1 == NEG_INF) ? 0.f : mn1;
     const float p0 = fast_exp2(t0 - ms0), p1 = fast_exp2(t1 - ms1);
     const float p2 = fast_exp2(t2 - ms0), p3 = fast_exp2(t3 - ms1);
@@ -190,260 +239,392 @@ __device__ __forceinline__ void consume_tile(const AttnParams& p, uint32_t ks, u
     const uint32_t pb0 = movmatrix_trans(pack_bf16(p0, p1));
     const uint32_t pb1 = movmatrix_trans(pack_bf16(p2, p3));
     // ---- O^T += V^T . P^T ------------------------------------------------------
-    // This lane needs rows 2tig, 2tig+1, 2tig+8, 2tig+9 and the 16-byte pieces gid and gid+8.
-    uint32_t vr[4][2][4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int r = 2 * tig + (i & 1) + ((i >> 1) << 3);
-        const uint32_t vswz = ((r >> 1) & 3) << 1;
-        lds128(vs + r * 256 + ((gid ^ vswz) << 4), vr[i][0]);
-        lds128(vs + r * 256 + (((gid + 8) ^ vswz) << 4), vr[i][1]);
-    }
+    // ldmatrix.trans hands out V^T fragments directly: for the 16 head-dim rows of block t the
+    // four matrices are (pos 0-7 | 8-15) x (16-byte pieces 2t | 2t+1) of the V tile. Lane l
+    // addresses row (l&7) + 8*(l>>4) and piece 2t + ((l>>3)&1); piece c of row r sits at c ^ (r&7).
+    const int lane = gid * 4 + tig;
+    const int rr = lane & 7, mb = (lane >> 3) & 1;
+    const uint32_t vlane = vs + (rr + ((lane >> 4) << 3)) * 256 + ((rr ^ mb) << 4);
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
-        const int u = t >> 1;
-        const uint32_t sel = (t & 1) ? 0x7632u : 0x5410u;
-        const uint32_t a0 = __byte_perm(vr[0][0][u], vr[1][0][u], sel);
-        const uint32_t a1 = __byte_perm(vr[0][1][u], vr[1][1][u], sel);
-        const uint32_t a2 = __byte_perm(vr[2][0][u], vr[3][0][u], sel);
-        const uint32_t a3 = __byte_perm(vr[2][1][u], vr[3][1][u], sel);
-        mma_bf16_16816(acc.o[t], a0, a1, a2, a3, pb0, pb1);
+        uint32_t a[4];
+        ldmatrix_x4_trans(vlane ^ (t << 5), a);       // ring slots are 256-byte aligned
+        mma_bf16_16816(acc.o[t], a[0], a[1], a[2], a[3], pb0, pb1);
     }
 }
 
+// Tiles of one (sequence, head group) item: at least one, so that an empty item still
+// produces its (all-zero) output row.
+__device__ __forceinline__ int item_tiles(int total) { return max(1, (total + TILE - 1) / TILE); }
+
 template <int MODE, int NW, int STAGES>
-__global__ void __launch_bounds__(NW * 32) attn_kernel(const AttnParams p) {
-    extern __shared__ __align__(128) uint8_t smem[];
+__global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    // Ring slots must be 256-byte aligned (the V fragment addressing XORs bits 5-7).
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     __shared__ uint32_t s_vmask[NW][STAGES];
     __shared__ int s_posbase[NW][STAGES];
     __shared__ int s_is_last;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = lane >> 2, tig = lane & 3;
-    const int b = blockIdx.z, item = blockIdx.y, split = blockIdx.x;
+    constexpr int RING_BYTES = NW * STAGES * STAGE_BYTES;
+    uint32_t* hist = reinterpret_cast<uint32_t*>(smem + RING_BYTES);   // MODE_SELECT: [columns][bins] counters
+    const bool hist_on = (MODE == MODE_SELECT) && p.hist != nullptr;
 
-    int head0, ncols, g;
-    if (MODE == MODE_SPARSE && p.Hi == p.Hq) { head0 = item; ncols = 1; g = item / p.G; }
-    else { g = item; head0 = g * p.G; ncols = p.G; }
-
-    const int N = min(p.ctx_lens[b], p.max_ctx);
-    int total = N;
-    const int* idx_row = nullptr;
-    if (MODE == MODE_SPARSE) {
-        int cnt = p.idx_count ? min(p.idx_count[b], p.budget) : p.budget;
-        total = max(cnt, 0);
-        const int hi = (p.Hi == p.Hq) ? item : ((p.Hi == p.Hkv) ? g : 0);
-        idx_row = p.idx + ((long long)b * p.Hi + hi) * p.budget;
-    }
-    total = max(total, 0);
-    const int nsplits = max(1, (total + p.chunk - 1) / p.chunk);
-    if (split >= nsplits) return;
-    const int e0 = split * p.chunk, e1 = min(total, e0 + p.chunk);
-    const int ntiles = (max(e1 - e0, 0) + TILE - 1) / TILE;
-
-    // Q^T fragments: column gid is head head0+gid; this lane holds the 16-byte
-    // pieces 4j+tig (j = 0..3) of that head's query row.
-    uint32_t qf[4][4];
-    {
-        const uint4* qp = reinterpret_cast<const uint4*>(p.q + ((long long)b * p.Hq + head0 + min(gid, ncols - 1)) * HEAD_DIM);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            uint4 t = __ldg(qp + 4 * j + tig);
-            const bool on = gid < ncols;
-            qf[j][0] = on ? t.x : 0u; qf[j][1] = on ? t.y : 0u; qf[j][2] = on ? t.z : 0u; qf[j][3] = on ? t.w : 0u;
+    // ---- this CTA's share of the flattened (sequence, item, tile) space ---------------------------
+    const bool per_qhead = (MODE == MODE_SPARSE) && (p.Hi == p.Hq);
+    const int IY = per_qhead ? p.Hq : p.Hkv;            // items per sequence
+    auto seq_total = [&](int b) -> int {
+        const int N = min(p.ctx_lens[b], p.max_ctx);
+        if (MODE != MODE_SPARSE) return max(N, 0);
+        const int cnt = p.idx_count ? min(p.idx_count[b], p.budget) : p.budget;
+        return max(cnt, 0);
+    };
+    long long per_cta, lo, hi, seq_start = 0;
+    int b = 0, tiles_b;
+    if (p.splits_per_item > 0) {
+        // Pooled split: CTAs c*S .. c*S+S-1 all work on item c and share its tiles dynamically, so
+        // that SMs that get less memory bandwidth simply take fewer tiles; no CTA spans two items.
+        const int item = blockIdx.x / p.splits_per_item, part = blockIdx.x % p.splits_per_item;
+        b = item / IY;
+        if (b >= p.batch) return;
+        tiles_b = item_tiles(seq_total(b));
+        per_cta = tiles_b;
+        // flat index of the item's first tile relative to sequence b (seq_start stays 0); the
+        // tiles themselves are handed out by the item's pool cursor
+        lo = (long long)(item % IY) * tiles_b;
+        hi = lo + 1;
+        (void)part;
+    } else {
+        long long T = 0;
+        for (int bb = 0; bb < p.batch; ++bb) T += (long long)IY * item_tiles(seq_total(bb));
+        per_cta = (T + gridDim.x - 1) / gridDim.x;
+        lo = (long long)blockIdx.x * per_cta;
+        hi = min(T, lo + per_cta);
+        tiles_b = item_tiles(seq_total(0));
+        if (lo < hi) {
+            while (seq_start + (long long)IY * tiles_b <= lo) {
+                seq_start += (long long)IY * tiles_b;
+                ++b;
+                tiles_b = item_tiles(seq_total(b));
+            }
         }
     }
-
-    float* score_row0 = nullptr;
-    float* score_row1 = nullptr;
-    if (MODE == MODE_SELECT) {
-        if (2 * tig < ncols) score_row0 = p.scores + ((long long)b * p.Hq + head0 + 2 * tig) * p.score_stride;
-        if (2 * tig + 1 < ncols) score_row1 = p.scores + ((long long)b * p.Hq + head0 + 2 * tig + 1) * p.score_stride;
+    if (lo >= hi && p.splits_per_item == 0) return;
+    if (hist_on) {
+        for (int i = threadIdx.x; i < HIST_SMEM_WORDS; i += NW * 32) hist[i] = 0;
+        __syncthreads();
     }
-
-    WarpAcc acc;
-    acc.m[0] = acc.m[1] = -INFINITY;
-    acc.l[0] = acc.l[1] = 0.f;
-#pragma unroll
-    for (int t = 0; t < 8; ++t) { acc.o[t][0] = acc.o[t][1] = acc.o[t][2] = acc.o[t][3] = 0.f; }
 
     uint8_t* wbase = smem + (size_t)warp * STAGES * STAGE_BYTES;
     const uint32_t wbase_u32 = smem_u32(wbase);
-    const long long head_off = (long long)g * p.stride_head;
-    const int my_tiles = (ntiles > warp) ? (ntiles - warp + NW - 1) / NW : 0;   // tiles warp, warp+NW, ...
+    const int c16 = lane & 15, rhalf = lane >> 4;
+    const long long lane_src = (long long)rhalf * p.stride_pos + c16 * 8;
+    const long long two_rows = 2 * p.stride_pos;
+    // Destination of this lane's piece inside a slot, row pair i adds 512 bytes:
+    //   K: row rhalf+2i, piece c16 ^ (rhalf<<2);   V: row rhalf+2i, piece (c16^rhalf) ^ ((i&3)<<1).
+    const uint32_t kdst = rhalf * 256 + ((c16 ^ (rhalf << 2)) << 4);
+    const uint32_t vdst = rhalf * 256;
+    const uint32_t vc = c16 ^ rhalf;
+    const bool pooled = p.splits_per_item > 0;
 
-    // Sparse: the index entry this lane will need for the next tile to be issued.
-    int pref_pos = -1;
-    auto prefetch_idx = [&](int it) {
+    do {
+        // ---- one segment: tiles [t0, t1) of item y of sequence b (pooled: whatever the warps grab) --
+        const int y = (int)((lo - seq_start) / tiles_b);
+        const int t0 = (int)((lo - seq_start) % tiles_b);
+        const int t1 = pooled ? tiles_b : (int)min((long long)tiles_b, t0 + (hi - lo));
+        const int total = seq_total(b);
+        const int N = max(min(p.ctx_lens[b], p.max_ctx), 0);
+        int head0, ncols, g;
+        if (per_qhead) { head0 = y; ncols = 1; g = y / p.G; }
+        else { g = y; head0 = g * p.G; ncols = p.G; }
+        const int* idx_row = nullptr;
         if (MODE == MODE_SPARSE) {
-            const int e = e0 + (warp + it * NW) * TILE + (lane & 15);
-            pref_pos = (it < my_tiles && e < e1) ? __ldg(idx_row + e) : -1;
+            const int hi_idx = per_qhead ? y : ((p.Hi == p.Hkv) ? g : 0);
+            idx_row = p.idx + ((long long)b * p.Hi + hi_idx) * p.budget;
         }
-    };
-    prefetch_idx(0);
+        int* pool = pooled ? p.tile_ctr + (long long)b * IY + y : nullptr;
 
-    // Issue the copies of this warp's `it`-th tile into ring slot `stage`.
-    // Shared layout of a slot: K rows then V rows, 256 B per row, 16-byte piece c of
-    // row r stored at piece c ^ ((r&1)<<2) for K and c ^ (((r>>1)&3)<<1) for V so that
-    // the fragment reads in consume_tile are bank-conflict free.
-    auto issue = [&](int it, int stage) {
-        const int tile = warp + it * NW;
-        const uint32_t ks = wbase_u32 + stage * STAGE_BYTES, vs = ks + TILE_BYTES;
-        const int c = lane & 15;
-        uint32_t vmask;
-        if (MODE != MODE_SPARSE) {
-            const int pos0 = e0 + tile * TILE;
-            long long off;
-            bool ok = true;
-            if (p.paged) {
-                const int page = __ldg(p.page_table + (long long)b * p.max_pages + (pos0 >> 4));
-                ok = (unsigned)page < (unsigned)p.num_pages;
-                if (!ok && lane == 0) atomicOr(p.status, STATUS_BAD_PAGE);
-                off = (ok ? (long long)page * p.stride_page : 0) + head_off;
-            } else {
-                off = (long long)b * p.stride_b + head_off + (long long)pos0 * p.stride_pos;
-            }
-            const int nvalid = ok ? min(TILE, e1 - pos0) : 0;
-            vmask = (1u << nvalid) - 1u;
+        // Q^T fragments: column gid is head head0+gid; this lane holds the 16-byte
+        // pieces 4j+tig (j = 0..3) of that head's query row.
+        uint32_t qf[4][4];
+        {
+            const uint4* qp = reinterpret_cast<const uint4*>(
+                p.q + ((long long)b * p.Hq + head0 + min(gid, ncols - 1)) * HEAD_DIM);
+            const bool on = gid < ncols;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int r = (lane >> 4) + 2 * i;
-                const bool rv = r < nvalid;
-                const long long eo = rv ? off + (long long)r * p.stride_pos + c * 8 : 0;
-                cp_async16(ks + r * 256 + ((c ^ ((r & 1) << 2)) << 4), p.k + eo, rv ? 16 : 0);
-                cp_async16(vs + r * 256 + ((c ^ (((r >> 1) & 3) << 1)) << 4), p.v + eo, rv ? 16 : 0);
+            for (int j = 0; j < 4; ++j) {
+                const uint4 t = __ldg(qp + 4 * j + tig);
+                qf[j][0] = on ? t.x : 0u; qf[j][1] = on ? t.y : 0u; qf[j][2] = on ? t.z : 0u; qf[j][3] = on ? t.w : 0u;
             }
-            if (lane == 0) { s_vmask[warp][stage] = vmask; s_posbase[warp][stage] = pos0; }
-        } else {
-            const int pos = pref_pos;
-            prefetch_idx(it + 1);
-            bool valid = pos >= 0 && pos < N;
-            if (pos >= N) atomicOr(p.status, STATUS_BAD_INDEX);
-            long long off = 0;
-            if (valid) {
+        }
+        float* score_row0 = nullptr;
+        float* score_row1 = nullptr;
+        if (MODE == MODE_SELECT) {
+            if (2 * tig < ncols) score_row0 = p.scores + ((long long)b * p.Hq + head0 + 2 * tig) * p.score_stride;
+            if (2 * tig + 1 < ncols) score_row1 = p.scores + ((long long)b * p.Hq + head0 + 2 * tig + 1) * p.score_stride;
+        }
+        WarpAcc acc;
+        acc.m[0] = acc.m[1] = -INFINITY;
+        acc.l[0] = acc.l[1] = 0.f;
+#pragma unroll
+        for (int t = 0; t < 8; ++t) { acc.o[t][0] = acc.o[t][1] = acc.o[t][2] = acc.o[t][3] = 0.f; }
+
+        const long long head_off = (long long)g * p.stride_head;
+        const long long item_off = (p.paged ? 0 : (long long)b * p.stride_b) + head_off;
+
+        // ---- this warp's tile sequence -----------------------------------------------------------------
+        // static: t0 + warp, + NW, ... below t1.  pooled: GRAB_TILES consecutive tiles at a time from the
+        // item's cursor; the next grab is requested one chunk ahead so that its latency is hidden.
+        int cur = t0 + warp, cur_end = t1;             // static walk
+        int grab_raw = 0;                              // lane 0: value returned by the outstanding grab
+        auto grab = [&]() { if (lane == 0) grab_raw = atomicAdd(pool, GRAB_TILES); };
+        if (pooled) {
+            grab();
+            cur = __shfl_sync(0xffffffffu, grab_raw, 0);
+            cur_end = min(tiles_b, cur + GRAB_TILES);
+            grab();
+        }
+        auto next_tile = [&]() -> int {                // -1 when this warp has no more tiles
+            if (!pooled) {
+                if (cur >= cur_end) return -1;
+                const int t = cur;
+                cur += NW;
+                return t;
+            }
+            if (cur >= cur_end) {
+                if (cur_end >= tiles_b) return -1;     // the pool ran dry on the previous grab
+                cur = __shfl_sync(0xffffffffu, grab_raw, 0);
+                if (cur >= tiles_b) { cur_end = tiles_b; return -1; }
+                cur_end = min(tiles_b, cur + GRAB_TILES);
+                grab();
+            }
+            return cur++;
+        };
+
+        // Sparse: the index entry this lane needs for the tile that will be issued next.
+        int pref_tile = next_tile();
+        int pref_pos = -1;
+        auto prefetch_idx = [&]() {
+            if (MODE == MODE_SPARSE) {
+                const int e = pref_tile * TILE + c16;
+                pref_pos = (pref_tile >= 0 && e < total) ? __ldg(idx_row + e) : -1;
+            }
+        };
+        prefetch_idx();
+
+        // Issue the copies of tile `pref_tile` into ring slot `stage`, then advance to the next tile.
+        // Shared layout of a slot: K rows then V rows, 256 B per row, 16-byte piece c of
+        // row r stored at piece c ^ ((r&1)<<2) for K and c ^ (r&7) for V so that the
+        // fragment reads in consume_tile are bank-conflict free. Lane l copies piece
+        // l&15 of rows (l>>4) + 2i, i = 0..7: one instruction moves two whole rows.
+        auto issue = [&](int stage) {
+            const int tile = pref_tile;
+            const uint32_t ks = wbase_u32 + stage * STAGE_BYTES, vs = ks + TILE_BYTES;
+            uint32_t vmask;
+            if (MODE != MODE_SPARSE) {
+                pref_tile = next_tile();
+                const int pos0 = tile * TILE;
+                long long off;
+                bool ok = true;
                 if (p.paged) {
-                    const int page = __ldg(p.page_table + (long long)b * p.max_pages + (pos >> 4));
-                    if ((unsigned)page < (unsigned)p.num_pages) {
-                        off = (long long)page * p.stride_page + (long long)(pos & 15) * p.stride_pos + head_off;
-                    } else {
-                        valid = false;
-                        atomicOr(p.status, STATUS_BAD_PAGE);
+                    const int page = __ldg(p.page_table + (long long)b * p.max_pages + tile);
+                    ok = (unsigned)page < (unsigned)p.num_pages;
+                    if (!ok && lane == 0) atomicOr(p.status, STATUS_BAD_PAGE);
+                    off = (ok ? (long long)page * p.stride_page : 0) + item_off + lane_src;
+                } else {
+                    off = item_off + (long long)pos0 * p.stride_pos + lane_src;
+                }
+                const int nvalid = ok ? max(0, min(TILE, total - pos0)) : 0;
+                vmask = (1u << nvalid) - 1u;
+                const __nv_bfloat16* ksrc = p.k + off;
+                const __nv_bfloat16* vsrc = p.v + off;
+                if (nvalid == TILE) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        cp_async16_full(ks + kdst + i * 512, ksrc + i * two_rows);
+                        cp_async16_full(vs + vdst + i * 512 + ((vc ^ ((i & 3) << 1)) << 4), vsrc + i * two_rows);
                     }
                 } else {
-                    off = (long long)b * p.stride_b + (long long)pos * p.stride_pos + head_off;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const bool rv = rhalf + 2 * i < nvalid;
+                        cp_async16(ks + kdst + i * 512, rv ? ksrc + i * two_rows : p.k, rv ? 16 : 0);
+                        cp_async16(vs + vdst + i * 512 + ((vc ^ ((i & 3) << 1)) << 4), rv ? vsrc + i * two_rows : p.v, rv ? 16 : 0);
+                    }
+                }
+                if (lane == 0) { s_vmask[warp][stage] = vmask; s_posbase[warp][stage] = pos0; }
+            } else {
+                const int pos = pref_pos;
+                pref_tile = next_tile();
+                prefetch_idx();
+                bool valid = pos >= 0 && pos < N;
+                if (pos >= N) atomicOr(p.status, STATUS_BAD_INDEX);
+                long long off = 0;
+                if (valid) {
+                    if (p.paged) {
+                        const int page = __ldg(p.page_table + (long long)b * p.max_pages + (pos >> 4));
+                        if ((unsigned)page < (unsigned)p.num_pages) {
+                            off = (long long)page * p.stride_page + (long long)(pos & 15) * p.stride_pos + head_off;
+                        } else {
+                            valid = false;
+                            atomicOr(p.status, STATUS_BAD_PAGE);
+                        }
+                    } else {
+                        off = item_off + (long long)pos * p.stride_pos;
+                    }
+                }
+                vmask = __ballot_sync(0xffffffffu, valid) & 0xffffu;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = rhalf + 2 * i;
+                    const long long ro = __shfl_sync(0xffffffffu, off, r);
+                    const bool rv = (vmask >> r) & 1u;
+                    const long long eo = rv ? ro + c16 * 8 : 0;
+                    cp_async16(ks + kdst + i * 512, p.k + eo, rv ? 16 : 0);
+                    cp_async16(vs + vdst + i * 512 + ((vc ^ ((i & 3) << 1)) << 4), p.v + eo, rv ? 16 : 0);
+                }
+                if (lane == 0) { s_vmask[warp][stage] = vmask; s_posbase[warp][stage] = 0; }
+            }
+        };
+
+        // ---- private cp.async ring -----------------------------------------------------------------------
+        int issued = 0;
+#pragma unroll
+        for (int s = 0; s < STAGES - 1; ++s) {
+            if (pref_tile >= 0) { issue(s); ++issued; }
+            cp_async_commit();
+        }
+        for (int it = 0; it < issued; ++it) {
+            cp_async_wait<STAGES - 2>();      // tile `it` has landed (this lane's copies)
+            __syncwarp();                     // ... and every other lane's; slot (it-1)%STAGES is free
+            if (pref_tile >= 0) { issue((it + STAGES - 1) % STAGES); ++issued; }
+            cp_async_commit();
+            const int stage = it % STAGES;
+            const uint32_t ks = wbase_u32 + stage * STAGE_BYTES;
+            consume_tile<MODE>(p, ks, ks + TILE_BYTES, qf, acc, s_vmask[warp][stage], gid, tig,
+                               score_row0, score_row1, s_posbase[warp][stage], hist_on ? hist : nullptr);
+        }
+        cp_async_wait<0>();
+        __syncwarp();
+
+        if (hist_on) {                        // add this segment's histogram to the global one
+            __syncthreads();
+            const int nb = 1 << (32 - p.hist_shift);
+            for (int i = threadIdx.x; i < ncols * nb; i += NW * 32) {
+                const uint32_t w = hist[i];
+                if (w) {
+                    atomicAdd(p.hist + ((long long)b * p.Hq + head0 + i / nb) * HIST_BINS + (i % nb), w);
+                    hist[i] = 0;
                 }
             }
-            vmask = __ballot_sync(0xffffffffu, valid) & 0xffffu;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int r = (lane >> 4) + 2 * i;
-                const long long ro = __shfl_sync(0xffffffffu, off, r);
-                const bool rv = (vmask >> r) & 1u;
-                const long long eo = rv ? ro + c * 8 : 0;
-                cp_async16(ks + r * 256 + ((c ^ ((r & 1) << 2)) << 4), p.k + eo, rv ? 16 : 0);
-                cp_async16(vs + r * 256 + ((c ^ (((r >> 1) & 3) << 1)) << 4), p.v + eo, rv ? 16 : 0);
-            }
-            if (lane == 0) { s_vmask[warp][stage] = vmask; s_posbase[warp][stage] = 0; }
+            __syncthreads();
         }
-    };
 
-    // ---- private cp.async ring --------------------------------------------------
+        // ---- merge the warps of this CTA ---------------------------------------------------------------
 #pragma unroll
-    for (int s = 0; s < STAGES - 1; ++s) {
-        if (s < my_tiles) issue(s, s);
-        cp_async_commit();
-    }
-    for (int it = 0; it < my_tiles; ++it) {
-        cp_async_wait<STAGES - 2>();      // tile `it` has landed (this lane's copies)
-        __syncwarp();                     // ... and every other lane's; slot (it-1)%STAGES is free
-        const int nxt = it + STAGES - 1;
-        if (nxt < my_tiles) issue(nxt, nxt % STAGES);
-        cp_async_commit();
-        const int stage = it % STAGES;
-        const uint32_t ks = wbase_u32 + stage * STAGE_BYTES;
-        consume_tile<MODE>(p, ks, ks + TILE_BYTES, qf, acc, s_vmask[warp][stage], gid, tig,
-                           score_row0, score_row1, s_posbase[warp][stage]);
-    }
-    cp_async_wait<0>();
-
-    // ---- merge the warps of this CTA ---------------------------------------------
-#pragma unroll
-    for (int sh = 4; sh <= 16; sh <<= 1) {
-        acc.l[0] += __shfl_xor_sync(0xffffffffu, acc.l[0], sh);
-        acc.l[1] += __shfl_xor_sync(0xffffffffu, acc.l[1], sh);
-    }
-    __syncthreads();                      // all rings drained; reuse the shared memory
-    float* mo = reinterpret_cast<float*>(smem);                   // [NW][8][128]
-    float2* mml = reinterpret_cast<float2*>(smem + NW * 8 * HEAD_DIM * 4);   // [NW][8]
-#pragma unroll
-    for (int t = 0; t < 8; ++t) {
-        float* w0 = mo + ((warp * 8 + 2 * tig) * HEAD_DIM);
-        float* w1 = w0 + HEAD_DIM;
-        w0[8 * gid + t] = acc.o[t][0];
-        w1[8 * gid + t] = acc.o[t][1];
-        w0[64 + 8 * gid + t] = acc.o[t][2];
-        w1[64 + 8 * gid + t] = acc.o[t][3];
-    }
-    if (gid == 0) {
-        mml[warp * 8 + 2 * tig] = make_float2(acc.m[0], acc.l[0]);
-        mml[warp * 8 + 2 * tig + 1] = make_float2(acc.m[1], acc.l[1]);
-    }
-    __syncthreads();
-
-    const long long row0 = (long long)b * p.Hq + head0;
-    for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) {
-        const int col = e >> 7, c = e & 127;
-        float M = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < NW; ++w) M = fmaxf(M, mml[w * 8 + col].x);
-        float L = 0.f, O = 0.f;
-        if (M != -INFINITY) {
-#pragma unroll
-            for (int w = 0; w < NW; ++w) {
-                const float2 ml = mml[w * 8 + col];
-                const float f = (ml.x == -INFINITY) ? 0.f : fast_exp2(ml.x - M);
-                L += ml.y * f;
-                O += mo[(w * 8 + col) * HEAD_DIM + c] * f;
-            }
+        for (int sh = 4; sh <= 16; sh <<= 1) {
+            acc.l[0] += __shfl_xor_sync(0xffffffffu, acc.l[0], sh);
+            acc.l[1] += __shfl_xor_sync(0xffffffffu, acc.l[1], sh);
         }
-        if (nsplits == 1) {
-            p.out[(row0 + col) * HEAD_DIM + c] = (L > 0.f) ? O / L : 0.f;
+        __syncthreads();                      // all rings drained; reuse the shared memory
+        float* mo = reinterpret_cast<float*>(smem);                                // [NW][8][128]
+        float2* mml = reinterpret_cast<float2*>(smem + NW * 8 * HEAD_DIM * 4);    // [NW][8]
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            float* w0 = mo + ((warp * 8 + 2 * tig) * HEAD_DIM);
+            float* w1 = w0 + HEAD_DIM;
+            w0[16 * t + gid] = acc.o[t][0];
+            w1[16 * t + gid] = acc.o[t][1];
+            w0[16 * t + 8 + gid] = acc.o[t][2];
+            w1[16 * t + 8 + gid] = acc.o[t][3];
+        }
+        if (gid == 0) {
+            mml[warp * 8 + 2 * tig] = make_float2(acc.m[0], acc.l[0]);
+            mml[warp * 8 + 2 * tig + 1] = make_float2(acc.m[1], acc.l[1]);
+        }
+        __syncthreads();
+
+        // CTAs that share this item: those whose range meets [item_lo, item_lo + tiles_b).
+        int nsplits, split;
+        if (pooled) {
+            nsplits = p.splits_per_item;          // every CTA of the item arrives, with or without tiles
+            split = blockIdx.x % p.splits_per_item;
         } else {
-            const long long pr = (row0 + col) * p.max_splits + split;
-            p.part_o[pr * HEAD_DIM + c] = O;
-            if (c == 0) p.part_ml[pr] = make_float2(M, L);
+            const long long item_lo = seq_start + (long long)y * tiles_b;
+            const int first_cta = (int)(item_lo / per_cta);
+            nsplits = (int)((item_lo + tiles_b - 1) / per_cta) - first_cta + 1;
+            split = (int)blockIdx.x - first_cta;
         }
-    }
-    if (nsplits == 1) return;
-
-    // ---- the last CTA of this (sequence, head group) combines the splits -----------
-    __threadfence();
-    __syncthreads();
-    int* ctr = p.counters + (long long)b * gridDim.y + item;
-    if (threadIdx.x == 0) {
-        const int old = atomicAdd(ctr, 1);
-        s_is_last = (old == nsplits - 1);
-    }
-    __syncthreads();
-    if (!s_is_last) return;
-    __threadfence();
-    for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) {
-        const int col = e >> 7, c = e & 127;
-        const long long pr = (row0 + col) * p.max_splits;
-        float M = -INFINITY;
-        for (int s = 0; s < nsplits; ++s) M = fmaxf(M, __ldcg(&p.part_ml[pr + s].x));
-        float L = 0.f, O = 0.f;
-        if (M != -INFINITY) {
-            for (int s = 0; s < nsplits; ++s) {
-                const float2 ml = __ldcg(&p.part_ml[pr + s]);
-                const float f = (ml.x == -INFINITY) ? 0.f : fast_exp2(ml.x - M);
-                L += ml.y * f;
-                O += __ldcg(&p.part_o[(pr + s) * HEAD_DIM + c]) * f;
+        const long long row0 = (long long)b * p.Hq + head0;
+        for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) {
+            const int col = e >> 7, c = e & 127;
+            float M = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) M = fmaxf(M, mml[w * 8 + col].x);
+            float L = 0.f, O = 0.f;
+            if (M != -INFINITY) {
+#pragma unroll
+                for (int w = 0; w < NW; ++w) {
+                    const float2 ml = mml[w * 8 + col];
+                    const float f = (ml.x == -INFINITY) ? 0.f : fast_exp2(ml.x - M);
+                    L += ml.y * f;
+                    O += mo[(w * 8 + col) * HEAD_DIM + c] * f;
+                }
+            }
+            if (nsplits == 1) {
+                p.out[(row0 + col) * HEAD_DIM + c] = (L > 0.f) ? O / L : 0.f;
+            } else if (split < p.max_splits) {
+                const long long pr = (row0 + col) * p.max_splits + split;
+                p.part_o[pr * HEAD_DIM + c] = O;
+                if (c == 0) p.part_ml[pr] = make_float2(M, L);
             }
         }
-        p.out[(row0 + col) * HEAD_DIM + c] = (L > 0.f) ? O / L : 0.f;
-    }
-    if (threadIdx.x == 0) *ctr = 0;       // ready for the next launch
+        if (nsplits == 1 && pooled && threadIdx.x == 0) *pool = 0;
+        if (nsplits > 1) {
+            // ---- the last CTA of this item to arrive combines the splits ---------------------------------
+            __threadfence();
+            __syncthreads();
+            int* ctr = p.counters + (long long)b * IY + y;
+            if (threadIdx.x == 0) {
+                const int old = atomicAdd(ctr, 1);
+                s_is_last = (old == nsplits - 1);
+            }
+            __syncthreads();
+            if (s_is_last) {
+                __threadfence();
+                const int ns = min(nsplits, p.max_splits);
+                for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) {
+                    const int col = e >> 7, c = e & 127;
+                    const long long pr = (row0 + col) * p.max_splits;
+                    float M = -INFINITY;
+                    for (int s = 0; s < ns; ++s) M = fmaxf(M, __ldcg(&p.part_ml[pr + s].x));
+                    float L = 0.f, O = 0.f;
+                    if (M != -INFINITY) {
+                        for (int s = 0; s < ns; ++s) {
+                            const float2 ml = __ldcg(&p.part_ml[pr + s]);
+                            const float f = (ml.x == -INFINITY) ? 0.f : fast_exp2(ml.x - M);
+                            L += ml.y * f;
+                            O += __ldcg(&p.part_o[(pr + s) * HEAD_DIM + c]) * f;
+                        }
+                    }
+                    p.out[(row0 + col) * HEAD_DIM + c] = (L > 0.f) ? O / L : 0.f;
+                }
+                if (threadIdx.x == 0) { *ctr = 0; if (pooled) *pool = 0; }   // ready for the next launch
+            }
+        }
+        __syncthreads();                          // shared memory is reused by the next segment
+
+        // ---- advance to the next segment -----------------------------------------------------------------
+        if (pooled) break;
+        lo += (t1 - t0);
+        if (lo < hi && lo >= seq_start + (long long)IY * tiles_b) {
+            seq_start += (long long)IY * tiles_b;
+            ++b;
+            tiles_b = item_tiles(seq_total(b));
+        }
+    } while (lo < hi);
 }
 
 }  // namespace tidal

@@ -20,16 +20,17 @@ using namespace tidal;
 namespace {
 
 constexpr int MAX_CTX = 262144;
-constexpr int MAX_SPLITS = 512;
+constexpr int GRID_MAX = 320;            // persistent CTAs per launch never exceed this (2 per SM on 148 SMs)
+constexpr int MIN_TILES_PER_CTA = 8;     // do not cut work finer than 128 positions per CTA
 constexpr int MAX_GROUP = 8;            // query heads per KV head that fit the 8 MMA columns
 
 // Streaming (full / selection) and gather (sparse) launch shapes.
 constexpr int DENSE_NW = 8, DENSE_STAGES = 3;
 constexpr int SPARSE_NW = 4, SPARSE_STAGES = 3;
+constexpr size_t HIST_SMEM = HIST_SMEM_WORDS * sizeof(uint32_t);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-struct Plan { int chunk; int nsplits; };
 
 }  // namespace
 
@@ -46,6 +47,7 @@ struct tidal_ctx {
     int state_rows = 0;                         // capacity in (sequence, head) rows
     int* status = nullptr;                      // device word, sticky
     int64_t launches = 0;
+    int tune_dense = 0, tune_sparse = 0;        // development switches (TIDAL_TUNE_DENSE / TIDAL_TUNE_SPARSE)
 };
 
 namespace {
@@ -54,35 +56,34 @@ struct WsLayout {
     size_t part_ml, part_o, scores, cand, idx, idx_count, q_stage, out_stage, total;
     long long cand_stride;
     long long score_stride;
+    int max_splits;
 };
 
-// Chunk of the context (or of the index list) per CTA. Single-sequence work is
-// split so that the CTAs fill whole waves of resident slots; batched work is cut
-// into more, smaller chunks so that the hardware scheduler evens out ragged lengths.
-Plan plan_split(int total_max, int items, int slots, int batch) {
-    total_max = std::max(total_max, 1);
-    const int tiles = (total_max + TILE - 1) / TILE;
-    int best_s = 1;
-    if (batch > 1) {
-        const int want = std::max(1, (6 * slots + items - 1) / items);
-        best_s = std::min(want, std::max(1, tiles / 32));           // at least 512 positions per CTA
-    } else {
-        double best = -1.0;
-        const int smax = std::max(1, std::min(MAX_SPLITS, tiles / 8));   // at least 128 positions per CTA
-        for (int s = 1; s <= smax; ++s) {
-            const long long ctas = (long long)items * s;
-            const long long waves = (ctas + slots - 1) / slots;
-            const double eff = (double)ctas / (double)(waves * slots) - 0.004 * (double)(waves - 1);
-            if (eff > best + 1e-9) { best = eff; best_s = s; }
-        }
-    }
-    best_s = std::max(1, std::min(best_s, MAX_SPLITS));
-    int chunk = (int)align_up((size_t)(total_max + best_s - 1) / best_s, TILE);
-    chunk = std::max(chunk, TILE);
-    Plan p;
-    p.chunk = chunk;
-    p.nsplits = (total_max + chunk - 1) / chunk;
-    return p;
+// Partial-result slots a (sequence, head) row can need: the CTAs of one launch are at most
+// GRID_MAX, and an item of `tiles_max` tiles is cut into at most tiles/per_cta + 2 pieces where
+// per_cta >= (one tile per item) * items / GRID_MAX.
+int max_splits_for(const tidal_kv_t* kv) {
+    const long long items = (long long)kv->batch * kv->num_kv_heads;
+    const long long tiles_max = (kv->max_ctx_len + TILE - 1) / TILE;
+    const long long bound = tiles_max * GRID_MAX / std::max(items, 1LL) + 2;
+    return (int)std::max(1LL, std::min<long long>(GRID_MAX, bound));
+}
+
+// Persistent grid: every resident slot gets an equal share of the tiles, but no CTA is
+// launched for fewer than MIN_TILES_PER_CTA tiles.
+int grid_for(long long tiles_upper_bound, int slots) {
+    const long long by_work = std::max(1LL, tiles_upper_bound / MIN_TILES_PER_CTA);
+    return (int)std::max(1LL, std::min<long long>(std::min(slots, GRID_MAX), by_work));
+}
+
+// 2048 histogram bins per head while the group's columns fit the shared histogram, else 1024.
+int hist_shift_for(const tidal_kv_t* kv) { return (kv->num_q_heads / kv->num_kv_heads) <= 4 ? 21 : 22; }
+
+// One sequence: all items have the same length, so whole groups of CTAs can share an item's tiles.
+int pooled_splits(const tidal_kv_t* kv, int items, int grid) {
+    if (kv->batch != 1) return 0;
+    const int S = grid / std::max(items, 1);
+    return S >= 2 ? S : 0;
 }
 
 int hi_of(const tidal_kv_t* kv, int granularity) {
@@ -127,8 +128,9 @@ WsLayout layout_ws(const tidal_kv_t* kv, int k, int num_layers_host) {
     WsLayout w;
     const size_t rows = (size_t)kv->batch * kv->num_q_heads;
     size_t at = 0;
-    w.part_ml = at;   at += align_up(rows * MAX_SPLITS * sizeof(float2), 256);
-    w.part_o = at;    at += align_up(rows * MAX_SPLITS * HEAD_DIM * sizeof(float), 256);
+    w.max_splits = max_splits_for(kv);
+    w.part_ml = at;   at += align_up(rows * w.max_splits * sizeof(float2), 256);
+    w.part_o = at;    at += align_up(rows * w.max_splits * HEAD_DIM * sizeof(float), 256);
     w.score_stride = (long long)align_up((size_t)kv->max_ctx_len, 16);
     w.scores = at;    at += align_up(rows * (size_t)w.score_stride * sizeof(float), 256);
     w.cand_stride = w.score_stride;
@@ -141,7 +143,6 @@ WsLayout layout_ws(const tidal_kv_t* kv, int k, int num_layers_host) {
     return w;
 }
 
-// part_o is sized for MAX_SPLITS per row only when that is small; otherwise bound it by the plan.
 size_t ws_bytes_for(const tidal_kv_t* kv, int k, int num_layers_host) {
     return layout_ws(kv, k, num_layers_host).total;
 }
@@ -157,18 +158,19 @@ tidal_status_t ensure_ws(tidal_ctx* ctx, size_t bytes) {
     return TIDAL_OK;
 }
 
-// State layout for a capacity of R rows: counters[R] | cursor[R] | done[R] | hist[R][TK_BINS].
+// State layout for a capacity of R rows: counters[R] | cursor[R] | done[R] | tile_ctr[R] | hist[R][TK_BINS].
 inline int* state_counters(const tidal_ctx* c) { return (int*)c->state; }
 inline int* state_cursor(const tidal_ctx* c) { return (int*)c->state + c->state_rows; }
 inline int* state_done(const tidal_ctx* c) { return (int*)c->state + 2 * (size_t)c->state_rows; }
-inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + 3 * (size_t)c->state_rows; }
+inline int* state_tile_ctr(const tidal_ctx* c) { return (int*)c->state + 3 * (size_t)c->state_rows; }
+inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + 4 * (size_t)c->state_rows; }
 
 tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     if (ctx->state_rows >= rows) return TIDAL_OK;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
     if (ctx->state) { cudaDeviceSynchronize(); cudaFree(ctx->state); ctx->state = nullptr; ctx->state_rows = 0; }
     const int cap = (int)align_up((size_t)rows, 64);
-    const size_t bytes = (size_t)cap * (3 + TK_BINS) * sizeof(int);
+    const size_t bytes = (size_t)cap * (4 + TK_BINS) * sizeof(int);
     void* p = nullptr;
     if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TIDAL_ERR_NOMEM; }
     if (cudaMemset(p, 0, bytes) != cudaSuccess) { cudaFree(p); return TIDAL_ERR_CUDA; }
@@ -202,34 +204,49 @@ void fill_common(AttnParams& a, const tidal_ctx* ctx, const tidal_kv_t* kv, cons
     a.counters = state_counters(ctx);
     a.part_ml = (float2*)(ws + w.part_ml);
     a.part_o = (float*)(ws + w.part_o);
-    a.max_splits = MAX_SPLITS;
+    a.max_splits = w.max_splits;
+    a.batch = kv->batch;
+    a.tile_ctr = state_tile_ctr(ctx);
+    a.hist_shift = hist_shift_for(kv);
     a.status = ctx->status;
 }
 
 template <int MODE, int NW, int STAGES>
-tidal_status_t launch_attn(tidal_ctx* ctx, const AttnParams& a, dim3 grid, cudaStream_t st) {
-    const size_t smem = (size_t)NW * STAGES * STAGE_BYTES;
-    attn_kernel<MODE, NW, STAGES><<<grid, NW * 32, smem, st>>>(a);
+constexpr size_t attn_smem() {
+    return (size_t)NW * STAGES * STAGE_BYTES + (MODE == MODE_SELECT ? HIST_SMEM : 0) + 1024;   // + alignment slack
+}
+
+template <int MODE, int NW, int STAGES>
+tidal_status_t launch_attn(tidal_ctx* ctx, const AttnParams& a, int grid, cudaStream_t st) {
+    attn_kernel<MODE, NW, STAGES><<<grid, NW * 32, attn_smem<MODE, NW, STAGES>(), st>>>(a);
     ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }
 
+// hist != nullptr: the kernel also accumulates the per-head histogram the top-k needs.
 tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, float* out, float* scores,
-                         long long score_stride, const WsLayout& w, cudaStream_t st) {
+                         long long score_stride, bool fuse_hist, const WsLayout& w, cudaStream_t st) {
     AttnParams a;
     fill_common(a, ctx, kv, q, out, w);
-    const int items = kv->batch * kv->num_kv_heads;
-    const Plan pl = plan_split(kv->max_ctx_len, items, ctx->dense_slots, kv->batch);
-    a.chunk = pl.chunk;
+    const long long tiles = (long long)kv->batch * kv->num_kv_heads * ((kv->max_ctx_len + TILE - 1) / TILE);
+    int grid = grid_for(tiles, ctx->dense_slots);
+    if (const int S = (ctx->tune_dense == 5) ? 0 : pooled_splits(kv, kv->batch * kv->num_kv_heads, grid)) {
+        a.splits_per_item = S;
+        grid = S * kv->batch * kv->num_kv_heads;
+    }
     a.scores = scores;
     a.score_stride = score_stride;
-    dim3 grid(pl.nsplits, kv->num_kv_heads, kv->batch);
+    a.hist = fuse_hist ? state_hist(ctx) : nullptr;
     if (scores) return launch_attn<MODE_SELECT, DENSE_NW, DENSE_STAGES>(ctx, a, grid, st);
+    if (ctx->tune_dense == 1) return launch_attn<MODE_FULL, 4, 6>(ctx, a, grid, st);
+    if (ctx->tune_dense == 2) return launch_attn<MODE_FULL, 6, 4>(ctx, a, grid, st);
+    if (ctx->tune_dense == 3) return launch_attn<MODE_FULL, 4, 3>(ctx, a, 2 * grid, st);
+    if (ctx->tune_dense == 4) return launch_attn<MODE_FULL, 9, 3>(ctx, a, grid, st);
     return launch_attn<MODE_FULL, DENSE_NW, DENSE_STAGES>(ctx, a, grid, st);
 }
 
 tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* scores, long long score_stride,
-                        int k, int Hi, int* idx, int* idx_count, const WsLayout& w, cudaStream_t st) {
+                        int k, int Hi, bool hist_done, int* idx, int* idx_count, const WsLayout& w, cudaStream_t st) {
     TopkParams t;
     std::memset(&t, 0, sizeof t);
     t.scores = scores; t.score_stride = score_stride;
@@ -245,14 +262,15 @@ tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* score
     const int items = kv->batch * Hi;
     if (items > 65535) return TIDAL_ERR_UNSUPPORTED;
     const int parts = (kv->max_ctx_len + TK_SLICE - 1) / TK_SLICE;
+    t.shift = hist_shift_for(kv);
     t.vec_ok = (((uintptr_t)scores & 15) == 0 && (score_stride & 3) == 0) ? 1 : 0;
     t.cand_smem = std::min(16384, std::max(4096, (int)align_up((size_t)k + 4096, 1024)));
     const size_t words = (size_t)(kv->max_ctx_len + 31) / 32;
     const size_t smem = 2 * words * sizeof(unsigned) + (size_t)t.cand_smem * sizeof(uint2);
     dim3 grid(parts, items, 1);
-    topk_hist_kernel<<<grid, TK_THREADS, 0, st>>>(t);
+    if (!hist_done) { topk_hist_kernel<<<grid, TK_THREADS, 0, st>>>(t); ctx->launches++; }
     topk_select_kernel<<<grid, TK_THREADS, smem, st>>>(t);
-    ctx->launches += 2;
+    ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }
 
@@ -262,10 +280,16 @@ tidal_status_t run_sparse(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, c
     AttnParams a;
     fill_common(a, ctx, kv, q, out, w);
     const int per_batch = (Hi == kv->num_q_heads) ? kv->num_q_heads : kv->num_kv_heads;
-    const Plan pl = plan_split(k, kv->batch * per_batch, ctx->sparse_slots, 1);
-    a.chunk = pl.chunk;
+    const long long tiles = (long long)kv->batch * per_batch * ((k + TILE - 1) / TILE);
+    int grid = grid_for(tiles, ctx->sparse_slots);
     a.idx = idx; a.idx_count = idx_count; a.budget = k; a.Hi = Hi;
-    dim3 grid(pl.nsplits, per_batch, kv->batch);
+    if (const int S = (ctx->tune_sparse == 4) ? 0 : pooled_splits(kv, kv->batch * per_batch, grid)) {
+        a.splits_per_item = S;
+        grid = S * kv->batch * per_batch;
+    }
+    if (ctx->tune_sparse == 1) return launch_attn<MODE_SPARSE, 4, 3>(ctx, a, 2 * grid, st);
+    if (ctx->tune_sparse == 2) return launch_attn<MODE_SPARSE, 4, 6>(ctx, a, grid, st);
+    if (ctx->tune_sparse == 3) return launch_attn<MODE_SPARSE, 6, 4>(ctx, a, grid, st);
     return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(ctx, a, grid, st);
 }
 
@@ -294,15 +318,22 @@ tidal_status_t tidal_create(tidal_ctx_t** out, int device, size_t workspace_byte
     if (!ctx) return TIDAL_ERR_NOMEM;
     ctx->device = device;
     ctx->sm_count = prop.multiProcessorCount;
-    const size_t dense_smem = (size_t)DENSE_NW * DENSE_STAGES * STAGE_BYTES;
-    const size_t sparse_smem = (size_t)SPARSE_NW * SPARSE_STAGES * STAGE_BYTES;
-    const int d0 = resident_ctas(attn_kernel<MODE_FULL, DENSE_NW, DENSE_STAGES>, DENSE_NW * 32, dense_smem, ctx->sm_count);
-    const int d1 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW, DENSE_STAGES>, DENSE_NW * 32, dense_smem, ctx->sm_count);
-    const int s0 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>, SPARSE_NW * 32, sparse_smem, ctx->sm_count);
+    const int d0 = resident_ctas(attn_kernel<MODE_FULL, DENSE_NW, DENSE_STAGES>, DENSE_NW * 32, attn_smem<MODE_FULL, DENSE_NW, DENSE_STAGES>(), ctx->sm_count);
+    const int d1 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW, DENSE_STAGES>, DENSE_NW * 32, attn_smem<MODE_SELECT, DENSE_NW, DENSE_STAGES>(), ctx->sm_count);
+    const int s0 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>, SPARSE_NW * 32, attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(), ctx->sm_count);
     const size_t topk_smem = 2 * (size_t)(MAX_CTX / 32) * sizeof(unsigned) + 16384 * sizeof(uint2);
     const bool topk_ok = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topk_smem) == cudaSuccess;
     if (d0 <= 0 || d1 <= 0 || s0 <= 0 || !topk_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
     ctx->dense_slots = std::min(d0, d1);
+    if (const char* e = std::getenv("TIDAL_TUNE_DENSE")) ctx->tune_dense = std::atoi(e);
+    if (const char* e = std::getenv("TIDAL_TUNE_SPARSE")) ctx->tune_sparse = std::atoi(e);
+    resident_ctas(attn_kernel<MODE_FULL, 4, 6>, 128, attn_smem<MODE_FULL, 4, 6>(), ctx->sm_count);
+    resident_ctas(attn_kernel<MODE_FULL, 6, 4>, 192, attn_smem<MODE_FULL, 6, 4>(), ctx->sm_count);
+    resident_ctas(attn_kernel<MODE_FULL, 4, 3>, 128, attn_smem<MODE_FULL, 4, 3>(), ctx->sm_count);
+    resident_ctas(attn_kernel<MODE_FULL, 9, 3>, 288, attn_smem<MODE_FULL, 9, 3>(), ctx->sm_count);
+    resident_ctas(attn_kernel<MODE_SPARSE, 4, 3>, 128, attn_smem<MODE_SPARSE, 4, 3>(), ctx->sm_count);
+    resident_ctas(attn_kernel<MODE_SPARSE, 4, 6>, 128, attn_smem<MODE_SPARSE, 4, 6>(), ctx->sm_count);
+    resident_ctas(attn_kernel<MODE_SPARSE, 6, 4>, 192, attn_smem<MODE_SPARSE, 6, 4>(), ctx->sm_count);
     ctx->sparse_slots = s0;
     if (cudaMalloc((void**)&ctx->status, 256) != cudaSuccess || cudaMemset(ctx->status, 0, 256) != cudaSuccess) {
         cudaGetLastError(); delete ctx; return TIDAL_ERR_NOMEM;
@@ -338,7 +369,7 @@ tidal_status_t tidal_full_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const voi
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
     const WsLayout w = layout_ws(kv, 1, 0);
     if ((rc = ensure_all(ctx, kv, w.total)) != TIDAL_OK) return rc;
-    return run_dense(ctx, kv, q, out, nullptr, 0, w, (cudaStream_t)stream);
+    return run_dense(ctx, kv, q, out, nullptr, 0, false, w, (cudaStream_t)stream);
 }
 
 tidal_status_t tidal_select_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const void* q, int32_t k,
@@ -356,8 +387,9 @@ tidal_status_t tidal_select_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const v
     float* scores = scores_opt ? scores_opt : (float*)((char*)ctx->ws + w.scores);
     const long long stride = scores_opt ? (long long)kv->max_ctx_len : w.score_stride;
     cudaStream_t st = (cudaStream_t)stream;
-    if ((rc = run_dense(ctx, kv, q, out, scores, stride, w, st)) != TIDAL_OK) return rc;
-    return run_topk(ctx, kv, scores, stride, k, Hi, idx, idx_count, w, st);
+    const bool fuse = Hi == kv->num_q_heads;     // per-head ranking: the attention kernel builds the histogram
+    if ((rc = run_dense(ctx, kv, q, out, scores, stride, fuse, w, st)) != TIDAL_OK) return rc;
+    return run_topk(ctx, kv, scores, stride, k, Hi, fuse, idx, idx_count, w, st);
 }
 
 tidal_status_t tidal_sparse_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const void* q, const int32_t* idx,
@@ -406,11 +438,12 @@ static tidal_status_t decode_step_impl(tidal_ctx_t* ctx, int32_t num_layers, con
         const tidal_kv_t* kv = &kvs[i];
         const WsLayout w = layout_ws(kv, k, host_layers);
         if (schedule[i] == TIDAL_LAYER_FULL) {
-            rc = run_dense(ctx, kv, qs[i], outs[i], nullptr, 0, w, st);
+            rc = run_dense(ctx, kv, qs[i], outs[i], nullptr, 0, false, w, st);
         } else if (schedule[i] == TIDAL_LAYER_SELECT) {
             float* scores = (float*)((char*)ctx->ws + w.scores);
-            rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, w, st);
-            if (rc == TIDAL_OK) rc = run_topk(ctx, kv, scores, w.score_stride, k, Hi, idx, idx_count, w, st);
+            const bool fuse = Hi == kv->num_q_heads;
+            rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, fuse, w, st);
+            if (rc == TIDAL_OK) rc = run_topk(ctx, kv, scores, w.score_stride, k, Hi, fuse, idx, idx_count, w, st);
         } else {
             rc = run_sparse(ctx, kv, qs[i], idx, idx_count, k, Hi, outs[i], w, st);
         }

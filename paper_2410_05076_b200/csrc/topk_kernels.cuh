@@ -3,7 +3,7 @@
 // toward the lower position, and write them in ascending position order.
 //
 // Scores become order-preserving 32-bit keys. The exact k'-th largest key is
-// found by a most-significant-digit radix select (11 + 11 + 10 bits):
+// found by a most-significant-digit radix select (11 + 11 + 10 bits, or 10 + 11 + 11):
 //   1. topk_hist_kernel: all SMs histogram the top 11 key bits of every score
 //      (shared-memory histograms, flushed to a global one per index head).
 //   2. topk_select_kernel, all SMs: every CTA derives the threshold bin from the
@@ -45,6 +45,7 @@ struct TopkParams {
     long long cand_stride;
     int cand_smem;             // candidates the last CTA can hold in shared memory
     int vec_ok;                // score rows are 16-byte aligned: float4 loads allowed
+    int shift;                 // first digit = key >> shift (21 or 22); the rest is split 11 + (shift-11) bits
 };
 
 // Larger float <=> larger key; -0 and +0 map to the same key.
@@ -163,7 +164,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_hist_kernel(const TopkParams 
     __syncthreads();
 #pragma unroll
     for (int e = 0; e < TK_VEC * 4; ++e)
-        if ((valid >> e) & 1u) atomicAdd(&sh[key[e] >> 21], 1u);
+        if ((valid >> e) & 1u) atomicAdd(&sh[key[e] >> p.shift], 1u);
     __syncthreads();
     unsigned* gh = p.hist + (long long)item * TK_BINS;
     for (int i = tid; i < TK_BINS; i += TK_THREADS) {
@@ -189,8 +190,12 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
 
     if (kk == N) {                                     // identity list, then padding
         for (int i = s0 + tid; i < s1; i += TK_THREADS) out[i] = i;
-        if (blockIdx.x == 0)
+        if (blockIdx.x == 0) {
             for (int i = N + tid; i < p.k; i += TK_THREADS) out[i] = -1;
+            // a selection layer's attention kernel may have filled the histogram regardless of k
+            unsigned* gh0 = p.hist + (long long)item * TK_BINS;
+            for (int i = tid; i < TK_BINS; i += TK_THREADS) gh0[i] = 0;
+        }
         return;
     }
     if (s0 >= s1) return;
@@ -214,7 +219,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     unsigned take = 0;
 #pragma unroll
     for (int e = 0; e < TK_VEC * 4; ++e)
-        if (((valid >> e) & 1u) && (int)(key[e] >> 21) >= b1) take |= 1u << e;
+        if (((valid >> e) & 1u) && (int)(key[e] >> p.shift) >= b1) take |= 1u << e;
     int cta_total;
     const int mine = __popc(take);
     int slot = block_scan_incl(mine, warp_sums, cta_total) - mine;
@@ -253,24 +258,25 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
     __syncthreads();
 
-    // second digit: key bits 20..10 among keys whose top 11 bits equal b1
+    // second digit: the next 11 key bits among keys whose first digit equals b1
+    const int s2 = p.shift - 11;                       // bits left for the third digit (10 or 11)
     for (int i = tid; i < M; i += TK_THREADS) {
         const uint32_t key = c[i].x;
-        if ((int)(key >> 21) == b1) atomicAdd(&sh_hist[(key >> 10) & 0x7ffu], 1u);
+        if ((int)(key >> p.shift) == b1) atomicAdd(&sh_hist[(key >> s2) & 0x7ffu], 1u);
     }
     __syncthreads();
     const int d2 = pick_digit(sh_hist, TK_BINS, warp_sums, bcast, need);
-    const uint32_t prefix2 = ((uint32_t)b1 << 21) | ((uint32_t)d2 << 10);
+    const uint32_t prefix2 = ((uint32_t)b1 << p.shift) | ((uint32_t)d2 << s2);
 
-    // third digit: key bits 9..0
-    for (int i = tid; i < 1024; i += TK_THREADS) sh_hist[i] = 0;
+    // third digit: the remaining low bits
+    for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
     __syncthreads();
     for (int i = tid; i < M; i += TK_THREADS) {
         const uint32_t key = c[i].x;
-        if ((key >> 10) == (prefix2 >> 10)) atomicAdd(&sh_hist[key & 0x3ffu], 1u);
+        if ((key >> s2) == (prefix2 >> s2)) atomicAdd(&sh_hist[key & ((1u << s2) - 1u)], 1u);
     }
     __syncthreads();
-    const int d3 = pick_digit(sh_hist, 1024, warp_sums, bcast, need);
+    const int d3 = pick_digit(sh_hist, 1 << s2, warp_sums, bcast, need);
     const uint32_t thr = prefix2 | (uint32_t)d3;       // the k'-th largest key; `need` keys equal to it are taken
 
     // bitmaps of positions above / equal to the threshold
