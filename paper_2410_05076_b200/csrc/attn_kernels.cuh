@@ -70,6 +70,8 @@ struct AttnParams {
     unsigned* hist;            // MODE_SELECT, optional: [B*Hq][HIST_BINS] += histogram of the top key bits
     int hist_shift;            // bin = key >> hist_shift (21: 2048 bins, 22: 1024 bins for groups above 4)
     int* tile_ctr;             // splits_per_item > 0: per-item pool cursor, zero between launches
+    int pdl;                   // launched with programmatic stream serialization: see pdl_wait()
+    int wait_first;            // the preceding kernel may have written ctx_lens / idx: wait before reading anything
     int* status;
 };
 
@@ -90,6 +92,12 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
+
+// Programmatic dependent launch: this grid may start while the previous kernel of the stream
+// is still draining. pdl_wait() blocks until that kernel has completed and its writes are
+// visible; pdl_trigger() lets the next kernel start filling SMs as our CTAs retire.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 
 __device__ __forceinline__ void lds128(uint32_t addr, uint32_t (&r)[4]) {
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n"
@@ -272,6 +280,9 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem + RING_BYTES);   // MODE_SELECT: [columns][bins] counters
     const bool hist_on = (MODE == MODE_SELECT) && p.hist != nullptr;
 
+    bool waited = !p.pdl;
+    if (p.pdl && p.wait_first) { pdl_wait(); pdl_trigger(); waited = true; }
+
     // ---- this CTA's share of the flattened (sequence, item, tile) space ---------------------------
     const bool per_qhead = (MODE == MODE_SPARSE) && (p.Hi == p.Hq);
     const int IY = per_qhead ? p.Hq : p.Hkv;            // items per sequence
@@ -284,11 +295,13 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
     long long per_cta, lo, hi, seq_start = 0;
     int b = 0, tiles_b;
     if (p.splits_per_item > 0) {
-        // Pooled split: CTAs c*S .. c*S+S-1 all work on item c and share its tiles dynamically, so
+        // Pooled split: S CTAs work on each item and share its tiles dynamically, so
         // that SMs that get less memory bandwidth simply take fewer tiles; no CTA spans two items.
-        const int item = blockIdx.x / p.splits_per_item, part = blockIdx.x % p.splits_per_item;
+        // CTA -> item round robin: the CTAs of one item are spread over the whole chip.
+        const int n_items = p.batch * IY;
+        const int item = blockIdx.x % n_items, part = blockIdx.x / n_items;
         b = item / IY;
-        if (b >= p.batch) return;
+        if (part >= p.splits_per_item) return;
         tiles_b = item_tiles(seq_total(b));
         per_cta = tiles_b;
         // flat index of the item's first tile relative to sequence b (seq_start stays 0); the
@@ -346,19 +359,6 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         }
         int* pool = pooled ? p.tile_ctr + (long long)b * IY + y : nullptr;
 
-        // Q^T fragments: column gid is head head0+gid; this lane holds the 16-byte
-        // pieces 4j+tig (j = 0..3) of that head's query row.
-        uint32_t qf[4][4];
-        {
-            const uint4* qp = reinterpret_cast<const uint4*>(
-                p.q + ((long long)b * p.Hq + head0 + min(gid, ncols - 1)) * HEAD_DIM);
-            const bool on = gid < ncols;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint4 t = __ldg(qp + 4 * j + tig);
-                qf[j][0] = on ? t.x : 0u; qf[j][1] = on ? t.y : 0u; qf[j][2] = on ? t.z : 0u; qf[j][3] = on ? t.w : 0u;
-            }
-        }
         float* score_row0 = nullptr;
         float* score_row1 = nullptr;
         if (MODE == MODE_SELECT) {
@@ -379,12 +379,13 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         // item's cursor; the next grab is requested one chunk ahead so that its latency is hidden.
         int cur = t0 + warp, cur_end = t1;             // static walk
         int grab_raw = 0;                              // lane 0: value returned by the outstanding grab
-        auto grab = [&]() { if (lane == 0) grab_raw = atomicAdd(pool, GRAB_TILES); };
+        // The first chunk of every warp is fixed (no round trip before the first load); the pool
+        // cursor hands out the tiles after those.
+        const int pool_base = p.splits_per_item * NW * GRAB_TILES;
+        auto grab = [&]() { if (lane == 0) grab_raw = pool_base + atomicAdd(pool, GRAB_TILES); };
         if (pooled) {
-            grab();
-            cur = __shfl_sync(0xffffffffu, grab_raw, 0);
+            cur = ((int)(blockIdx.x / (p.batch * IY)) * NW + warp) * GRAB_TILES;
             cur_end = min(tiles_b, cur + GRAB_TILES);
-            grab();
         }
         auto next_tile = [&]() -> int {                // -1 when this warp has no more tiles
             if (!pooled) {
@@ -413,6 +414,25 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             }
         };
         prefetch_idx();
+
+        // Everything above read only the index list, lengths and launch geometry; the query, the
+        // pool cursor and the scratch buffers belong to the kernels before us.
+        if (!waited) { pdl_wait(); pdl_trigger(); waited = true; }
+        if (pooled) grab();
+
+        // Q^T fragments: column gid is head head0+gid; this lane holds the 16-byte
+        // pieces 4j+tig (j = 0..3) of that head's query row.
+        uint32_t qf[4][4];
+        {
+            const uint4* qp = reinterpret_cast<const uint4*>(
+                p.q + ((long long)b * p.Hq + head0 + min(gid, ncols - 1)) * HEAD_DIM);
+            const bool on = gid < ncols;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint4 t = __ldg(qp + 4 * j + tig);
+                qf[j][0] = on ? t.x : 0u; qf[j][1] = on ? t.y : 0u; qf[j][2] = on ? t.z : 0u; qf[j][3] = on ? t.w : 0u;
+            }
+        }
 
         // Issue the copies of tile `pref_tile` into ring slot `stage`, then advance to the next tile.
         // Shared layout of a slot: K rows then V rows, 256 B per row, 16-byte piece c of
@@ -550,7 +570,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         int nsplits, split;
         if (pooled) {
             nsplits = p.splits_per_item;          // every CTA of the item arrives, with or without tiles
-            split = blockIdx.x % p.splits_per_item;
+            split = blockIdx.x / (p.batch * IY);
         } else {
             const long long item_lo = seq_start + (long long)y * tiles_b;
             const int first_cta = (int)(item_lo / per_cta);
@@ -595,21 +615,43 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             if (s_is_last) {
                 __threadfence();
                 const int ns = min(nsplits, p.max_splits);
-                for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) {
-                    const int col = e >> 7, c = e & 127;
+                // Scale factors of all splits first (shared memory), then every thread sums its
+                // output elements over the splits with the loads batched eight at a time.
+                float* fsc = reinterpret_cast<float*>(smem);              // [ncols][ns] exp2(m_s - M)
+                float* linv = fsc + 8 * p.max_splits;                    // [ncols] 1 / sum
+                for (int col = warp; col < ncols; col += NW) {
                     const long long pr = (row0 + col) * p.max_splits;
                     float M = -INFINITY;
-                    for (int s = 0; s < ns; ++s) M = fmaxf(M, __ldcg(&p.part_ml[pr + s].x));
-                    float L = 0.f, O = 0.f;
-                    if (M != -INFINITY) {
-                        for (int s = 0; s < ns; ++s) {
-                            const float2 ml = __ldcg(&p.part_ml[pr + s]);
-                            const float f = (ml.x == -INFINITY) ? 0.f : fast_exp2(ml.x - M);
-                            L += ml.y * f;
-                            O += __ldcg(&p.part_o[(pr + s) * HEAD_DIM + c]) * f;
-                        }
+                    for (int s = lane; s < ns; s += 32) M = fmaxf(M, __ldcg(&p.part_ml[pr + s].x));
+#pragma unroll
+                    for (int sh = 16; sh >= 1; sh >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sh));
+                    float L = 0.f;
+                    for (int s = lane; s < ns; s += 32) {
+                        const float2 ml = __ldcg(&p.part_ml[pr + s]);
+                        const float f = (ml.x == -INFINITY || M == -INFINITY) ? 0.f : fast_exp2(ml.x - M);
+                        fsc[col * p.max_splits + s] = f;
+                        L += ml.y * f;
                     }
-                    p.out[(row0 + col) * HEAD_DIM + c] = (L > 0.f) ? O / L : 0.f;
+#pragma unroll
+                    for (int sh = 16; sh >= 1; sh >>= 1) L += __shfl_xor_sync(0xffffffffu, L, sh);
+                    if (lane == 0) linv[col] = (L > 0.f) ? 1.f / L : 0.f;
+                }
+                __syncthreads();
+                for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) {
+                    const int col = e >> 7, c = e & 127;
+                    const float* po = p.part_o + ((row0 + col) * p.max_splits) * HEAD_DIM + c;
+                    const float* fs = fsc + col * p.max_splits;
+                    float O = 0.f;
+                    int s = 0;
+                    for (; s + 8 <= ns; s += 8) {
+                        float v[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) v[u] = __ldcg(po + (long long)(s + u) * HEAD_DIM);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) O += v[u] * fs[s + u];
+                    }
+                    for (; s < ns; ++s) O += __ldcg(po + (long long)s * HEAD_DIM) * fs[s];
+                    p.out[(row0 + col) * HEAD_DIM + c] = O * linv[col];
                 }
                 if (threadIdx.x == 0) { *ctr = 0; if (pooled) *pool = 0; }   // ready for the next launch
             }

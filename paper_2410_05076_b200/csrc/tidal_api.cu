@@ -217,17 +217,31 @@ constexpr size_t attn_smem() {
 }
 
 template <int MODE, int NW, int STAGES>
-tidal_status_t launch_attn(tidal_ctx* ctx, const AttnParams& a, int grid, cudaStream_t st) {
-    attn_kernel<MODE, NW, STAGES><<<grid, NW * 32, attn_smem<MODE, NW, STAGES>(), st>>>(a);
+tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, cudaStream_t st) {
+    // Programmatic dependent launch: the kernel may begin while its predecessor in the stream
+    // drains; it waits (griddepcontrol.wait) before touching anything that predecessor wrote.
+    a.pdl = 1;
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(NW * 32, 1, 1);
+    cfg.dynamicSmemBytes = attn_smem<MODE, NW, STAGES>();
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     ctx->launches++;
-    return cudaGetLastError() == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, attn_kernel<MODE, NW, STAGES>, a) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }
 
 // hist != nullptr: the kernel also accumulates the per-head histogram the top-k needs.
 tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, float* out, float* scores,
-                         long long score_stride, bool fuse_hist, const WsLayout& w, cudaStream_t st) {
+                         long long score_stride, bool fuse_hist, bool wait_first, const WsLayout& w, cudaStream_t st) {
     AttnParams a;
     fill_common(a, ctx, kv, q, out, w);
+    a.wait_first = wait_first;
     const long long tiles = (long long)kv->batch * kv->num_kv_heads * ((kv->max_ctx_len + TILE - 1) / TILE);
     int grid = grid_for(tiles, ctx->dense_slots);
     if (const int S = (ctx->tune_dense == 5) ? 0 : pooled_splits(kv, kv->batch * kv->num_kv_heads, grid)) {
@@ -275,10 +289,11 @@ tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* score
 }
 
 tidal_status_t run_sparse(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, const int* idx,
-                          const int* idx_count, int k, int Hi, float* out, const WsLayout& w,
+                          const int* idx_count, int k, int Hi, float* out, bool wait_first, const WsLayout& w,
                           cudaStream_t st) {
     AttnParams a;
     fill_common(a, ctx, kv, q, out, w);
+    a.wait_first = wait_first;
     const int per_batch = (Hi == kv->num_q_heads) ? kv->num_q_heads : kv->num_kv_heads;
     const long long tiles = (long long)kv->batch * per_batch * ((k + TILE - 1) / TILE);
     int grid = grid_for(tiles, ctx->sparse_slots);
@@ -369,7 +384,7 @@ tidal_status_t tidal_full_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const voi
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
     const WsLayout w = layout_ws(kv, 1, 0);
     if ((rc = ensure_all(ctx, kv, w.total)) != TIDAL_OK) return rc;
-    return run_dense(ctx, kv, q, out, nullptr, 0, false, w, (cudaStream_t)stream);
+    return run_dense(ctx, kv, q, out, nullptr, 0, false, true, w, (cudaStream_t)stream);
 }
 
 tidal_status_t tidal_select_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const void* q, int32_t k,
@@ -388,7 +403,7 @@ tidal_status_t tidal_select_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const v
     const long long stride = scores_opt ? (long long)kv->max_ctx_len : w.score_stride;
     cudaStream_t st = (cudaStream_t)stream;
     const bool fuse = Hi == kv->num_q_heads;     // per-head ranking: the attention kernel builds the histogram
-    if ((rc = run_dense(ctx, kv, q, out, scores, stride, fuse, w, st)) != TIDAL_OK) return rc;
+    if ((rc = run_dense(ctx, kv, q, out, scores, stride, fuse, true, w, st)) != TIDAL_OK) return rc;
     return run_topk(ctx, kv, scores, stride, k, Hi, fuse, idx, idx_count, w, st);
 }
 
@@ -404,7 +419,7 @@ tidal_status_t tidal_sparse_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const v
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
     const WsLayout w = layout_ws(kv, k, 0);
     if ((rc = ensure_all(ctx, kv, w.total)) != TIDAL_OK) return rc;
-    return run_sparse(ctx, kv, q, idx, idx_count, k, Hi, out, w, (cudaStream_t)stream);
+    return run_sparse(ctx, kv, q, idx, idx_count, k, Hi, out, true, w, (cudaStream_t)stream);
 }
 
 static tidal_status_t decode_step_impl(tidal_ctx_t* ctx, int32_t num_layers, const uint8_t* schedule,
@@ -438,14 +453,15 @@ static tidal_status_t decode_step_impl(tidal_ctx_t* ctx, int32_t num_layers, con
         const tidal_kv_t* kv = &kvs[i];
         const WsLayout w = layout_ws(kv, k, host_layers);
         if (schedule[i] == TIDAL_LAYER_FULL) {
-            rc = run_dense(ctx, kv, qs[i], outs[i], nullptr, 0, false, w, st);
+            rc = run_dense(ctx, kv, qs[i], outs[i], nullptr, 0, false, i == 0, w, st);
         } else if (schedule[i] == TIDAL_LAYER_SELECT) {
             float* scores = (float*)((char*)ctx->ws + w.scores);
             const bool fuse = Hi == kv->num_q_heads;
-            rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, fuse, w, st);
+            rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, fuse, i == 0, w, st);
             if (rc == TIDAL_OK) rc = run_topk(ctx, kv, scores, w.score_stride, k, Hi, fuse, idx, idx_count, w, st);
         } else {
-            rc = run_sparse(ctx, kv, qs[i], idx, idx_count, k, Hi, outs[i], w, st);
+            // the index list is fresh when the previous layer selected it
+            rc = run_sparse(ctx, kv, qs[i], idx, idx_count, k, Hi, outs[i], i == 0 || schedule[i - 1] == TIDAL_LAYER_SELECT, w, st);
         }
         if (rc != TIDAL_OK) return rc;
     }
