@@ -404,47 +404,55 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             return cur++;
         };
 
-        // Sparse: the index entry this lane needs for the tile that will be issued next.
-        int pref_tile = next_tile();
-        int pref_pos = -1;
-        auto prefetch_idx = [&]() {
-            if (MODE == MODE_SPARSE) {
-                const int e = pref_tile * TILE + c16;
-                pref_pos = (pref_tile >= 0 && e < total) ? __ldg(idx_row + e) : -1;
+        // Tile queue with a lookahead of two: tA is issued next, tB after it. In the sparse mode the
+        // row offset of tA is already resolved (offA / validA, including the page lookup) and the index
+        // entry of tB is in flight (posB), so neither load ever delays a copy.
+        int tA = next_tile();
+        int tB = (tA >= 0) ? next_tile() : -1;
+        auto load_pos = [&](int tile) -> int {
+            if (MODE != MODE_SPARSE || tile < 0) return -1;
+            const int e = tile * TILE + c16;
+            return (e < total) ? __ldg(idx_row + e) : -1;
+        };
+        long long offA = 0;
+        bool validA = false;
+        auto resolve = [&](int pos) {
+            validA = pos >= 0 && pos < N;
+            if (pos >= N) atomicOr(p.status, STATUS_BAD_INDEX);
+            offA = 0;
+            if (validA) {
+                if (p.paged) {
+                    const int page = __ldg(p.page_table + (long long)b * p.max_pages + (pos >> 4));
+                    if ((unsigned)page < (unsigned)p.num_pages) {
+                        offA = (long long)page * p.stride_page + (long long)(pos & 15) * p.stride_pos + head_off;
+                    } else {
+                        validA = false;
+                        atomicOr(p.status, STATUS_BAD_PAGE);
+                    }
+                } else {
+                    offA = item_off + (long long)pos * p.stride_pos;
+                }
             }
         };
-        prefetch_idx();
-
-        // Everything above read only the index list, lengths and launch geometry; the query, the
-        // pool cursor and the scratch buffers belong to the kernels before us.
-        if (!waited) { pdl_wait(); pdl_trigger(); waited = true; }
-        if (pooled) grab();
-
-        // Q^T fragments: column gid is head head0+gid; this lane holds the 16-byte
-        // pieces 4j+tig (j = 0..3) of that head's query row.
-        uint32_t qf[4][4];
-        {
-            const uint4* qp = reinterpret_cast<const uint4*>(
-                p.q + ((long long)b * p.Hq + head0 + min(gid, ncols - 1)) * HEAD_DIM);
-            const bool on = gid < ncols;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint4 t = __ldg(qp + 4 * j + tig);
-                qf[j][0] = on ? t.x : 0u; qf[j][1] = on ? t.y : 0u; qf[j][2] = on ? t.z : 0u; qf[j][3] = on ? t.w : 0u;
-            }
+        int posB = -1;
+        if (MODE == MODE_SPARSE) {
+            const int posA = load_pos(tA);
+            posB = load_pos(tB);
+            resolve(posA);
         }
 
-        // Issue the copies of tile `pref_tile` into ring slot `stage`, then advance to the next tile.
+        // Issue the copies of tile tA into ring slot `stage`, then advance the queue.
         // Shared layout of a slot: K rows then V rows, 256 B per row, 16-byte piece c of
         // row r stored at piece c ^ ((r&1)<<2) for K and c ^ (r&7) for V so that the
         // fragment reads in consume_tile are bank-conflict free. Lane l copies piece
         // l&15 of rows (l>>4) + 2i, i = 0..7: one instruction moves two whole rows.
         auto issue = [&](int stage) {
-            const int tile = pref_tile;
+            const int tile = tA;
             const uint32_t ks = wbase_u32 + stage * STAGE_BYTES, vs = ks + TILE_BYTES;
             uint32_t vmask;
             if (MODE != MODE_SPARSE) {
-                pref_tile = next_tile();
+                tA = tB;
+                tB = (tA >= 0) ? next_tile() : -1;
                 const int pos0 = tile * TILE;
                 long long off;
                 bool ok = true;
@@ -476,25 +484,12 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                 }
                 if (lane == 0) { s_vmask[warp][stage] = vmask; s_posbase[warp][stage] = pos0; }
             } else {
-                const int pos = pref_pos;
-                pref_tile = next_tile();
-                prefetch_idx();
-                bool valid = pos >= 0 && pos < N;
-                if (pos >= N) atomicOr(p.status, STATUS_BAD_INDEX);
-                long long off = 0;
-                if (valid) {
-                    if (p.paged) {
-                        const int page = __ldg(p.page_table + (long long)b * p.max_pages + (pos >> 4));
-                        if ((unsigned)page < (unsigned)p.num_pages) {
-                            off = (long long)page * p.stride_page + (long long)(pos & 15) * p.stride_pos + head_off;
-                        } else {
-                            valid = false;
-                            atomicOr(p.status, STATUS_BAD_PAGE);
-                        }
-                    } else {
-                        off = item_off + (long long)pos * p.stride_pos;
-                    }
-                }
+                const long long off = offA;
+                const bool valid = validA;
+                tA = tB;
+                resolve(posB);                       // the page lookup of the next tile starts now
+                tB = (tA >= 0) ? next_tile() : -1;
+                posB = load_pos(tB);
                 vmask = __ballot_sync(0xffffffffu, valid) & 0xffffu;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
@@ -510,16 +505,48 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         };
 
         // ---- private cp.async ring -----------------------------------------------------------------------
-        int issued = 0;
+        // Until the grid dependency is resolved, only tiles that cannot hold the token appended for
+        // this layer may be fetched: every tile but the last one of the item (index lists produced by
+        // the selection kernel are ascending). The query, the pool cursor and the scratch buffers
+        // belong to the kernels before us and are touched only after the wait.
+        int issued = 0, commits = 0;
+        if (!waited) {
+            while (commits < STAGES - 1 && tA >= 0 && tA < tiles_b - 1) {
+                issue(issued % STAGES);
+                ++issued;
+                cp_async_commit();
+                ++commits;
+            }
+            pdl_wait();
+            pdl_trigger();
+            waited = true;
+        }
+        if (pooled) grab();
+
+        // Q^T fragments: column gid is head head0+gid; this lane holds the 16-byte
+        // pieces 4j+tig (j = 0..3) of that head's query row.
+        uint32_t qf[4][4];
+        {
+            const uint4* qp = reinterpret_cast<const uint4*>(
+                p.q + ((long long)b * p.Hq + head0 + min(gid, ncols - 1)) * HEAD_DIM);
+            const bool on = gid < ncols;
 #pragma unroll
-        for (int s = 0; s < STAGES - 1; ++s) {
-            if (pref_tile >= 0) { issue(s); ++issued; }
+            for (int j = 0; j < 4; ++j) {
+                const uint4 t = __ldg(qp + 4 * j + tig);
+                qf[j][0] = on ? t.x : 0u; qf[j][1] = on ? t.y : 0u; qf[j][2] = on ? t.z : 0u; qf[j][3] = on ? t.w : 0u;
+            }
+        }
+
+
+        while (commits < STAGES - 1) {
+            if (tA >= 0) { issue(issued % STAGES); ++issued; }
             cp_async_commit();
+            ++commits;
         }
         for (int it = 0; it < issued; ++it) {
             cp_async_wait<STAGES - 2>();      // tile `it` has landed (this lane's copies)
             __syncwarp();                     // ... and every other lane's; slot (it-1)%STAGES is free
-            if (pref_tile >= 0) { issue((it + STAGES - 1) % STAGES); ++issued; }
+            if (tA >= 0) { issue((it + STAGES - 1) % STAGES); ++issued; }
             cp_async_commit();
             const int stage = it % STAGES;
             const uint32_t ks = wbase_u32 + stage * STAGE_BYTES;
@@ -604,10 +631,10 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         if (nsplits == 1 && pooled && threadIdx.x == 0) *pool = 0;
         if (nsplits > 1) {
             // ---- the last CTA of this item to arrive combines the splits ---------------------------------
-            __threadfence();
             __syncthreads();
             int* ctr = p.counters + (long long)b * IY + y;
             if (threadIdx.x == 0) {
+                __threadfence();                  // cumulative: orders the whole CTA's partial stores
                 const int old = atomicAdd(ctr, 1);
                 s_is_last = (old == nsplits - 1);
             }
