@@ -42,7 +42,8 @@ constexpr int TILE_BYTES = TILE * HEAD_DIM * 2;   // 4 KB of K, same of V
 constexpr int STAGE_BYTES = 2 * TILE_BYTES;
 constexpr int HIST_BINS = 2048;          // global histogram row: up to 11 top bits of the score key
 constexpr int HIST_SMEM_WORDS = 8192;    // shared histogram: columns x bins <= 8192 counters (32 KB)
-constexpr int GRAB_TILES = 4;            // tiles a warp takes from its item's pool at a time
+constexpr int FIRST_TILES = 4;           // tiles of a warp's fixed first chunk (known before any pool access)
+constexpr int GRAB_TILES = 4;            // tiles a warp takes from its item's pool at a time afterwards
 
 struct AttnParams {
     const __nv_bfloat16* q;
@@ -375,17 +376,18 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         const long long item_off = (p.paged ? 0 : (long long)b * p.stride_b) + head_off;
 
         // ---- this warp's tile sequence -----------------------------------------------------------------
-        // static: t0 + warp, + NW, ... below t1.  pooled: GRAB_TILES consecutive tiles at a time from the
-        // item's cursor; the next grab is requested one chunk ahead so that its latency is hidden.
+        // static: t0 + warp, + NW, ... below t1.  pooled: a fixed first chunk, then GRAB_TILES consecutive
+        // tiles at a time from the item's cursor; the next grab is requested one chunk ahead so that its
+        // latency is hidden.
         int cur = t0 + warp, cur_end = t1;             // static walk
         int grab_raw = 0;                              // lane 0: value returned by the outstanding grab
         // The first chunk of every warp is fixed (no round trip before the first load); the pool
         // cursor hands out the tiles after those.
-        const int pool_base = p.splits_per_item * NW * GRAB_TILES;
+        const int pool_base = p.splits_per_item * NW * FIRST_TILES;
         auto grab = [&]() { if (lane == 0) grab_raw = pool_base + atomicAdd(pool, GRAB_TILES); };
         if (pooled) {
-            cur = ((int)(blockIdx.x / (p.batch * IY)) * NW + warp) * GRAB_TILES;
-            cur_end = min(tiles_b, cur + GRAB_TILES);
+            cur = ((int)(blockIdx.x / (p.batch * IY)) * NW + warp) * FIRST_TILES;
+            cur_end = min(tiles_b, cur + FIRST_TILES);
         }
         auto next_tile = [&]() -> int {                // -1 when this warp has no more tiles
             if (!pooled) {
@@ -642,10 +644,18 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             if (s_is_last) {
                 __threadfence();
                 const int ns = min(nsplits, p.max_splits);
-                // Scale factors of all splits first (shared memory), then every thread sums its
-                // output elements over the splits with the loads batched eight at a time.
-                float* fsc = reinterpret_cast<float*>(smem);              // [ncols][ns] exp2(m_s - M)
+                // Every thread first puts the loads of its output elements in flight (up to 16 splits
+                // at once), the warps meanwhile reduce the (max, sum) pairs to per-split scale factors
+                // in shared memory: one round trip to L2 instead of three.
+                float* fsc = reinterpret_cast<float*>(smem);              // [ncols][max_splits] exp2(m_s - M)
                 float* linv = fsc + 8 * p.max_splits;                    // [ncols] 1 / sum
+                constexpr int CB = 16;
+                const int e0 = threadIdx.x;                               // first (col, c) element of this thread
+                const bool has0 = e0 < ncols * HEAD_DIM;
+                const float* po0 = p.part_o + ((row0 + (e0 >> 7)) * p.max_splits) * HEAD_DIM + (e0 & 127);
+                float v0[CB];
+#pragma unroll
+                for (int u = 0; u < CB; ++u) v0[u] = (has0 && u < ns) ? __ldcg(po0 + (long long)u * HEAD_DIM) : 0.f;
                 for (int col = warp; col < ncols; col += NW) {
                     const long long pr = (row0 + col) * p.max_splits;
                     float M = -INFINITY;
@@ -670,6 +680,11 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                     const float* fs = fsc + col * p.max_splits;
                     float O = 0.f;
                     int s = 0;
+                    if (e == e0) {
+#pragma unroll
+                        for (int u = 0; u < CB; ++u) if (u < ns) O += v0[u] * fs[u];
+                        s = min(ns, CB);
+                    }
                     for (; s + 8 <= ns; s += 8) {
                         float v[8];
 #pragma unroll
