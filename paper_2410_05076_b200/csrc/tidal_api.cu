@@ -53,8 +53,8 @@ struct tidal_ctx {
 namespace {
 
 struct WsLayout {
-    size_t part_ml, part_o, scores, cand, idx, idx_count, q_stage, out_stage, total;
-    long long cand_stride;
+    size_t part_ml, part_o, scores, cand, bitmap, idx, idx_count, q_stage, out_stage, total;
+    long long cand_stride, bitmap_stride;
     long long score_stride;
     int max_splits;
 };
@@ -135,6 +135,8 @@ WsLayout layout_ws(const tidal_kv_t* kv, int k, int num_layers_host) {
     w.scores = at;    at += align_up(rows * (size_t)w.score_stride * sizeof(float), 256);
     w.cand_stride = w.score_stride;
     w.cand = at;      at += align_up(rows * (size_t)w.cand_stride * sizeof(uint2), 256);
+    w.bitmap_stride = (long long)align_up((size_t)kv->max_ctx_len, TK_SLICE) / 32;
+    w.bitmap = at;    at += align_up(rows * (size_t)w.bitmap_stride * sizeof(unsigned), 256);
     w.idx = at;       at += align_up(rows * (size_t)std::max(k, 1) * sizeof(int), 256);
     w.idx_count = at; at += align_up((size_t)kv->batch * sizeof(int), 256);
     w.q_stage = at;   at += align_up((size_t)num_layers_host * rows * HEAD_DIM * 2, 256);
@@ -273,12 +275,14 @@ tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* score
     t.done = state_done(ctx);
     t.cand = (uint2*)(ws + w.cand);
     t.cand_stride = w.cand_stride;
+    t.bitmap = (unsigned*)(ws + w.bitmap);
+    t.bitmap_stride = w.bitmap_stride;
     const int items = kv->batch * Hi;
     if (items > 65535) return TIDAL_ERR_UNSUPPORTED;
     const int parts = (kv->max_ctx_len + TK_SLICE - 1) / TK_SLICE;
     t.shift = hist_shift_for(kv);
     t.vec_ok = (((uintptr_t)scores & 15) == 0 && (score_stride & 3) == 0) ? 1 : 0;
-    t.cand_smem = std::min(16384, std::max(4096, (int)align_up((size_t)k + 4096, 1024)));
+    t.cand_smem = 8192;          // one histogram bin's population; larger lists are read from global memory
     const size_t words = (size_t)(kv->max_ctx_len + 31) / 32;
     const size_t smem = 2 * words * sizeof(unsigned) + (size_t)t.cand_smem * sizeof(uint2);
     dim3 grid(parts, items, 1);
@@ -336,7 +340,7 @@ tidal_status_t tidal_create(tidal_ctx_t** out, int device, size_t workspace_byte
     const int d0 = resident_ctas(attn_kernel<MODE_FULL, DENSE_NW, DENSE_STAGES>, DENSE_NW * 32, attn_smem<MODE_FULL, DENSE_NW, DENSE_STAGES>(), ctx->sm_count);
     const int d1 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW, DENSE_STAGES>, DENSE_NW * 32, attn_smem<MODE_SELECT, DENSE_NW, DENSE_STAGES>(), ctx->sm_count);
     const int s0 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>, SPARSE_NW * 32, attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(), ctx->sm_count);
-    const size_t topk_smem = 2 * (size_t)(MAX_CTX / 32) * sizeof(unsigned) + 16384 * sizeof(uint2);
+    const size_t topk_smem = 2 * (size_t)(MAX_CTX / 32) * sizeof(unsigned) + 8192 * sizeof(uint2);
     const bool topk_ok = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topk_smem) == cudaSuccess;
     if (d0 <= 0 || d1 <= 0 || s0 <= 0 || !topk_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
     ctx->dense_slots = std::min(d0, d1);

@@ -4,15 +4,17 @@
 //
 // Scores become order-preserving 32-bit keys. The exact k'-th largest key is
 // found by a most-significant-digit radix select (11 + 11 + 10 bits, or 10 + 11 + 11):
-//   1. topk_hist_kernel: all SMs histogram the top 11 key bits of every score
-//      (shared-memory histograms, flushed to a global one per index head).
-//   2. topk_select_kernel, all SMs: every CTA derives the threshold bin from the
-//      global histogram and appends the few scores at or above that bin —
-//      about k' plus the population of one bin — to a candidate list.
-//      The last CTA of an index head to finish then resolves the remaining 21
-//      bits on the candidate list alone (in shared memory), marks the winners
-//      in a position bitmap, taking only as many keys equal to the threshold as
-//      are still needed, lowest positions first, and enumerates the bitmap in
+//   1. The histogram of the first digit comes from the selection layer's attention
+//      kernel (fused, per query head) or from topk_hist_kernel (summed scores of a
+//      head group).
+//   2. topk_select_kernel, all SMs: every CTA derives the threshold bin from that
+//      histogram; positions in higher bins are winners outright and go straight
+//      into a position bitmap (each CTA owns whole words of it), positions in the
+//      threshold bin itself — one bin's population — are appended to a
+//      candidate list. The last CTA of an index head to finish resolves the
+//      remaining 21 bits on the candidate list alone (in shared memory), adds the
+//      candidates above the final threshold and as many equal to it as are still
+//      needed (lowest positions first) to the bitmap, and enumerates the bitmap in
 //      order. The result is the unique set that a full sort by (score desc,
 //      position asc) gives.
 // No CTA ever waits for another one; the per-head histogram, cursor and
@@ -25,9 +27,10 @@
 namespace tidal {
 
 constexpr int TK_THREADS = 512;
-constexpr int TK_BINS = 2048;          // top 11 bits of the key
+constexpr int TK_BINS = 2048;          // first digit: up to 11 top bits of the key
 constexpr int TK_VEC = 4;              // float4 loads per thread per slice
-constexpr int TK_SLICE = TK_THREADS * TK_VEC * 4;   // positions per CTA
+constexpr int TK_SLICE = TK_THREADS * TK_VEC * 4;   // positions per CTA (8192)
+constexpr int TK_KEYS = TK_VEC * 4;    // keys per thread
 
 struct TopkParams {
     const float* scores;       // [B, Hq, score_stride]
@@ -41,8 +44,10 @@ struct TopkParams {
     unsigned* hist;            // [items, TK_BINS], zero between calls
     int* cursor;               // [items], zero between calls
     int* done;                 // [items], zero between calls
-    uint2* cand;               // [items, cand_stride] (key, position)
+    uint2* cand;               // [items, cand_stride] (key, position) of the threshold bin
     long long cand_stride;
+    unsigned* bitmap;          // [items, bitmap_stride] winners above the threshold bin, one bit per position
+    long long bitmap_stride;   // words per item (covers max_ctx rounded up to a whole slice)
     int cand_smem;             // candidates the last CTA can hold in shared memory
     int vec_ok;                // score rows are 16-byte aligned: float4 loads allowed
     int shift;                 // first digit = key >> shift (21 or 22); the rest is split 11 + (shift-11) bits
@@ -55,12 +60,12 @@ __device__ __forceinline__ uint32_t score_key(float s) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Keys of this thread's 16 positions of the slice starting at s0: four groups of four
+// Keys of this thread's positions of the slice starting at s0: TK_VEC groups of four
 // consecutive positions, group j at s0 + 4*(j*TK_THREADS + tid). All loads are issued
 // before any is used. Positions at or beyond n get key 0 and valid bit 0.
 __device__ __forceinline__ unsigned load_slice_keys(const TopkParams& p, const float* srow, int members,
-                                                    int s0, int n, uint32_t (&key)[TK_VEC * 4]) {
-    float v[TK_VEC * 4];
+                                                    int s0, int n, uint32_t (&key)[TK_KEYS]) {
+    float v[TK_KEYS];
 #pragma unroll
     for (int j = 0; j < TK_VEC; ++j) {
         const int pos = s0 + 4 * (j * TK_THREADS + (int)threadIdx.x);
@@ -96,21 +101,22 @@ __device__ __forceinline__ unsigned load_slice_keys(const TopkParams& p, const f
     return valid;
 }
 
-// Inclusive scan of one int per thread over a TK_THREADS block.
-__device__ __forceinline__ int block_scan_incl(int v, int* warp_sums, int& total) {
+// Inclusive scan of one value per thread over a TK_THREADS block.
+template <typename T>
+__device__ __forceinline__ T block_scan_incl(T v, T* warp_sums, T& total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, v, d);
+        const T t = __shfl_up_sync(0xffffffffu, v, d);
         if (lane >= d) v += t;
     }
     __syncthreads();                       // warp_sums may still be read from a previous call
     if (lane == 31) warp_sums[warp] = v;
     __syncthreads();
-    int before = 0, all = 0;
+    T before = 0, all = 0;
 #pragma unroll
     for (int w = 0; w < TK_THREADS / 32; ++w) {
-        const int s = warp_sums[w];
+        const T s = warp_sums[w];
         if (w < warp) before += s;
         all += s;
     }
@@ -131,7 +137,7 @@ __device__ __forceinline__ int pick_digit(const unsigned* hist, int nbins, int* 
         if (bin >= 0) mine += (int)hist[bin];
     }
     int total;
-    const int incl = block_scan_incl(mine, warp_sums, total);
+    const int incl = block_scan_incl<int>(mine, warp_sums, total);
     const int excl = incl - mine;
     if (excl < need && need <= incl) {
         int above = excl;
@@ -149,6 +155,8 @@ __device__ __forceinline__ int pick_digit(const unsigned* hist, int nbins, int* 
     return digit;
 }
 
+// Histogram of the first digit for rankings that sum several heads' scores (the attention
+// kernel cannot build those: the member heads live in different CTAs).
 __global__ void __launch_bounds__(TK_THREADS) topk_hist_kernel(const TopkParams p) {
     __shared__ unsigned sh[TK_BINS];
     const int item = blockIdx.y, b = item / p.Hi, hi = item % p.Hi, tid = threadIdx.x;
@@ -159,11 +167,11 @@ __global__ void __launch_bounds__(TK_THREADS) topk_hist_kernel(const TopkParams 
     for (int i = tid; i < TK_BINS; i += TK_THREADS) sh[i] = 0;
     const int members = p.Hq / p.Hi;
     const float* srow = p.scores + ((long long)b * p.Hq + (long long)hi * members) * p.score_stride;
-    uint32_t key[TK_VEC * 4];
+    uint32_t key[TK_KEYS];
     const unsigned valid = load_slice_keys(p, srow, members, s0, N, key);
     __syncthreads();
 #pragma unroll
-    for (int e = 0; e < TK_VEC * 4; ++e)
+    for (int e = 0; e < TK_KEYS; ++e)
         if ((valid >> e) & 1u) atomicAdd(&sh[key[e] >> p.shift], 1u);
     __syncthreads();
     unsigned* gh = p.hist + (long long)item * TK_BINS;
@@ -178,23 +186,25 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     __shared__ __align__(16) unsigned sh_hist[TK_BINS];
     static_assert(TK_BINS == 4 * TK_THREADS, "one uint4 of the histogram per thread");
     __shared__ int warp_sums[TK_THREADS / 32];
+    __shared__ unsigned long long warp_sums64[TK_THREADS / 32];
     __shared__ int bcast[2];
     __shared__ int s_last;
 
     const int item = blockIdx.y, b = item / p.Hi, hi = item % p.Hi, tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5;
     const int N = max(0, min(p.ctx_lens[b], p.max_ctx));
     const int kk = min(p.k, N);
     int* out = p.idx + (long long)item * p.k;
     const int s0 = blockIdx.x * TK_SLICE, s1 = min(N, s0 + TK_SLICE);
     if (blockIdx.x == 0 && hi == 0 && tid == 0 && p.idx_count) p.idx_count[b] = kk;
+    unsigned* gh = p.hist + (long long)item * TK_BINS;
 
     if (kk == N) {                                     // identity list, then padding
         for (int i = s0 + tid; i < s1; i += TK_THREADS) out[i] = i;
         if (blockIdx.x == 0) {
             for (int i = N + tid; i < p.k; i += TK_THREADS) out[i] = -1;
             // a selection layer's attention kernel may have filled the histogram regardless of k
-            unsigned* gh0 = p.hist + (long long)item * TK_BINS;
-            for (int i = tid; i < TK_BINS; i += TK_THREADS) gh0[i] = 0;
+            for (int i = tid; i < TK_BINS; i += TK_THREADS) gh[i] = 0;
         }
         return;
     }
@@ -204,66 +214,92 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     // ---- this CTA's keys (all loads in flight at once), then the threshold bin ------------------
     const int members = p.Hq / p.Hi;
     const float* srow = p.scores + ((long long)b * p.Hq + (long long)hi * members) * p.score_stride;
-    uint32_t key[TK_VEC * 4];
+    uint32_t key[TK_KEYS];
     const unsigned valid = load_slice_keys(p, srow, members, s0, N, key);
-    unsigned* gh = p.hist + (long long)item * TK_BINS;
     {
-        const uint4 h4 = __ldcg(reinterpret_cast<const uint4*>(gh) + tid);     // TK_BINS == 4 * TK_THREADS
+        const uint4 h4 = __ldcg(reinterpret_cast<const uint4*>(gh) + tid);
         reinterpret_cast<uint4*>(sh_hist)[tid] = h4;
     }
     __syncthreads();
     int need = kk;
     const int b1 = pick_digit(sh_hist, TK_BINS, warp_sums, bcast, need);
+    // `need` of the keys in bin b1 are still to be taken; every key in a higher bin is a winner.
 
-    // ---- append every score at or above that bin to the candidate list: one cursor bump per CTA ----
-    unsigned take = 0;
+    // ---- winners above the threshold bin: straight into the position bitmap ------------------------
+    // Group j of a warp covers 128 consecutive positions, lane l the four at 4l: the 8 lanes of a
+    // word OR their nibbles together and one of them stores the word (zeros included, so the
+    // bitmap needs no clearing).
+    unsigned* bm = p.bitmap + (long long)item * p.bitmap_stride;
+    unsigned eq_mask = 0;
 #pragma unroll
-    for (int e = 0; e < TK_VEC * 4; ++e)
-        if (((valid >> e) & 1u) && (int)(key[e] >> p.shift) >= b1) take |= 1u << e;
+    for (int j = 0; j < TK_VEC; ++j) {
+        unsigned nib = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int i = 4 * j + e;
+            const int bin = (int)(key[i] >> p.shift);
+            const bool ok = (valid >> i) & 1u;
+            if (ok && bin > b1) nib |= 1u << e;
+            if (ok && bin == b1) eq_mask |= 1u << i;
+        }
+        unsigned word = nib << (4 * (lane & 7));
+        word |= __shfl_xor_sync(0xffffffffu, word, 1);
+        word |= __shfl_xor_sync(0xffffffffu, word, 2);
+        word |= __shfl_xor_sync(0xffffffffu, word, 4);
+        if ((lane & 7) == 0) bm[(s0 >> 5) + j * (TK_THREADS / 8) + warp * 4 + (lane >> 3)] = word;
+    }
+
+    // ---- the threshold bin's own keys: append to the candidate list, one cursor bump per CTA -------
     int cta_total;
-    const int mine = __popc(take);
-    int slot = block_scan_incl(mine, warp_sums, cta_total) - mine;
+    const int mine = __popc(eq_mask);
+    int slot = block_scan_incl<int>(mine, warp_sums, cta_total) - mine;
     if (tid == 0) bcast[0] = cta_total ? atomicAdd(&p.cursor[item], cta_total) : 0;
     __syncthreads();
     slot += bcast[0];
     uint2* cand = p.cand + (long long)item * p.cand_stride;
 #pragma unroll
-    for (int e = 0; e < TK_VEC * 4; ++e)
-        if ((take >> e) & 1u) {
+    for (int e = 0; e < TK_KEYS; ++e)
+        if ((eq_mask >> e) & 1u) {
             const int pos = s0 + 4 * ((e >> 2) * TK_THREADS + tid) + (e & 3);
             if (slot < p.cand_stride) cand[slot] = make_uint2(key[e], (unsigned)pos);
             ++slot;
         }
 
     // ---- the last CTA of this index head resolves the rest ------------------------------------------
-    __threadfence();
     __syncthreads();
-    if (tid == 0) s_last = (atomicAdd(&p.done[item], 1) == nparts - 1);
+    if (tid == 0) {
+        __threadfence();                               // cumulative: orders the CTA's bitmap and candidate stores
+        s_last = (atomicAdd(&p.done[item], 1) == nparts - 1);
+    }
     __syncthreads();
     if (!s_last) return;
     __threadfence();
 
-    const int M = min((long long)__ldcg(&p.cursor[item]), p.cand_stride);
+    const int M = (int)min((long long)__ldcg(&p.cursor[item]), p.cand_stride);
     const int words = (N + 31) >> 5;
-    unsigned* sel = reinterpret_cast<unsigned*>(tk_smem);          // [words] keys above the threshold
-    unsigned* eqm = sel + words;                                    // [words] keys equal to it
-    uint2* scand = reinterpret_cast<uint2*>(eqm + words);          // [cand_smem]; 8*words bytes in: 8-byte aligned
+    unsigned* cgt = reinterpret_cast<unsigned*>(tk_smem);          // [words] candidates above the final threshold
+    unsigned* ceq = cgt + words;                                    // [words] candidates equal to it
+    uint2* scand = reinterpret_cast<uint2*>(ceq + words);          // [cand_smem]; 8*words bytes in: 8-byte aligned
     const uint2* c = cand;
     if (M <= p.cand_smem) {
 #pragma unroll 4
         for (int i = tid; i < M; i += TK_THREADS) scand[i] = __ldcg(&cand[i]);
         c = scand;
     }
-    for (int i = tid; i < words; i += TK_THREADS) { sel[i] = 0; eqm[i] = 0; }
+    // this thread's bitmap words for the enumeration: loads in flight while the digits are resolved
+    constexpr int WB = 8;
+    const int per = (words + TK_THREADS - 1) / TK_THREADS;
+    const int w0 = min(words, tid * per), w1 = min(words, w0 + per);
+    unsigned bw[WB];
+#pragma unroll
+    for (int u = 0; u < WB; ++u) bw[u] = (w0 + u < w1) ? __ldcg(&bm[w0 + u]) : 0u;
+    for (int i = tid; i < words; i += TK_THREADS) { cgt[i] = 0; ceq[i] = 0; }
     for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
     __syncthreads();
 
-    // second digit: the next 11 key bits among keys whose first digit equals b1
+    // second digit: the next 11 key bits (every candidate already has first digit b1)
     const int s2 = p.shift - 11;                       // bits left for the third digit (10 or 11)
-    for (int i = tid; i < M; i += TK_THREADS) {
-        const uint32_t key = c[i].x;
-        if ((int)(key >> p.shift) == b1) atomicAdd(&sh_hist[(key >> s2) & 0x7ffu], 1u);
-    }
+    for (int i = tid; i < M; i += TK_THREADS) atomicAdd(&sh_hist[(c[i].x >> s2) & 0x7ffu], 1u);
     __syncthreads();
     const int d2 = pick_digit(sh_hist, TK_BINS, warp_sums, bcast, need);
     const uint32_t prefix2 = ((uint32_t)b1 << p.shift) | ((uint32_t)d2 << s2);
@@ -272,45 +308,52 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
     __syncthreads();
     for (int i = tid; i < M; i += TK_THREADS) {
-        const uint32_t key = c[i].x;
-        if ((key >> s2) == (prefix2 >> s2)) atomicAdd(&sh_hist[key & ((1u << s2) - 1u)], 1u);
+        const uint32_t k32 = c[i].x;
+        if ((k32 >> s2) == (prefix2 >> s2)) atomicAdd(&sh_hist[k32 & ((1u << s2) - 1u)], 1u);
     }
     __syncthreads();
     const int d3 = pick_digit(sh_hist, 1 << s2, warp_sums, bcast, need);
     const uint32_t thr = prefix2 | (uint32_t)d3;       // the k'-th largest key; `need` keys equal to it are taken
 
-    // bitmaps of positions above / equal to the threshold
+    // candidates above / equal to the threshold, as position bitmaps
     for (int i = tid; i < M; i += TK_THREADS) {
         const uint2 e = c[i];
-        if (e.x > thr) atomicOr(&sel[e.y >> 5], 1u << (e.y & 31));
-        else if (e.x == thr) atomicOr(&eqm[e.y >> 5], 1u << (e.y & 31));
+        if (e.x > thr) atomicOr(&cgt[e.y >> 5], 1u << (e.y & 31));
+        else if (e.x == thr) atomicOr(&ceq[e.y >> 5], 1u << (e.y & 31));
     }
     __syncthreads();
 
-    // ordered enumeration
-    const int per = (words + TK_THREADS - 1) / TK_THREADS;
-    const int w0 = min(words, tid * per), w1 = min(words, w0 + per);
-    int ngt = 0, neq = 0;
-    for (int w = w0; w < w1; ++w) { ngt += __popc(sel[w]); neq += __popc(eqm[w]); }
-    int tot_gt, tot_eq;
-    const int gt_excl = block_scan_incl(ngt, warp_sums, tot_gt) - ngt;
-    const int eq_excl = block_scan_incl(neq, warp_sums, tot_eq) - neq;
-    int eq_seen = eq_excl;
-    int at = gt_excl + min(eq_seen, need);
-    for (int w = w0; w < w1; ++w) {
-        unsigned e = eqm[w];
+    // ordered enumeration: (winner count, equal count) scanned together in one 64-bit value
+    unsigned long long cnt = 0;
+    auto count_word = [&](int w, unsigned base) {
+        cnt += ((unsigned long long)__popc(base | cgt[w]) << 32) | (unsigned long long)__popc(ceq[w]);
+    };
+#pragma unroll
+    for (int u = 0; u < WB; ++u)
+        if (w0 + u < w1) count_word(w0 + u, bw[u]);
+    for (int w = w0 + WB; w < w1; ++w) count_word(w, __ldcg(&bm[w]));
+    unsigned long long tot;
+    const unsigned long long excl = block_scan_incl<unsigned long long>(cnt, warp_sums64, tot) - cnt;
+    int eq_seen = (int)(excl & 0xffffffffu);
+    int at = (int)(excl >> 32) + min(eq_seen, need);
+    auto emit_word = [&](int w, unsigned base) {
+        unsigned e = ceq[w];
         const int ne = __popc(e);
-        int keep = min(max(need - eq_seen, 0), ne);    // lowest `keep` equal-key positions of this word
+        const int keep = min(max(need - eq_seen, 0), ne);   // lowest `keep` equal-key positions of this word
         eq_seen += ne;
         while (__popc(e) > keep) e &= ~(0x80000000u >> __clz(e));
-        unsigned bits = sel[w] | e;
+        unsigned bits = base | cgt[w] | e;
         while (bits) {
             const int pbit = __ffs(bits) - 1;
             if (at < p.k) out[at] = (w << 5) + pbit;
             ++at;
             bits &= bits - 1;
         }
-    }
+    };
+#pragma unroll
+    for (int u = 0; u < WB; ++u)
+        if (w0 + u < w1) emit_word(w0 + u, bw[u]);
+    for (int w = w0 + WB; w < w1; ++w) emit_word(w, __ldcg(&bm[w]));
     for (int i = kk + tid; i < p.k; i += TK_THREADS) out[i] = -1;
 
     // leave the shared state clean for the next call
