@@ -48,7 +48,8 @@ enum {
     TIDAL_ERR_NOMEM = -3,         /* workspace allocation failed */
     TIDAL_ERR_CUDA = -4,          /* a CUDA runtime call failed */
     TIDAL_ERR_TIMEOUT = -5,       /* reserved: a bounded device-side wait expired */
-    TIDAL_ERR_INDEX = -6          /* device saw a token index or page id out of range */
+    TIDAL_ERR_INDEX = -6,         /* device saw a token index or page id out of range */
+    TIDAL_ERR_TOO_LARGE = -7      /* tidal_sparse_attn_noalloc only: problem exceeds its fixed scratch */
 };
 
 enum { TIDAL_KV_CONTIG = 0, TIDAL_KV_PAGED = 1 };
@@ -145,6 +146,31 @@ tidal_status_t tidal_decode_step(tidal_ctx_t *ctx, int32_t num_layers, const uin
 tidal_status_t tidal_decode_step_host(tidal_ctx_t *ctx, int32_t num_layers, const uint8_t *schedule,
                                       const tidal_kv_t *kv_per_layer, const void *q_host,
                                       float *out_host, int32_t k, int32_t granularity, void *stream);
+
+/* tidal_sparse_attn for callers that are not allowed to allocate device memory. (The paper has
+ * no counterpart to this call; it exists for integration, not for the method.) Such callers are,
+ * for example, a serving process that handed all device memory to its own pool at start-up, so
+ * that a later cudaMalloc fails or is forbidden by policy; code running inside a latency-critical
+ * loop where the implicit synchronisation of cudaMalloc/cudaFree is unacceptable; or a plug-in
+ * that is called with the device already in a state where allocation is not permitted. The other
+ * entry points need a context whose workspace is allocated (and may grow) behind the caller's back.
+ *
+ * This one takes no context and never calls cudaMalloc, cudaFree or any allocating routine: its
+ * scratch (split partial results, arrival counters, pool cursors) is one static device array of
+ * about 2.07 MiB (4096 partial rows) that every GPU loading the library holds until the process
+ * exits. It runs on the CURRENT device. Arguments and results are those of tidal_sparse_attn,
+ * with these differences:
+ *   - batch * num_q_heads must not exceed 4096, otherwise TIDAL_ERR_TOO_LARGE (nothing enqueued);
+ *   - an index entry >= ctx_lens[b] or a page id outside the pool is skipped but cannot be
+ *     reported (there is no context to hold the status word);
+ *   - all calls on a device share the one scratch array: two calls whose kernels can overlap on
+ *     the GPU (different streams, no dependency) race; keep them on one stream or order them;
+ *   - the first call on each device also does the one-time set-up (it resolves the array's device
+ *     address and prepares the kernel, still without allocating): that first call should come
+ *     before any stream capture. */
+tidal_status_t tidal_sparse_attn_noalloc(const tidal_kv_t *kv, const void *q, const int32_t *idx,
+                                         const int32_t *idx_count, int32_t k, int32_t num_index_heads,
+                                         float *out, void *stream);
 
 /* Waits for `stream`, then returns and clears the sticky device status word:
  * TIDAL_OK, TIDAL_ERR_INDEX, or TIDAL_ERR_CUDA if the stream reports an error. */

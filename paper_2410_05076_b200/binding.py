@@ -17,6 +17,7 @@ from . import build as _build
 
 OK = 0
 ERR_INVALID, ERR_UNSUPPORTED, ERR_NOMEM, ERR_CUDA, ERR_TIMEOUT, ERR_INDEX = -1, -2, -3, -4, -5, -6
+ERR_TOO_LARGE = -7
 KV_CONTIG, KV_PAGED = 0, 1
 SEL_PER_QHEAD, SEL_PER_KVHEAD, SEL_SHARED = 0, 1, 2
 LAYER_FULL, LAYER_SELECT, LAYER_SPARSE = 0, 1, 2
@@ -24,7 +25,7 @@ LAYER_FULL, LAYER_SELECT, LAYER_SPARSE = 0, 1, 2
 EXPORTS = [
     "tidal_create", "tidal_destroy", "tidal_workspace_bytes", "tidal_full_attn", "tidal_select_attn",
     "tidal_sparse_attn", "tidal_decode_step", "tidal_decode_step_host", "tidal_device_status",
-    "tidal_launch_count", "tidal_strerror",
+    "tidal_launch_count", "tidal_strerror", "tidal_sparse_attn_noalloc",
 ]
 
 
@@ -77,6 +78,8 @@ def load() -> C.CDLL:
     L.tidal_select_attn.restype = I32
     L.tidal_sparse_attn.argtypes = [P, KVP, P, P, P, I32, I32, P, P]
     L.tidal_sparse_attn.restype = I32
+    L.tidal_sparse_attn_noalloc.argtypes = [KVP, P, P, P, I32, I32, P, P]
+    L.tidal_sparse_attn_noalloc.restype = I32
     L.tidal_decode_step.argtypes = [P, I32, P, KVP, C.POINTER(P), C.POINTER(P), I32, I32, P, P, P]
     L.tidal_decode_step.restype = I32
     L.tidal_decode_step_host.argtypes = [P, I32, P, KVP, P, P, I32, I32, P]
@@ -123,6 +126,22 @@ def _stream() -> int:
 def _check(status: int, what: str) -> None:
     if status != OK:
         raise TidalError(status, what)
+
+
+def sparse_attn_noalloc(layer, q: torch.Tensor, idx: torch.Tensor, idx_count: Optional[torch.Tensor] = None,
+                        out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """tidal_sparse_attn_noalloc on the current device and stream: sparse attention for callers that
+    may not allocate device memory. No context is involved; the library's fixed static scratch is
+    used, so batch * num_q_heads is limited to 4096 and overlapping calls on one GPU race. `out`
+    should be passed by such callers (this wrapper allocates it with torch only as a convenience)."""
+    if out is None:
+        out = torch.empty(layer.batch, layer.num_q_heads, layer.head_dim, dtype=torch.float32, device=q.device)
+    s = kv_struct(layer)
+    _, hi, k = idx.shape
+    _check(load().tidal_sparse_attn_noalloc(C.byref(s), q.data_ptr(), idx.data_ptr(),
+                                            idx_count.data_ptr() if idx_count is not None else None, k, hi,
+                                            out.data_ptr(), _stream()), "tidal_sparse_attn_noalloc")
+    return out
 
 
 class Tidal:

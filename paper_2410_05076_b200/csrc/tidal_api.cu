@@ -10,6 +10,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "attn_kernels.cuh"
@@ -547,8 +548,128 @@ const char* tidal_strerror(tidal_status_t s) {
         case TIDAL_ERR_CUDA: return "CUDA runtime error";
         case TIDAL_ERR_TIMEOUT: return "device-side wait timed out";
         case TIDAL_ERR_INDEX: return "token index or page id out of range";
+        case TIDAL_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of the allocation-free entry point";
         default: return "unknown status";
     }
 }
 
 }  // extern "C"
+
+// =====================================================================================================
+// Sparse attention for callers that must not allocate.
+//
+// Everything the kernel needs beyond the caller's inputs and outputs (the split partial results,
+// the arrival counters, the pool cursors and a status word) lives in one file-scope device array
+// of fixed size, so this entry point never calls cudaMalloc, cudaFree or anything that allocates.
+// =====================================================================================================
+namespace {
+
+constexpr int NOALLOC_MAX_ROWS = 4096;      // (sequence, query head) rows; also the number of partial slots
+constexpr size_t NOALLOC_PART_O = (size_t)NOALLOC_MAX_ROWS * HEAD_DIM * sizeof(float);   // 2 MiB
+constexpr size_t NOALLOC_PART_ML = (size_t)NOALLOC_MAX_ROWS * sizeof(float2);           // 32 KiB
+constexpr size_t NOALLOC_WORDS = 2 * (size_t)NOALLOC_MAX_ROWS * sizeof(int) + 256;      // counters, cursors, status
+constexpr size_t NOALLOC_BYTES = NOALLOC_PART_O + NOALLOC_PART_ML + NOALLOC_WORDS;      // about 2.07 MiB
+
+// Held by every GPU that loads the library until the process exits. In host code this name is
+// only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_BYTES];
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+struct NoallocDevice {
+    bool ready = false;
+    unsigned char* scratch = nullptr;       // device address of g_noalloc_scratch on this GPU
+    int slots = 0;                          // resident CTAs of the sparse kernel on this GPU
+};
+NoallocDevice g_noalloc_dev[NOALLOC_MAX_DEVICES];
+std::mutex g_noalloc_mutex;
+
+// Once per device, with that device current: resolve the scratch array's device address and
+// prepare the kernel (shared-memory opt-in, occupancy). Allocates nothing.
+tidal_status_t noalloc_setup(int device, const NoallocDevice** out) {
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    NoallocDevice& d = g_noalloc_dev[device];
+    if (!d.ready) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) {
+            cudaGetLastError();
+            return TIDAL_ERR_CUDA;
+        }
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return TIDAL_ERR_CUDA;
+        const int slots = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>, SPARSE_NW * 32,
+                                        attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(), sms);
+        if (slots <= 0) { cudaGetLastError(); return TIDAL_ERR_CUDA; }
+        d.scratch = static_cast<unsigned char*>(ptr);
+        d.slots = slots;
+        d.ready = true;
+    }
+    *out = &d;
+    return TIDAL_OK;
+}
+
+}  // namespace
+
+extern "C" tidal_status_t tidal_sparse_attn_noalloc(const tidal_kv_t* kv, const void* q, const int32_t* idx,
+                                                    const int32_t* idx_count, int32_t k,
+                                                    int32_t num_index_heads, float* out, void* stream) {
+    if (!q || !out || !idx || ((uintptr_t)q & 15)) return TIDAL_ERR_INVALID;
+    tidal_status_t rc = check_kv(kv);
+    if (rc != TIDAL_OK) return rc;
+    if (k <= 0) return TIDAL_ERR_INVALID;
+    const int Hi = num_index_heads;
+    if (Hi != kv->num_q_heads && Hi != kv->num_kv_heads && Hi != 1) return TIDAL_ERR_INVALID;
+    const long long rows = (long long)kv->batch * kv->num_q_heads;
+    if (rows > NOALLOC_MAX_ROWS) return TIDAL_ERR_TOO_LARGE;
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return TIDAL_ERR_CUDA; }
+    if (device < 0 || device >= NOALLOC_MAX_DEVICES) return TIDAL_ERR_UNSUPPORTED;
+    const NoallocDevice* dev = nullptr;
+    if ((rc = noalloc_setup(device, &dev)) != TIDAL_OK) return rc;
+
+    // Every item (one query head, or one KV head's group) is shared by S CTAs through its pool
+    // cursor; a row then needs S partial slots and the scratch holds NOALLOC_MAX_ROWS of them.
+    const int per_batch = (Hi == kv->num_q_heads) ? kv->num_q_heads : kv->num_kv_heads;
+    const int items = kv->batch * per_batch;
+    const int tiles_item = (k + TILE - 1) / TILE;
+    int S = std::max(1, std::min(dev->slots, GRID_MAX) / items);
+    S = std::min(S, std::max(1, tiles_item / MIN_TILES_PER_CTA));
+    while (S > 1 && rows * S > NOALLOC_MAX_ROWS) --S;
+
+    unsigned char* base = dev->scratch;
+    int* words = reinterpret_cast<int*>(base + NOALLOC_PART_O + NOALLOC_PART_ML);
+    AttnParams a;
+    std::memset(&a, 0, sizeof a);
+    a.q = (const __nv_bfloat16*)q;
+    a.k = (const __nv_bfloat16*)kv->k;
+    a.v = (const __nv_bfloat16*)kv->v;
+    a.out = out;
+    a.stride_b = kv->stride_b; a.stride_pos = kv->stride_pos; a.stride_head = kv->stride_head;
+    a.stride_page = kv->stride_page;
+    a.page_table = kv->page_table; a.max_pages = kv->max_pages_per_seq; a.num_pages = kv->num_pages;
+    a.paged = kv->kv_layout == TIDAL_KV_PAGED;
+    a.ctx_lens = kv->ctx_lens;
+    a.max_ctx = kv->max_ctx_len;
+    a.Hq = kv->num_q_heads; a.Hkv = kv->num_kv_heads; a.G = a.Hq / a.Hkv;
+    a.scale = kv->sm_scale > 0.f ? kv->sm_scale : 1.0f / std::sqrt((float)kv->head_dim);
+    a.scale_log2 = a.scale * 1.4426950408889634f;
+    a.batch = kv->batch;
+    a.splits_per_item = S;
+    a.idx = idx; a.idx_count = idx_count; a.budget = k; a.Hi = Hi;
+    a.part_o = reinterpret_cast<float*>(base);
+    a.part_ml = reinterpret_cast<float2*>(base + NOALLOC_PART_O);
+    a.counters = words;
+    a.tile_ctr = words + NOALLOC_MAX_ROWS;
+    a.status = words + 2 * NOALLOC_MAX_ROWS;
+    a.max_splits = S;
+    a.hist_shift = 21;
+    a.pdl = 0;
+    a.wait_first = 1;
+
+    cudaStream_t st = (cudaStream_t)stream;
+    // The array keeps whatever the previous call left behind: the counters and cursors must read
+    // zero when the kernel starts (the partial results are always written before they are read).
+    if (cudaMemsetAsync(words, 0, NOALLOC_WORDS, st) != cudaSuccess) { cudaGetLastError(); return TIDAL_ERR_CUDA; }
+    attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>
+        <<<S * items, SPARSE_NW * 32, attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(), st>>>(a);
+    return cudaGetLastError() == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+}
