@@ -120,8 +120,9 @@ def physical_gpu_index(local: int) -> int:
     return local
 
 
-def oracle_sample(w: synth.Workload, qs, layers):
-    """Time the CPU oracle, as it stands, on one layer of each type and scale by the layer mix."""
+def oracle_sample(w: synth.Workload, qs, layers, host_cache=None):
+    """Time the CPU oracle, as it stands, on one layer of each type and scale by the layer mix.
+    Only the oracle calls are timed; the host copies of the sampled layers may be cached by the caller."""
     import oracle
     from oracle import adapter
 
@@ -129,7 +130,12 @@ def oracle_sample(w: synth.Workload, qs, layers):
     times, rho = {}, None
     order = sorted(first.items(), key=lambda kv: (kv[0] == 2, kv[1]))    # selection before sparse
     for t, i in order:
-        okv, qb = adapter.kv_from_layer(layers[i]), adapter.bits(qs[i])
+        if host_cache is not None and i in host_cache:
+            okv, qb = host_cache[i]
+        else:
+            okv, qb = adapter.kv_from_layer(layers[i]), adapter.bits(qs[i])
+            if host_cache is not None:
+                host_cache[i] = (okv, qb)
         t0 = time.perf_counter()
         if t == 0:
             oracle.full_attn(okv, qb)
@@ -163,9 +169,9 @@ def run_reference(args, w, rank):
         pt, total = synth.make_page_table(w)
         layers = {i: synth.make_layer(w, i, dev, layout="paged", q=qs[i], page_table=pt, num_pages=total)
                   for i in need}
-    vals = []
+    vals, cache = [], {}
     for it in range(args.warmup + args.steps):
-        us, cores, sample, _ = oracle_sample(w, qs, layers)
+        us, cores, sample, _ = oracle_sample(w, qs, layers, cache)
         if it >= args.warmup:
             vals.append(us)
     v = sum(vals) / len(vals)
@@ -198,14 +204,61 @@ def profile_case(td, w, dev, steps):
     print(json.dumps({"profile_case": w.name, "steps": steps, "launches": td.launch_count()}))
 
 
+def sweep(td, dev, reps):
+    """Configuration 5: context 4K..256K x budget 512..8192. Every point rotates over enough distinct
+    copies of the two layers that each launch finds its KV cache cold in L2."""
+    points = []
+    for ctx in synth.SWEEP_CTX:
+        w0 = synth.sweep_point(ctx, 512)
+        layer_bytes = ctx * w0.num_kv_heads * 512
+        copies = max(2, min(24, -(-400 * 2 ** 20 // layer_bytes)))
+        qs = [synth.make_q(w0, 0, dev), synth.make_q(w0, 1, dev)]
+        sel_layers, sp_layers = [], []
+        for c in range(copies):
+            wc = synth.sweep_point(ctx, 512)
+            wc.seed += 1000 * c
+            sel_layers.append(synth.make_layer(wc, 0, dev, q=qs[0]))
+            sp_layers.append(synth.make_layer(wc, 1, dev, q=qs[1]))
+        for k in synth.SWEEP_K:
+            kk = min(k, ctx)
+            outs = torch.empty(1, w0.num_q_heads, w0.head_dim, dtype=torch.float32, device=dev)
+            idx = torch.empty(1, w0.num_q_heads, kk, dtype=torch.int32, device=dev)
+            cnt = torch.empty(1, dtype=torch.int32, device=dev)
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(3 * (reps + 2))]
+            for r in range(reps + 2):
+                c = r % copies
+                ev[3 * r].record()
+                td.select_attn(sel_layers[c], qs[0], kk, out=outs, idx=idx, idx_count=cnt)
+                ev[3 * r + 1].record()
+                td.sparse_attn(sp_layers[c], qs[1], idx, cnt, out=outs)
+                ev[3 * r + 2].record()
+            torch.cuda.synchronize()
+            sel = [ev[3 * r].elapsed_time(ev[3 * r + 1]) * 1e3 for r in range(2, reps + 2)]
+            sp = [ev[3 * r + 1].elapsed_time(ev[3 * r + 2]) * 1e3 for r in range(2, reps + 2)]
+            sel_us, sp_us = statistics.median(sel), statistics.median(sp)
+            points.append({"ctx": ctx, "k": k, "select_us_incl_topk": sel_us, "sparse_us": sp_us,
+                           "select_GBs": layer_bytes / sel_us / 1e3,
+                           "sparse_GBs": w0.num_q_heads * kk * 516 / sp_us / 1e3,
+                           "select_over_sparse": sel_us / sp_us, "copies": copies})
+        del sel_layers, sp_layers
+        torch.cuda.empty_cache()
+    assert td.device_status() == 0
+    print(json.dumps({"sweep": "cfg5: B1 32q/8kv d128, one selection layer + one sparse layer, per-layer "
+                      "CUDA-event medians, KV cold in L2 (rotating copies)", "reps": reps, "points": points}),
+          flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="tidal", choices=["tidal", "reference"])
     ap.add_argument("--workload", default="cfg3")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="context x budget sweep (Llama-3-8B head shapes, one selection + one sparse layer): "
+                         "prints one JSON line with the selection-layer and sparse-layer cost of every point")
     ap.add_argument("--profile-case", action="store_true",
                     help="small capture target for ncu: one full, one selection and one sparse layer of "
                          "the workload, each run --steps times, nothing else")
@@ -241,6 +294,9 @@ def main():
     td = binding.Tidal(local)
     if args.profile_case:
         profile_case(td, w, dev, args.steps)
+        return
+    if args.sweep:
+        sweep(td, dev, max(3, min(args.steps, 30)))
         return
     qs, layers = build_workload(w, dev)
     outs = [torch.empty(w.batch, w.num_q_heads, w.head_dim, dtype=torch.float32, device=dev) for _ in layers]
