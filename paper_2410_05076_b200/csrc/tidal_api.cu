@@ -136,7 +136,7 @@ WsLayout layout_ws(const tidal_kv_t* kv, int k, int num_layers_host) {
     w.scores = at;    at += align_up(rows * (size_t)w.score_stride * sizeof(float), 256);
     w.cand_stride = w.score_stride;
     w.cand = at;      at += align_up(rows * (size_t)w.cand_stride * sizeof(uint2), 256);
-    w.bitmap_stride = (long long)align_up((size_t)kv->max_ctx_len, TK_SLICE) / 32;
+    w.bitmap_stride = (long long)align_up((size_t)kv->max_ctx_len, TK_SPAN) / 32;
     w.bitmap = at;    at += align_up(rows * (size_t)w.bitmap_stride * sizeof(unsigned), 256);
     w.idx = at;       at += align_up(rows * (size_t)std::max(k, 1) * sizeof(int), 256);
     w.idx_count = at; at += align_up((size_t)kv->batch * sizeof(int), 256);
@@ -280,7 +280,8 @@ tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* score
     t.bitmap_stride = w.bitmap_stride;
     const int items = kv->batch * Hi;
     if (items > 65535) return TIDAL_ERR_UNSUPPORTED;
-    const int parts = (kv->max_ctx_len + TK_SLICE - 1) / TK_SLICE;
+    const int parts = (kv->max_ctx_len + TK_SLICE - 1) / TK_SLICE;        // histogram kernel
+    const int sel_parts = (kv->max_ctx_len + TK_SPAN - 1) / TK_SPAN;     // select kernel
     t.shift = hist_shift_for(kv);
     t.vec_ok = (((uintptr_t)scores & 15) == 0 && (score_stride & 3) == 0) ? 1 : 0;
     t.cand_smem = 8192;          // one histogram bin's population; larger lists are read from global memory
@@ -288,7 +289,7 @@ tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* score
     const size_t smem = 2 * words * sizeof(unsigned) + (size_t)t.cand_smem * sizeof(uint2);
     dim3 grid(parts, items, 1);
     if (!hist_done) { topk_hist_kernel<<<grid, TK_THREADS, 0, st>>>(t); ctx->launches++; }
-    topk_select_kernel<<<grid, TK_THREADS, smem, st>>>(t);
+    topk_select_kernel<<<dim3(sel_parts, items, 1), TK_THREADS, smem, st>>>(t);
     ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }

@@ -30,7 +30,9 @@ constexpr int TK_THREADS = 512;
 constexpr int TK_BINS = 2048;          // first digit: up to 11 top bits of the key
 constexpr int TK_VEC = 4;              // float4 loads per thread per slice
 constexpr int TK_SLICE = TK_THREADS * TK_VEC * 4;   // positions per CTA (8192)
-constexpr int TK_KEYS = TK_VEC * 4;    // keys per thread
+constexpr int TK_KEYS = TK_VEC * 4;    // keys per thread per slice
+constexpr int TK_BATCHES = 2;          // slices a CTA of the select kernel walks through, one after the other
+constexpr int TK_SPAN = TK_BATCHES * TK_SLICE;      // positions per CTA of the select kernel
 
 struct TopkParams {
     const float* scores;       // [B, Hq, score_stride]
@@ -195,7 +197,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     const int N = max(0, min(p.ctx_lens[b], p.max_ctx));
     const int kk = min(p.k, N);
     int* out = p.idx + (long long)item * p.k;
-    const int s0 = blockIdx.x * TK_SLICE, s1 = min(N, s0 + TK_SLICE);
+    const int s0 = blockIdx.x * TK_SPAN, s1 = min(N, s0 + TK_SPAN);
     if (blockIdx.x == 0 && hi == 0 && tid == 0 && p.idx_count) p.idx_count[b] = kk;
     unsigned* gh = p.hist + (long long)item * TK_BINS;
 
@@ -209,13 +211,13 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         return;
     }
     if (s0 >= s1) return;
-    const int nparts = (N + TK_SLICE - 1) / TK_SLICE;  // CTAs that reach the arrival counter
+    const int nparts = (N + TK_SPAN - 1) / TK_SPAN;    // CTAs that reach the arrival counter
 
-    // ---- this CTA's keys (all loads in flight at once), then the threshold bin ------------------
+    // ---- the first slice's keys (all loads in flight at once) and the threshold bin ----------------
     const int members = p.Hq / p.Hi;
     const float* srow = p.scores + ((long long)b * p.Hq + (long long)hi * members) * p.score_stride;
     uint32_t key[TK_KEYS];
-    const unsigned valid = load_slice_keys(p, srow, members, s0, N, key);
+    unsigned valid = load_slice_keys(p, srow, members, s0, N, key);
     {
         const uint4 h4 = __ldcg(reinterpret_cast<const uint4*>(gh) + tid);
         reinterpret_cast<uint4*>(sh_hist)[tid] = h4;
@@ -228,42 +230,58 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     // ---- winners above the threshold bin: straight into the position bitmap ------------------------
     // Group j of a warp covers 128 consecutive positions, lane l the four at 4l: the 8 lanes of a
     // word OR their nibbles together and one of them stores the word (zeros included, so the
-    // bitmap needs no clearing).
+    // bitmap needs no clearing). Keys of the threshold bin itself are only marked here.
     unsigned* bm = p.bitmap + (long long)item * p.bitmap_stride;
-    unsigned eq_mask = 0;
+    unsigned eq_mask[TK_BATCHES];
 #pragma unroll
-    for (int j = 0; j < TK_VEC; ++j) {
-        unsigned nib = 0;
+    for (int bt = 0; bt < TK_BATCHES; ++bt) {
+        const int base = s0 + bt * TK_SLICE;
+        if (bt > 0) valid = load_slice_keys(p, srow, members, base, N, key);
+        unsigned eqm = 0;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int i = 4 * j + e;
-            const int bin = (int)(key[i] >> p.shift);
-            const bool ok = (valid >> i) & 1u;
-            if (ok && bin > b1) nib |= 1u << e;
-            if (ok && bin == b1) eq_mask |= 1u << i;
+        for (int j = 0; j < TK_VEC; ++j) {
+            unsigned nib = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int i = 4 * j + e;
+                const int bin = (int)(key[i] >> p.shift);
+                const bool ok = (valid >> i) & 1u;
+                if (ok && bin > b1) nib |= 1u << e;
+                if (ok && bin == b1) eqm |= 1u << i;
+            }
+            unsigned word = nib << (4 * (lane & 7));
+            word |= __shfl_xor_sync(0xffffffffu, word, 1);
+            word |= __shfl_xor_sync(0xffffffffu, word, 2);
+            word |= __shfl_xor_sync(0xffffffffu, word, 4);
+            if ((lane & 7) == 0) bm[(base >> 5) + j * (TK_THREADS / 8) + warp * 4 + (lane >> 3)] = word;
         }
-        unsigned word = nib << (4 * (lane & 7));
-        word |= __shfl_xor_sync(0xffffffffu, word, 1);
-        word |= __shfl_xor_sync(0xffffffffu, word, 2);
-        word |= __shfl_xor_sync(0xffffffffu, word, 4);
-        if ((lane & 7) == 0) bm[(s0 >> 5) + j * (TK_THREADS / 8) + warp * 4 + (lane >> 3)] = word;
+        eq_mask[bt] = eqm;
     }
 
     // ---- the threshold bin's own keys: append to the candidate list, one cursor bump per CTA -------
+    // (the few keys involved are read again: the registers only hold the last slice)
     int cta_total;
-    const int mine = __popc(eq_mask);
+    int mine = 0;
+#pragma unroll
+    for (int bt = 0; bt < TK_BATCHES; ++bt) mine += __popc(eq_mask[bt]);
     int slot = block_scan_incl<int>(mine, warp_sums, cta_total) - mine;
     if (tid == 0) bcast[0] = cta_total ? atomicAdd(&p.cursor[item], cta_total) : 0;
     __syncthreads();
     slot += bcast[0];
     uint2* cand = p.cand + (long long)item * p.cand_stride;
 #pragma unroll
-    for (int e = 0; e < TK_KEYS; ++e)
-        if ((eq_mask >> e) & 1u) {
-            const int pos = s0 + 4 * ((e >> 2) * TK_THREADS + tid) + (e & 3);
-            if (slot < p.cand_stride) cand[slot] = make_uint2(key[e], (unsigned)pos);
+    for (int bt = 0; bt < TK_BATCHES; ++bt) {
+        unsigned m = eq_mask[bt];
+        while (m) {
+            const int e = __ffs(m) - 1;
+            m &= m - 1;
+            const int pos = s0 + bt * TK_SLICE + 4 * ((e >> 2) * TK_THREADS + tid) + (e & 3);
+            float sc = __ldcg(srow + pos);
+            for (int mm = 1; mm < members; ++mm) sc += __ldcg(srow + mm * p.score_stride + pos);
+            if (slot < p.cand_stride) cand[slot] = make_uint2(score_key(sc), (unsigned)pos);
             ++slot;
         }
+    }
 
     // ---- the last CTA of this index head resolves the rest ------------------------------------------
     __syncthreads();
