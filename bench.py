@@ -110,6 +110,19 @@ class ClockSampler(threading.Thread):
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def max_over_ranks(value: float, dist, device) -> float:
+    """Slowest rank's figure: every multi-GPU time is the max over ranks (replicas finish together)."""
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_us_per_step(ms_per_step: float, world: int) -> float:
+    """N replicas complete N decode steps in the time of the slowest one."""
+    return ms_per_step * 1e3 / world
+
+
 def physical_gpu_index(local: int) -> int:
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -319,10 +332,7 @@ def main():
     clocks = sampler.stop()
     launches = td.launch_count() - launches0
     ms_total = e0.elapsed_time(e1)
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
+    ms_step = max_over_ranks(ms_total, dist, dev) / args.steps
     status = td.device_status()
     if status != binding.OK:
         raise SystemExit(f"device status {status} after the timed region")
@@ -380,10 +390,7 @@ def main():
         step_host()
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e_us = float(te.item()) / args.steps * 1e6
+    e2e_us = max_over_ranks(e2e_s, dist, dev) / args.steps * 1e6
     if not torch.allclose(out_host[0].to(dev), outs[0], rtol=0, atol=1e-3):
         raise SystemExit("host-buffer step and device step disagree")
 
@@ -394,7 +401,7 @@ def main():
 
     if rank == 0:
         line = {
-            "metric": METRIC, "value": ms_step * 1e3 / world, "unit": "us", "n_gpus": world,
+            "metric": METRIC, "value": whole_job_us_per_step(ms_step, world), "unit": "us", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": describe(w), "replicas": world,
