@@ -378,6 +378,33 @@ def main():
     }
     step_bytes = sum(kv_bytes[i] if tk != synth.LAYER_SPARSE else sparse_bytes for i, tk in enumerate(w.sched))
 
+    # ---- the same layers in situ: sub-schedules run through tidal_decode_step (no host gaps between
+    # launches, programmatic dependent launch active), differences of CUDA-event times ------------------
+    def time_schedule(ids, kinds):
+        st = td.make_step(kinds, [layers[i] for i in ids], [qs[i] for i in ids], [outs[i] for i in ids], w.k)
+        for _ in range(3):
+            st()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(nrep):
+            st()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3 / nrep
+
+    sel_ids = [i for i, tk in enumerate(w.sched) if tk == synth.LAYER_SELECT]
+    sp_ids = [i for i, tk in enumerate(w.sched) if tk == synth.LAYER_SPARSE]
+    if sel_ids and len(sp_ids) >= 2:
+        t_sel = time_schedule(sel_ids[:1], [synth.LAYER_SELECT])
+        t_chain = time_schedule(sel_ids[:1] + sp_ids, [synth.LAYER_SELECT] + [synth.LAYER_SPARSE] * len(sp_ids))
+        sp_in = (t_chain - t_sel) / len(sp_ids)
+        layers_report.update({
+            "select_us_alone_in_decode_step_call": t_sel,
+            "sparse_us_in_step": sp_in,
+            "sparse_in_step_GBs": sparse_bytes / sp_in / 1e3,
+            "sparse_in_step_frac_of_8TBs": sparse_bytes / sp_in / 1e3 / NOMINAL_HBM_GBS,
+        })
+
     # ---- end to end through the host-buffer entry point ----------------------------------------------
     q_host = torch.stack([q.cpu() for q in qs]).contiguous().pin_memory()
     out_host = torch.empty(w.num_layers, w.batch, w.num_q_heads, w.head_dim, dtype=torch.float32).pin_memory()
