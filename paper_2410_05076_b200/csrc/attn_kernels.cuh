@@ -31,6 +31,12 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+// Development hook: a tracing build (never the shipped library) defines this to record a
+// timestamp per warp at the numbered point; normally it expands to nothing.
+#ifndef TIDAL_TRACE
+#define TIDAL_TRACE(point)
+#endif
+
 namespace tidal {
 
 enum { MODE_FULL = 0, MODE_SELECT = 1, MODE_SPARSE = 2 };
@@ -277,6 +283,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = lane >> 2, tig = lane & 3;
+    TIDAL_TRACE(0);
     constexpr int RING_BYTES = NW * STAGES * STAGE_BYTES;
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem + RING_BYTES);   // MODE_SELECT: [columns][bins] counters
     const bool hist_on = (MODE == MODE_SELECT) && p.hist != nullptr;
@@ -382,7 +389,9 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         int cur = t0 + warp, cur_end = t1;             // static walk
         int grab_raw = 0;                              // lane 0: value returned by the outstanding grab
         // The first chunk of every warp is fixed (no round trip before the first load); the pool
-        // cursor hands out the tiles after those.
+        // cursor hands out the tiles after those. Requests to one cursor are served one after the
+        // other by the L2 (roughly 15-20 per microsecond), so chunks must not be too small: two-tile
+        // and single-tile requests made the kernels slower, not better balanced.
         const int pool_base = p.splits_per_item * NW * FIRST_TILES;
         auto grab = [&]() { if (lane == 0) grab_raw = pool_base + atomicAdd(pool, GRAB_TILES); };
         if (pooled) {
@@ -523,6 +532,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             pdl_trigger();
             waited = true;
         }
+        TIDAL_TRACE(1);
         if (pooled) grab();
 
         // Q^T fragments: column gid is head head0+gid; this lane holds the 16-byte
@@ -545,9 +555,11 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             cp_async_commit();
             ++commits;
         }
+        TIDAL_TRACE(2);
         for (int it = 0; it < issued; ++it) {
             cp_async_wait<STAGES - 2>();      // tile `it` has landed (this lane's copies)
-            __syncwarp();                     // ... and every other lane's; slot (it-1)%STAGES is free
+            __syncwarp();
+            if (it == 0) { TIDAL_TRACE(3); }                     // ... and every other lane's; slot (it-1)%STAGES is free
             if (tA >= 0) { issue((it + STAGES - 1) % STAGES); ++issued; }
             cp_async_commit();
             const int stage = it % STAGES;
@@ -557,6 +569,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         }
         cp_async_wait<0>();
         __syncwarp();
+        TIDAL_TRACE(4);
 
         if (hist_on) {                        // add this segment's histogram to the global one
             __syncthreads();
@@ -630,6 +643,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                 if (c == 0) p.part_ml[pr] = make_float2(M, L);
             }
         }
+        TIDAL_TRACE(5);
         if (nsplits == 1 && pooled && threadIdx.x == 0) *pool = 0;
         if (nsplits > 1) {
             // ---- the last CTA of this item to arrive combines the splits ---------------------------------
@@ -699,6 +713,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             }
         }
         __syncthreads();                          // shared memory is reused by the next segment
+        TIDAL_TRACE(6);
 
         // ---- advance to the next segment -----------------------------------------------------------------
         if (pooled) break;

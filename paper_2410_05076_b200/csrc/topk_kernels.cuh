@@ -24,6 +24,10 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#ifndef TIDAL_TRACE2
+#define TIDAL_TRACE2(point)        // development hook, see attn_kernels.cuh
+#endif
+
 namespace tidal {
 
 constexpr int TK_THREADS = 512;
@@ -197,6 +201,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     const int N = max(0, min(p.ctx_lens[b], p.max_ctx));
     const int kk = min(p.k, N);
     int* out = p.idx + (long long)item * p.k;
+    TIDAL_TRACE2(0);
     const int s0 = blockIdx.x * TK_SPAN, s1 = min(N, s0 + TK_SPAN);
     if (blockIdx.x == 0 && hi == 0 && tid == 0 && p.idx_count) p.idx_count[b] = kk;
     unsigned* gh = p.hist + (long long)item * TK_BINS;
@@ -223,8 +228,10 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         reinterpret_cast<uint4*>(sh_hist)[tid] = h4;
     }
     __syncthreads();
+    TIDAL_TRACE2(1);
     int need = kk;
     const int b1 = pick_digit(sh_hist, TK_BINS, warp_sums, bcast, need);
+    TIDAL_TRACE2(2);
     // `need` of the keys in bin b1 are still to be taken; every key in a higher bin is a winner.
 
     // ---- winners above the threshold bin: straight into the position bitmap ------------------------
@@ -258,6 +265,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         eq_mask[bt] = eqm;
     }
 
+    TIDAL_TRACE2(10);
     // ---- the threshold bin's own keys: append to the candidate list, one cursor bump per CTA -------
     // (the few keys involved are read again: the registers only hold the last slice)
     int cta_total;
@@ -283,6 +291,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         }
     }
 
+    TIDAL_TRACE2(3);
     // ---- the last CTA of this index head resolves the rest ------------------------------------------
     __syncthreads();
     if (tid == 0) {
@@ -290,6 +299,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         s_last = (atomicAdd(&p.done[item], 1) == nparts - 1);
     }
     __syncthreads();
+    TIDAL_TRACE2(4);
     if (!s_last) return;
     __threadfence();
 
@@ -315,6 +325,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
     __syncthreads();
 
+    TIDAL_TRACE2(5);
     // second digit: the next 11 key bits (every candidate already has first digit b1)
     const int s2 = p.shift - 11;                       // bits left for the third digit (10 or 11)
     for (int i = tid; i < M; i += TK_THREADS) atomicAdd(&sh_hist[(c[i].x >> s2) & 0x7ffu], 1u);
@@ -322,6 +333,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     const int d2 = pick_digit(sh_hist, TK_BINS, warp_sums, bcast, need);
     const uint32_t prefix2 = ((uint32_t)b1 << p.shift) | ((uint32_t)d2 << s2);
 
+    TIDAL_TRACE2(6);
     // third digit: the remaining low bits
     for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
     __syncthreads();
@@ -333,6 +345,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     const int d3 = pick_digit(sh_hist, 1 << s2, warp_sums, bcast, need);
     const uint32_t thr = prefix2 | (uint32_t)d3;       // the k'-th largest key; `need` keys equal to it are taken
 
+    TIDAL_TRACE2(7);
     // candidates above / equal to the threshold, as position bitmaps
     for (int i = tid; i < M; i += TK_THREADS) {
         const uint2 e = c[i];
@@ -341,6 +354,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     }
     __syncthreads();
 
+    TIDAL_TRACE2(8);
     // ordered enumeration: (winner count, equal count) scanned together in one 64-bit value
     unsigned long long cnt = 0;
     auto count_word = [&](int w, unsigned base) {
@@ -374,6 +388,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     for (int w = w0 + WB; w < w1; ++w) emit_word(w, __ldcg(&bm[w]));
     for (int i = kk + tid; i < p.k; i += TK_THREADS) out[i] = -1;
 
+    TIDAL_TRACE2(9);
     // leave the shared state clean for the next call
     for (int i = tid; i < TK_BINS; i += TK_THREADS) gh[i] = 0;
     if (tid == 0) { p.cursor[item] = 0; p.done[item] = 0; }
