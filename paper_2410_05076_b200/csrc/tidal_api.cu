@@ -48,7 +48,6 @@ struct tidal_ctx {
     int state_rows = 0;                         // capacity in (sequence, head) rows
     int* status = nullptr;                      // device word, sticky
     int64_t launches = 0;
-    int tune_dense = 0, tune_sparse = 0;        // development switches (TIDAL_TUNE_DENSE / TIDAL_TUNE_SPARSE)
 };
 
 namespace {
@@ -247,7 +246,7 @@ tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, fl
     a.wait_first = wait_first;
     const long long tiles = (long long)kv->batch * kv->num_kv_heads * ((kv->max_ctx_len + TILE - 1) / TILE);
     int grid = grid_for(tiles, ctx->dense_slots);
-    if (const int S = (ctx->tune_dense == 5) ? 0 : pooled_splits(kv, kv->batch * kv->num_kv_heads, grid)) {
+    if (const int S = pooled_splits(kv, kv->batch * kv->num_kv_heads, grid)) {
         a.splits_per_item = S;
         grid = S * kv->batch * kv->num_kv_heads;
     }
@@ -255,10 +254,6 @@ tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, fl
     a.score_stride = score_stride;
     a.hist = fuse_hist ? state_hist(ctx) : nullptr;
     if (scores) return launch_attn<MODE_SELECT, DENSE_NW, DENSE_STAGES>(ctx, a, grid, st);
-    if (ctx->tune_dense == 1) return launch_attn<MODE_FULL, 4, 6>(ctx, a, grid, st);
-    if (ctx->tune_dense == 2) return launch_attn<MODE_FULL, 6, 4>(ctx, a, grid, st);
-    if (ctx->tune_dense == 3) return launch_attn<MODE_FULL, 4, 3>(ctx, a, 2 * grid, st);
-    if (ctx->tune_dense == 4) return launch_attn<MODE_FULL, 9, 3>(ctx, a, grid, st);
     return launch_attn<MODE_FULL, DENSE_NW, DENSE_STAGES>(ctx, a, grid, st);
 }
 
@@ -304,13 +299,10 @@ tidal_status_t run_sparse(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, c
     const long long tiles = (long long)kv->batch * per_batch * ((k + TILE - 1) / TILE);
     int grid = grid_for(tiles, ctx->sparse_slots);
     a.idx = idx; a.idx_count = idx_count; a.budget = k; a.Hi = Hi;
-    if (const int S = (ctx->tune_sparse == 4) ? 0 : pooled_splits(kv, kv->batch * per_batch, grid)) {
+    if (const int S = pooled_splits(kv, kv->batch * per_batch, grid)) {
         a.splits_per_item = S;
         grid = S * kv->batch * per_batch;
     }
-    if (ctx->tune_sparse == 1) return launch_attn<MODE_SPARSE, 4, 3>(ctx, a, 2 * grid, st);
-    if (ctx->tune_sparse == 2) return launch_attn<MODE_SPARSE, 4, 6>(ctx, a, grid, st);
-    if (ctx->tune_sparse == 3) return launch_attn<MODE_SPARSE, 6, 4>(ctx, a, grid, st);
     return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(ctx, a, grid, st);
 }
 
@@ -346,15 +338,6 @@ tidal_status_t tidal_create(tidal_ctx_t** out, int device, size_t workspace_byte
     const bool topk_ok = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topk_smem) == cudaSuccess;
     if (d0 <= 0 || d1 <= 0 || s0 <= 0 || !topk_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
     ctx->dense_slots = std::min(d0, d1);
-    if (const char* e = std::getenv("TIDAL_TUNE_DENSE")) ctx->tune_dense = std::atoi(e);
-    if (const char* e = std::getenv("TIDAL_TUNE_SPARSE")) ctx->tune_sparse = std::atoi(e);
-    resident_ctas(attn_kernel<MODE_FULL, 4, 6>, 128, attn_smem<MODE_FULL, 4, 6>(), ctx->sm_count);
-    resident_ctas(attn_kernel<MODE_FULL, 6, 4>, 192, attn_smem<MODE_FULL, 6, 4>(), ctx->sm_count);
-    resident_ctas(attn_kernel<MODE_FULL, 4, 3>, 128, attn_smem<MODE_FULL, 4, 3>(), ctx->sm_count);
-    resident_ctas(attn_kernel<MODE_FULL, 9, 3>, 288, attn_smem<MODE_FULL, 9, 3>(), ctx->sm_count);
-    resident_ctas(attn_kernel<MODE_SPARSE, 4, 3>, 128, attn_smem<MODE_SPARSE, 4, 3>(), ctx->sm_count);
-    resident_ctas(attn_kernel<MODE_SPARSE, 4, 6>, 128, attn_smem<MODE_SPARSE, 4, 6>(), ctx->sm_count);
-    resident_ctas(attn_kernel<MODE_SPARSE, 6, 4>, 192, attn_smem<MODE_SPARSE, 6, 4>(), ctx->sm_count);
     ctx->sparse_slots = s0;
     if (cudaMalloc((void**)&ctx->status, 256) != cudaSuccess || cudaMemset(ctx->status, 0, 256) != cudaSuccess) {
         cudaGetLastError(); delete ctx; return TIDAL_ERR_NOMEM;

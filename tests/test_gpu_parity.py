@@ -269,3 +269,72 @@ def test_results_are_reproducible(td):
     b = td.select_attn(lay, q, w.k)
     assert torch.equal(a[1], b[1])                       # the selected sets are reproducible bit for bit
     assert torch.allclose(a[0], b[0], rtol=0, atol=1e-4)  # outputs up to fp32 summation order
+
+
+def test_many_short_sequences_use_the_flat_split(td):
+    """A batch of 37 ragged short sequences: every CTA walks several (sequence, head) segments."""
+    w = wl(37, 4, 2, 700, 33, ragged=True, ctx_min=20, seed=21)
+    q, lay = build(w, "paged")
+    okv, qb = util.oracle_kv(lay), synth.bits(q)
+    lens = lay.ctx_lens.cpu().numpy()
+    out, idx, cnt = td.select_attn(lay, q, w.k)
+    ref, sc = oracle.full_attn(okv, qb, want_scores=True)
+    util.check_out(out.cpu().numpy(), ref, "batch.select")
+    idx_h = idx.cpu().numpy()
+    for b in range(w.batch):
+        for h in range(w.num_q_heads):
+            util.check_idx_row(idx_h[b, h], sc[b, h], w.k, int(lens[b]), f"batch.idx[{b},{h}]")
+    sp = td.sparse_attn(lay, q, idx, cnt)
+    util.check_out(sp.cpu().numpy(), oracle.sparse_attn(okv, qb, idx_h, cnt.cpu().numpy()), "batch.sparse")
+    assert td.device_status() == binding.OK
+
+
+def test_explicit_softmax_scale(td):
+    w = wl(1, 8, 2, 600, 30, seed=23)
+    q, lay = build(w, "hnd_interleaved")
+    lay.sm_scale = 0.05
+    okv, qb = util.oracle_kv(lay), synth.bits(q)
+    scores = torch.empty(1, 8, 600, dtype=torch.float32, device=DEV)
+    out, idx, cnt = td.select_attn(lay, q, w.k, scores=scores)
+    ref, sc = oracle.full_attn(okv, qb, want_scores=True)
+    util.check_out(out.cpu().numpy(), ref, "scale.out")
+    assert np.abs(scores.cpu().numpy() - sc).max() <= 1e-4
+    # the stored logits scale with sm_scale: compare with the default scale 1/sqrt(128)
+    lay.sm_scale = 0.0
+    _, sc_default = oracle.full_attn(util.oracle_kv(lay), qb, want_scores=True)
+    assert np.allclose(sc, sc_default * (0.05 * np.sqrt(128.0)), atol=1e-5)
+
+
+def test_group_of_eight_with_shared_sets_at_32k(td):
+    """64 query heads over 8 KV heads (Llama-3-70B-like), context 32768, one token set per KV head:
+    the sparse layer then runs all eight heads of a group as MMA columns over the same gathered rows."""
+    w = synth.Workload("g8", 1, 64, 8, 2, 32768, 1024, 64, [1, 2], synth.BASE_SEED + 777)
+    q, lay = build(w, "hnd_interleaved")
+    okv, qb = util.oracle_kv(lay), synth.bits(q)
+    out, idx, cnt = td.select_attn(lay, q, w.k, granularity=binding.SEL_PER_KVHEAD)
+    ref, ref_idx, ref_cnt, sc = oracle.select_attn(okv, qb, w.k, 8, want_scores=True)
+    util.check_out(out.cpu().numpy(), ref, "g8.select")
+    idx_h = idx.cpu().numpy()
+    for g in range(8):
+        agg = sc[0, 8 * g: 8 * g + 8].astype(np.float64).sum(0).astype(np.float32)
+        util.check_idx_row(idx_h[0, g], agg, w.k, w.ctx, f"g8.idx[{g}]")
+    sp = td.sparse_attn(lay, q, idx, cnt)
+    util.check_out(sp.cpu().numpy(), oracle.sparse_attn(okv, qb, idx_h, cnt.cpu().numpy()), "g8.sparse")
+    # the paper's per-head sets on the same cache (histogram with 1024 bins for a group of 8)
+    out2, idx2, cnt2 = td.select_attn(lay, q, w.k)
+    idx2_h = idx2.cpu().numpy()
+    for h in range(0, 64, 7):
+        util.check_idx_row(idx2_h[0, h], sc[0, h], w.k, w.ctx, f"g8.idx_q[{h}]")
+    sp2 = td.sparse_attn(lay, q, idx2, cnt2)
+    util.check_out(sp2.cpu().numpy(), oracle.sparse_attn(okv, qb, idx2_h, cnt2.cpu().numpy()), "g8.sparse_q")
+
+
+def test_budget_equal_to_a_long_context_keeps_everything(td):
+    w = synth.sweep_point(65536, 65536)
+    q, lay = build(w, "hnd_interleaved")
+    out, idx, cnt = td.select_attn(lay, q, w.k)
+    assert cnt.item() == 65536
+    assert torch.equal(idx[0, 5], torch.arange(65536, dtype=torch.int32, device=DEV))
+    sp = td.sparse_attn(lay, q, idx, cnt)
+    torch.cuda.synchronize()
+    assert torch.allclose(sp, out, rtol=0, atol=2e-4)       # sparse over everything is full attention
