@@ -281,7 +281,9 @@ tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* score
     t.vec_ok = (((uintptr_t)scores & 15) == 0 && (score_stride & 3) == 0) ? 1 : 0;
     t.cand_smem = 8192;          // one histogram bin's population; larger lists are read from global memory
     const size_t words = (size_t)(kv->max_ctx_len + 31) / 32;
-    const size_t smem = 2 * words * sizeof(unsigned) + (size_t)t.cand_smem * sizeof(uint2);
+    // the last CTA's bitmaps and candidate buffer, or every CTA's score staging area, whichever is larger
+    const size_t smem = std::max(2 * words * sizeof(unsigned) + (size_t)t.cand_smem * sizeof(uint2),
+                                 (size_t)TK_SPAN * sizeof(float));
     dim3 grid(parts, items, 1);
     if (!hist_done) { topk_hist_kernel<<<grid, TK_THREADS, 0, st>>>(t); ctx->launches++; }
     topk_select_kernel<<<dim3(sel_parts, items, 1), TK_THREADS, smem, st>>>(t);

@@ -218,11 +218,42 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     if (s0 >= s1) return;
     const int nparts = (N + TK_SPAN - 1) / TK_SPAN;    // CTAs that reach the arrival counter
 
-    // ---- the first slice's keys (all loads in flight at once) and the threshold bin ----------------
+    // ---- stage this CTA's scores in shared memory, every load in flight at once -------------------------
+    // (the staging area is the head of the dynamic shared memory, which only the last CTA of an
+    // index head uses again later, for other things)
     const int members = p.Hq / p.Hi;
     const float* srow = p.scores + ((long long)b * p.Hq + (long long)hi * members) * p.score_stride;
-    uint32_t key[TK_KEYS];
-    unsigned valid = load_slice_keys(p, srow, members, s0, N, key);
+    float* raw = reinterpret_cast<float*>(tk_smem);                // [TK_SPAN]
+    if (p.vec_ok && members == 1) {
+#pragma unroll
+        for (int j = 0; j < TK_BATCHES * TK_VEC; ++j) {
+            const int off = 4 * (j * TK_THREADS + tid);
+            const int pos = s0 + off;
+            const int nbytes = max(0, min(4, N - pos)) * 4;        // zero-fill past the end of the cache
+            const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(raw + off));
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n"
+                         ::"r"(dst), "l"(nbytes ? srow + pos : srow), "r"(nbytes) : "memory");
+        }
+        asm volatile("cp.async.commit_group;\n" ::: "memory");
+    } else {
+#pragma unroll
+        for (int bt = 0; bt < TK_BATCHES; ++bt) {                  // summed member heads or unaligned rows
+            float v[TK_KEYS];
+#pragma unroll
+            for (int e = 0; e < TK_KEYS; ++e) {
+                const int pos = s0 + bt * TK_SLICE + 4 * ((e >> 2) * TK_THREADS + tid) + (e & 3);
+                float t = 0.f;
+                if (pos < N) {
+                    t = __ldcg(srow + pos);
+                    for (int m = 1; m < members; ++m) t += __ldcg(srow + m * p.score_stride + pos);
+                }
+                v[e] = t;
+            }
+#pragma unroll
+            for (int e = 0; e < TK_KEYS; ++e)
+                raw[bt * TK_SLICE + 4 * ((e >> 2) * TK_THREADS + tid) + (e & 3)] = v[e];
+        }
+    }
     {
         const uint4 h4 = __ldcg(reinterpret_cast<const uint4*>(gh) + tid);
         reinterpret_cast<uint4*>(sh_hist)[tid] = h4;
@@ -233,60 +264,51 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     const int b1 = pick_digit(sh_hist, TK_BINS, warp_sums, bcast, need);
     TIDAL_TRACE2(2);
     // `need` of the keys in bin b1 are still to be taken; every key in a higher bin is a winner.
+    asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+    __syncthreads();
 
     // ---- winners above the threshold bin: straight into the position bitmap ------------------------
     // Group j of a warp covers 128 consecutive positions, lane l the four at 4l: the 8 lanes of a
     // word OR their nibbles together and one of them stores the word (zeros included, so the
     // bitmap needs no clearing). Keys of the threshold bin itself are only marked here.
     unsigned* bm = p.bitmap + (long long)item * p.bitmap_stride;
-    unsigned eq_mask[TK_BATCHES];
+    unsigned eq_mask = 0;                                          // bit 4j+e: group j, element e
 #pragma unroll
-    for (int bt = 0; bt < TK_BATCHES; ++bt) {
-        const int base = s0 + bt * TK_SLICE;
-        if (bt > 0) valid = load_slice_keys(p, srow, members, base, N, key);
-        unsigned eqm = 0;
+    for (int j = 0; j < TK_BATCHES * TK_VEC; ++j) {
+        const int off = 4 * (j * TK_THREADS + tid);
+        const float4 f = *reinterpret_cast<const float4*>(raw + off);
+        const float fe[4] = {f.x, f.y, f.z, f.w};
+        unsigned nib = 0;
 #pragma unroll
-        for (int j = 0; j < TK_VEC; ++j) {
-            unsigned nib = 0;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int i = 4 * j + e;
-                const int bin = (int)(key[i] >> p.shift);
-                const bool ok = (valid >> i) & 1u;
-                if (ok && bin > b1) nib |= 1u << e;
-                if (ok && bin == b1) eqm |= 1u << i;
-            }
-            unsigned word = nib << (4 * (lane & 7));
-            word |= __shfl_xor_sync(0xffffffffu, word, 1);
-            word |= __shfl_xor_sync(0xffffffffu, word, 2);
-            word |= __shfl_xor_sync(0xffffffffu, word, 4);
-            if ((lane & 7) == 0) bm[(base >> 5) + j * (TK_THREADS / 8) + warp * 4 + (lane >> 3)] = word;
+        for (int e = 0; e < 4; ++e) {
+            const bool ok = s0 + off + e < N;
+            const int bin = (int)(score_key(fe[e]) >> p.shift);
+            if (ok && bin > b1) nib |= 1u << e;
+            if (ok && bin == b1) eq_mask |= 1u << (4 * j + e);
         }
-        eq_mask[bt] = eqm;
+        unsigned word = nib << (4 * (lane & 7));
+        word |= __shfl_xor_sync(0xffffffffu, word, 1);
+        word |= __shfl_xor_sync(0xffffffffu, word, 2);
+        word |= __shfl_xor_sync(0xffffffffu, word, 4);
+        if ((lane & 7) == 0) bm[(s0 >> 5) + j * (TK_THREADS / 8) + warp * 4 + (lane >> 3)] = word;
     }
-
     TIDAL_TRACE2(10);
+
     // ---- the threshold bin's own keys: append to the candidate list, one cursor bump per CTA -------
-    // (the few keys involved are read again: the registers only hold the last slice)
     int cta_total;
-    int mine = 0;
-#pragma unroll
-    for (int bt = 0; bt < TK_BATCHES; ++bt) mine += __popc(eq_mask[bt]);
+    const int mine = __popc(eq_mask);
     int slot = block_scan_incl<int>(mine, warp_sums, cta_total) - mine;
     if (tid == 0) bcast[0] = cta_total ? atomicAdd(&p.cursor[item], cta_total) : 0;
     __syncthreads();
     slot += bcast[0];
     uint2* cand = p.cand + (long long)item * p.cand_stride;
-#pragma unroll
-    for (int bt = 0; bt < TK_BATCHES; ++bt) {
-        unsigned m = eq_mask[bt];
+    {
+        unsigned m = eq_mask;
         while (m) {
             const int e = __ffs(m) - 1;
             m &= m - 1;
-            const int pos = s0 + bt * TK_SLICE + 4 * ((e >> 2) * TK_THREADS + tid) + (e & 3);
-            float sc = __ldcg(srow + pos);
-            for (int mm = 1; mm < members; ++mm) sc += __ldcg(srow + mm * p.score_stride + pos);
-            if (slot < p.cand_stride) cand[slot] = make_uint2(score_key(sc), (unsigned)pos);
+            const int off = 4 * ((e >> 2) * TK_THREADS + tid) + (e & 3);
+            if (slot < p.cand_stride) cand[slot] = make_uint2(score_key(raw[off]), (unsigned)(s0 + off));
             ++slot;
         }
     }
@@ -305,8 +327,8 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
 
     const int M = (int)min((long long)__ldcg(&p.cursor[item]), p.cand_stride);
     const int words = (N + 31) >> 5;
-    unsigned* cgt = reinterpret_cast<unsigned*>(tk_smem);          // [words] candidates above the final threshold
-    unsigned* ceq = cgt + words;                                    // [words] candidates equal to it
+    unsigned* cgt = reinterpret_cast<unsigned*>(tk_smem);          // [words] winners: higher bins + winning candidates
+    unsigned* ceq = cgt + words;                                    // [words] candidates equal to the threshold key
     uint2* scand = reinterpret_cast<uint2*>(ceq + words);          // [cand_smem]; 8*words bytes in: 8-byte aligned
     const uint2* c = cand;
     if (M <= p.cand_smem) {
@@ -314,14 +336,11 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         for (int i = tid; i < M; i += TK_THREADS) scand[i] = __ldcg(&cand[i]);
         c = scand;
     }
-    // this thread's bitmap words for the enumeration: loads in flight while the digits are resolved
-    constexpr int WB = 8;
+    // The winners' bitmap written by all CTAs of this head is pulled into shared memory once
+    // (coalesced); candidates that turn out to be winners are ORed into the same words.
     const int per = (words + TK_THREADS - 1) / TK_THREADS;
     const int w0 = min(words, tid * per), w1 = min(words, w0 + per);
-    unsigned bw[WB];
-#pragma unroll
-    for (int u = 0; u < WB; ++u) bw[u] = (w0 + u < w1) ? __ldcg(&bm[w0 + u]) : 0u;
-    for (int i = tid; i < words; i += TK_THREADS) { cgt[i] = 0; ceq[i] = 0; }
+    for (int i = tid; i < words; i += TK_THREADS) { cgt[i] = __ldcg(&bm[i]); ceq[i] = 0; }
     for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
     __syncthreads();
 
@@ -332,60 +351,83 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     __syncthreads();
     const int d2 = pick_digit(sh_hist, TK_BINS, warp_sums, bcast, need);
     const uint32_t prefix2 = ((uint32_t)b1 << p.shift) | ((uint32_t)d2 << s2);
+    const int in_bin = (int)sh_hist[d2];               // candidates that share both digits with the threshold key
+    __syncthreads();                                   // sh_hist is recycled below
 
     TIDAL_TRACE2(6);
-    // third digit: the remaining low bits
-    for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
-    __syncthreads();
-    for (int i = tid; i < M; i += TK_THREADS) {
-        const uint32_t k32 = c[i].x;
-        if ((k32 >> s2) == (prefix2 >> s2)) atomicAdd(&sh_hist[k32 & ((1u << s2) - 1u)], 1u);
+    constexpr int SMALL = 64;
+    if (in_bin <= SMALL) {
+        // A handful of keys are left: rank them directly. Entry i is taken iff fewer than `need` of the
+        // others beat it (larger key, or equal key at a lower position).
+        uint2* few = reinterpret_cast<uint2*>(sh_hist);            // [SMALL]
+        int* nfew = &bcast[0];
+        if (tid == 0) *nfew = 0;
+        __syncthreads();
+        for (int i = tid; i < M; i += TK_THREADS) {
+            const uint2 e = c[i];
+            if ((e.x >> s2) == (prefix2 >> s2)) few[atomicAdd(nfew, 1)] = e;
+            else if ((e.x >> s2) > (prefix2 >> s2)) atomicOr(&cgt[e.y >> 5], 1u << (e.y & 31));
+        }
+        __syncthreads();
+        const int n = *nfew;
+        if (tid < n) {
+            const uint2 me = few[tid];
+            int beaten_by = 0;
+            for (int j = 0; j < n; ++j) {
+                const uint2 o = few[j];
+                beaten_by += (o.x > me.x) || (o.x == me.x && o.y < me.y);
+            }
+            if (beaten_by < need) atomicOr(&cgt[me.y >> 5], 1u << (me.y & 31));
+        }
+        need = 0;                                      // nothing is taken through the equal-key bitmap
+        __syncthreads();
+    } else {
+        // third digit: the remaining low bits
+        for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
+        __syncthreads();
+        for (int i = tid; i < M; i += TK_THREADS) {
+            const uint32_t k32 = c[i].x;
+            if ((k32 >> s2) == (prefix2 >> s2)) atomicAdd(&sh_hist[k32 & ((1u << s2) - 1u)], 1u);
+        }
+        __syncthreads();
+        const int d3 = pick_digit(sh_hist, 1 << s2, warp_sums, bcast, need);
+        const uint32_t thr = prefix2 | (uint32_t)d3;   // the k'-th largest key; `need` keys equal to it are taken
+        TIDAL_TRACE2(7);
+        // candidates above / equal to the threshold, as position bitmaps
+        for (int i = tid; i < M; i += TK_THREADS) {
+            const uint2 e = c[i];
+            if (e.x > thr) atomicOr(&cgt[e.y >> 5], 1u << (e.y & 31));
+            else if (e.x == thr) atomicOr(&ceq[e.y >> 5], 1u << (e.y & 31));
+        }
+        __syncthreads();
     }
-    __syncthreads();
-    const int d3 = pick_digit(sh_hist, 1 << s2, warp_sums, bcast, need);
-    const uint32_t thr = prefix2 | (uint32_t)d3;       // the k'-th largest key; `need` keys equal to it are taken
-
-    TIDAL_TRACE2(7);
-    // candidates above / equal to the threshold, as position bitmaps
-    for (int i = tid; i < M; i += TK_THREADS) {
-        const uint2 e = c[i];
-        if (e.x > thr) atomicOr(&cgt[e.y >> 5], 1u << (e.y & 31));
-        else if (e.x == thr) atomicOr(&ceq[e.y >> 5], 1u << (e.y & 31));
-    }
-    __syncthreads();
 
     TIDAL_TRACE2(8);
     // ordered enumeration: (winner count, equal count) scanned together in one 64-bit value
     unsigned long long cnt = 0;
-    auto count_word = [&](int w, unsigned base) {
-        cnt += ((unsigned long long)__popc(base | cgt[w]) << 32) | (unsigned long long)__popc(ceq[w]);
-    };
-#pragma unroll
-    for (int u = 0; u < WB; ++u)
-        if (w0 + u < w1) count_word(w0 + u, bw[u]);
-    for (int w = w0 + WB; w < w1; ++w) count_word(w, __ldcg(&bm[w]));
+    for (int w = w0; w < w1; ++w)
+        cnt += ((unsigned long long)__popc(cgt[w]) << 32) | (unsigned long long)__popc(ceq[w]);
+    TIDAL_TRACE2(11);
     unsigned long long tot;
     const unsigned long long excl = block_scan_incl<unsigned long long>(cnt, warp_sums64, tot) - cnt;
+    TIDAL_TRACE2(12);
     int eq_seen = (int)(excl & 0xffffffffu);
     int at = (int)(excl >> 32) + min(eq_seen, need);
-    auto emit_word = [&](int w, unsigned base) {
+    for (int w = w0; w < w1; ++w) {
         unsigned e = ceq[w];
         const int ne = __popc(e);
         const int keep = min(max(need - eq_seen, 0), ne);   // lowest `keep` equal-key positions of this word
         eq_seen += ne;
         while (__popc(e) > keep) e &= ~(0x80000000u >> __clz(e));
-        unsigned bits = base | cgt[w] | e;
+        unsigned bits = cgt[w] | e;
         while (bits) {
             const int pbit = __ffs(bits) - 1;
             if (at < p.k) out[at] = (w << 5) + pbit;
             ++at;
             bits &= bits - 1;
         }
-    };
-#pragma unroll
-    for (int u = 0; u < WB; ++u)
-        if (w0 + u < w1) emit_word(w0 + u, bw[u]);
-    for (int w = w0 + WB; w < w1; ++w) emit_word(w, __ldcg(&bm[w]));
+    }
+    TIDAL_TRACE2(13);
     for (int i = kk + tid; i < p.k; i += TK_THREADS) out[i] = -1;
 
     TIDAL_TRACE2(9);
