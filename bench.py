@@ -226,38 +226,49 @@ def sweep(td, dev, reps):
         layer_bytes = ctx * w0.num_kv_heads * 512
         copies = max(2, min(24, -(-400 * 2 ** 20 // layer_bytes)))
         qs = [synth.make_q(w0, 0, dev), synth.make_q(w0, 1, dev)]
+        # sparse layers gather as little as 8 MiB each: 20 distinct caches keep a chain of them cold
+        sp_copies = max(copies, 20)
         sel_layers, sp_layers = [], []
-        for c in range(copies):
+        for c in range(sp_copies):
             wc = synth.sweep_point(ctx, 512)
             wc.seed += 1000 * c
-            sel_layers.append(synth.make_layer(wc, 0, dev, q=qs[0]))
+            if c < copies:
+                sel_layers.append(synth.make_layer(wc, 0, dev, q=qs[0]))
             sp_layers.append(synth.make_layer(wc, 1, dev, q=qs[1]))
+        outs = [torch.empty(1, w0.num_q_heads, w0.head_dim, dtype=torch.float32, device=dev)
+                for _ in range(max(copies, sp_copies) + 1)]
+
+        def timed(kinds, lays, qq, k):
+            st = td.make_step(kinds, lays, qq, outs[:len(kinds)], k)
+            for _ in range(2):
+                st()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(reps):
+                st()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) * 1e3 / reps
+
         for k in synth.SWEEP_K:
             kk = min(k, ctx)
-            outs = torch.empty(1, w0.num_q_heads, w0.head_dim, dtype=torch.float32, device=dev)
-            idx = torch.empty(1, w0.num_q_heads, kk, dtype=torch.int32, device=dev)
-            cnt = torch.empty(1, dtype=torch.int32, device=dev)
-            ev = [torch.cuda.Event(enable_timing=True) for _ in range(3 * (reps + 2))]
-            for r in range(reps + 2):
-                c = r % copies
-                ev[3 * r].record()
-                td.select_attn(sel_layers[c], qs[0], kk, out=outs, idx=idx, idx_count=cnt)
-                ev[3 * r + 1].record()
-                td.sparse_attn(sp_layers[c], qs[1], idx, cnt, out=outs)
-                ev[3 * r + 2].record()
-            torch.cuda.synchronize()
-            sel = [ev[3 * r].elapsed_time(ev[3 * r + 1]) * 1e3 for r in range(2, reps + 2)]
-            sp = [ev[3 * r + 1].elapsed_time(ev[3 * r + 2]) * 1e3 for r in range(2, reps + 2)]
-            sel_us, sp_us = statistics.median(sel), statistics.median(sp)
+            # all launches go through tidal_decode_step (no host gaps): a chain of selection layers over
+            # the distinct copies, and one selection layer followed by a chain of sparse layers
+            t_sel_chain = timed([synth.LAYER_SELECT] * copies, sel_layers, [qs[0]] * copies, kk)
+            t_one = timed([synth.LAYER_SELECT], sel_layers[:1], qs[:1], kk)
+            t_sp_chain = timed([synth.LAYER_SELECT] + [synth.LAYER_SPARSE] * sp_copies,
+                               sel_layers[:1] + sp_layers, [qs[0]] + [qs[1]] * sp_copies, kk)
+            sel_us, sp_us = t_sel_chain / copies, (t_sp_chain - t_one) / sp_copies
             points.append({"ctx": ctx, "k": k, "select_us_incl_topk": sel_us, "sparse_us": sp_us,
                            "select_GBs": layer_bytes / sel_us / 1e3,
                            "sparse_GBs": w0.num_q_heads * kk * 516 / sp_us / 1e3,
-                           "select_over_sparse": sel_us / sp_us, "copies": copies})
+                           "select_over_sparse": sel_us / sp_us, "copies": [copies, sp_copies]})
         del sel_layers, sp_layers
         torch.cuda.empty_cache()
     assert td.device_status() == 0
-    print(json.dumps({"sweep": "cfg5: B1 32q/8kv d128, one selection layer + one sparse layer, per-layer "
-                      "CUDA-event medians, KV cold in L2 (rotating copies)", "reps": reps, "points": points}),
+    print(json.dumps({"sweep": "cfg5: B1 32q/8kv d128; per-layer cost of a selection layer (attention + top-k) and "
+                      "of a sparse layer, from chains of layers run through tidal_decode_step over distinct "
+                      "KV copies (cold in L2), CUDA events", "reps": reps, "points": points}),
           flush=True)
 
 

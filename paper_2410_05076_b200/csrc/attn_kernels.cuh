@@ -392,11 +392,15 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         // cursor hands out the tiles after those. Requests to one cursor are served one after the
         // other by the L2 (roughly 15-20 per microsecond), so chunks must not be too small: two-tile
         // and single-tile requests made the kernels slower, not better balanced.
-        const int pool_base = p.splits_per_item * NW * FIRST_TILES;
+        // Short items are spread evenly over all the item's warps instead (nothing left for the pool).
+        const int item_warps = p.splits_per_item * NW;
+        const int first_tiles = (tiles_b <= item_warps * FIRST_TILES)
+                                    ? max(1, (tiles_b + item_warps - 1) / max(item_warps, 1)) : FIRST_TILES;
+        const int pool_base = item_warps * first_tiles;
         auto grab = [&]() { if (lane == 0) grab_raw = pool_base + atomicAdd(pool, GRAB_TILES); };
         if (pooled) {
-            cur = ((int)(blockIdx.x / (p.batch * IY)) * NW + warp) * FIRST_TILES;
-            cur_end = min(tiles_b, cur + FIRST_TILES);
+            cur = ((int)(blockIdx.x / (p.batch * IY)) * NW + warp) * first_tiles;
+            cur_end = min(tiles_b, cur + first_tiles);
         }
         auto next_tile = [&]() -> int {                // -1 when this warp has no more tiles
             if (!pooled) {
@@ -406,7 +410,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                 return t;
             }
             if (cur >= cur_end) {
-                if (cur_end >= tiles_b) return -1;     // the pool ran dry on the previous grab
+                if (cur_end >= tiles_b || pool_base >= tiles_b) return -1;   // nothing (left) in the pool
                 cur = __shfl_sync(0xffffffffu, grab_raw, 0);
                 if (cur >= tiles_b) { cur_end = tiles_b; return -1; }
                 cur_end = min(tiles_b, cur + GRAB_TILES);
