@@ -94,6 +94,19 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int sr
 __device__ __forceinline__ void cp_async16_full(uint32_t dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
 }
+// The same with an L2 eviction hint: the KV stream is read once, so its lines should be the first
+// to go and leave the scores, index lists and partial results of the step in L2.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void cp_async16_hint(uint32_t dst, const void* src, int src_bytes, uint64_t pol) {
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;\n" ::"r"(dst), "l"(src), "r"(src_bytes), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void cp_async16_full_hint(uint32_t dst, const void* src, uint64_t pol) {
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "l"(pol) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
@@ -349,6 +362,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
     const uint32_t vdst = rhalf * 256;
     const uint32_t vc = c16 ^ rhalf;
     const bool pooled = p.splits_per_item > 0;
+    const uint64_t kv_policy = l2_evict_first_policy();
 
     do {
         // ---- one segment: tiles [t0, t1) of item y of sequence b (pooled: whatever the warps grab) --
@@ -486,8 +500,8 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                 if (nvalid == TILE) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        cp_async16_full(ks + kdst + i * 512, ksrc + i * two_rows);
-                        cp_async16_full(vs + vdst + i * 512 + ((vc ^ ((i & 3) << 1)) << 4), vsrc + i * two_rows);
+                        cp_async16_full_hint(ks + kdst + i * 512, ksrc + i * two_rows, kv_policy);
+                        cp_async16_full_hint(vs + vdst + i * 512 + ((vc ^ ((i & 3) << 1)) << 4), vsrc + i * two_rows, kv_policy);
                     }
                 } else {
 #pragma unroll
@@ -512,8 +526,8 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                     const long long ro = __shfl_sync(0xffffffffu, off, r);
                     const bool rv = (vmask >> r) & 1u;
                     const long long eo = rv ? ro + c16 * 8 : 0;
-                    cp_async16(ks + kdst + i * 512, p.k + eo, rv ? 16 : 0);
-                    cp_async16(vs + vdst + i * 512 + ((vc ^ ((i & 3) << 1)) << 4), p.v + eo, rv ? 16 : 0);
+                    cp_async16_hint(ks + kdst + i * 512, p.k + eo, rv ? 16 : 0, kv_policy);
+                    cp_async16_hint(vs + vdst + i * 512 + ((vc ^ ((i & 3) << 1)) << 4), p.v + eo, rv ? 16 : 0, kv_policy);
                 }
                 if (lane == 0) { s_vmask[warp][stage] = vmask; s_posbase[warp][stage] = 0; }
             }
