@@ -64,7 +64,8 @@ struct AttnParams {
     int Hq, Hkv, G;
     float scale, scale_log2;
     int batch;
-    int splits_per_item;       // S > 0: CTAs c*S..c*S+S-1 share item c's tiles through a pool cursor; 0: static flat split
+    int splits_per_item;       // > 0: pooled mode, CTA c works on item c % items; an item is served by every CTA
+                               // of the grid that maps to it (this many, or one more); 0: static flat split
     float* scores;             // MODE_SELECT: [B, Hq, score_stride]
     long long score_stride;
     const int* idx;            // MODE_SPARSE: [B, Hi, k]
@@ -315,6 +316,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
     };
     long long per_cta, lo, hi, seq_start = 0;
     int b = 0, tiles_b;
+    int part_idx = 0, item_ctas = 0;                   // pooled: which of the item's CTAs this is, out of how many
     if (p.splits_per_item > 0) {
         // Pooled split: S CTAs work on each item and share its tiles dynamically, so
         // that SMs that get less memory bandwidth simply take fewer tiles; no CTA spans two items.
@@ -322,14 +324,15 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         const int n_items = p.batch * IY;
         const int item = blockIdx.x % n_items, part = blockIdx.x / n_items;
         b = item / IY;
-        if (part >= p.splits_per_item) return;
+        part_idx = part;
+        item_ctas = ((int)gridDim.x - item + n_items - 1) / n_items;
         tiles_b = item_tiles(seq_total(b));
         per_cta = tiles_b;
         // flat index of the item's first tile relative to sequence b (seq_start stays 0); the
         // tiles themselves are handed out by the item's pool cursor
         lo = (long long)(item % IY) * tiles_b;
         hi = lo + 1;
-        (void)part;
+
     } else {
         long long T = 0;
         for (int bb = 0; bb < p.batch; ++bb) T += (long long)IY * item_tiles(seq_total(bb));
@@ -407,13 +410,13 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         // other by the L2 (roughly 15-20 per microsecond), so chunks must not be too small: two-tile
         // and single-tile requests made the kernels slower, not better balanced.
         // Short items are spread evenly over all the item's warps instead (nothing left for the pool).
-        const int item_warps = p.splits_per_item * NW;
+        const int item_warps = item_ctas * NW;
         const int first_tiles = (tiles_b <= item_warps * FIRST_TILES)
                                     ? max(1, (tiles_b + item_warps - 1) / max(item_warps, 1)) : FIRST_TILES;
         const int pool_base = item_warps * first_tiles;
         auto grab = [&]() { if (lane == 0) grab_raw = pool_base + atomicAdd(pool, GRAB_TILES); };
         if (pooled) {
-            cur = ((int)(blockIdx.x / (p.batch * IY)) * NW + warp) * first_tiles;
+            cur = (part_idx * NW + warp) * first_tiles;
             cur_end = min(tiles_b, cur + first_tiles);
         }
         auto next_tile = [&]() -> int {                // -1 when this warp has no more tiles
@@ -629,8 +632,8 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         // CTAs that share this item: those whose range meets [item_lo, item_lo + tiles_b).
         int nsplits, split;
         if (pooled) {
-            nsplits = p.splits_per_item;          // every CTA of the item arrives, with or without tiles
-            split = blockIdx.x / (p.batch * IY);
+            nsplits = item_ctas;                  // every CTA of the item arrives, with or without tiles
+            split = part_idx;
         } else {
             const long long item_lo = seq_start + (long long)y * tiles_b;
             const int first_cta = (int)(item_lo / per_cta);

@@ -247,8 +247,7 @@ tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, fl
     const long long tiles = (long long)kv->batch * kv->num_kv_heads * ((kv->max_ctx_len + TILE - 1) / TILE);
     int grid = grid_for(tiles, ctx->dense_slots);
     if (const int S = pooled_splits(kv, kv->batch * kv->num_kv_heads, grid)) {
-        a.splits_per_item = S;
-        grid = S * kv->batch * kv->num_kv_heads;
+        a.splits_per_item = S;        // the grid keeps its size: some items get one CTA more than others
     }
     a.scores = scores;
     a.score_stride = score_stride;
@@ -303,7 +302,6 @@ tidal_status_t run_sparse(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, c
     a.idx = idx; a.idx_count = idx_count; a.budget = k; a.Hi = Hi;
     if (const int S = pooled_splits(kv, kv->batch * per_batch, grid)) {
         a.splits_per_item = S;
-        grid = S * kv->batch * per_batch;
     }
     return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(ctx, a, grid, st);
 }
