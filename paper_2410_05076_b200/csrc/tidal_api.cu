@@ -283,10 +283,27 @@ tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* score
     // the last CTA's bitmaps and candidate buffer, or every CTA's score staging area, whichever is larger
     const size_t smem = std::max(2 * words * sizeof(unsigned) + (size_t)t.cand_smem * sizeof(uint2),
                                  (size_t)TK_SPAN * sizeof(float));
-    dim3 grid(parts, items, 1);
-    if (!hist_done) { topk_hist_kernel<<<grid, TK_THREADS, 0, st>>>(t); ctx->launches++; }
-    topk_select_kernel<<<dim3(sel_parts, items, 1), TK_THREADS, smem, st>>>(t);
+    // Both kernels may become resident while the kernel before them drains (they wait for it first).
+    t.pdl = 1;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.blockDim = dim3(TK_THREADS, 1, 1);
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (!hist_done) {
+        cfg.gridDim = dim3(parts, items, 1);
+        cfg.dynamicSmemBytes = 0;
+        ctx->launches++;
+        if (cudaLaunchKernelEx(&cfg, topk_hist_kernel, t) != cudaSuccess) return TIDAL_ERR_CUDA;
+    }
+    cfg.gridDim = dim3(sel_parts, items, 1);
+    cfg.dynamicSmemBytes = smem;
     ctx->launches++;
+    if (cudaLaunchKernelEx(&cfg, topk_select_kernel, t) != cudaSuccess) return TIDAL_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }
 

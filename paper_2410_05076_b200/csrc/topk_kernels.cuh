@@ -57,6 +57,7 @@ struct TopkParams {
     int cand_smem;             // candidates the last CTA can hold in shared memory
     int vec_ok;                // score rows are 16-byte aligned: float4 loads allowed
     int shift;                 // first digit = key >> shift (21 or 22); the rest is split 11 + (shift-11) bits
+    int pdl;                   // launched with programmatic stream serialization: wait for the producer of the scores
 };
 
 // Larger float <=> larger key; -0 and +0 map to the same key.
@@ -166,6 +167,10 @@ __device__ __forceinline__ int pick_digit(const unsigned* hist, int nbins, int* 
 __global__ void __launch_bounds__(TK_THREADS) topk_hist_kernel(const TopkParams p) {
     __shared__ unsigned sh[TK_BINS];
     const int item = blockIdx.y, b = item / p.Hi, hi = item % p.Hi, tid = threadIdx.x;
+    if (p.pdl) {
+        asm volatile("griddepcontrol.wait;\n" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+    }
     const int N = max(0, min(p.ctx_lens[b], p.max_ctx));
     if (min(p.k, N) == N) return;                      // everything is kept: no ranking needed
     const int s0 = blockIdx.x * TK_SLICE;
@@ -198,6 +203,11 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
 
     const int item = blockIdx.y, b = item / p.Hi, hi = item % p.Hi, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
+    if (p.pdl) {
+        // resident early, but nothing is read before the kernel that produced scores and histogram is done
+        asm volatile("griddepcontrol.wait;\n" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+    }
     const int N = max(0, min(p.ctx_lens[b], p.max_ctx));
     const int kk = min(p.k, N);
     int* out = p.idx + (long long)item * p.k;
