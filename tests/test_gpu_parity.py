@@ -338,3 +338,29 @@ def test_budget_equal_to_a_long_context_keeps_everything(td):
     sp = td.sparse_attn(lay, q, idx, cnt)
     torch.cuda.synchronize()
     assert torch.allclose(sp, out, rtol=0, atol=2e-4)       # sparse over everything is full attention
+
+
+def test_sixty_four_layer_schedule_matches_the_oracle_step(td):
+    """The 64-layer composition of Section 4.3 (2 full + 2 selection + 60 sparse layers, selection at
+    layers 2 and 13) as one tidal_decode_step call against the oracle's own step driver."""
+    L = 64
+    sched = synth.schedule(L, 13)
+    assert (sched.count(0), sched.count(1), sched.count(2)) == (2, 2, 60)
+    w = synth.Workload("l64", 1, 8, 2, L, 320, 40, 8, sched, synth.BASE_SEED + 64)
+    qs = [synth.make_q(w, i, DEV) for i in range(L)]
+    layers = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(L)]
+    outs, idx, cnt = td.decode_step(sched, layers, qs, w.k)
+    ref_outs, ref_idx, ref_cnt = oracle.decode_step(sched, [util.oracle_kv(l) for l in layers],
+                                                    [synth.bits(q) for q in qs], w.k)
+    # with well separated scores the selected sets agree exactly and every layer can be compared directly
+    assert np.array_equal(cnt.cpu().numpy(), ref_cnt)
+    if np.array_equal(idx.cpu().numpy(), ref_idx):
+        for i in range(L):
+            util.check_out(outs[i].cpu().numpy(), ref_outs[i], f"l64.layer{i}")
+    else:       # a legal swap inside the tie band at the last selection layer: compare on the GPU's sets
+        for i in (0, 1, 2, 13):
+            util.check_out(outs[i].cpu().numpy(), ref_outs[i], f"l64.layer{i}")
+        for i in range(14, L):
+            ref = oracle.sparse_attn(util.oracle_kv(layers[i]), synth.bits(qs[i]), idx.cpu().numpy(), cnt.cpu().numpy())
+            util.check_out(outs[i].cpu().numpy(), ref, f"l64.layer{i}")
+    assert td.launch_count() > 0 and td.device_status() == binding.OK
