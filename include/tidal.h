@@ -95,6 +95,17 @@ tidal_status_t tidal_destroy(tidal_ctx_t *ctx);
  * partial results, the score buffer of a selection layer, top-k histograms). */
 size_t tidal_workspace_bytes(const tidal_kv_t *kv, int32_t k);
 
+/* C.append(k, v) of Algorithm 1 for one layer: writes the new token's key and value rows
+ * (k_new, v_new: device bf16 [batch, num_kv_heads, head_dim], contiguous, 16-byte aligned) into
+ * the cache at position ctx_lens[b] - 1, the slot that the lengths already count, through the
+ * layout described by `kv` (contiguous or paged). The cache memory behind kv->k / kv->v is
+ * WRITTEN by this call although the descriptor declares it const. Sequences with
+ * ctx_lens[b] < 1 or > max_ctx_len and page ids outside the pool are skipped (the latter is
+ * reported by tidal_device_status). q and k are expected position-encoded already: rotary or
+ * other position encodings are the caller's. */
+tidal_status_t tidal_kv_append(tidal_ctx_t *ctx, const tidal_kv_t *kv, const void *k_new,
+                               const void *v_new, void *stream);
+
 /* FullAttention(q, C[:]) of Algorithm 1, Eq. 1 per head:
  *   out[b,h,:] = softmax_j(q[b,h,:] . K[b,j,g,:] * sm_scale) V[b,j,g,:],  j < ctx_lens[b], g = h / (Hq/Hkv).
  * The single decode query sees every cached token (no mask). */

@@ -72,6 +72,8 @@ def lib():
         L.oracle_sparse_attn.restype = I
         L.oracle_decode_step.argtypes = [I, P, C.POINTER(_KV), C.POINTER(P), C.POINTER(P), I, I, P, P]
         L.oracle_decode_step.restype = I
+        L.oracle_kv_append.argtypes = [C.POINTER(_KV), P, P]
+        L.oracle_kv_append.restype = None
         L.oracle_schedule.argtypes = [I, I, P]
         L.oracle_schedule.restype = None
         L.oracle_num_threads.restype = I
@@ -197,6 +199,13 @@ def sparse_attn(kv: KV, q: np.ndarray, idx: np.ndarray, idx_count: Optional[np.n
     if rc:
         raise ValueError("oracle_sparse_attn: bad arguments")
     return out
+
+
+def kv_append(kv: KV, k_new: np.ndarray, v_new: np.ndarray) -> None:
+    """C.append(k, v): writes the rows [B, Hkv, d] at position ctx_lens[b] - 1 of kv's arrays, in place."""
+    k_new, v_new = _q(k_new), _q(v_new)
+    st = kv.c_struct()
+    lib().oracle_kv_append(C.byref(st), k_new.ctypes.data, v_new.ctypes.data)
 
 
 def schedule(num_layers: int, reselect_layer: int) -> np.ndarray:

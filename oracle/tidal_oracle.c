@@ -208,6 +208,21 @@ int oracle_decode_step(int num_layers, const uint8_t *schedule, const oracle_kv_
     return 0;
 }
 
+void oracle_kv_append(const oracle_kv_t *kv, const uint16_t *k_new, const uint16_t *v_new) {
+    int d = kv->head_dim;
+    for (int b = 0; b < kv->batch; ++b) {
+        int pos = kv->ctx_lens[b] - 1;
+        if (pos < 0) continue;
+        for (int g = 0; g < kv->num_kv_heads; ++g) {
+            uint16_t *kr = (uint16_t *)kv_row(kv, kv->k, b, pos, g);
+            uint16_t *vr = (uint16_t *)kv_row(kv, kv->v, b, pos, g);
+            const uint16_t *ks = k_new + ((int64_t)b * kv->num_kv_heads + g) * d;
+            const uint16_t *vs = v_new + ((int64_t)b * kv->num_kv_heads + g) * d;
+            for (int c = 0; c < d; ++c) { kr[c] = ks[c]; vr[c] = vs[c]; }
+        }
+    }
+}
+
 void oracle_schedule(int num_layers, int reselect_layer, uint8_t *schedule) {
     for (int i = 0; i < num_layers; ++i) {
         if (i < 2) schedule[i] = ORACLE_LAYER_FULL;

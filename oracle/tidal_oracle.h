@@ -104,6 +104,11 @@ int oracle_decode_step(int num_layers, const uint8_t *schedule, const oracle_kv_
                        const uint16_t *const *q_per_layer, float *const *out_per_layer,
                        int k, int num_index_heads, int32_t *idx, int32_t *idx_count);
 
+/* C.append(k, v) of Algorithm 1 for one layer: the new token's key and value rows (bf16
+ * [B, Hkv, d]) are written at position ctx_lens[b] - 1, the slot the lengths already count.
+ * The cache arrays are written through the descriptor's (const) base pointers. */
+void oracle_kv_append(const oracle_kv_t *kv, const uint16_t *k_new, const uint16_t *v_new);
+
 /* Layer schedule of Sections 3 and 4.3: the first two layers full, layer 2 and
  * one middle layer (0-based `reselect_layer`) select, every other layer sparse. */
 void oracle_schedule(int num_layers, int reselect_layer, uint8_t *schedule);

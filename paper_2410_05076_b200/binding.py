@@ -25,7 +25,7 @@ LAYER_FULL, LAYER_SELECT, LAYER_SPARSE = 0, 1, 2
 EXPORTS = [
     "tidal_create", "tidal_destroy", "tidal_workspace_bytes", "tidal_full_attn", "tidal_select_attn",
     "tidal_sparse_attn", "tidal_decode_step", "tidal_decode_step_host", "tidal_device_status",
-    "tidal_launch_count", "tidal_strerror", "tidal_sparse_attn_noalloc",
+    "tidal_launch_count", "tidal_strerror", "tidal_sparse_attn_noalloc", "tidal_kv_append",
 ]
 
 
@@ -72,6 +72,8 @@ def load() -> C.CDLL:
     L.tidal_destroy.restype = I32
     L.tidal_workspace_bytes.argtypes = [KVP, I32]
     L.tidal_workspace_bytes.restype = C.c_size_t
+    L.tidal_kv_append.argtypes = [P, KVP, P, P, P]
+    L.tidal_kv_append.restype = I32
     L.tidal_full_attn.argtypes = [P, KVP, P, P, P]
     L.tidal_full_attn.restype = I32
     L.tidal_select_attn.argtypes = [P, KVP, P, I32, I32, P, P, P, P, P]
@@ -168,6 +170,12 @@ class Tidal:
     def workspace_bytes(layer, k: int) -> int:
         s = kv_struct(layer)
         return load().tidal_workspace_bytes(C.byref(s), k)
+
+    def kv_append(self, layer, k_new: torch.Tensor, v_new: torch.Tensor) -> None:
+        """Write the new token's rows (bf16 [B, Hkv, d]) at position ctx_lens[b] - 1 of the layer's cache."""
+        s = kv_struct(layer)
+        _check(self.lib.tidal_kv_append(self.ctx, C.byref(s), k_new.data_ptr(), v_new.data_ptr(), _stream()),
+               "tidal_kv_append")
 
     def full_attn(self, layer, q: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
         if out is None:

@@ -747,4 +747,40 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
     } while (lo < hi);
 }
 
+// C.append(k, v): one warp per (sequence, KV head) copies the two 256-byte rows of the new token
+// to position ctx_lens[b] - 1 of the cache.
+struct AppendParams {
+    __nv_bfloat16* k;
+    __nv_bfloat16* v;
+    const __nv_bfloat16* k_new;
+    const __nv_bfloat16* v_new;
+    long long stride_b, stride_pos, stride_head, stride_page;
+    const int* page_table;
+    int max_pages, num_pages, paged;
+    const int* ctx_lens;
+    int max_ctx, batch, Hkv;
+    int* status;
+};
+
+__global__ void __launch_bounds__(128) kv_append_kernel(const AppendParams p) {
+    const int pair = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (pair >= p.batch * p.Hkv) return;
+    const int b = pair / p.Hkv, g = pair % p.Hkv;
+    const int pos = p.ctx_lens[b] - 1;
+    if (pos < 0 || pos >= p.max_ctx) return;
+    long long off;
+    if (p.paged) {
+        const int page = p.page_table[(long long)b * p.max_pages + (pos >> 4)];
+        if ((unsigned)page >= (unsigned)p.num_pages) { if (lane == 0) atomicOr(p.status, STATUS_BAD_PAGE); return; }
+        off = (long long)page * p.stride_page + (long long)(pos & 15) * p.stride_pos + (long long)g * p.stride_head;
+    } else {
+        off = (long long)b * p.stride_b + (long long)pos * p.stride_pos + (long long)g * p.stride_head;
+    }
+    const long long src = (long long)pair * HEAD_DIM;
+    // lanes 0-15 move the key row, lanes 16-31 the value row, 16 bytes each
+    const uint4* from = reinterpret_cast<const uint4*>((lane < 16 ? p.k_new : p.v_new) + src) + (lane & 15);
+    uint4* to = reinterpret_cast<uint4*>((lane < 16 ? p.k : p.v) + off) + (lane & 15);
+    *to = __ldg(from);
+}
+
 }  // namespace tidal

@@ -383,6 +383,31 @@ size_t tidal_workspace_bytes(const tidal_kv_t* kv, int32_t k) {
     return ws_bytes_for(kv, k, 0);
 }
 
+tidal_status_t tidal_kv_append(tidal_ctx_t* ctx, const tidal_kv_t* kv, const void* k_new, const void* v_new,
+                               void* stream) {
+    if (!ctx || !k_new || !v_new || (((uintptr_t)k_new | (uintptr_t)v_new) & 15)) return TIDAL_ERR_INVALID;
+    const tidal_status_t rc = check_kv(kv);
+    if (rc != TIDAL_OK) return rc;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    AppendParams a;
+    std::memset(&a, 0, sizeof a);
+    a.k = (__nv_bfloat16*)const_cast<void*>(kv->k);
+    a.v = (__nv_bfloat16*)const_cast<void*>(kv->v);
+    a.k_new = (const __nv_bfloat16*)k_new;
+    a.v_new = (const __nv_bfloat16*)v_new;
+    a.stride_b = kv->stride_b; a.stride_pos = kv->stride_pos; a.stride_head = kv->stride_head;
+    a.stride_page = kv->stride_page;
+    a.page_table = kv->page_table; a.max_pages = kv->max_pages_per_seq; a.num_pages = kv->num_pages;
+    a.paged = kv->kv_layout == TIDAL_KV_PAGED;
+    a.ctx_lens = kv->ctx_lens; a.max_ctx = kv->max_ctx_len;
+    a.batch = kv->batch; a.Hkv = kv->num_kv_heads;
+    a.status = ctx->status;
+    const int pairs = kv->batch * kv->num_kv_heads;
+    kv_append_kernel<<<(pairs + 3) / 4, 128, 0, (cudaStream_t)stream>>>(a);
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+}
+
 tidal_status_t tidal_full_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const void* q, float* out, void* stream) {
     if (!ctx || !q || !out || ((uintptr_t)q & 15)) return TIDAL_ERR_INVALID;
     tidal_status_t rc = check_kv(kv);

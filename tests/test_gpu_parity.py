@@ -364,3 +364,22 @@ def test_sixty_four_layer_schedule_matches_the_oracle_step(td):
             ref = oracle.sparse_attn(util.oracle_kv(layers[i]), synth.bits(qs[i]), idx.cpu().numpy(), cnt.cpu().numpy())
             util.check_out(outs[i].cpu().numpy(), ref, f"l64.layer{i}")
     assert td.launch_count() > 0 and td.device_status() == binding.OK
+
+
+@pytest.mark.parametrize("layout", ["hnd_interleaved", "nhd_separate", "paged"])
+def test_kv_append_writes_the_same_rows_as_the_oracle(td, layout):
+    """C.append of Algorithm 1: the whole cache is bit-identical to the oracle's after the append, and
+    full attention over it matches."""
+    w = wl(3, 8, 2, 333, 32, ragged=True, ctx_min=1)
+    q, lay = build(w, layout)
+    okv = util.oracle_kv(lay)                     # host copy taken BEFORE the append
+    g = torch.Generator(device="cpu").manual_seed(99)
+    kn = torch.randn(w.batch, w.num_kv_heads, w.head_dim, generator=g).to(torch.bfloat16)
+    vn = torch.randn(w.batch, w.num_kv_heads, w.head_dim, generator=g).to(torch.bfloat16)
+    oracle.kv_append(okv, synth.bits(kn), synth.bits(vn))
+    td.kv_append(lay, kn.to(DEV), vn.to(DEV))
+    torch.cuda.synchronize()
+    after = util.oracle_kv(lay)                   # host copy of what the kernel wrote
+    assert np.array_equal(after.k, okv.k) and np.array_equal(after.v, okv.v)
+    util.check_out(td.full_attn(lay, q).cpu().numpy(), oracle.full_attn(okv, synth.bits(q)), "full after append")
+    assert td.device_status() == binding.OK

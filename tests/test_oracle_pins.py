@@ -381,3 +381,66 @@ def test_decode_step_keeps_rho_until_the_next_selection_layer():
     assert np.array_equal(outs[6], oracle.sparse_attn(kvs[6], qs[6], rho4, c4))
     with pytest.raises(ValueError):
         oracle.decode_step([0, 2], kvs[:2], qs[:2], k)
+
+
+# ---- KV append (Algorithm 1, C.append) ------------------------------------
+def test_append_writes_exactly_the_last_counted_row():
+    """Independent numpy slice assignment on the [B, N, Hkv, D] arrays gives the same cache."""
+    B, Hq, Hkv, N = 3, 4, 2, 37
+    lens = [37, 1, 20]
+    q, k, v, kv = make(B, Hq, Hkv, N, 41, lens=lens)
+    r = np.random.default_rng(5)
+    kn, vn = bf16_bits(r.standard_normal((B, Hkv, D))), bf16_bits(r.standard_normal((B, Hkv, D)))
+    k_ref, v_ref = k.copy(), v.copy()
+    for b in range(B):
+        k_ref[b, lens[b] - 1] = kn[b]
+        v_ref[b, lens[b] - 1] = vn[b]
+    oracle.kv_append(kv, kn, vn)
+    assert np.array_equal(kv.k.reshape(k.shape), k_ref)
+    assert np.array_equal(kv.v.reshape(v.shape), v_ref)
+
+
+def test_appended_dominant_key_returns_the_appended_value():
+    """Closed form: a new key that dominates every logit makes Eq. 1 return the new value row."""
+    B, Hq, Hkv, N = 2, 4, 2, 50
+    lens = [50, 13]
+    q, k, v, kv = make(B, Hq, Hkv, N, 43, lens=lens)
+    qv = bf16_val(q)
+    kn = np.zeros((B, Hkv, D))
+    for b in range(B):
+        for g in range(Hkv):
+            kn[b, g] = 40.0 * (qv[b, 2 * g] + qv[b, 2 * g + 1])   # aligned with both heads of the group
+    r = np.random.default_rng(6)
+    kn, vn = bf16_bits(kn), bf16_bits(r.standard_normal((B, Hkv, D)))
+    oracle.kv_append(kv, kn, vn)
+    out = oracle.full_attn(kv, q)
+    for b in range(B):
+        for h in range(Hq):
+            assert np.allclose(out[b, h], bf16_val(vn)[b, h // 2], atol=1e-6)
+
+
+def test_append_through_a_page_table_equals_contiguous_append():
+    B, Hq, Hkv, N, PS = 2, 2, 2, 40, 16
+    lens = [40, 17]
+    q, k, v, kv = make(B, Hq, Hkv, N, 47, lens=lens)
+    r = np.random.default_rng(7)
+    pages_per_seq = (N + PS - 1) // PS
+    perm = r.permutation(B * pages_per_seq + 3)[: B * pages_per_seq].reshape(B, pages_per_seq)
+    pool_k = np.zeros((B * pages_per_seq + 3, PS, Hkv, D), np.uint16)
+    pool_v = np.zeros_like(pool_k)
+    for b in range(B):
+        for p in range(pages_per_seq):
+            n = min(PS, N - p * PS)
+            pool_k[perm[b, p], :n] = k[b, p * PS: p * PS + n]
+            pool_v[perm[b, p], :n] = v[b, p * PS: p * PS + n]
+    pkv = oracle.KV(k=pool_k.reshape(-1), v=pool_v.reshape(-1), batch=B, num_q_heads=Hq, num_kv_heads=Hkv,
+                    head_dim=D, ctx_lens=np.asarray(lens, np.int32), stride_pos=Hkv * D, stride_head=D,
+                    stride_page=PS * Hkv * D, page_table=perm.astype(np.int32), page_size=PS,
+                    max_pages_per_seq=pages_per_seq)
+    kn, vn = bf16_bits(r.standard_normal((B, Hkv, D))), bf16_bits(r.standard_normal((B, Hkv, D)))
+    oracle.kv_append(kv, kn, vn)
+    oracle.kv_append(pkv, kn, vn)
+    assert np.array_equal(oracle.full_attn(kv, q), oracle.full_attn(pkv, q))
+    for b in range(B):
+        pos = lens[b] - 1
+        assert np.array_equal(pkv.k.reshape(pool_k.shape)[perm[b, pos // PS], pos % PS], kn[b])
