@@ -48,7 +48,8 @@ constexpr int TILE_BYTES = TILE * HEAD_DIM * 2;   // 4 KB of K, same of V
 constexpr int STAGE_BYTES = 2 * TILE_BYTES;
 constexpr int HIST_BINS = 2048;          // global histogram row: up to 11 top bits of the score key
 constexpr int HIST_SMEM_WORDS = 8192;    // shared histogram: columns x bins <= 8192 counters (32 KB)
-constexpr int FIRST_TILES = 4;           // tiles of a warp's fixed first chunk (known before any pool access)
+constexpr int FIRST_TILES = 5;           // tiles of a warp's fixed first chunk (known before any pool access):
+                                         // a three-slot ring filled before the wait plus a lookahead of two
 constexpr int GRAB_TILES = 4;            // tiles a warp takes from its item's pool at a time afterwards
 
 struct AttnParams {
@@ -543,7 +544,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         // belong to the kernels before us and are touched only after the wait.
         int issued = 0, commits = 0;
         if (!waited) {
-            while (commits < STAGES - 1 && tA >= 0 && tA < tiles_b - 1) {
+            while (commits < STAGES && tA >= 0 && tA < tiles_b - 1) {
                 issue(issued % STAGES);
                 ++issued;
                 cp_async_commit();
@@ -571,6 +572,9 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         }
 
 
+        // Before the grid dependency was resolved the whole ring may have been filled (one slot more
+        // than the loop keeps in flight): the first iteration then has no free slot and issues nothing.
+        const bool ring_full = commits == STAGES;
         while (commits < STAGES - 1) {
             if (tA >= 0) { issue(issued % STAGES); ++issued; }
             cp_async_commit();
@@ -578,11 +582,16 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         }
         TIDAL_TRACE(2);
         for (int it = 0; it < issued; ++it) {
-            cp_async_wait<STAGES - 2>();      // tile `it` has landed (this lane's copies)
-            __syncwarp();
-            if (it == 0) { TIDAL_TRACE(3); }                     // ... and every other lane's; slot (it-1)%STAGES is free
-            if (tA >= 0) { issue((it + STAGES - 1) % STAGES); ++issued; }
-            cp_async_commit();
+            if (it == 0 && ring_full) {
+                cp_async_wait<STAGES - 1>();
+                __syncwarp();
+            } else {
+                cp_async_wait<STAGES - 2>();      // tile `it` has landed (this lane's copies)
+                __syncwarp();                     // ... and every other lane's; slot (it-1)%STAGES is free
+                if (tA >= 0) { issue((it + STAGES - 1) % STAGES); ++issued; }
+                cp_async_commit();
+            }
+            if (it == 0) { TIDAL_TRACE(3); }
             const int stage = it % STAGES;
             const uint32_t ks = wbase_u32 + stage * STAGE_BYTES;
             consume_tile<MODE>(p, ks, ks + TILE_BYTES, qf, acc, s_vmask[warp][stage], gid, tig,
