@@ -133,7 +133,7 @@ def physical_gpu_index(local: int) -> int:
     return local
 
 
-def oracle_sample(w: synth.Workload, qs, layers, host_cache=None):
+def oracle_sample(w: synth.Workload, qs, layers, host_cache=None, index_heads=None):
     """Time the CPU oracle, as it stands, on one layer of each type and scale by the layer mix.
     Only the oracle calls are timed; the host copies of the sampled layers may be cached by the caller."""
     import oracle
@@ -153,11 +153,11 @@ def oracle_sample(w: synth.Workload, qs, layers, host_cache=None):
         if t == 0:
             oracle.full_attn(okv, qb)
         elif t == 1:
-            _, idx, cnt = oracle.select_attn(okv, qb, w.k)
+            _, idx, cnt = oracle.select_attn(okv, qb, w.k, index_heads)
             rho = (idx, cnt)
         else:
             if rho is None:
-                _, idx, cnt = oracle.select_attn(okv, qb, w.k)
+                _, idx, cnt = oracle.select_attn(okv, qb, w.k, index_heads)
                 rho = (idx, cnt)
                 t0 = time.perf_counter()
             oracle.sparse_attn(okv, qb, rho[0], rho[1])
@@ -184,7 +184,7 @@ def run_reference(args, w, rank):
                   for i in need}
     vals, cache = [], {}
     for it in range(args.warmup + args.steps):
-        us, cores, sample, _ = oracle_sample(w, qs, layers, cache)
+        us, cores, sample, _ = oracle_sample(w, qs, layers, cache, index_heads={'qhead': w.num_q_heads, 'kvhead': w.num_kv_heads, 'shared': 1}[args.granularity])
         if it >= args.warmup:
             vals.append(us)
     v = sum(vals) / len(vals)
@@ -280,6 +280,9 @@ def main():
     ap.add_argument("--impl", default="tidal", choices=["tidal", "reference"])
     ap.add_argument("--workload", default="cfg3")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--granularity", default="qhead", choices=["qhead", "kvhead", "shared"],
+                    help="one token set per query head (default), per KV head, or shared by all heads "
+                         "(the latter two rank by the sum of the member heads' scaled logits)")
     ap.add_argument("--sweep", action="store_true",
                     help="context x budget sweep (Llama-3-8B head shapes, one selection + one sparse layer): "
                          "prints one JSON line with the selection-layer and sparse-layer cost of every point")
@@ -324,7 +327,11 @@ def main():
         return
     qs, layers = build_workload(w, dev)
     outs = [torch.empty(w.batch, w.num_q_heads, w.head_dim, dtype=torch.float32, device=dev) for _ in layers]
-    step = td.make_step(w.sched, layers, qs, outs, w.k)
+    gran = {"qhead": binding.SEL_PER_QHEAD, "kvhead": binding.SEL_PER_KVHEAD, "shared": binding.SEL_SHARED}[args.granularity]
+    index_heads = {"qhead": w.num_q_heads, "kvhead": w.num_kv_heads, "shared": 1}[args.granularity]
+    # rows a sparse layer gathers: one list per index head, read once per KV head it serves
+    gather_lists = w.num_q_heads if args.granularity == "qhead" else w.num_kv_heads
+    step = td.make_step(w.sched, layers, qs, outs, w.k, gran)
     kv_bytes = [l.kv_bytes() for l in layers]
 
     # ---- device-resident timing: the headline value -------------------------------------------
@@ -360,7 +367,7 @@ def main():
             if tkind == synth.LAYER_FULL:
                 td.full_attn(layers[i], qs[i], out=outs[i])
             elif tkind == synth.LAYER_SELECT:
-                td.select_attn(layers[i], qs[i], w.k, out=outs[i], idx=idx, idx_count=cnt)
+                td.select_attn(layers[i], qs[i], w.k, gran, out=outs[i], idx=idx, idx_count=cnt)
             else:
                 td.sparse_attn(layers[i], qs[i], idx, cnt, out=outs[i])
             evs[r][i + 1].record()
@@ -375,7 +382,7 @@ def main():
     dense_us = layer_us[0] if layer_us[0] else layer_us[1]
     peak, peak_kind = measured_peak_gbs()
     achieved = dense_bytes / (dense_us * 1e-6) / 1e9
-    sparse_bytes = w.batch * w.num_q_heads * min(w.k, w.ctx) * (512 + 4)
+    sparse_bytes = w.batch * gather_lists * min(w.k, w.ctx) * 512 + w.batch * index_heads * min(w.k, w.ctx) * 4
     roofline = {"bound": "hbm", "kernel": "attn_kernel<FULL> (full-attention layers; the selection layers run the same loop)",
                 "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                 "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
@@ -394,7 +401,7 @@ def main():
     # ---- the same layers in situ: sub-schedules run through tidal_decode_step (no host gaps between
     # launches, programmatic dependent launch active), differences of CUDA-event times ------------------
     def time_schedule(ids, kinds):
-        st = td.make_step(kinds, [layers[i] for i in ids], [qs[i] for i in ids], [outs[i] for i in ids], w.k)
+        st = td.make_step(kinds, [layers[i] for i in ids], [qs[i] for i in ids], [outs[i] for i in ids], w.k, gran)
         for _ in range(3):
             st()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -437,7 +444,7 @@ def main():
     # ---- end to end through the host-buffer entry point ----------------------------------------------
     q_host = torch.stack([q.cpu() for q in qs]).contiguous().pin_memory()
     out_host = torch.empty(w.num_layers, w.batch, w.num_q_heads, w.head_dim, dtype=torch.float32).pin_memory()
-    step_host = td.make_step_host(w.sched, layers, q_host, out_host, w.k)
+    step_host = td.make_step_host(w.sched, layers, q_host, out_host, w.k, gran)
     for _ in range(args.warmup):
         step_host()
     barrier()
@@ -452,7 +459,7 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        us, cores, sample, _ = oracle_sample(w, qs, layers)
+        us, cores, sample, _ = oracle_sample(w, qs, layers, index_heads=index_heads)
         cpu = {"value": us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample}
 
     if rank == 0:
@@ -460,7 +467,7 @@ def main():
             "metric": METRIC, "value": whole_job_us_per_step(ms_step, world), "unit": "us", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": describe(w), "replicas": world,
+            "config": {"workload": describe(w), "replicas": world, "granularity": args.granularity,
                        "l2": "every layer has its own KV cache (16 GiB per step at cfg3), far larger than L2",
                        "step_bytes": step_bytes,
                        "step_frac_of_8TBs": step_bytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS},

@@ -79,6 +79,9 @@ def workload(name: str) -> Workload:
     if name == "cfg4":    # batched paged decode, ragged lengths
         return Workload(name, 8, 32, 8, 32, 65536, 2048, 64, schedule(32, 13), BASE_SEED + 4,
                         paged=True, ragged=True, ctx_min=8192)
+    if name == "cfg64":   # the 64-layer variant of Section 4.3 (2 + 2 + 60): Llama-3-70B attention shapes, GQA group 8,
+        #                   32K context (the longest the paper runs that model at), re-selection at layer 31
+        return Workload(name, 1, 64, 8, 64, 32768, 2048, 64, schedule(64, 31), BASE_SEED + 6)
     raise KeyError(name)
 
 

@@ -75,6 +75,14 @@ def test_config4_paged_ragged_batch(td):
     select_then_sparse(td, w, 2, 3)
 
 
+def test_sixty_four_layer_variant_group_of_eight(td):
+    """The 64-layer variant of Section 4.3 at Llama-3-70B attention shapes: its re-selection layer and the
+    sparse layer after it."""
+    w = synth.workload("cfg64")
+    assert w.sched.count(0) == 2 and w.sched.count(1) == 2 and w.sched.count(2) == 60 and w.sched[31] == 1
+    select_then_sparse(td, w, 31, 32)
+
+
 @pytest.mark.parametrize("ctx,k", [(262144, 8192), (65536, 512), (4096, 8192), (16384, 1024)])
 def test_config5_sweep_points(td, ctx, k):
     w = synth.sweep_point(ctx, min(k, ctx))      # the API takes k <= max_ctx_len; k' = min(k, N)
