@@ -67,7 +67,8 @@ struct AttnParams {
     int batch;
     int splits_per_item;       // > 0: pooled mode, CTA c works on item c % items; an item is served by every CTA
                                // of the grid that maps to it (this many, or one more); 0: static flat split
-    float* scores;             // MODE_SELECT: [B, Hq, score_stride]
+    float* scores;             // MODE_SELECT: [B, Hq, score_stride], or [B, Hkv, score_stride] with agg
+    int agg;                   // MODE_SELECT: store one row per KV head, the sum of its group's scaled logits
     long long score_stride;
     const int* idx;            // MODE_SPARSE: [B, Hi, k]
     const int* idx_count;      // MODE_SPARSE: [B] or null
@@ -211,6 +212,23 @@ __device__ __forceinline__ void consume_tile(const AttnParams& p, uint32_t ks, u
     if (MODE == MODE_SELECT) {
         // s[0],s[1]: (pos gid; heads 2tig, 2tig+1)   s[2],s[3]: (pos gid+8; same heads)
         const float f0 = s[0] * p.scale, f1 = s[1] * p.scale, f2 = s[2] * p.scale, f3 = s[3] * p.scale;
+        if (p.agg) {
+            // One ranking score per (position, KV head): the group's columns summed (unused columns
+            // hold zeros). Lanes that differ only in tig hold the columns of one position.
+            float a0 = f0 + f1, a1 = f2 + f3;
+            a0 += __shfl_xor_sync(0xffffffffu, a0, 1);
+            a1 += __shfl_xor_sync(0xffffffffu, a1, 1);
+            a0 += __shfl_xor_sync(0xffffffffu, a0, 2);
+            a1 += __shfl_xor_sync(0xffffffffu, a1, 2);
+            if (tig == 0) {
+                if (v0) score_row0[pos_base + gid] = a0;
+                if (v1) score_row0[pos_base + gid + 8] = a1;
+                if (hist) {
+                    if (v0) atomicAdd(hist + (score_key_bits(a0) >> p.hist_shift), 1u);
+                    if (v1) atomicAdd(hist + (score_key_bits(a1) >> p.hist_shift), 1u);
+                }
+            }
+        } else {
         if (score_row0) {
             if (v0) score_row0[pos_base + gid] = f0;
             if (v1) score_row0[pos_base + gid + 8] = f2;
@@ -231,6 +249,7 @@ __device__ __forceinline__ void consume_tile(const AttnParams& p, uint32_t ks, u
                 if (v0) atomicAdd(h1 + (score_key_bits(f1) >> p.hist_shift), 1u);
                 if (v1) atomicAdd(h1 + (score_key_bits(f3) >> p.hist_shift), 1u);
             }
+        }
         }
     }
     // ---- running softmax (base 2) ---------------------------------------------
@@ -387,7 +406,9 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
 
         float* score_row0 = nullptr;
         float* score_row1 = nullptr;
-        if (MODE == MODE_SELECT) {
+        if (MODE == MODE_SELECT && p.agg) {
+            score_row0 = p.scores + ((long long)b * p.Hkv + g) * p.score_stride;
+        } else if (MODE == MODE_SELECT) {
             if (2 * tig < ncols) score_row0 = p.scores + ((long long)b * p.Hq + head0 + 2 * tig) * p.score_stride;
             if (2 * tig + 1 < ncols) score_row1 = p.scores + ((long long)b * p.Hq + head0 + 2 * tig + 1) * p.score_stride;
         }
@@ -604,10 +625,11 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         if (hist_on) {                        // add this segment's histogram to the global one
             __syncthreads();
             const int nb = 1 << (32 - p.hist_shift);
-            for (int i = threadIdx.x; i < ncols * nb; i += NW * 32) {
+            const long long hrow0 = p.agg ? (long long)b * p.Hkv + g : (long long)b * p.Hq + head0;
+            for (int i = threadIdx.x; i < (p.agg ? 1 : ncols) * nb; i += NW * 32) {
                 const uint32_t w = hist[i];
                 if (w) {
-                    atomicAdd(p.hist + ((long long)b * p.Hq + head0 + i / nb) * HIST_BINS + (i % nb), w);
+                    atomicAdd(p.hist + (hrow0 + i / nb) * HIST_BINS + (i % nb), w);
                     hist[i] = 0;
                 }
             }

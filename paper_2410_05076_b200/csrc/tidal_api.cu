@@ -238,9 +238,23 @@ tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, cudaStream_t
     return cudaLaunchKernelEx(&cfg, attn_kernel<MODE, NW, STAGES>, a) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }
 
+// How a selection layer produces its ranking scores. Per query head: one row per head, histogram
+// fused. Fewer index heads than query heads: the ranking score is the sum of the member heads'
+// scaled logits; unless the caller wants the per-head scores, the attention kernel stores the
+// group sums directly (one row per KV head; histogram fused when a set belongs to one KV head).
+struct SelectPlan { bool agg, fuse; int rows; };
+SelectPlan select_plan(const tidal_kv_t* kv, int Hi, bool caller_scores) {
+    SelectPlan s;
+    s.agg = Hi != kv->num_q_heads && !caller_scores;
+    s.rows = s.agg ? kv->num_kv_heads : kv->num_q_heads;
+    s.fuse = Hi == s.rows;
+    return s;
+}
+
 // hist != nullptr: the kernel also accumulates the per-head histogram the top-k needs.
 tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, float* out, float* scores,
-                         long long score_stride, bool fuse_hist, bool wait_first, const WsLayout& w, cudaStream_t st) {
+                         long long score_stride, bool fuse_hist, bool wait_first, const WsLayout& w, cudaStream_t st,
+                         bool agg = false) {
     AttnParams a;
     fill_common(a, ctx, kv, q, out, w);
     a.wait_first = wait_first;
@@ -251,18 +265,21 @@ tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, fl
     }
     a.scores = scores;
     a.score_stride = score_stride;
+    a.agg = agg ? 1 : 0;
     a.hist = fuse_hist ? state_hist(ctx) : nullptr;
     if (scores) return launch_attn<MODE_SELECT, DENSE_NW, DENSE_STAGES>(ctx, a, grid, st);
     return launch_attn<MODE_FULL, DENSE_NW, DENSE_STAGES>(ctx, a, grid, st);
 }
 
+// `rows`: score rows per sequence (query heads, or KV heads when the attention kernel stored group sums).
 tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* scores, long long score_stride,
-                        int k, int Hi, bool hist_done, int* idx, int* idx_count, const WsLayout& w, cudaStream_t st) {
+                        int k, int rows, int Hi, bool hist_done, int* idx, int* idx_count, const WsLayout& w,
+                        cudaStream_t st) {
     TopkParams t;
     std::memset(&t, 0, sizeof t);
     t.scores = scores; t.score_stride = score_stride;
     t.ctx_lens = kv->ctx_lens; t.max_ctx = kv->max_ctx_len;
-    t.Hq = kv->num_q_heads; t.Hi = Hi; t.k = k;
+    t.Hq = rows; t.Hi = Hi; t.k = k;
     t.idx = idx; t.idx_count = idx_count;
     char* ws = (char*)ctx->ws;
     t.hist = state_hist(ctx);
@@ -433,9 +450,9 @@ tidal_status_t tidal_select_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const v
     float* scores = scores_opt ? scores_opt : (float*)((char*)ctx->ws + w.scores);
     const long long stride = scores_opt ? (long long)kv->max_ctx_len : w.score_stride;
     cudaStream_t st = (cudaStream_t)stream;
-    const bool fuse = Hi == kv->num_q_heads;     // per-head ranking: the attention kernel builds the histogram
-    if ((rc = run_dense(ctx, kv, q, out, scores, stride, fuse, true, w, st)) != TIDAL_OK) return rc;
-    return run_topk(ctx, kv, scores, stride, k, Hi, fuse, idx, idx_count, w, st);
+    const SelectPlan sp = select_plan(kv, Hi, scores_opt != nullptr);
+    if ((rc = run_dense(ctx, kv, q, out, scores, stride, sp.fuse, true, w, st, sp.agg)) != TIDAL_OK) return rc;
+    return run_topk(ctx, kv, scores, stride, k, sp.rows, Hi, sp.fuse, idx, idx_count, w, st);
 }
 
 tidal_status_t tidal_sparse_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const void* q, const int32_t* idx,
@@ -487,9 +504,9 @@ static tidal_status_t decode_step_impl(tidal_ctx_t* ctx, int32_t num_layers, con
             rc = run_dense(ctx, kv, qs[i], outs[i], nullptr, 0, false, i == 0, w, st);
         } else if (schedule[i] == TIDAL_LAYER_SELECT) {
             float* scores = (float*)((char*)ctx->ws + w.scores);
-            const bool fuse = Hi == kv->num_q_heads;
-            rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, fuse, i == 0, w, st);
-            if (rc == TIDAL_OK) rc = run_topk(ctx, kv, scores, w.score_stride, k, Hi, fuse, idx, idx_count, w, st);
+            const SelectPlan sp = select_plan(kv, Hi, false);
+            rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, sp.fuse, i == 0, w, st, sp.agg);
+            if (rc == TIDAL_OK) rc = run_topk(ctx, kv, scores, w.score_stride, k, sp.rows, Hi, sp.fuse, idx, idx_count, w, st);
         } else {
             // the index list is fresh when the previous layer selected it
             rc = run_sparse(ctx, kv, qs[i], idx, idx_count, k, Hi, outs[i], i == 0 || schedule[i - 1] == TIDAL_LAYER_SELECT, w, st);

@@ -75,6 +75,29 @@ def test_config4_paged_ragged_batch(td):
     select_then_sparse(td, w, 2, 3)
 
 
+@pytest.mark.parametrize("gran,hi", [(binding.SEL_PER_KVHEAD, 8), (binding.SEL_SHARED, 1)])
+def test_config3_with_one_set_per_kv_head_or_one_shared_set(td, gran, hi):
+    """128K selection layer ranking by the summed logits of a KV head's group (or of all heads), then a sparse
+    layer over those sets, against the oracle."""
+    w = synth.workload("cfg3")
+    q = synth.make_q(w, 2, DEV)
+    lay = synth.make_layer(w, 2, DEV, q=q)
+    out, idx, cnt = td.select_attn(lay, q, w.k, granularity=gran)
+    sp = td.sparse_attn(lay, q, idx, cnt)
+    torch.cuda.synchronize()
+    okv, qb = util.oracle_kv(lay), synth.bits(q)
+    ref, sc = oracle.full_attn(okv, qb, want_scores=True)
+    util.check_out(out.cpu().numpy(), ref, "select")
+    idx_h, cnt_h = idx.cpu().numpy(), cnt.cpu().numpy()
+    assert idx_h.shape == (1, hi, w.k) and cnt_h.tolist() == [w.k]
+    members = w.num_q_heads // hi
+    for h in range(hi):
+        agg = sc[0, h * members:(h + 1) * members].astype(np.float64).sum(0).astype(np.float32)
+        assert util.check_idx_row(idx_h[0, h], agg, w.k, w.ctx, f"idx[{h}]") <= 64
+    util.check_out(sp.cpu().numpy(), oracle.sparse_attn(okv, qb, idx_h, cnt_h), "sparse")
+    assert td.device_status() == binding.OK
+
+
 def test_sixty_four_layer_variant_group_of_eight(td):
     """The 64-layer variant of Section 4.3 at Llama-3-70B attention shapes: its re-selection layer and the
     sparse layer after it."""

@@ -127,17 +127,25 @@ def test_aggregated_granularities(td, gran, hi_of):
     q, lay = build(w, "hnd_interleaved")
     okv, qb = util.oracle_kv(lay), synth.bits(q)
     Hi = hi_of(w)
-    out, idx, cnt = td.select_attn(lay, q, w.k, granularity=gran)
     ref_out, ref_idx, ref_cnt, ref_sc = oracle.select_attn(okv, qb, w.k, Hi, want_scores=True)
-    util.check_out(out.cpu().numpy(), ref_out, "agg.out")
     lens = lay.ctx_lens.cpu().numpy()
     members = w.num_q_heads // Hi
-    idx_h = idx.cpu().numpy()
-    for b in range(w.batch):
-        n = int(lens[b])
-        for hi in range(Hi):
-            agg = ref_sc[b, hi * members:(hi + 1) * members, :n].astype(np.float64).sum(0).astype(np.float32)
-            util.check_idx_row(idx_h[b, hi], agg, w.k, n, f"agg.idx[{b},{hi}]")
+    # without a score buffer the attention kernel stores the group sums itself; with one it stores the
+    # per-head scores and the top-k sums them: both must give the oracle's sets
+    for scores in (None, torch.full((w.batch, w.num_q_heads, w.ctx), float("nan"), dtype=torch.float32, device=DEV)):
+        out, idx, cnt = td.select_attn(lay, q, w.k, granularity=gran, scores=scores)
+        util.check_out(out.cpu().numpy(), ref_out, "agg.out")
+        idx_h = idx.cpu().numpy()
+        assert cnt.cpu().numpy().tolist() == ref_cnt.tolist()
+        for b in range(w.batch):
+            n = int(lens[b])
+            for hi in range(Hi):
+                agg = ref_sc[b, hi * members:(hi + 1) * members, :n].astype(np.float64).sum(0).astype(np.float32)
+                util.check_idx_row(idx_h[b, hi], agg, w.k, n, f"agg.idx[{b},{hi}]")
+        if scores is not None:
+            for b in range(w.batch):
+                n = int(lens[b])
+                assert np.abs(scores[b, :, :n].cpu().numpy() - ref_sc[b, :, :n]).max() <= 1e-4
     sp = td.sparse_attn(lay, q, torch.from_numpy(ref_idx).to(DEV), torch.from_numpy(ref_cnt).to(DEV))
     util.check_out(sp.cpu().numpy(), oracle.sparse_attn(okv, qb, ref_idx, ref_cnt), "agg.sparse")
 
