@@ -391,3 +391,29 @@ def test_kv_append_writes_the_same_rows_as_the_oracle(td, layout):
     assert np.array_equal(after.k, okv.k) and np.array_equal(after.v, okv.v)
     util.check_out(td.full_attn(lay, q).cpu().numpy(), oracle.full_attn(okv, synth.bits(q)), "full after append")
     assert td.device_status() == binding.OK
+
+
+@pytest.mark.parametrize("layout", ["hnd_interleaved", "paged"])
+def test_batch_with_an_empty_and_a_one_token_sequence(td, layout):
+    """Degenerate lengths inside a batch: an empty cache gives a zero output row, no indices and a count
+    of 0; a one-token cache returns v_0; the other sequences are unaffected."""
+    w = wl(4, 8, 2, 200, 24, ragged=False, seed=11)
+    q, lay = build(w, layout)
+    lay.ctx_lens = torch.tensor([200, 0, 1, 77], dtype=torch.int32, device=DEV)
+    okv, qb = util.oracle_kv(lay), synth.bits(q)
+    ref_out, ref_idx, ref_cnt, ref_sc = oracle.select_attn(okv, qb, w.k, want_scores=True)
+    assert ref_cnt.tolist() == [24, 0, 1, 24] and (ref_out[1] == 0).all()
+    util.check_out(td.full_attn(lay, q).cpu().numpy(), ref_out, "full")
+    out, idx, cnt = td.select_attn(lay, q, w.k)
+    util.check_out(out.cpu().numpy(), ref_out, "select")
+    assert (out.cpu().numpy()[1] == 0).all()
+    assert cnt.cpu().numpy().tolist() == ref_cnt.tolist()
+    idx_h = idx.cpu().numpy()
+    assert (idx_h[1] == -1).all() and (idx_h[2, :, 0] == 0).all() and (idx_h[2, :, 1:] == -1).all()
+    for b in (0, 3):
+        for h in range(w.num_q_heads):
+            util.check_idx_row(idx_h[b, h], ref_sc[b, h], w.k, int(lay.ctx_lens[b]), f"idx[{b},{h}]")
+    sp = td.sparse_attn(lay, q, idx, cnt)
+    util.check_out(sp.cpu().numpy(), oracle.sparse_attn(okv, qb, idx_h, cnt.cpu().numpy()), "sparse")
+    assert (sp.cpu().numpy()[1] == 0).all()
+    assert td.device_status() == binding.OK
