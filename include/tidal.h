@@ -149,6 +149,19 @@ tidal_status_t tidal_decode_step(tidal_ctx_t *ctx, int32_t num_layers, const uin
                                  float *const *out_per_layer, int32_t k, int32_t granularity,
                                  int32_t *idx, int32_t *idx_count, void *stream);
 
+/* The step of Algorithm 1 including its cache update: layer i's new key and value rows
+ * (k_new_per_layer[i], v_new_per_layer[i]: device bf16 [batch, Hkv, head_dim], as for
+ * tidal_kv_append) are written at position ctx_lens[b] - 1 of layer i's cache, then the layers
+ * run as in tidal_decode_step. All layers' rows are written by one launch ahead of the first
+ * layer, which is equivalent because every layer's inputs are given up front. The caches are
+ * WRITTEN although the descriptors declare them const. */
+tidal_status_t tidal_decode_step_append(tidal_ctx_t *ctx, int32_t num_layers, const uint8_t *schedule,
+                                        const tidal_kv_t *kv_per_layer, const void *const *q_per_layer,
+                                        const void *const *k_new_per_layer,
+                                        const void *const *v_new_per_layer, float *const *out_per_layer,
+                                        int32_t k, int32_t granularity, int32_t *idx,
+                                        int32_t *idx_count, void *stream);
+
 /* The same step for a caller whose queries and outputs live in HOST memory
  * (pinned for full speed): q_host is bf16 [num_layers, batch, Hq, head_dim],
  * out_host fp32 of the same shape. Copies q to the device, runs

@@ -26,6 +26,7 @@ EXPORTS = [
     "tidal_create", "tidal_destroy", "tidal_workspace_bytes", "tidal_full_attn", "tidal_select_attn",
     "tidal_sparse_attn", "tidal_decode_step", "tidal_decode_step_host", "tidal_device_status",
     "tidal_launch_count", "tidal_strerror", "tidal_sparse_attn_noalloc", "tidal_kv_append",
+    "tidal_decode_step_append",
 ]
 
 
@@ -72,6 +73,8 @@ def load() -> C.CDLL:
     L.tidal_destroy.restype = I32
     L.tidal_workspace_bytes.argtypes = [KVP, I32]
     L.tidal_workspace_bytes.restype = C.c_size_t
+    L.tidal_decode_step_append.argtypes = [P, I32, P, KVP, P, P, P, P, I32, I32, P, P, P]
+    L.tidal_decode_step_append.restype = I32
     L.tidal_kv_append.argtypes = [P, KVP, P, P, P]
     L.tidal_kv_append.restype = I32
     L.tidal_full_attn.argtypes = [P, KVP, P, P, P]
@@ -233,6 +236,22 @@ class Tidal:
 
         step.idx, step.idx_count, step.keep = idx, cnt, keep
         return step
+
+    def decode_step_append(self, sched, layers, qs, k_new, v_new, k: int, granularity: int = SEL_PER_QHEAD):
+        """One step including the cache update: k_new[i], v_new[i] (bf16 [B, Hkv, d]) go to position
+        ctx_lens[b] - 1 of layer i's cache before the layers run. Returns (outs, idx, idx_count)."""
+        L = len(sched)
+        outs = [torch.empty(l.batch, l.num_q_heads, l.head_dim, dtype=torch.float32, device=qs[0].device)
+                for l in layers]
+        hi = {SEL_PER_QHEAD: layers[0].num_q_heads, SEL_PER_KVHEAD: layers[0].num_kv_heads, SEL_SHARED: 1}[granularity]
+        idx = torch.full((layers[0].batch, hi, k), -1, dtype=torch.int32, device=qs[0].device)
+        cnt = torch.zeros(layers[0].batch, dtype=torch.int32, device=qs[0].device)
+        ptrs = lambda ts: (C.c_void_p * L)(*[t.data_ptr() for t in ts])
+        _check(self.lib.tidal_decode_step_append(
+            self.ctx, L, (C.c_uint8 * L)(*sched), (tidal_kv_t * L)(*[kv_struct(l) for l in layers]), ptrs(qs),
+            ptrs(k_new), ptrs(v_new), ptrs(outs), k, granularity, idx.data_ptr(), cnt.data_ptr(), _stream()),
+            "tidal_decode_step_append")
+        return outs, idx, cnt
 
     def decode_step(self, sched, layers, qs, k: int, granularity: int = SEL_PER_QHEAD):
         outs = [torch.empty(l.batch, l.num_q_heads, l.head_dim, dtype=torch.float32, device=qs[0].device)

@@ -793,7 +793,7 @@ struct AppendParams {
     int* status;
 };
 
-__global__ void __launch_bounds__(128) kv_append_kernel(const AppendParams p) {
+__device__ __forceinline__ void kv_append_rows(const AppendParams& p) {
     const int pair = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (pair >= p.batch * p.Hkv) return;
     const int b = pair / p.Hkv, g = pair % p.Hkv;
@@ -812,6 +812,17 @@ __global__ void __launch_bounds__(128) kv_append_kernel(const AppendParams p) {
     const uint4* from = reinterpret_cast<const uint4*>((lane < 16 ? p.k_new : p.v_new) + src) + (lane & 15);
     uint4* to = reinterpret_cast<uint4*>((lane < 16 ? p.k : p.v) + off) + (lane & 15);
     *to = __ldg(from);
+}
+
+__global__ void __launch_bounds__(128) kv_append_kernel(const AppendParams p) { kv_append_rows(p); }
+
+// The same for several layers in one launch: blockIdx.y picks the layer.
+constexpr int APPEND_MAX_LAYERS = 24;
+struct AppendBatchParams {
+    AppendParams layer[APPEND_MAX_LAYERS];
+};
+__global__ void __launch_bounds__(128) kv_append_layers_kernel(const __grid_constant__ AppendBatchParams p) {
+    kv_append_rows(p.layer[blockIdx.y]);
 }
 
 }  // namespace tidal

@@ -400,6 +400,9 @@ size_t tidal_workspace_bytes(const tidal_kv_t* kv, int32_t k) {
     return ws_bytes_for(kv, k, 0);
 }
 
+static void fill_append(AppendParams& a, const tidal_ctx* ctx, const tidal_kv_t* kv, const void* k_new,
+                        const void* v_new);
+
 tidal_status_t tidal_kv_append(tidal_ctx_t* ctx, const tidal_kv_t* kv, const void* k_new, const void* v_new,
                                void* stream) {
     if (!ctx || !k_new || !v_new || (((uintptr_t)k_new | (uintptr_t)v_new) & 15)) return TIDAL_ERR_INVALID;
@@ -407,6 +410,15 @@ tidal_status_t tidal_kv_append(tidal_ctx_t* ctx, const tidal_kv_t* kv, const voi
     if (rc != TIDAL_OK) return rc;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
     AppendParams a;
+    fill_append(a, ctx, kv, k_new, v_new);
+    const int pairs = kv->batch * kv->num_kv_heads;
+    kv_append_kernel<<<(pairs + 3) / 4, 128, 0, (cudaStream_t)stream>>>(a);
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+}
+
+static void fill_append(AppendParams& a, const tidal_ctx* ctx, const tidal_kv_t* kv, const void* k_new,
+                        const void* v_new) {
     std::memset(&a, 0, sizeof a);
     a.k = (__nv_bfloat16*)const_cast<void*>(kv->k);
     a.v = (__nv_bfloat16*)const_cast<void*>(kv->v);
@@ -419,10 +431,6 @@ tidal_status_t tidal_kv_append(tidal_ctx_t* ctx, const tidal_kv_t* kv, const voi
     a.ctx_lens = kv->ctx_lens; a.max_ctx = kv->max_ctx_len;
     a.batch = kv->batch; a.Hkv = kv->num_kv_heads;
     a.status = ctx->status;
-    const int pairs = kv->batch * kv->num_kv_heads;
-    kv_append_kernel<<<(pairs + 3) / 4, 128, 0, (cudaStream_t)stream>>>(a);
-    ctx->launches++;
-    return cudaGetLastError() == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }
 
 tidal_status_t tidal_full_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const void* q, float* out, void* stream) {
@@ -514,6 +522,37 @@ static tidal_status_t decode_step_impl(tidal_ctx_t* ctx, int32_t num_layers, con
         if (rc != TIDAL_OK) return rc;
     }
     return TIDAL_OK;
+}
+
+tidal_status_t tidal_decode_step_append(tidal_ctx_t* ctx, int32_t num_layers, const uint8_t* schedule,
+                                        const tidal_kv_t* kv_per_layer, const void* const* q_per_layer,
+                                        const void* const* k_new_per_layer, const void* const* v_new_per_layer,
+                                        float* const* out_per_layer, int32_t k, int32_t granularity, int32_t* idx,
+                                        int32_t* idx_count, void* stream) {
+    if (!ctx || num_layers <= 0 || !schedule || !kv_per_layer || !q_per_layer || !out_per_layer || !idx || !idx_count ||
+        !k_new_per_layer || !v_new_per_layer || k <= 0)
+        return TIDAL_ERR_INVALID;
+    for (int i = 0; i < num_layers; ++i) {
+        const tidal_status_t rc = check_kv(&kv_per_layer[i]);
+        if (rc != TIDAL_OK) return rc;
+        if (!k_new_per_layer[i] || !v_new_per_layer[i] ||
+            (((uintptr_t)k_new_per_layer[i] | (uintptr_t)v_new_per_layer[i]) & 15)) return TIDAL_ERR_INVALID;
+        if (kv_per_layer[i].batch != kv_per_layer[0].batch || kv_per_layer[i].num_kv_heads != kv_per_layer[0].num_kv_heads)
+            return TIDAL_ERR_INVALID;
+    }
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    const int pairs = kv_per_layer[0].batch * kv_per_layer[0].num_kv_heads;
+    for (int l0 = 0; l0 < num_layers; l0 += APPEND_MAX_LAYERS) {
+        const int n = std::min(APPEND_MAX_LAYERS, num_layers - l0);
+        AppendBatchParams bp;
+        std::memset(&bp, 0, sizeof bp);
+        for (int j = 0; j < n; ++j) fill_append(bp.layer[j], ctx, &kv_per_layer[l0 + j], k_new_per_layer[l0 + j], v_new_per_layer[l0 + j]);
+        kv_append_layers_kernel<<<dim3((pairs + 3) / 4, n, 1), 128, 0, (cudaStream_t)stream>>>(bp);
+        ctx->launches++;
+        if (cudaGetLastError() != cudaSuccess) return TIDAL_ERR_CUDA;
+    }
+    return tidal_decode_step(ctx, num_layers, schedule, kv_per_layer, q_per_layer, out_per_layer, k, granularity, idx,
+                             idx_count, stream);
 }
 
 tidal_status_t tidal_decode_step(tidal_ctx_t* ctx, int32_t num_layers, const uint8_t* schedule,

@@ -417,3 +417,42 @@ def test_batch_with_an_empty_and_a_one_token_sequence(td, layout):
     util.check_out(sp.cpu().numpy(), oracle.sparse_attn(okv, qb, idx_h, cnt.cpu().numpy()), "sparse")
     assert (sp.cpu().numpy()[1] == 0).all()
     assert td.device_status() == binding.OK
+
+
+def test_decode_step_with_the_cache_update(td):
+    """Algorithm 1's loop with C.append: every layer's new rows are written, then F,S,sp,S,sp run; compared
+    with the oracle appending to host copies of the caches and stepping over them."""
+    sched = [0, 1, 2, 1, 2]
+    w = wl(2, 8, 2, 500, 48, ragged=True, ctx_min=100, seed=21, layers=len(sched))
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    layers = [synth.make_layer(w, i, DEV, layout="nhd_separate" if i % 2 else "hnd_interleaved", q=qs[i])
+              for i in range(len(sched))]
+    g = torch.Generator(device="cpu").manual_seed(5)
+    k_new = [(3.0 * torch.randn(w.batch, w.num_kv_heads, w.head_dim, generator=g)).to(torch.bfloat16) for _ in sched]
+    v_new = [torch.randn(w.batch, w.num_kv_heads, w.head_dim, generator=g).to(torch.bfloat16) for _ in sched]
+    okvs = [util.oracle_kv(l) for l in layers]                     # host copies taken before the update
+    for okv, kn, vn in zip(okvs, k_new, v_new):
+        oracle.kv_append(okv, synth.bits(kn), synth.bits(vn))
+    outs, idx, cnt = td.decode_step_append(sched, layers, qs, [t.to(DEV) for t in k_new], [t.to(DEV) for t in v_new], w.k)
+    torch.cuda.synchronize()
+    for l, okv in zip(layers, okvs):                               # the caches themselves
+        after = util.oracle_kv(l)
+        assert np.array_equal(after.k, okv.k) and np.array_equal(after.v, okv.v)
+    lens = layers[0].ctx_lens.cpu().numpy()
+    cur = None
+    for i, t in enumerate(sched):
+        qb = synth.bits(qs[i])
+        got = outs[i].cpu().numpy()
+        if t in (0, 1):
+            ref, sc = oracle.full_attn(okvs[i], qb, want_scores=True)
+            util.check_out(got, ref, f"layer{i}")
+            if t == 1:
+                _, gi, gc = td.select_attn(layers[i], qs[i], w.k)      # the cache now holds the new rows
+                cur = (gi.cpu().numpy(), gc.cpu().numpy())
+                for b in range(w.batch):
+                    for h in range(w.num_q_heads):
+                        util.check_idx_row(cur[0][b, h], sc[b, h], w.k, int(lens[b]), f"idx{i}")
+        else:
+            util.check_out(got, oracle.sparse_attn(okvs[i], qb, cur[0], cur[1]), f"layer{i}")
+    assert np.array_equal(idx.cpu().numpy(), cur[0])
+    assert td.device_status() == binding.OK
