@@ -48,8 +48,6 @@ constexpr int TILE_BYTES = TILE * HEAD_DIM * 2;   // 4 KB of K, same of V
 constexpr int STAGE_BYTES = 2 * TILE_BYTES;
 constexpr int HIST_BINS = 2048;          // global histogram row: up to 11 top bits of the score key
 constexpr int HIST_SMEM_WORDS = 8192;    // shared histogram: columns x bins <= 8192 counters (32 KB)
-constexpr int FIRST_TILES = 5;           // tiles of a warp's fixed first chunk (known before any pool access):
-                                         // a three-slot ring filled before the wait plus a lookahead of two
 constexpr int GRAB_TILES = 4;            // tiles a warp takes from its item's pool at a time afterwards
 
 struct AttnParams {
@@ -433,6 +431,8 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         // and single-tile requests made the kernels slower, not better balanced.
         // Short items are spread evenly over all the item's warps instead (nothing left for the pool).
         const int item_warps = item_ctas * NW;
+        // (fixed chunk: the ring's slots, all filled before the wait, plus the lookahead of two)
+        constexpr int FIRST_TILES = STAGES + 2;
         const int first_tiles = (tiles_b <= item_warps * FIRST_TILES)
                                     ? max(1, (tiles_b + item_warps - 1) / max(item_warps, 1)) : FIRST_TILES;
         const int pool_base = item_warps * first_tiles;
