@@ -456,3 +456,42 @@ def test_decode_step_with_the_cache_update(td):
             util.check_out(got, oracle.sparse_attn(okvs[i], qb, cur[0], cur[1]), f"layer{i}")
     assert np.array_equal(idx.cpu().numpy(), cur[0])
     assert td.device_status() == binding.OK
+
+
+def _fuzz_cases(n, seed):
+    r = np.random.default_rng(seed)
+    out = []
+    for _ in range(n):
+        hkv = int(r.choice([1, 2, 3, 4, 8]))
+        g = int(r.choice([1, 2, 4, 8]))
+        batch = int(r.integers(1, 5))
+        ctx = int(r.choice([int(r.integers(1, 40)), int(r.integers(40, 700)), int(r.integers(700, 5000))]))
+        k = int(r.integers(1, ctx + 1)) if r.random() < 0.7 else ctx
+        out.append((batch, hkv * g, hkv, ctx, k, bool(r.random() < 0.6), str(r.choice(["hnd_interleaved", "nhd_separate", "paged"])),
+                    int(r.choice([binding.SEL_PER_QHEAD, binding.SEL_PER_KVHEAD, binding.SEL_SHARED]))))
+    return out
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,N,k,ragged,layout,gran", _fuzz_cases(36, 20241005))
+def test_random_shapes_match_the_oracle(td, B, Hq, Hkv, N, k, ragged, layout, gran):
+    """Seeded random shapes: head counts, groups 1-8, batch, context from one token to a few thousand, budget,
+    layout and index granularity all vary; selection and sparse layers against the oracle."""
+    w = wl(B, Hq, Hkv, N, k, planted=min(8, N), ragged=ragged, ctx_min=max(1, N // 4), seed=N + k)
+    q, lay = build(w, layout)
+    okv, qb = util.oracle_kv(lay), synth.bits(q)
+    Hi = {binding.SEL_PER_QHEAD: Hq, binding.SEL_PER_KVHEAD: Hkv, binding.SEL_SHARED: 1}[gran]
+    ref_out, ref_idx, ref_cnt, ref_sc = oracle.select_attn(okv, qb, k, Hi, want_scores=True)
+    out, idx, cnt = td.select_attn(lay, q, k, granularity=gran)
+    util.check_out(out.cpu().numpy(), ref_out, "select")
+    assert cnt.cpu().numpy().tolist() == ref_cnt.tolist()
+    lens = lay.ctx_lens.cpu().numpy()
+    idx_h = idx.cpu().numpy()
+    members = Hq // Hi
+    for b in range(B):
+        n = int(lens[b])
+        for hi in range(Hi):
+            agg = ref_sc[b, hi * members:(hi + 1) * members, :n].astype(np.float64).sum(0).astype(np.float32)
+            util.check_idx_row(idx_h[b, hi], agg, k, n, f"idx[{b},{hi}]")
+    sp = td.sparse_attn(lay, q, idx, cnt)
+    util.check_out(sp.cpu().numpy(), oracle.sparse_attn(okv, qb, idx_h, cnt.cpu().numpy()), "sparse")
+    assert td.device_status() == binding.OK
