@@ -7,7 +7,8 @@
  * full attention that also ranks every cached token by its query-key inner
  * product and keeps the top k (token selection layers), and sparse attention
  * over only the positions kept by the last selection layer (all other
- * layers). Projections, FFN and the KV append are the caller's.
+ * layers), and the cache update (the new token's key and value rows written
+ * into the cache). Projections, position encodings and FFN are the caller's.
  *
  * Conventions shared by every call
  *   - All tensor pointers are DEVICE pointers unless a parameter says "host".
@@ -121,7 +122,8 @@ tidal_status_t tidal_full_attn(tidal_ctx_t *ctx, const tidal_kv_t *kv, const voi
  *   idx_count int32 [batch] or NULL: receives k'.
  *   scores_opt float [batch, Hq, max_ctx_len] or NULL: receives the scaled
  *             logits q.k*sm_scale (entries at and beyond ctx_lens[b] are unspecified);
- *             with NULL they live in the workspace. */
+ *             with NULL they live in the workspace (with fewer index heads than
+ *             query heads the workspace then holds only the per-KV-head sums). */
 tidal_status_t tidal_select_attn(tidal_ctx_t *ctx, const tidal_kv_t *kv, const void *q,
                                  int32_t k, int32_t granularity, float *out, int32_t *idx,
                                  int32_t *idx_count, float *scores_opt, void *stream);
