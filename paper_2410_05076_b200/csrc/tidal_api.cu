@@ -298,8 +298,13 @@ tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* score
     t.cand_smem = 8192;          // one histogram bin's population; larger lists are read from global memory
     const size_t words = (size_t)(kv->max_ctx_len + 31) / 32;
     // the last CTA's bitmaps and candidate buffer, or every CTA's score staging area, whichever is larger
-    const size_t smem = std::max(2 * words * sizeof(unsigned) + (size_t)t.cand_smem * sizeof(uint2),
-                                 (size_t)TK_SPAN * sizeof(float));
+    size_t smem = std::max(2 * words * sizeof(unsigned) + (size_t)t.cand_smem * sizeof(uint2),
+                           (size_t)TK_SPAN * sizeof(float));
+    if (kv->max_ctx_len <= TK_SPAN) {
+        // every row fits one CTA: staged scores, two bitmaps and 4096 candidates in shared memory
+        t.solo_cand = 4096;
+        smem = (size_t)TK_SPAN * sizeof(float) + 2 * (TK_SPAN / 32) * sizeof(unsigned) + (size_t)t.solo_cand * sizeof(uint2);
+    }
     // Both kernels may become resident while the kernel before them drains (they wait for it first).
     t.pdl = 1;
     cudaLaunchAttribute attr[1];

@@ -55,6 +55,8 @@ struct TopkParams {
     unsigned* bitmap;          // [items, bitmap_stride] winners above the threshold bin, one bit per position
     long long bitmap_stride;   // words per item (covers max_ctx rounded up to a whole slice)
     int cand_smem;             // candidates the last CTA can hold in shared memory
+    int solo_cand;             // > 0: rows of at most TK_SPAN positions are resolved by their single CTA entirely in
+                               // shared memory, which then holds this many candidates behind the staged scores
     int vec_ok;                // score rows are 16-byte aligned: float4 loads allowed
     int shift;                 // first digit = key >> shift (21 or 22); the rest is split 11 + (shift-11) bits
     int pdl;                   // launched with programmatic stream serialization: wait for the producer of the scores
@@ -281,7 +283,14 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     // Group j of a warp covers 128 consecutive positions, lane l the four at 4l: the 8 lanes of a
     // word OR their nibbles together and one of them stores the word (zeros included, so the
     // bitmap needs no clearing). Keys of the threshold bin itself are only marked here.
-    unsigned* bm = p.bitmap + (long long)item * p.bitmap_stride;
+    // A row that fits one CTA never leaves shared memory: bitmap and candidates are built behind the
+    // staged scores, and the arrival protocol is skipped.
+    const bool solo = p.solo_cand > 0 && nparts == 1;
+    unsigned* solo_bm = reinterpret_cast<unsigned*>(tk_smem + (size_t)TK_SPAN * sizeof(float));
+    const int solo_words = TK_SPAN / 32;
+    uint2* solo_cand = reinterpret_cast<uint2*>(solo_bm + 2 * solo_words);
+    unsigned* bm = solo ? solo_bm : p.bitmap + (long long)item * p.bitmap_stride;
+    const int bm_base = solo ? 0 : (s0 >> 5);
     unsigned eq_mask = 0;                                          // bit 4j+e: group j, element e
 #pragma unroll
     for (int j = 0; j < TK_BATCHES * TK_VEC; ++j) {
@@ -300,7 +309,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         word |= __shfl_xor_sync(0xffffffffu, word, 1);
         word |= __shfl_xor_sync(0xffffffffu, word, 2);
         word |= __shfl_xor_sync(0xffffffffu, word, 4);
-        if ((lane & 7) == 0) bm[(s0 >> 5) + j * (TK_THREADS / 8) + warp * 4 + (lane >> 3)] = word;
+        if ((lane & 7) == 0) bm[bm_base + j * (TK_THREADS / 8) + warp * 4 + (lane >> 3)] = word;
     }
     TIDAL_TRACE2(10);
 
@@ -308,11 +317,20 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     int cta_total;
     const int mine = __popc(eq_mask);
     int slot = block_scan_incl<int>(mine, warp_sums, cta_total) - mine;
-    if (tid == 0) bcast[0] = cta_total ? atomicAdd(&p.cursor[item], cta_total) : 0;
+    const bool solo_cands = solo && cta_total <= p.solo_cand;      // else the list goes through global memory
+    if (tid == 0) bcast[0] = (cta_total && !solo) ? atomicAdd(&p.cursor[item], cta_total) : 0;
     __syncthreads();
     slot += bcast[0];
-    uint2* cand = p.cand + (long long)item * p.cand_stride;
-    {
+    uint2* cand = solo_cands ? solo_cand : p.cand + (long long)item * p.cand_stride;
+    if (solo_cands) {
+        unsigned m = eq_mask;
+        while (m) {
+            const int e = __ffs(m) - 1;
+            m &= m - 1;
+            const int off = 4 * ((e >> 2) * TK_THREADS + tid) + (e & 3);
+            cand[slot++] = make_uint2(score_key(raw[off]), (unsigned)(s0 + off));
+        }
+    } else {
         unsigned m = eq_mask;
         while (m) {
             const int e = __ffs(m) - 1;
@@ -326,33 +344,47 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     TIDAL_TRACE2(3);
     // ---- the last CTA of this index head resolves the rest ------------------------------------------
     __syncthreads();
-    if (tid == 0) {
-        __threadfence();                               // cumulative: orders the CTA's bitmap and candidate stores
-        s_last = (atomicAdd(&p.done[item], 1) == nparts - 1);
-    }
-    __syncthreads();
-    TIDAL_TRACE2(4);
-    if (!s_last) return;
-    __threadfence();
-
-    const int M = (int)min((long long)__ldcg(&p.cursor[item]), p.cand_stride);
     const int words = (N + 31) >> 5;
-    unsigned* cgt = reinterpret_cast<unsigned*>(tk_smem);          // [words] winners: higher bins + winning candidates
-    unsigned* ceq = cgt + words;                                    // [words] candidates equal to the threshold key
-    uint2* scand = reinterpret_cast<uint2*>(ceq + words);          // [cand_smem]; 8*words bytes in: 8-byte aligned
-    const uint2* c = cand;
-    if (M <= p.cand_smem) {
-#pragma unroll 4
-        for (int i = tid; i < M; i += TK_THREADS) scand[i] = __ldcg(&cand[i]);
-        c = scand;
-    }
-    // The winners' bitmap written by all CTAs of this head is pulled into shared memory once
-    // (coalesced); candidates that turn out to be winners are ORed into the same words.
     const int per = (words + TK_THREADS - 1) / TK_THREADS;
     const int w0 = min(words, tid * per), w1 = min(words, w0 + per);
-    for (int i = tid; i < words; i += TK_THREADS) { cgt[i] = __ldcg(&bm[i]); ceq[i] = 0; }
-    for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
-    __syncthreads();
+    unsigned* cgt;                                                  // [words] winners: higher bins + winning candidates
+    unsigned* ceq;                                                  // [words] candidates equal to the threshold key
+    const uint2* c;
+    int M;
+    if (solo) {
+        cgt = solo_bm;
+        ceq = solo_bm + solo_words;
+        M = solo_cands ? cta_total : (int)min((long long)cta_total, p.cand_stride);
+        c = cand;                                                   // shared memory, or this CTA's own global list
+        for (int i = tid; i < words; i += TK_THREADS) ceq[i] = 0;
+        for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
+        __syncthreads();
+    } else {
+        if (tid == 0) {
+            __threadfence();                           // cumulative: orders the CTA's bitmap and candidate stores
+            s_last = (atomicAdd(&p.done[item], 1) == nparts - 1);
+        }
+        __syncthreads();
+        TIDAL_TRACE2(4);
+        if (!s_last) return;
+        __threadfence();
+
+        M = (int)min((long long)__ldcg(&p.cursor[item]), p.cand_stride);
+        cgt = reinterpret_cast<unsigned*>(tk_smem);
+        ceq = cgt + words;
+        uint2* scand = reinterpret_cast<uint2*>(ceq + words);      // [cand_smem]; 8*words bytes in: 8-byte aligned
+        c = cand;
+        if (M <= p.cand_smem) {
+#pragma unroll 4
+            for (int i = tid; i < M; i += TK_THREADS) scand[i] = __ldcg(&cand[i]);
+            c = scand;
+        }
+        // The winners' bitmap written by all CTAs of this head is pulled into shared memory once
+        // (coalesced); candidates that turn out to be winners are ORed into the same words.
+        for (int i = tid; i < words; i += TK_THREADS) { cgt[i] = __ldcg(&bm[i]); ceq[i] = 0; }
+        for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
+        __syncthreads();
+    }
 
     TIDAL_TRACE2(5);
     // second digit: the next 11 key bits (every candidate already has first digit b1)
@@ -443,7 +475,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     TIDAL_TRACE2(9);
     // leave the shared state clean for the next call
     for (int i = tid; i < TK_BINS; i += TK_THREADS) gh[i] = 0;
-    if (tid == 0) { p.cursor[item] = 0; p.done[item] = 0; }
+    if (tid == 0 && !solo) { p.cursor[item] = 0; p.done[item] = 0; }
 }
 
 }  // namespace tidal

@@ -201,13 +201,16 @@ def test_decode_step_host_buffers(td):
         assert torch.allclose(out_host[i], outs[i].cpu(), rtol=0, atol=1e-4)
 
 
-def test_ties_and_constant_scores(td):
-    """q = 0: every score is equal, so the lowest positions win and the output is the mean of V."""
-    w = wl(1, 4, 2, 333, 20, seed=13)
+@pytest.mark.parametrize("N,k", [(333, 20), (9000, 700), (40000, 5000)])
+def test_ties_and_constant_scores(td, N, k):
+    """q = 0: every score is equal, so the lowest positions win and the output is the mean of V. The sizes
+    cover a threshold bin that fits shared memory, one that overflows it in a single CTA, and one that
+    overflows it across several CTAs."""
+    w = wl(1, 4, 2, N, k, seed=13)
     q, lay = build(w, "hnd_interleaved")
     q.zero_()
     out, idx, _ = td.select_attn(lay, q, w.k)
-    assert idx.cpu().numpy()[0].tolist() == [list(range(20))] * 4
+    assert idx.cpu().numpy()[0].tolist() == [list(range(k))] * 4
     ref = oracle.full_attn(util.oracle_kv(lay), synth.bits(q))
     util.check_out(out.cpu().numpy(), ref, "ties.out")
 
