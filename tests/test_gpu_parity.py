@@ -348,7 +348,10 @@ def test_budget_equal_to_a_long_context_keeps_everything(td):
     assert torch.equal(idx[0, 5], torch.arange(65536, dtype=torch.int32, device=DEV))
     sp = td.sparse_attn(lay, q, idx, cnt)
     torch.cuda.synchronize()
-    assert torch.allclose(sp, out, rtol=0, atol=2e-4)       # sparse over everything is full attention
+    # sparse over everything is full attention; the two kernels round the softmax weights to bf16 at
+    # different running maxima and sum in different orders (each is within about 1.5e-4 of the exact
+    # result at this size), so they agree to a few 1e-4, not bit for bit
+    assert torch.allclose(sp, out, rtol=0, atol=1e-3)
 
 
 def test_sixty_four_layer_schedule_matches_the_oracle_step(td):
