@@ -198,7 +198,7 @@ def test_decode_step_host_buffers(td):
     # tiles are handed to warps dynamically, so the fp32 summation order (not the result
     # beyond rounding) may differ between two runs
     for i in range(len(sched)):
-        assert torch.allclose(out_host[i], outs[i].cpu(), rtol=0, atol=1e-4)
+        assert torch.allclose(out_host[i], outs[i].cpu(), rtol=0, atol=5e-4)
 
 
 @pytest.mark.parametrize("N,k", [(333, 20), (9000, 700), (40000, 5000)])
@@ -279,7 +279,7 @@ def test_results_are_reproducible(td):
     a = td.select_attn(lay, q, w.k)
     b = td.select_attn(lay, q, w.k)
     assert torch.equal(a[1], b[1])                       # the selected sets are reproducible bit for bit
-    assert torch.allclose(a[0], b[0], rtol=0, atol=1e-4)  # outputs up to fp32 summation order
+    assert torch.allclose(a[0], b[0], rtol=0, atol=5e-4)  # outputs up to fp32 summation order
 
 
 def test_many_short_sequences_use_the_flat_split(td):
