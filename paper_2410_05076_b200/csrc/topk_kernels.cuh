@@ -80,6 +80,7 @@ __device__ __forceinline__ unsigned load_slice_keys(const TopkParams& p, const f
         const int pos = s0 + 4 * (j * TK_THREADS + (int)threadIdx.x);
         if (p.vec_ok && pos + 3 < n) {
             float4 t = __ldcg(reinterpret_cast<const float4*>(srow + pos));
+#pragma unroll 4
             for (int m = 1; m < members; ++m) {
                 const float4 u = __ldcg(reinterpret_cast<const float4*>(srow + m * p.score_stride + pos));
                 t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
@@ -91,6 +92,7 @@ __device__ __forceinline__ unsigned load_slice_keys(const TopkParams& p, const f
                 float t = 0.f;
                 if (pos + e < n) {
                     t = __ldcg(srow + pos + e);
+#pragma unroll 1
                     for (int m = 1; m < members; ++m) t += __ldcg(srow + m * p.score_stride + pos + e);
                 }
                 v[4 * j + e] = t;
@@ -111,8 +113,10 @@ __device__ __forceinline__ unsigned load_slice_keys(const TopkParams& p, const f
 }
 
 // Inclusive scan of one value per thread over a TK_THREADS block.
+// (Not inlined, like pick_digit below: these kernels run most of their code exactly once, so their speed
+// is set by instruction fetch and every repeated copy of a helper costs more misses than a call.)
 template <typename T>
-__device__ __forceinline__ T block_scan_incl(T v, T* warp_sums, T& total) {
+__device__ __noinline__ T block_scan_incl(T v, T* warp_sums, T& total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
@@ -136,8 +140,8 @@ __device__ __forceinline__ T block_scan_incl(T v, T* warp_sums, T& total) {
 // Given a histogram of `nbins` digits (shared memory), find the digit holding
 // the `need`-th largest remaining key; on return `need` is reduced by the number
 // of keys in higher digits. Identical result in every thread.
-__device__ __forceinline__ int pick_digit(const unsigned* hist, int nbins, int* warp_sums, int* bcast,
-                                          int& need) {
+__device__ __noinline__ int pick_digit(const unsigned* hist, int nbins, int* warp_sums, int* bcast,
+                                       int& need) {
     const int per = (nbins + TK_THREADS - 1) / TK_THREADS;
     const int hi_bin = nbins - 1 - (int)threadIdx.x * per;      // this thread's highest bin
     int mine = 0;
@@ -247,23 +251,34 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
                          ::"r"(dst), "l"(nbytes ? srow + pos : srow), "r"(nbytes) : "memory");
         }
         asm volatile("cp.async.commit_group;\n" ::: "memory");
-    } else {
-#pragma unroll
-        for (int bt = 0; bt < TK_BATCHES; ++bt) {                  // summed member heads or unaligned rows
-            float v[TK_KEYS];
-#pragma unroll
-            for (int e = 0; e < TK_KEYS; ++e) {
-                const int pos = s0 + bt * TK_SLICE + 4 * ((e >> 2) * TK_THREADS + tid) + (e & 3);
-                float t = 0.f;
-                if (pos < N) {
-                    t = __ldcg(srow + pos);
-                    for (int m = 1; m < members; ++m) t += __ldcg(srow + m * p.score_stride + pos);
+    } else if (p.vec_ok) {
+        // summed member heads: the same groups of four positions, the members' rows added up
+#pragma unroll 2
+        for (int j = 0; j < TK_BATCHES * TK_VEC; ++j) {
+            const int off = 4 * (j * TK_THREADS + tid);
+            const int pos = s0 + off;
+            float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (pos < N) {                                         // rows are padded to a multiple of four
+                t = __ldcg(reinterpret_cast<const float4*>(srow + pos));
+#pragma unroll 4
+                for (int m = 1; m < members; ++m) {
+                    const float4 u = __ldcg(reinterpret_cast<const float4*>(srow + m * p.score_stride + pos));
+                    t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
                 }
-                v[e] = t;
             }
-#pragma unroll
-            for (int e = 0; e < TK_KEYS; ++e)
-                raw[bt * TK_SLICE + 4 * ((e >> 2) * TK_THREADS + tid) + (e & 3)] = v[e];
+            *reinterpret_cast<float4*>(raw + off) = t;
+        }
+    } else {
+        // unaligned score rows (a caller's buffer): one position at a time
+#pragma unroll 1
+        for (int i = tid; i < TK_SPAN; i += TK_THREADS) {
+            const int pos = s0 + i;
+            float t = 0.f;
+            if (pos < N) {
+#pragma unroll 1
+                for (int m = 0; m < members; ++m) t += __ldcg(srow + m * p.score_stride + pos);
+            }
+            raw[i] = t;
         }
     }
     {
