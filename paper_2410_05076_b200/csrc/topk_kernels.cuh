@@ -460,36 +460,25 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     }
 
     TIDAL_TRACE2(8);
-    constexpr int PER_MAX = 16;                        // bitmap words per thread at the longest supported context
-    if (need == 0 && per <= PER_MAX) {
-        // No equal-key positions are pending (the usual case): only the winners' bitmap is enumerated,
-        // and each thread keeps its words in registers between counting and writing. When the words
-        // divide evenly they are fetched as 16-byte pieces (consecutive threads are `per` words apart,
-        // which scalar reads would turn into an 8-way bank conflict).
-        unsigned wg[PER_MAX];
-        const bool even = (per & 3) == 0 && words == per * TK_THREADS;
-        if (even) {
-            const uint4* src = reinterpret_cast<const uint4*>(cgt + w0);
-#pragma unroll
-            for (int j = 0; j < PER_MAX / 4; ++j) {
-                uint4 t = make_uint4(0u, 0u, 0u, 0u);
-                if (4 * j < per) t = src[j];
-                wg[4 * j] = t.x; wg[4 * j + 1] = t.y; wg[4 * j + 2] = t.z; wg[4 * j + 3] = t.w;
-            }
-        } else {
-#pragma unroll
-            for (int j = 0; j < PER_MAX; ++j) wg[j] = (w0 + j < w1) ? cgt[w0 + j] : 0u;
-        }
+    if (need == 0 && (per & 3) == 0 && words == per * TK_THREADS) {
+        // No equal-key positions are pending (the usual case) and the words divide evenly: only the
+        // winners' bitmap is enumerated, fetched as 16-byte pieces (consecutive threads are `per` words
+        // apart, which scalar reads turn into an 8-way bank conflict). The loops stay rolled: this
+        // code runs once, so every instruction costs a fetch.
+        const uint4* src = reinterpret_cast<const uint4*>(cgt + w0);
         int mine = 0;
-#pragma unroll
-        for (int j = 0; j < PER_MAX; ++j) mine += __popc(wg[j]);
+#pragma unroll 1
+        for (int j = 0; j < per / 4; ++j) {
+            const uint4 t = src[j];
+            mine += __popc(t.x) + __popc(t.y) + __popc(t.z) + __popc(t.w);
+        }
         TIDAL_TRACE2(11);
         int tot;
         int at = block_scan_incl<int>(mine, warp_sums, tot) - mine;
         TIDAL_TRACE2(12);
-#pragma unroll
-        for (int j = 0; j < PER_MAX; ++j) {
-            unsigned bits = wg[j];
+#pragma unroll 1
+        for (int j = 0; j < per; ++j) {
+            unsigned bits = cgt[w0 + j];
             while (bits) {
                 const int pbit = __ffs(bits) - 1;
                 if (at < p.k) out[at] = ((w0 + j) << 5) + pbit;
