@@ -501,3 +501,33 @@ def test_random_shapes_match_the_oracle(td, B, Hq, Hkv, N, k, ragged, layout, gr
     sp = td.sparse_attn(lay, q, idx, cnt)
     util.check_out(sp.cpu().numpy(), oracle.sparse_attn(okv, qb, idx_h, cnt.cpu().numpy()), "sparse")
     assert td.device_status() == binding.OK
+
+
+def test_decode_step_replays_from_a_cuda_graph(td):
+    """The step allocates nothing once its workspace exists, so it can be captured into a CUDA graph
+    (programmatic dependent launches included) and replayed: same token sets, same outputs."""
+    sched = [0, 1, 2, 2, 1, 2]
+    w = wl(1, 8, 2, 3000, 128, seed=23, layers=len(sched))
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    layers = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(len(sched))]
+    outs = [torch.zeros(1, 8, 128, dtype=torch.float32, device=DEV) for _ in sched]
+    step = td.make_step(sched, layers, qs, outs, w.k)
+    step()                                                    # sizes the workspace outside the capture
+    torch.cuda.synchronize()
+    eager = [o.clone() for o in outs]
+    eager_idx = step.idx.clone()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    for o in outs:
+        o.zero_()
+    step.idx.fill_(-7)
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(step.idx, eager_idx)
+    for o, e in zip(outs, eager):
+        assert torch.allclose(o, e, rtol=0, atol=5e-4)
+    assert td.device_status() == binding.OK
