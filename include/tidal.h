@@ -151,6 +151,14 @@ tidal_status_t tidal_decode_step(tidal_ctx_t *ctx, int32_t num_layers, const uin
                                  float *const *out_per_layer, int32_t k, int32_t granularity,
                                  int32_t *idx, int32_t *idx_count, void *stream);
 
+/* Step graphs. When `stream` is an ordinary stream (not the legacy or per-thread default, and not
+ * being captured by the caller), tidal_decode_step and tidal_decode_step_host record their launches
+ * once as a CUDA graph and replay it for as long as every argument (schedule, descriptors, pointers,
+ * k, granularity) stays byte-for-byte the same: lengths and page tables live in device memory and
+ * may change freely. Up to 16 recordings are kept per context. On by default; enabled = 0 turns it
+ * off and frees the recordings. */
+tidal_status_t tidal_set_graphs(tidal_ctx_t *ctx, int32_t enabled);
+
 /* The step of Algorithm 1 including its cache update: layer i's new key and value rows
  * (k_new_per_layer[i], v_new_per_layer[i]: device bf16 [batch, Hkv, head_dim], as for
  * tidal_kv_append) are written at position ctx_lens[b] - 1 of layer i's cache, then the layers

@@ -26,7 +26,7 @@ EXPORTS = [
     "tidal_create", "tidal_destroy", "tidal_workspace_bytes", "tidal_full_attn", "tidal_select_attn",
     "tidal_sparse_attn", "tidal_decode_step", "tidal_decode_step_host", "tidal_device_status",
     "tidal_launch_count", "tidal_strerror", "tidal_sparse_attn_noalloc", "tidal_kv_append",
-    "tidal_decode_step_append",
+    "tidal_decode_step_append", "tidal_set_graphs",
 ]
 
 
@@ -75,6 +75,8 @@ def load() -> C.CDLL:
     L.tidal_workspace_bytes.restype = C.c_size_t
     L.tidal_decode_step_append.argtypes = [P, I32, P, KVP, P, P, P, P, I32, I32, P, P, P]
     L.tidal_decode_step_append.restype = I32
+    L.tidal_set_graphs.argtypes = [P, I32]
+    L.tidal_set_graphs.restype = I32
     L.tidal_kv_append.argtypes = [P, KVP, P, P, P]
     L.tidal_kv_append.restype = I32
     L.tidal_full_attn.argtypes = [P, KVP, P, P, P]
@@ -276,6 +278,10 @@ class Tidal:
 
         step.keep = (sched_arr, kvs, list(layers), q_host, out_host)
         return step
+
+    def set_graphs(self, enabled: bool) -> None:
+        """Record whole steps as CUDA graphs and replay them (on by default; needs a non-default stream)."""
+        _check(self.lib.tidal_set_graphs(self.ctx, 1 if enabled else 0), "tidal_set_graphs")
 
     def device_status(self) -> int:
         return self.lib.tidal_device_status(self.ctx, _stream())

@@ -11,6 +11,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <vector>
 #include <new>
 
 #include "attn_kernels.cuh"
@@ -48,6 +49,18 @@ struct tidal_ctx {
     int state_rows = 0;                         // capacity in (sequence, head) rows
     int* status = nullptr;                      // device word, sticky
     int64_t launches = 0;
+    // Whole steps are recorded once as CUDA graphs (programmatic dependent launches included) and
+    // replayed while every host-visible argument stays the same: one launch per step instead of one
+    // per kernel. Keyed by the bytes of all arguments plus the workspace addresses they bake in.
+    struct StepGraph {
+        std::vector<unsigned char> key;
+        cudaGraphExec_t exec = nullptr;
+        int launches = 0;
+        uint64_t last_use = 0;
+    };
+    std::vector<StepGraph> graphs;
+    uint64_t graph_clock = 0;
+    bool graphs_enabled = true;
 };
 
 namespace {
@@ -149,9 +162,17 @@ size_t ws_bytes_for(const tidal_kv_t* kv, int k, int num_layers_host) {
     return layout_ws(kv, k, num_layers_host).total;
 }
 
+void drop_graphs(tidal_ctx* ctx) {
+    if (ctx->graphs.empty()) return;
+    cudaDeviceSynchronize();
+    for (auto& g : ctx->graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
+    ctx->graphs.clear();
+}
+
 tidal_status_t ensure_ws(tidal_ctx* ctx, size_t bytes) {
     if (ctx->ws_bytes >= bytes) return TIDAL_OK;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    drop_graphs(ctx);                           // they carry addresses inside the old workspace
     if (ctx->ws) { cudaDeviceSynchronize(); cudaFree(ctx->ws); ctx->ws = nullptr; ctx->ws_bytes = 0; }
     void* p = nullptr;
     if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TIDAL_ERR_NOMEM; }
@@ -170,6 +191,7 @@ inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + 4
 tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     if (ctx->state_rows >= rows) return TIDAL_OK;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    drop_graphs(ctx);
     if (ctx->state) { cudaDeviceSynchronize(); cudaFree(ctx->state); ctx->state = nullptr; ctx->state_rows = 0; }
     const int cap = (int)align_up((size_t)rows, 64);
     const size_t bytes = (size_t)cap * (4 + TK_BINS) * sizeof(int);
@@ -353,6 +375,92 @@ int resident_ctas(K kernel, int threads, size_t smem, int sm_count) {
     return per_sm * sm_count;
 }
 
+// ---- step graphs ------------------------------------------------------------------------------------
+struct KeyBuilder {
+    std::vector<unsigned char> bytes;
+    template <typename T> void add(const T& v) {
+        const unsigned char* p = reinterpret_cast<const unsigned char*>(&v);
+        bytes.insert(bytes.end(), p, p + sizeof(T));
+    }
+    void add_raw(const void* p, size_t n) {
+        const unsigned char* c = static_cast<const unsigned char*>(p);
+        bytes.insert(bytes.end(), c, c + n);
+    }
+};
+
+void step_key(KeyBuilder& kb, const tidal_ctx* ctx, int tag, int32_t num_layers, const uint8_t* schedule,
+                     const tidal_kv_t* kvs, int32_t k, int32_t granularity, int host_layers) {
+    kb.add(tag); kb.add(num_layers); kb.add(k); kb.add(granularity); kb.add(host_layers);
+    kb.add(ctx->ws); kb.add(ctx->state);
+    kb.add_raw(schedule, (size_t)num_layers);
+    for (int i = 0; i < num_layers; ++i) {
+        // field by field: the struct has padding whose bytes are not the caller's to define
+        const tidal_kv_t& v = kvs[i];
+        kb.add(v.batch); kb.add(v.num_q_heads); kb.add(v.num_kv_heads); kb.add(v.head_dim); kb.add(v.kv_layout);
+        kb.add(v.k); kb.add(v.v); kb.add(v.stride_b); kb.add(v.stride_pos); kb.add(v.stride_head); kb.add(v.stride_page);
+        kb.add(v.page_table); kb.add(v.page_size); kb.add(v.max_pages_per_seq); kb.add(v.num_pages);
+        kb.add(v.ctx_lens); kb.add(v.max_ctx_len); kb.add(v.sm_scale);
+    }
+}
+
+// A stream can record a graph if it is a real stream (not the legacy or per-thread default) that is
+// not already being captured by the caller.
+bool graphable(const tidal_ctx* ctx, cudaStream_t st) {
+    if (!ctx->graphs_enabled || st == nullptr || st == cudaStreamLegacy || st == cudaStreamPerThread) return false;
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) { cudaGetLastError(); return false; }
+    return cs == cudaStreamCaptureStatusNone;
+}
+
+// Replays the recorded graph of `key`, or records one from `enqueue` (which must only launch work on
+// `st`). Falls back to plain enqueueing when recording is not possible.
+template <typename F>
+tidal_status_t run_graphed(tidal_ctx* ctx, KeyBuilder& kb, cudaStream_t st, F&& enqueue) {
+    constexpr size_t MAX_GRAPHS = 16;
+    if (!graphable(ctx, st)) return enqueue();
+    ++ctx->graph_clock;
+    for (auto& g : ctx->graphs) {
+        if (g.key == kb.bytes) {
+            g.last_use = ctx->graph_clock;
+            if (cudaGraphLaunch(g.exec, st) != cudaSuccess) return TIDAL_ERR_CUDA;
+            ctx->launches += g.launches;
+            return TIDAL_OK;
+        }
+    }
+    if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); return enqueue(); }
+    const int64_t before = ctx->launches;
+    const tidal_status_t rc = enqueue();
+    cudaGraph_t graph = nullptr;
+    const cudaError_t end = cudaStreamEndCapture(st, &graph);
+    const int recorded = (int)(ctx->launches - before);
+    ctx->launches = before;                     // nothing has run yet
+    if (rc != TIDAL_OK || end != cudaSuccess || !graph) {
+        if (graph) cudaGraphDestroy(graph);
+        cudaGetLastError();
+        return rc != TIDAL_OK ? rc : enqueue();
+    }
+    cudaGraphExec_t exec = nullptr;
+    const cudaError_t inst = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (inst != cudaSuccess || !exec) { cudaGetLastError(); return enqueue(); }
+    if (ctx->graphs.size() >= MAX_GRAPHS) {     // forget the entry that has gone unused the longest
+        size_t victim = 0;
+        for (size_t i = 1; i < ctx->graphs.size(); ++i)
+            if (ctx->graphs[i].last_use < ctx->graphs[victim].last_use) victim = i;
+        cudaGraphExecDestroy(ctx->graphs[victim].exec);   // deferred by the runtime while a launch is in flight
+        ctx->graphs.erase(ctx->graphs.begin() + victim);
+    }
+    tidal_ctx::StepGraph g;
+    g.key = std::move(kb.bytes);
+    g.exec = exec;
+    g.launches = recorded;
+    g.last_use = ctx->graph_clock;
+    ctx->graphs.push_back(std::move(g));
+    if (cudaGraphLaunch(exec, st) != cudaSuccess) return TIDAL_ERR_CUDA;
+    ctx->launches += recorded;
+    return TIDAL_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -393,6 +501,7 @@ tidal_status_t tidal_destroy(tidal_ctx_t* ctx) {
     if (!ctx) return TIDAL_ERR_INVALID;
     cudaSetDevice(ctx->device);
     cudaDeviceSynchronize();
+    drop_graphs(ctx);
     if (ctx->ws) cudaFree(ctx->ws);
     if (ctx->state) cudaFree(ctx->state);
     if (ctx->status) cudaFree(ctx->status);
@@ -483,10 +592,10 @@ tidal_status_t tidal_sparse_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const v
     return run_sparse(ctx, kv, q, idx, idx_count, k, Hi, out, true, w, (cudaStream_t)stream);
 }
 
-static tidal_status_t decode_step_impl(tidal_ctx_t* ctx, int32_t num_layers, const uint8_t* schedule,
-                                       const tidal_kv_t* kvs, const void* const* qs, float* const* outs,
-                                       int32_t k, int32_t granularity, int32_t* idx, int32_t* idx_count,
-                                       int host_layers, cudaStream_t st) {
+// Validates a step and sizes the workspace for it (may allocate and synchronise).
+static tidal_status_t decode_step_prepare(tidal_ctx_t* ctx, int32_t num_layers, const uint8_t* schedule,
+                                          const tidal_kv_t* kvs, const void* const* qs, float* const* outs,
+                                          int32_t k, int32_t granularity, int host_layers) {
     // Validate everything before enqueuing anything.
     bool have_rho = false;
     size_t need = 0;
@@ -506,10 +615,17 @@ static tidal_status_t decode_step_impl(tidal_ctx_t* ctx, int32_t num_layers, con
         }
         need = std::max(need, ws_bytes_for(&kvs[i], k, host_layers));
     }
+    if (hi_of(&kvs[0], granularity) <= 0) return TIDAL_ERR_INVALID;
+    return ensure_all(ctx, &kvs[0], need);
+}
+
+// Enqueues the layers of a prepared step: launches only, nothing that a stream capture forbids.
+static tidal_status_t decode_step_enqueue(tidal_ctx_t* ctx, int32_t num_layers, const uint8_t* schedule,
+                                          const tidal_kv_t* kvs, const void* const* qs, float* const* outs,
+                                          int32_t k, int32_t granularity, int32_t* idx, int32_t* idx_count,
+                                          int host_layers, cudaStream_t st) {
     const int Hi = hi_of(&kvs[0], granularity);
-    if (Hi <= 0) return TIDAL_ERR_INVALID;
-    tidal_status_t rc = ensure_all(ctx, &kvs[0], need);
-    if (rc != TIDAL_OK) return rc;
+    tidal_status_t rc = TIDAL_OK;
     for (int i = 0; i < num_layers; ++i) {
         const tidal_kv_t* kv = &kvs[i];
         const WsLayout w = layout_ws(kv, k, host_layers);
@@ -567,8 +683,27 @@ tidal_status_t tidal_decode_step(tidal_ctx_t* ctx, int32_t num_layers, const uin
     if (!ctx || num_layers <= 0 || !schedule || !kv_per_layer || !q_per_layer || !out_per_layer || !idx || k <= 0)
         return TIDAL_ERR_INVALID;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
-    return decode_step_impl(ctx, num_layers, schedule, kv_per_layer, q_per_layer, out_per_layer, k,
-                            granularity, idx, idx_count, 0, (cudaStream_t)stream);
+    cudaStream_t st = (cudaStream_t)stream;
+    tidal_status_t rc = decode_step_prepare(ctx, num_layers, schedule, kv_per_layer, q_per_layer, out_per_layer, k,
+                                            granularity, 0);
+    if (rc != TIDAL_OK) return rc;
+    KeyBuilder kb;
+    step_key(kb, ctx, 0, num_layers, schedule, kv_per_layer, k, granularity, 0);
+    kb.add_raw(q_per_layer, sizeof(void*) * (size_t)num_layers);
+    kb.add_raw(out_per_layer, sizeof(void*) * (size_t)num_layers);
+    kb.add(idx); kb.add(idx_count);
+    return run_graphed(ctx, kb, st, [&]() {
+        return decode_step_enqueue(ctx, num_layers, schedule, kv_per_layer, q_per_layer, out_per_layer, k, granularity,
+                                   idx, idx_count, 0, st);
+    });
+}
+
+tidal_status_t tidal_set_graphs(tidal_ctx_t* ctx, int32_t enabled) {
+    if (!ctx) return TIDAL_ERR_INVALID;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    ctx->graphs_enabled = enabled != 0;
+    if (!ctx->graphs_enabled) drop_graphs(ctx);
+    return TIDAL_OK;
 }
 
 tidal_status_t tidal_decode_step_host(tidal_ctx_t* ctx, int32_t num_layers, const uint8_t* schedule,
@@ -597,19 +732,39 @@ tidal_status_t tidal_decode_step_host(tidal_ctx_t* ctx, int32_t num_layers, cons
     char* ws = (char*)ctx->ws;
     char* qd = ws + w.q_stage;
     float* od = (float*)(ws + w.out_stage);
-    if (cudaMemcpyAsync(qd, q_host, (size_t)num_layers * rows * HEAD_DIM * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return TIDAL_ERR_CUDA;
     const void* qs[1024];
     float* outs[1024];
     for (int i = 0; i < num_layers; ++i) {
         qs[i] = qd + (size_t)i * rows * HEAD_DIM * 2;
         outs[i] = od + (size_t)i * rows * HEAD_DIM;
     }
-    rc = decode_step_impl(ctx, num_layers, schedule, kv_per_layer, qs, outs, k, granularity,
-                          (int*)(ws + w.idx), (int*)(ws + w.idx_count), num_layers, st);
+    if ((rc = decode_step_prepare(ctx, num_layers, schedule, kv_per_layer, qs, outs, k, granularity, num_layers)) != TIDAL_OK)
+        return rc;
+    auto enqueue = [&]() -> tidal_status_t {
+        if (cudaMemcpyAsync(qd, q_host, (size_t)num_layers * rows * HEAD_DIM * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return TIDAL_ERR_CUDA;
+        const tidal_status_t r = decode_step_enqueue(ctx, num_layers, schedule, kv_per_layer, qs, outs, k, granularity,
+                                                     (int*)(ws + w.idx), (int*)(ws + w.idx_count), num_layers, st);
+        if (r != TIDAL_OK) return r;
+        if (cudaMemcpyAsync(out_host, od, (size_t)num_layers * rows * HEAD_DIM * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return TIDAL_ERR_CUDA;
+        return TIDAL_OK;
+    };
+    // The copies can be recorded with the layers only when both host buffers are page-locked.
+    auto pinned = [](const void* p) {
+        cudaPointerAttributes at;
+        if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return false; }
+        return at.type == cudaMemoryTypeHost;
+    };
+    if (pinned(q_host) && pinned(out_host)) {
+        KeyBuilder kb;
+        step_key(kb, ctx, 1, num_layers, schedule, kv_per_layer, k, granularity, num_layers);
+        kb.add(q_host); kb.add(out_host);
+        rc = run_graphed(ctx, kb, st, enqueue);
+    } else {
+        rc = enqueue();
+    }
     if (rc != TIDAL_OK) return rc;
-    if (cudaMemcpyAsync(out_host, od, (size_t)num_layers * rows * HEAD_DIM * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-        return TIDAL_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }
 

@@ -531,3 +531,55 @@ def test_decode_step_replays_from_a_cuda_graph(td):
     for o, e in zip(outs, eager):
         assert torch.allclose(o, e, rtol=0, atol=5e-4)
     assert td.device_status() == binding.OK
+
+
+def test_library_records_and_replays_step_graphs(td):
+    """On an ordinary stream the step is recorded once and replayed; lengths live in device memory, so a
+    replay follows them when they change. Compared with the same step enqueued kernel by kernel."""
+    sched = [0, 1, 2, 2]
+    w = wl(2, 8, 2, 2000, 64, ragged=True, ctx_min=500, seed=29, layers=len(sched))
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    layers = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(len(sched))]
+    lens0 = layers[0].ctx_lens.clone()
+    for l in layers:
+        l.ctx_lens = layers[0].ctx_lens                   # one length vector for all layers, changed in place below
+    outs = [torch.zeros(2, 8, 128, dtype=torch.float32, device=DEV) for _ in sched]
+    step = td.make_step(sched, layers, qs, outs, w.k)
+    q_host = torch.stack([q.cpu() for q in qs]).contiguous().pin_memory()
+    out_host = torch.zeros(len(sched), 2, 8, 128, dtype=torch.float32).pin_memory()
+    step_host = td.make_step_host(sched, layers, q_host, out_host, w.k)
+
+    def run_direct():
+        step()                                            # default stream: kernel by kernel
+        torch.cuda.synchronize()
+        return [o.clone() for o in outs], step.idx.clone()
+
+    side = torch.cuda.Stream()
+    for new_lens in (lens0, (lens0 // 2).clamp(min=70), lens0):
+        layers[0].ctx_lens.copy_(new_lens)
+        ref_outs, ref_idx = run_direct()
+        for o in outs:
+            o.zero_()
+        with torch.cuda.stream(side):
+            n0 = td.launch_count()
+            step()
+            n1 = td.launch_count()
+            step()                                        # a replay at the latest
+            n2 = td.launch_count()
+            side.synchronize()
+            assert n1 - n0 == n2 - n1 == 5                # 4 attention kernels + 1 top-k
+            assert torch.equal(step.idx, ref_idx)
+            for o, r in zip(outs, ref_outs):
+                assert torch.allclose(o, r, rtol=0, atol=5e-4)
+            step_host()
+            step_host()
+            for i, r in enumerate(ref_outs):
+                assert torch.allclose(out_host[i].to(DEV), r, rtol=0, atol=5e-4)
+    td.set_graphs(False)
+    with torch.cuda.stream(side):
+        step()
+        side.synchronize()
+    td.set_graphs(True)
+    for o, r in zip(outs, ref_outs):
+        assert torch.allclose(o, r, rtol=0, atol=5e-4)
+    assert td.device_status() == binding.OK
