@@ -473,7 +473,10 @@ def main():
             "config": {"workload": describe(w), "replicas": world, "granularity": args.granularity,
                        "launch": "tidal_decode_step on a non-default stream: the step's kernels are recorded once as a "
                                  "CUDA graph by the library and replayed (gpu_launches counts the kernels, not the graphs)",
-                       "l2": "every layer has its own KV cache (16 GiB per step at cfg3), far larger than L2",
+                       "l2": ("every layer has its own KV cache: %.2f GiB are streamed or gathered from per step, %s the "
+                              "126 MB L2%s" % (sum(kv_bytes) / 2**30,
+                                              "far more than" if sum(kv_bytes) > 4 * 126e6 else "NOT more than a few times",
+                                              "" if sum(kv_bytes) > 4 * 126e6 else ": this workload is L2-warm and not a bandwidth figure")),
                        "step_bytes": step_bytes,
                        "step_frac_of_8TBs": step_bytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
             "clocks": clocks, "gpu_launches": launches,
