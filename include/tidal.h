@@ -130,8 +130,9 @@ tidal_status_t tidal_select_attn(tidal_ctx_t *ctx, const tidal_kv_t *kv, const v
 
 /* SparseAttention(q, C[rho]) of Algorithm 1: Eq. 1 restricted to the positions
  * listed for the query head's index head hi = h * Hi / Hq, softmax renormalised
- * over them. Entries < 0 are padding and skipped; an entry >= ctx_lens[b] is
- * skipped and reported as TIDAL_ERR_INDEX by tidal_device_status(); a repeated
+ * over them. -1 is padding and skipped; any other entry outside
+ * [0, ctx_lens[b]) is skipped too and reported as TIDAL_ERR_INDEX by
+ * tidal_device_status(); a repeated
  * entry counts once per occurrence. Only the first idx_count[b] entries are
  * read when idx_count is given, else k. A head with no valid entry gets zeros.
  * num_index_heads must be Hq, Hkv or 1. */

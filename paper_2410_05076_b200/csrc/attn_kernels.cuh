@@ -472,7 +472,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         bool validA = false;
         auto resolve = [&](int pos) {
             validA = pos >= 0 && pos < N;
-            if (pos >= N) atomicOr(p.status, STATUS_BAD_INDEX);
+            if (pos >= N || pos < -1) atomicOr(p.status, STATUS_BAD_INDEX);   // -1 is padding, anything else is not a token
             offA = 0;
             if (validA) {
                 if (p.paged) {

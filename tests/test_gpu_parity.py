@@ -233,6 +233,10 @@ def test_sparse_skips_padding_duplicates_and_flags_bad_indices(td):
     assert td.device_status() == binding.ERR_INDEX
     assert td.device_status() == binding.OK       # sticky word was cleared
     util.check_out(sp.cpu().numpy(), ref, "sparse.badidx")   # the bad entry was skipped
+    idx[0, 1, 1] = -5                             # negative but not the padding value
+    sp = td.sparse_attn(lay, q, torch.from_numpy(idx).to(DEV))
+    assert td.device_status() == binding.ERR_INDEX
+    util.check_out(sp.cpu().numpy(), ref, "sparse.negidx")   # skipped as well
 
 
 def test_host_side_argument_errors(td):
