@@ -702,13 +702,14 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             __syncthreads();
             int* ctr = p.counters + (long long)b * IY + y;
             if (threadIdx.x == 0) {
-                __threadfence();                  // cumulative: orders the whole CTA's partial stores
-                const int old = atomicAdd(ctr, 1);
+                // release: orders the whole CTA's partial stores (made visible to this thread by the barrier)
+                // before the arrival; acquire: the last arrival sees every earlier part's stores
+                int old;
+                asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;\n" : "=r"(old) : "l"(ctr) : "memory");
                 s_is_last = (old == nsplits - 1);
             }
             __syncthreads();
             if (s_is_last) {
-                __threadfence();
                 const int ns = min(nsplits, p.max_splits);
                 // Every thread first puts the loads of its output elements in flight (up to 16 splits
                 // at once), the warps meanwhile reduce the (max, sum) pairs to per-split scale factors

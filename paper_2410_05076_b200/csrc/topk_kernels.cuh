@@ -376,13 +376,15 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         __syncthreads();
     } else {
         if (tid == 0) {
-            __threadfence();                           // cumulative: orders the CTA's bitmap and candidate stores
-            s_last = (atomicAdd(&p.done[item], 1) == nparts - 1);
+            // release: orders the CTA's bitmap and candidate stores (seen by this thread through the barrier)
+            // before the arrival; acquire: the last arrival sees every other CTA's
+            int old;
+            asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;\n" : "=r"(old) : "l"(&p.done[item]) : "memory");
+            s_last = (old == nparts - 1);
         }
         __syncthreads();
         TIDAL_TRACE2(4);
         if (!s_last) return;
-        __threadfence();
 
         M = (int)min((long long)__ldcg(&p.cursor[item]), p.cand_stride);
         cgt = reinterpret_cast<unsigned*>(tk_smem);
