@@ -102,6 +102,16 @@ __device__ __forceinline__ uint64_t l2_evict_first_policy() {
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(pol));
     return pol;
 }
+// Scores are written once and read back by the top-k right after: they are asked to stay in L2
+// (evict-last), so that they are not written out to DRAM in between.
+__device__ __forceinline__ uint64_t l2_evict_last_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;\n" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void st_keep(float* ptr, float v, uint64_t pol) {
+    asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;\n" ::"l"(ptr), "f"(v), "l"(pol) : "memory");
+}
 __device__ __forceinline__ void cp_async16_hint(uint32_t dst, const void* src, int src_bytes, uint64_t pol) {
     asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;\n" ::"r"(dst), "l"(src), "r"(src_bytes), "l"(pol) : "memory");
 }
@@ -210,6 +220,7 @@ __device__ __forceinline__ void consume_tile(const AttnParams& p, uint32_t ks, u
     if (MODE == MODE_SELECT) {
         // s[0],s[1]: (pos gid; heads 2tig, 2tig+1)   s[2],s[3]: (pos gid+8; same heads)
         const float f0 = s[0] * p.scale, f1 = s[1] * p.scale, f2 = s[2] * p.scale, f3 = s[3] * p.scale;
+        const uint64_t keep = l2_evict_last_policy();
         if (p.agg) {
             // One ranking score per (position, KV head): the group's columns summed (unused columns
             // hold zeros). Lanes that differ only in tig hold the columns of one position.
@@ -219,8 +230,8 @@ __device__ __forceinline__ void consume_tile(const AttnParams& p, uint32_t ks, u
             a0 += __shfl_xor_sync(0xffffffffu, a0, 2);
             a1 += __shfl_xor_sync(0xffffffffu, a1, 2);
             if (tig == 0) {
-                if (v0) score_row0[pos_base + gid] = a0;
-                if (v1) score_row0[pos_base + gid + 8] = a1;
+                if (v0) st_keep(score_row0 + pos_base + gid, a0, keep);
+                if (v1) st_keep(score_row0 + pos_base + gid + 8, a1, keep);
                 if (hist) {
                     if (v0) atomicAdd(hist + (score_key_bits(a0) >> p.hist_shift), 1u);
                     if (v1) atomicAdd(hist + (score_key_bits(a1) >> p.hist_shift), 1u);
@@ -228,12 +239,12 @@ __device__ __forceinline__ void consume_tile(const AttnParams& p, uint32_t ks, u
             }
         } else {
         if (score_row0) {
-            if (v0) score_row0[pos_base + gid] = f0;
-            if (v1) score_row0[pos_base + gid + 8] = f2;
+            if (v0) st_keep(score_row0 + pos_base + gid, f0, keep);
+            if (v1) st_keep(score_row0 + pos_base + gid + 8, f2, keep);
         }
         if (score_row1) {
-            if (v0) score_row1[pos_base + gid] = f1;
-            if (v1) score_row1[pos_base + gid + 8] = f3;
+            if (v0) st_keep(score_row1 + pos_base + gid, f1, keep);
+            if (v1) st_keep(score_row1 + pos_base + gid + 8, f3, keep);
         }
         if (hist) {      // histogram of the top key bits of every stored score, per head
             const int nb = 1 << (32 - p.hist_shift);
