@@ -48,7 +48,8 @@ constexpr int TILE_BYTES = TILE * HEAD_DIM * 2;   // 4 KB of K, same of V
 constexpr int STAGE_BYTES = 2 * TILE_BYTES;
 constexpr int HIST_BINS = 2048;          // global histogram row: up to 11 top bits of the score key
 constexpr int HIST_SMEM_WORDS = 8192;    // shared histogram: columns x bins <= 8192 counters (32 KB)
-constexpr int GRAB_TILES = 4;            // tiles a warp takes from its item's pool at a time afterwards
+constexpr int GRAB_TILES = 4;            // tiles a warp takes from its item's pool at a time afterwards (gather kernel)
+constexpr int GRAB_TILES_DENSE = 2;      // the same for the streaming kernels, whose items hold thousands of tiles
 
 struct AttnParams {
     const __nv_bfloat16* q;
@@ -78,6 +79,7 @@ struct AttnParams {
     unsigned* hist;            // MODE_SELECT, optional: [B*Hq][HIST_BINS] += histogram of the top key bits
     int hist_shift;            // bin = key >> hist_shift (21: 2048 bins, 22: 1024 bins for groups above 4)
     int* tile_ctr;             // splits_per_item > 0: per-item pool cursor, zero between launches
+    int ctr_stride;            // ints between the cursors of consecutive items (32: one 128-byte line each)
     int pdl;                   // launched with programmatic stream serialization: see pdl_wait()
     int wait_first;            // the preceding kernel may have written ctx_lens / idx: wait before reading anything
     int* status;
@@ -411,7 +413,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             const int hi_idx = per_qhead ? y : ((p.Hi == p.Hkv) ? g : 0);
             idx_row = p.idx + ((long long)b * p.Hi + hi_idx) * p.budget;
         }
-        int* pool = pooled ? p.tile_ctr + (long long)b * IY + y : nullptr;
+        int* pool = pooled ? p.tile_ctr + ((long long)b * IY + y) * p.ctr_stride : nullptr;
 
         float* score_row0 = nullptr;
         float* score_row1 = nullptr;
@@ -446,8 +448,9 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         constexpr int FIRST_TILES = STAGES + 2;
         const int first_tiles = (tiles_b <= item_warps * FIRST_TILES)
                                     ? max(1, (tiles_b + item_warps - 1) / max(item_warps, 1)) : FIRST_TILES;
+        constexpr int GRAB = (MODE == MODE_SPARSE) ? GRAB_TILES : GRAB_TILES_DENSE;
         const int pool_base = item_warps * first_tiles;
-        auto grab = [&]() { if (lane == 0) grab_raw = pool_base + atomicAdd(pool, GRAB_TILES); };
+        auto grab = [&]() { if (lane == 0) grab_raw = pool_base + atomicAdd(pool, GRAB); };
         if (pooled) {
             cur = (part_idx * NW + warp) * first_tiles;
             cur_end = min(tiles_b, cur + first_tiles);
@@ -463,7 +466,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                 if (cur_end >= tiles_b || pool_base >= tiles_b) return -1;   // nothing (left) in the pool
                 cur = __shfl_sync(0xffffffffu, grab_raw, 0);
                 if (cur >= tiles_b) { cur_end = tiles_b; return -1; }
-                cur_end = min(tiles_b, cur + GRAB_TILES);
+                cur_end = min(tiles_b, cur + GRAB);
                 grab();
             }
             return cur++;
@@ -711,7 +714,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         if (nsplits > 1) {
             // ---- the last CTA of this item to arrive combines the splits ---------------------------------
             __syncthreads();
-            int* ctr = p.counters + (long long)b * IY + y;
+            int* ctr = p.counters + ((long long)b * IY + y) * p.ctr_stride;
             if (threadIdx.x == 0) {
                 // release: orders the whole CTA's partial stores (made visible to this thread by the barrier)
                 // before the arrival; acquire: the last arrival sees every earlier part's stores

@@ -181,12 +181,15 @@ tidal_status_t ensure_ws(tidal_ctx* ctx, size_t bytes) {
     return TIDAL_OK;
 }
 
-// State layout for a capacity of R rows: counters[R] | cursor[R] | done[R] | tile_ctr[R] | hist[R][TK_BINS].
+// State layout for a capacity of R rows: counters | cursor | done | tile_ctr, each [R][CTR_STRIDE], then hist[R][TK_BINS].
+// Every counter has a 128-byte line of its own: hundreds of warps hit them at once, and atomics to one
+// line are served one after the other.
+constexpr int CTR_STRIDE = 32;
 inline int* state_counters(const tidal_ctx* c) { return (int*)c->state; }
-inline int* state_cursor(const tidal_ctx* c) { return (int*)c->state + c->state_rows; }
-inline int* state_done(const tidal_ctx* c) { return (int*)c->state + 2 * (size_t)c->state_rows; }
-inline int* state_tile_ctr(const tidal_ctx* c) { return (int*)c->state + 3 * (size_t)c->state_rows; }
-inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + 4 * (size_t)c->state_rows; }
+inline int* state_cursor(const tidal_ctx* c) { return (int*)c->state + (size_t)CTR_STRIDE * c->state_rows; }
+inline int* state_done(const tidal_ctx* c) { return (int*)c->state + 2 * (size_t)CTR_STRIDE * c->state_rows; }
+inline int* state_tile_ctr(const tidal_ctx* c) { return (int*)c->state + 3 * (size_t)CTR_STRIDE * c->state_rows; }
+inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + 4 * (size_t)CTR_STRIDE * c->state_rows; }
 
 tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     if (ctx->state_rows >= rows) return TIDAL_OK;
@@ -194,7 +197,7 @@ tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     drop_graphs(ctx);
     if (ctx->state) { cudaDeviceSynchronize(); cudaFree(ctx->state); ctx->state = nullptr; ctx->state_rows = 0; }
     const int cap = (int)align_up((size_t)rows, 64);
-    const size_t bytes = (size_t)cap * (4 + TK_BINS) * sizeof(int);
+    const size_t bytes = (size_t)cap * (4 * CTR_STRIDE + TK_BINS) * sizeof(int);
     void* p = nullptr;
     if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TIDAL_ERR_NOMEM; }
     if (cudaMemset(p, 0, bytes) != cudaSuccess) { cudaFree(p); return TIDAL_ERR_CUDA; }
@@ -231,6 +234,7 @@ void fill_common(AttnParams& a, const tidal_ctx* ctx, const tidal_kv_t* kv, cons
     a.max_splits = w.max_splits;
     a.batch = kv->batch;
     a.tile_ctr = state_tile_ctr(ctx);
+    a.ctr_stride = CTR_STRIDE;
     a.hist_shift = hist_shift_for(kv);
     a.status = ctx->status;
 }
@@ -306,6 +310,7 @@ tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* score
     char* ws = (char*)ctx->ws;
     t.hist = state_hist(ctx);
     t.cursor = state_cursor(ctx);
+    t.ctr_stride = CTR_STRIDE;
     t.done = state_done(ctx);
     t.cand = (uint2*)(ws + w.cand);
     t.cand_stride = w.cand_stride;
@@ -901,6 +906,7 @@ extern "C" tidal_status_t tidal_sparse_attn_noalloc(const tidal_kv_t* kv, const 
     a.part_ml = reinterpret_cast<float2*>(base + NOALLOC_PART_O);
     a.counters = words;
     a.tile_ctr = words + NOALLOC_MAX_ROWS;
+    a.ctr_stride = 1;
     a.status = words + 2 * NOALLOC_MAX_ROWS;
     a.max_splits = S;
     a.hist_shift = 21;

@@ -48,8 +48,9 @@ struct TopkParams {
     int* idx;                  // [B, Hi, k]
     int* idx_count;            // [B] or null
     unsigned* hist;            // [items, TK_BINS], zero between calls
-    int* cursor;               // [items], zero between calls
-    int* done;                 // [items], zero between calls
+    int* cursor;               // [items][ctr_stride], zero between calls
+    int* done;                 // [items][ctr_stride], zero between calls
+    int ctr_stride;            // ints between consecutive items' counters (one 128-byte line each)
     uint2* cand;               // [items, cand_stride] (key, position) of the threshold bin
     long long cand_stride;
     unsigned* bitmap;          // [items, bitmap_stride] winners above the threshold bin, one bit per position
@@ -333,7 +334,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     const int mine = __popc(eq_mask);
     int slot = block_scan_incl<int>(mine, warp_sums, cta_total) - mine;
     const bool solo_cands = solo && cta_total <= p.solo_cand;      // else the list goes through global memory
-    if (tid == 0) bcast[0] = (cta_total && !solo) ? atomicAdd(&p.cursor[item], cta_total) : 0;
+    if (tid == 0) bcast[0] = (cta_total && !solo) ? atomicAdd(&p.cursor[(size_t)item * p.ctr_stride], cta_total) : 0;
     __syncthreads();
     slot += bcast[0];
     uint2* cand = solo_cands ? solo_cand : p.cand + (long long)item * p.cand_stride;
@@ -379,14 +380,14 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
             // release: orders the CTA's bitmap and candidate stores (seen by this thread through the barrier)
             // before the arrival; acquire: the last arrival sees every other CTA's
             int old;
-            asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;\n" : "=r"(old) : "l"(&p.done[item]) : "memory");
+            asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;\n" : "=r"(old) : "l"(&p.done[(size_t)item * p.ctr_stride]) : "memory");
             s_last = (old == nparts - 1);
         }
         __syncthreads();
         TIDAL_TRACE2(4);
         if (!s_last) return;
 
-        M = (int)min((long long)__ldcg(&p.cursor[item]), p.cand_stride);
+        M = (int)min((long long)__ldcg(&p.cursor[(size_t)item * p.ctr_stride]), p.cand_stride);
         cgt = reinterpret_cast<unsigned*>(tk_smem);
         ceq = cgt + words;
         uint2* scand = reinterpret_cast<uint2*>(ceq + words);      // [cand_smem]; 8*words bytes in: 8-byte aligned
@@ -520,7 +521,7 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     TIDAL_TRACE2(9);
     // leave the shared state clean for the next call
     for (int i = tid; i < TK_BINS; i += TK_THREADS) gh[i] = 0;
-    if (tid == 0 && !solo) { p.cursor[item] = 0; p.done[item] = 0; }
+    if (tid == 0 && !solo) { p.cursor[(size_t)item * p.ctr_stride] = 0; p.done[(size_t)item * p.ctr_stride] = 0; }
 }
 
 }  // namespace tidal
