@@ -575,9 +575,15 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         // ---- private cp.async ring -----------------------------------------------------------------------
         // Until the grid dependency is resolved, only tiles that cannot hold the token appended for
         // this layer may be fetched: every tile but the last one of the item (index lists produced by
-        // the selection kernel are ascending). The query, the pool cursor and the scratch buffers
-        // belong to the kernels before us and are touched only after the wait.
+        // the selection kernel are ascending). The query and the scratch buffers belong to the kernels
+        // before us and are touched only after the wait.
         int issued = 0, commits = 0;
+        // The first pool request goes out at once, even before the grid dependency resolves: consecutive
+        // launches use alternating sets of cursors, and the set of this launch was last touched two
+        // launches ago (its last user reset it, and had finished before our predecessor could start us).
+        // By the time the fixed chunk runs out the answer is there; asked for only after the wait, the
+        // forty-odd warps of an item queue up on one address and stall at that point.
+        if (pooled) grab();
         if (!waited) {
             while (commits < STAGES && tA >= 0 && tA < tiles_b - 1) {
                 issue(issued % STAGES);
@@ -590,7 +596,6 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             waited = true;
         }
         TIDAL_TRACE(1);
-        if (pooled) grab();
 
         // Q^T fragments: column gid is head head0+gid; this lane holds the 16-byte
         // pieces 4j+tig (j = 0..3) of that head's query row.

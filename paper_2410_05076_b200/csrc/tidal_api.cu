@@ -48,6 +48,7 @@ struct tidal_ctx {
     void* state = nullptr;
     int state_rows = 0;                         // capacity in (sequence, head) rows
     int* status = nullptr;                      // device word, sticky
+    int cursor_set = 0;                         // which of the two sets of pool cursors the last attention launch used
     int64_t launches = 0;
     // Whole steps are recorded once as CUDA graphs (programmatic dependent launches included) and
     // replayed while every host-visible argument stays the same: one launch per step instead of one
@@ -181,7 +182,9 @@ tidal_status_t ensure_ws(tidal_ctx* ctx, size_t bytes) {
     return TIDAL_OK;
 }
 
-// State layout for a capacity of R rows: counters | cursor | done | tile_ctr, each [R][CTR_STRIDE], then hist[R][TK_BINS].
+// State layout for a capacity of R rows: counters | cursor | done | tile_ctr set 0 | tile_ctr set 1, each
+// [R][CTR_STRIDE], then hist[R][TK_BINS]. Consecutive attention launches alternate between the two sets of
+// pool cursors, so that a launch may use its set before its predecessor has finished with the other.
 // Every counter has a 128-byte line of its own: hundreds of warps hit them at once, and atomics to one
 // line are served one after the other.
 constexpr int CTR_STRIDE = 32;
@@ -189,7 +192,7 @@ inline int* state_counters(const tidal_ctx* c) { return (int*)c->state; }
 inline int* state_cursor(const tidal_ctx* c) { return (int*)c->state + (size_t)CTR_STRIDE * c->state_rows; }
 inline int* state_done(const tidal_ctx* c) { return (int*)c->state + 2 * (size_t)CTR_STRIDE * c->state_rows; }
 inline int* state_tile_ctr(const tidal_ctx* c) { return (int*)c->state + 3 * (size_t)CTR_STRIDE * c->state_rows; }
-inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + 4 * (size_t)CTR_STRIDE * c->state_rows; }
+inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + 5 * (size_t)CTR_STRIDE * c->state_rows; }
 
 tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     if (ctx->state_rows >= rows) return TIDAL_OK;
@@ -197,7 +200,7 @@ tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     drop_graphs(ctx);
     if (ctx->state) { cudaDeviceSynchronize(); cudaFree(ctx->state); ctx->state = nullptr; ctx->state_rows = 0; }
     const int cap = (int)align_up((size_t)rows, 64);
-    const size_t bytes = (size_t)cap * (4 * CTR_STRIDE + TK_BINS) * sizeof(int);
+    const size_t bytes = (size_t)cap * (5 * CTR_STRIDE + TK_BINS) * sizeof(int);
     void* p = nullptr;
     if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TIDAL_ERR_NOMEM; }
     if (cudaMemset(p, 0, bytes) != cudaSuccess) { cudaFree(p); return TIDAL_ERR_CUDA; }
@@ -249,6 +252,8 @@ tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, cudaStream_t
     // Programmatic dependent launch: the kernel may begin while its predecessor in the stream
     // drains; it waits (griddepcontrol.wait) before touching anything that predecessor wrote.
     a.pdl = 1;
+    ctx->cursor_set ^= 1;
+    a.tile_ctr = state_tile_ctr(ctx) + (size_t)ctx->cursor_set * CTR_STRIDE * ctx->state_rows;
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(grid, 1, 1);
