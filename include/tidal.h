@@ -152,6 +152,13 @@ tidal_status_t tidal_decode_step(tidal_ctx_t *ctx, int32_t num_layers, const uin
                                  float *const *out_per_layer, int32_t k, int32_t granularity,
                                  int32_t *idx, int32_t *idx_count, void *stream);
 
+/* Output type of every later call on this context: TIDAL_OUT_F32 (default; `out` arguments are
+ * float*) or TIDAL_OUT_BF16 (the same `out` arguments then point to bf16 [batch, Hq, head_dim],
+ * each value the fp32 result rounded to nearest even; out_host of tidal_decode_step_host likewise).
+ * tidal_sparse_attn_noalloc always writes fp32. */
+enum { TIDAL_OUT_F32 = 0, TIDAL_OUT_BF16 = 1 };
+tidal_status_t tidal_set_output_dtype(tidal_ctx_t *ctx, int32_t dtype);
+
 /* Step graphs. When `stream` is an ordinary stream (not the legacy or per-thread default, and not
  * being captured by the caller), tidal_decode_step and tidal_decode_step_host record their launches
  * once as a CUDA graph and replay it for as long as every argument (schedule, descriptors, pointers,

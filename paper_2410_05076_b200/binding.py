@@ -26,7 +26,7 @@ EXPORTS = [
     "tidal_create", "tidal_destroy", "tidal_workspace_bytes", "tidal_full_attn", "tidal_select_attn",
     "tidal_sparse_attn", "tidal_decode_step", "tidal_decode_step_host", "tidal_device_status",
     "tidal_launch_count", "tidal_strerror", "tidal_sparse_attn_noalloc", "tidal_kv_append",
-    "tidal_decode_step_append", "tidal_set_graphs",
+    "tidal_decode_step_append", "tidal_set_graphs", "tidal_set_output_dtype",
 ]
 
 
@@ -75,6 +75,8 @@ def load() -> C.CDLL:
     L.tidal_workspace_bytes.restype = C.c_size_t
     L.tidal_decode_step_append.argtypes = [P, I32, P, KVP, P, P, P, P, I32, I32, P, P, P]
     L.tidal_decode_step_append.restype = I32
+    L.tidal_set_output_dtype.argtypes = [P, I32]
+    L.tidal_set_output_dtype.restype = I32
     L.tidal_set_graphs.argtypes = [P, I32]
     L.tidal_set_graphs.restype = I32
     L.tidal_kv_append.argtypes = [P, KVP, P, P, P]
@@ -159,6 +161,7 @@ class Tidal:
         self.ctx = C.c_void_p()
         _check(self.lib.tidal_create(C.byref(self.ctx), device, workspace_bytes), "tidal_create")
         self.device = device
+        self.out_dtype = torch.float32
 
     def close(self) -> None:
         if getattr(self, "ctx", None) and self.ctx.value:
@@ -184,7 +187,7 @@ class Tidal:
 
     def full_attn(self, layer, q: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
         if out is None:
-            out = torch.empty(layer.batch, layer.num_q_heads, layer.head_dim, dtype=torch.float32, device=q.device)
+            out = torch.empty(layer.batch, layer.num_q_heads, layer.head_dim, dtype=self.out_dtype, device=q.device)
         s = kv_struct(layer)
         _check(self.lib.tidal_full_attn(self.ctx, C.byref(s), q.data_ptr(), out.data_ptr(), _stream()),
                "tidal_full_attn")
@@ -195,7 +198,7 @@ class Tidal:
                     idx_count: Optional[torch.Tensor] = None, scores: Optional[torch.Tensor] = None):
         hi = {SEL_PER_QHEAD: layer.num_q_heads, SEL_PER_KVHEAD: layer.num_kv_heads, SEL_SHARED: 1}.get(granularity, 1)
         if out is None:
-            out = torch.empty(layer.batch, layer.num_q_heads, layer.head_dim, dtype=torch.float32, device=q.device)
+            out = torch.empty(layer.batch, layer.num_q_heads, layer.head_dim, dtype=self.out_dtype, device=q.device)
         if idx is None:
             idx = torch.empty(layer.batch, hi, max(k, 1), dtype=torch.int32, device=q.device)
         if idx_count is None:
@@ -210,7 +213,7 @@ class Tidal:
     def sparse_attn(self, layer, q: torch.Tensor, idx: torch.Tensor, idx_count: Optional[torch.Tensor] = None,
                     out: Optional[torch.Tensor] = None) -> torch.Tensor:
         if out is None:
-            out = torch.empty(layer.batch, layer.num_q_heads, layer.head_dim, dtype=torch.float32, device=q.device)
+            out = torch.empty(layer.batch, layer.num_q_heads, layer.head_dim, dtype=self.out_dtype, device=q.device)
         s = kv_struct(layer)
         _, hi, k = idx.shape
         _check(self.lib.tidal_sparse_attn(self.ctx, C.byref(s), q.data_ptr(), idx.data_ptr(),
@@ -243,7 +246,7 @@ class Tidal:
         """One step including the cache update: k_new[i], v_new[i] (bf16 [B, Hkv, d]) go to position
         ctx_lens[b] - 1 of layer i's cache before the layers run. Returns (outs, idx, idx_count)."""
         L = len(sched)
-        outs = [torch.empty(l.batch, l.num_q_heads, l.head_dim, dtype=torch.float32, device=qs[0].device)
+        outs = [torch.empty(l.batch, l.num_q_heads, l.head_dim, dtype=self.out_dtype, device=qs[0].device)
                 for l in layers]
         hi = {SEL_PER_QHEAD: layers[0].num_q_heads, SEL_PER_KVHEAD: layers[0].num_kv_heads, SEL_SHARED: 1}[granularity]
         idx = torch.full((layers[0].batch, hi, k), -1, dtype=torch.int32, device=qs[0].device)
@@ -256,7 +259,7 @@ class Tidal:
         return outs, idx, cnt
 
     def decode_step(self, sched, layers, qs, k: int, granularity: int = SEL_PER_QHEAD):
-        outs = [torch.empty(l.batch, l.num_q_heads, l.head_dim, dtype=torch.float32, device=qs[0].device)
+        outs = [torch.empty(l.batch, l.num_q_heads, l.head_dim, dtype=self.out_dtype, device=qs[0].device)
                 for l in layers]
         step = self.make_step(sched, layers, qs, outs, k, granularity)
         step()
@@ -278,6 +281,11 @@ class Tidal:
 
         step.keep = (sched_arr, kvs, list(layers), q_host, out_host)
         return step
+
+    def set_output_bf16(self, enabled: bool) -> None:
+        """Later calls write bf16 outputs (pass bf16 `out` tensors) instead of fp32."""
+        _check(self.lib.tidal_set_output_dtype(self.ctx, 1 if enabled else 0), "tidal_set_output_dtype")
+        self.out_dtype = torch.bfloat16 if enabled else torch.float32
 
     def set_graphs(self, enabled: bool) -> None:
         """Record whole steps as CUDA graphs and replay them (on by default; needs a non-default stream)."""

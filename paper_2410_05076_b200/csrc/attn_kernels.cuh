@@ -55,7 +55,8 @@ struct AttnParams {
     const __nv_bfloat16* q;
     const __nv_bfloat16* k;
     const __nv_bfloat16* v;
-    float* out;
+    float* out;                // [B, Hq, 128]; bf16 instead of fp32 when out_bf16 is set
+    int out_bf16;
     long long stride_b, stride_pos, stride_head, stride_page;
     const int* page_table;
     int max_pages, num_pages, paged;
@@ -129,6 +130,11 @@ __device__ __forceinline__ void cp_async_wait() {
 // Programmatic dependent launch: this grid may start while the previous kernel of the stream
 // is still draining. pdl_wait() blocks until that kernel has completed and its writes are
 // visible; pdl_trigger() lets the next kernel start filling SMs as our CTAs retire.
+// One output element: fp32, or rounded to bf16 (nearest even) for callers that feed a bf16 GEMM next.
+__device__ __forceinline__ void store_out(const AttnParams& p, long long i, float v) {
+    if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[i] = __float2bfloat16_rn(v);
+    else p.out[i] = v;
+}
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 
@@ -707,7 +713,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                 }
             }
             if (nsplits == 1) {
-                p.out[(row0 + col) * HEAD_DIM + c] = (L > 0.f) ? O / L : 0.f;
+                store_out(p, (row0 + col) * HEAD_DIM + c, (L > 0.f) ? O / L : 0.f);
             } else if (split < p.max_splits) {
                 const long long pr = (row0 + col) * p.max_splits + split;
                 p.part_o[pr * HEAD_DIM + c] = O;
@@ -779,7 +785,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                         for (int u = 0; u < 8; ++u) O += v[u] * fs[s + u];
                     }
                     for (; s < ns; ++s) O += __ldcg(po + (long long)s * HEAD_DIM) * fs[s];
-                    p.out[(row0 + col) * HEAD_DIM + c] = O * linv[col];
+                    store_out(p, (row0 + col) * HEAD_DIM + c, O * linv[col]);
                 }
                 if (threadIdx.x == 0) { *ctr = 0; if (pooled) *pool = 0; }   // ready for the next launch
             }

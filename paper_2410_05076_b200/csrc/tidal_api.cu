@@ -48,6 +48,7 @@ struct tidal_ctx {
     void* state = nullptr;
     int state_rows = 0;                         // capacity in (sequence, head) rows
     int* status = nullptr;                      // device word, sticky
+    int out_bf16 = 0;                           // outputs are written as bf16 instead of fp32
     int cursor_set = 0;                         // which of the two sets of pool cursors the last attention launch used
     int64_t launches = 0;
     // Whole steps are recorded once as CUDA graphs (programmatic dependent launches included) and
@@ -221,6 +222,7 @@ void fill_common(AttnParams& a, const tidal_ctx* ctx, const tidal_kv_t* kv, cons
     a.k = (const __nv_bfloat16*)kv->k;
     a.v = (const __nv_bfloat16*)kv->v;
     a.out = out;
+    a.out_bf16 = ctx->out_bf16;
     a.stride_b = kv->stride_b; a.stride_pos = kv->stride_pos; a.stride_head = kv->stride_head;
     a.stride_page = kv->stride_page;
     a.page_table = kv->page_table; a.max_pages = kv->max_pages_per_seq; a.num_pages = kv->num_pages;
@@ -401,7 +403,7 @@ struct KeyBuilder {
 void step_key(KeyBuilder& kb, const tidal_ctx* ctx, int tag, int32_t num_layers, const uint8_t* schedule,
                      const tidal_kv_t* kvs, int32_t k, int32_t granularity, int host_layers) {
     kb.add(tag); kb.add(num_layers); kb.add(k); kb.add(granularity); kb.add(host_layers);
-    kb.add(ctx->ws); kb.add(ctx->state);
+    kb.add(ctx->ws); kb.add(ctx->state); kb.add(ctx->out_bf16);
     kb.add_raw(schedule, (size_t)num_layers);
     for (int i = 0; i < num_layers; ++i) {
         // field by field: the struct has padding whose bytes are not the caller's to define
@@ -708,6 +710,12 @@ tidal_status_t tidal_decode_step(tidal_ctx_t* ctx, int32_t num_layers, const uin
     });
 }
 
+tidal_status_t tidal_set_output_dtype(tidal_ctx_t* ctx, int32_t dtype) {
+    if (!ctx || (dtype != TIDAL_OUT_F32 && dtype != TIDAL_OUT_BF16)) return TIDAL_ERR_INVALID;
+    ctx->out_bf16 = dtype == TIDAL_OUT_BF16;
+    return TIDAL_OK;
+}
+
 tidal_status_t tidal_set_graphs(tidal_ctx_t* ctx, int32_t enabled) {
     if (!ctx) return TIDAL_ERR_INVALID;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
@@ -742,11 +750,12 @@ tidal_status_t tidal_decode_step_host(tidal_ctx_t* ctx, int32_t num_layers, cons
     char* ws = (char*)ctx->ws;
     char* qd = ws + w.q_stage;
     float* od = (float*)(ws + w.out_stage);
+    const size_t out_elem = ctx->out_bf16 ? 2 : 4;            // bytes per output element, device and host side
     const void* qs[1024];
     float* outs[1024];
     for (int i = 0; i < num_layers; ++i) {
         qs[i] = qd + (size_t)i * rows * HEAD_DIM * 2;
-        outs[i] = od + (size_t)i * rows * HEAD_DIM;
+        outs[i] = (float*)((char*)od + (size_t)i * rows * HEAD_DIM * out_elem);
     }
     if ((rc = decode_step_prepare(ctx, num_layers, schedule, kv_per_layer, qs, outs, k, granularity, num_layers)) != TIDAL_OK)
         return rc;
@@ -756,7 +765,7 @@ tidal_status_t tidal_decode_step_host(tidal_ctx_t* ctx, int32_t num_layers, cons
         const tidal_status_t r = decode_step_enqueue(ctx, num_layers, schedule, kv_per_layer, qs, outs, k, granularity,
                                                      (int*)(ws + w.idx), (int*)(ws + w.idx_count), num_layers, st);
         if (r != TIDAL_OK) return r;
-        if (cudaMemcpyAsync(out_host, od, (size_t)num_layers * rows * HEAD_DIM * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        if (cudaMemcpyAsync(out_host, od, (size_t)num_layers * rows * HEAD_DIM * out_elem, cudaMemcpyDeviceToHost, st) != cudaSuccess)
             return TIDAL_ERR_CUDA;
         return TIDAL_OK;
     };

@@ -587,3 +587,39 @@ def test_library_records_and_replays_step_graphs(td):
     for o, r in zip(outs, ref_outs):
         assert torch.allclose(o, r, rtol=0, atol=5e-4)
     assert td.device_status() == binding.OK
+
+
+def test_bf16_outputs_are_the_fp32_results_rounded(td):
+    """With the bf16 output type every call writes the rounded fp32 result; everything else is unchanged."""
+    sched = [0, 1, 2]
+    w = wl(2, 8, 2, 700, 64, ragged=True, ctx_min=300, seed=31, layers=len(sched))
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    layers = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(len(sched))]
+    ref_outs, ref_idx, _ = td.decode_step(sched, layers, qs, w.k)
+    ref_full = td.full_attn(layers[0], qs[0])
+    torch.cuda.synchronize()
+    td.set_output_bf16(True)
+    try:
+        outs, idx, cnt = td.decode_step(sched, layers, qs, w.k)
+        full = td.full_attn(layers[0], qs[0])
+        _, idx2, cnt2 = td.select_attn(layers[1], qs[1], w.k)
+        sp = td.sparse_attn(layers[2], qs[2], idx2, cnt2)
+        q_host = torch.stack([q.cpu() for q in qs]).contiguous().pin_memory()
+        out_host = torch.zeros(len(sched), 2, 8, 128, dtype=torch.bfloat16).pin_memory()
+        td.make_step_host(sched, layers, q_host, out_host, w.k)()
+        torch.cuda.synchronize()
+    finally:
+        td.set_output_bf16(False)
+    assert torch.equal(idx, ref_idx) and torch.equal(idx2, ref_idx)
+    for o, r, h in zip(outs, ref_outs, out_host):
+        assert o.dtype == torch.bfloat16
+        # equal to the rounded fp32 result up to the run-to-run variation of the fp32 value (one bf16 step)
+        assert torch.allclose(o.float(), r.to(torch.bfloat16).float(), rtol=2 ** -7, atol=5e-4)
+        assert torch.allclose(h.to(DEV).float(), r, rtol=2 ** -7, atol=5e-4)
+    assert torch.allclose(full.float(), ref_full, rtol=2 ** -7, atol=5e-4)
+    assert torch.allclose(sp.float(), ref_outs[2], rtol=2 ** -7, atol=5e-4)
+    okv, qb = util.oracle_kv(layers[0]), synth.bits(qs[0])
+    util.check_out(full.float().cpu().numpy(), oracle.full_attn(okv, qb), "bf16 full vs oracle")
+    again = td.full_attn(layers[0], qs[0])
+    assert again.dtype == torch.float32
+    assert td.device_status() == binding.OK
