@@ -623,3 +623,33 @@ def test_bf16_outputs_are_the_fp32_results_rounded(td):
     again = td.full_attn(layers[0], qs[0])
     assert again.dtype == torch.float32
     assert td.device_status() == binding.OK
+
+
+def test_two_contexts_on_two_streams_do_not_interfere(td):
+    """Each context owns its workspace, counters and step graphs: two of them driven alternately on two
+    streams give the results of one."""
+    sched = [0, 1, 2, 2]
+    w = wl(1, 8, 2, 2500, 96, seed=37, layers=len(sched))
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    layers = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(len(sched))]
+    ref_outs, ref_idx, _ = td.decode_step(sched, layers, qs, w.k)
+    torch.cuda.synchronize()
+    other = binding.Tidal(0)
+    try:
+        sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+        outs_a = [torch.zeros_like(o) for o in ref_outs]
+        outs_b = [torch.zeros_like(o) for o in ref_outs]
+        step_a = td.make_step(sched, layers, qs, outs_a, w.k)
+        step_b = other.make_step(sched, layers, qs, outs_b, w.k)
+        for _ in range(4):
+            with torch.cuda.stream(sa):
+                step_a()
+            with torch.cuda.stream(sb):
+                step_b()
+        torch.cuda.synchronize()
+        for oa, ob, r in zip(outs_a, outs_b, ref_outs):
+            assert torch.allclose(oa, r, rtol=0, atol=5e-4) and torch.allclose(ob, r, rtol=0, atol=5e-4)
+        assert torch.equal(step_a.idx, ref_idx) and torch.equal(step_b.idx, ref_idx)
+        assert other.device_status() == binding.OK
+    finally:
+        other.close()
