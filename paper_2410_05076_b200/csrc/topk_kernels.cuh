@@ -70,6 +70,11 @@ __device__ __forceinline__ uint32_t score_key(float s) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// The value whose key is `key` (inverse of score_key; -0 never occurs as a key).
+__device__ __forceinline__ float key_score(uint32_t key) {
+    return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+
 // Keys of this thread's positions of the slice starting at s0: TK_VEC groups of four
 // consecutive positions, group j at s0 + 4*(j*TK_THREADS + tid). All loads are issued
 // before any is used. Positions at or beyond n get key 0 and valid bit 0.
@@ -308,19 +313,20 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     unsigned* bm = solo ? solo_bm : p.bitmap + (long long)item * p.bitmap_stride;
     const int bm_base = solo ? 0 : (s0 >> 5);
     unsigned eq_mask = 0;                                          // bit 4j+e: group j, element e
+    // the values whose keys open bin b1 and bin b1 + 1 (nothing lies above the last bin: NaN compares false)
+    const float f_lo = key_score((uint32_t)b1 << p.shift);
+    const float f_hi = (b1 + 1 >= (1 << (32 - p.shift))) ? __uint_as_float(0x7fc00000u) : key_score((uint32_t)(b1 + 1) << p.shift);
 #pragma unroll
     for (int j = 0; j < TK_BATCHES * TK_VEC; ++j) {
         const int off = 4 * (j * TK_THREADS + tid);
         const float4 f = *reinterpret_cast<const float4*>(raw + off);
-        const float fe[4] = {f.x, f.y, f.z, f.w};
-        unsigned nib = 0;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const bool ok = s0 + off + e < N;
-            const int bin = (int)(score_key(fe[e]) >> p.shift);
-            if (ok && bin > b1) nib |= 1u << e;
-            if (ok && bin == b1) eq_mask |= 1u << (4 * j + e);
-        }
+        // bin > b1 <=> f >= f_hi and bin >= b1 <=> f >= f_lo: the key is monotone in the value, so two
+        // float comparisons per score replace the key transform
+        const unsigned ok = (1u << max(0, min(4, N - (s0 + off)))) - 1u;
+        const unsigned hi4 = (f.x >= f_hi ? 1u : 0u) | (f.y >= f_hi ? 2u : 0u) | (f.z >= f_hi ? 4u : 0u) | (f.w >= f_hi ? 8u : 0u);
+        const unsigned lo4 = (f.x >= f_lo ? 1u : 0u) | (f.y >= f_lo ? 2u : 0u) | (f.z >= f_lo ? 4u : 0u) | (f.w >= f_lo ? 8u : 0u);
+        const unsigned nib = hi4 & ok;
+        eq_mask |= (lo4 & ~hi4 & ok) << (4 * j);
         unsigned word = nib << (4 * (lane & 7));
         word |= __shfl_xor_sync(0xffffffffu, word, 1);
         word |= __shfl_xor_sync(0xffffffffu, word, 2);
