@@ -393,19 +393,43 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         TIDAL_TRACE2(4);
         if (!s_last) return;
 
-        M = (int)min((long long)__ldcg(&p.cursor[(size_t)item * p.ctr_stride]), p.cand_stride);
+        // One round trip for everything the last CTA needs: the candidate count, the winners' bitmap
+        // written by all CTAs of this head (pulled into shared memory; candidates that turn out to be
+        // winners are ORed into the same words) and, without waiting for the count, the first 2048
+        // candidate slots (a usual threshold bin holds about that many; unused slots are in bounds).
+        constexpr int BM_REGS = 16, CAND_REGS = 4;             // 16 x 512 words = the longest supported context
         cgt = reinterpret_cast<unsigned*>(tk_smem);
         ceq = cgt + words;
         uint2* scand = reinterpret_cast<uint2*>(ceq + words);      // [cand_smem]; 8*words bytes in: 8-byte aligned
+        unsigned bmreg[BM_REGS];
+        uint2 creg[CAND_REGS];
+#pragma unroll
+        for (int j = 0; j < BM_REGS; ++j) {
+            const int i = tid + j * TK_THREADS;
+            bmreg[j] = (i < words) ? __ldcg(&bm[i]) : 0u;
+        }
+#pragma unroll
+        for (int j = 0; j < CAND_REGS; ++j) {
+            const int i = tid + j * TK_THREADS;
+            creg[j] = (i < p.cand_stride && i < p.cand_smem) ? __ldcg(&cand[i]) : make_uint2(0u, 0u);
+        }
+        M = (int)min((long long)__ldcg(&p.cursor[(size_t)item * p.ctr_stride]), p.cand_stride);
         c = cand;
         if (M <= p.cand_smem) {
+#pragma unroll
+            for (int j = 0; j < CAND_REGS; ++j) {
+                const int i = tid + j * TK_THREADS;
+                if (i < M) scand[i] = creg[j];
+            }
 #pragma unroll 4
-            for (int i = tid; i < M; i += TK_THREADS) scand[i] = __ldcg(&cand[i]);
+            for (int i = tid + CAND_REGS * TK_THREADS; i < M; i += TK_THREADS) scand[i] = __ldcg(&cand[i]);
             c = scand;
         }
-        // The winners' bitmap written by all CTAs of this head is pulled into shared memory once
-        // (coalesced); candidates that turn out to be winners are ORed into the same words.
-        for (int i = tid; i < words; i += TK_THREADS) { cgt[i] = __ldcg(&bm[i]); ceq[i] = 0; }
+#pragma unroll
+        for (int j = 0; j < BM_REGS; ++j) {
+            const int i = tid + j * TK_THREADS;
+            if (i < words) { cgt[i] = bmreg[j]; ceq[i] = 0; }
+        }
         for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
         __syncthreads();
     }
