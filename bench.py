@@ -33,7 +33,7 @@ METRIC = "us_per_decode_step_attention_all_layers"
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) of one full-attention launch at the cfg3 shape, from the ncu
 # capture summarised in profiles/attn_topk_kernels_cfg3_ncu_full.md (dram__bytes_read.sum + dram__bytes_write.sum).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg3": 536.96e6 + 3.90e6}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg3": 536.94e6 + 3.86e6}
 
 
 def describe(w: synth.Workload) -> str:
