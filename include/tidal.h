@@ -26,6 +26,9 @@
  *   - q is bf16 [batch, num_q_heads, head_dim] contiguous; outputs are fp32
  *     [batch, num_q_heads, head_dim] contiguous. Arithmetic: bf16 inputs,
  *     fp32 accumulation.
+ *   - A context holds scratch memory and counters that its calls share: use it
+ *     from one host thread and on one stream at a time (work of consecutive
+ *     calls may overlap on that stream; calls on two streams need two contexts).
  *   - There is no CPU path: on a machine without a usable GPU tidal_create()
  *     fails with TIDAL_ERR_CUDA.
  */
