@@ -155,6 +155,12 @@ tidal_status_t tidal_decode_step(tidal_ctx_t *ctx, int32_t num_layers, const uin
                                  float *const *out_per_layer, int32_t k, int32_t granularity,
                                  int32_t *idx, int32_t *idx_count, void *stream);
 
+/* Optional deviation from Algorithm 1 (off by default): with enabled != 0 every later sparse layer on
+ * this context also attends the newest token, position ctx_lens[b] - 1, whether or not it was
+ * selected. A list that already ends with that position (lists from tidal_select_attn are ascending) is
+ * left as it is, so the token never counts twice. tidal_sparse_attn then needs idx_count. */
+tidal_status_t tidal_set_attend_newest(tidal_ctx_t *ctx, int32_t enabled);
+
 /* Output type of every later call on this context: TIDAL_OUT_F32 (default; `out` arguments are
  * float*) or TIDAL_OUT_BF16 (the same `out` arguments then point to bf16 [batch, Hq, head_dim],
  * each value the fp32 result rounded to nearest even; out_host of tidal_decode_step_host likewise).

@@ -201,6 +201,23 @@ def sparse_attn(kv: KV, q: np.ndarray, idx: np.ndarray, idx_count: Optional[np.n
     return out
 
 
+def with_newest(kv: KV, idx: np.ndarray, idx_count: np.ndarray):
+    """Index lists for the optional 'always attend the newest token' variant (not in the paper): every
+    list gets one more slot holding position ctx_len - 1, or -1 if the list already ends with it. Data
+    preparation only; the attention itself is sparse_attn on the returned lists."""
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    B, hi, k = idx.shape
+    out = np.full((B, hi, k + 1), -1, dtype=np.int32)
+    cnt = np.asarray(idx_count, dtype=np.int32)
+    for b in range(B):
+        c, n = int(min(cnt[b], k)), int(kv.ctx_lens[b])
+        out[b, :, :c] = idx[b, :, :c]
+        for h in range(hi):
+            last = idx[b, h, c - 1] if c > 0 else -1
+            out[b, h, c] = n - 1 if (n > 0 and last != n - 1) else -1
+    return out, cnt + 1
+
+
 def kv_append(kv: KV, k_new: np.ndarray, v_new: np.ndarray) -> None:
     """C.append(k, v): writes the rows [B, Hkv, d] at position ctx_lens[b] - 1 of kv's arrays, in place."""
     k_new, v_new = _q(k_new), _q(v_new)

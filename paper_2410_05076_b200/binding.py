@@ -26,7 +26,7 @@ EXPORTS = [
     "tidal_create", "tidal_destroy", "tidal_workspace_bytes", "tidal_full_attn", "tidal_select_attn",
     "tidal_sparse_attn", "tidal_decode_step", "tidal_decode_step_host", "tidal_device_status",
     "tidal_launch_count", "tidal_strerror", "tidal_sparse_attn_noalloc", "tidal_kv_append",
-    "tidal_decode_step_append", "tidal_set_graphs", "tidal_set_output_dtype",
+    "tidal_decode_step_append", "tidal_set_graphs", "tidal_set_output_dtype", "tidal_set_attend_newest",
 ]
 
 
@@ -75,6 +75,8 @@ def load() -> C.CDLL:
     L.tidal_workspace_bytes.restype = C.c_size_t
     L.tidal_decode_step_append.argtypes = [P, I32, P, KVP, P, P, P, P, I32, I32, P, P, P]
     L.tidal_decode_step_append.restype = I32
+    L.tidal_set_attend_newest.argtypes = [P, I32]
+    L.tidal_set_attend_newest.restype = I32
     L.tidal_set_output_dtype.argtypes = [P, I32]
     L.tidal_set_output_dtype.restype = I32
     L.tidal_set_graphs.argtypes = [P, I32]
@@ -281,6 +283,10 @@ class Tidal:
 
         step.keep = (sched_arr, kvs, list(layers), q_host, out_host)
         return step
+
+    def set_attend_newest(self, enabled: bool) -> None:
+        """Sparse layers also attend the newest token (an optional deviation from the paper's algorithm)."""
+        _check(self.lib.tidal_set_attend_newest(self.ctx, 1 if enabled else 0), "tidal_set_attend_newest")
 
     def set_output_bf16(self, enabled: bool) -> None:
         """Later calls write bf16 outputs (pass bf16 `out` tensors) instead of fp32."""

@@ -323,7 +323,8 @@ __device__ __forceinline__ void consume_tile(const AttnParams& p, uint32_t ks, u
 // produces its (all-zero) output row.
 __device__ __forceinline__ int item_tiles(int total) { return max(1, (total + TILE - 1) / TILE); }
 
-template <int MODE, int NW, int STAGES>
+// NEWEST (gather kernel only): every list has one more slot that stands for the newest token.
+template <int MODE, int NW, int STAGES, bool NEWEST = false>
 __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     // Ring slots must be 256-byte aligned (the V fragment addressing XORs bits 5-7).
@@ -349,7 +350,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         const int N = min(p.ctx_lens[b], p.max_ctx);
         if (MODE != MODE_SPARSE) return max(N, 0);
         const int cnt = p.idx_count ? min(p.idx_count[b], p.budget) : p.budget;
-        return max(cnt, 0);
+        return max(cnt, 0) + (NEWEST ? 1 : 0);
     };
     long long per_cta, lo, hi, seq_start = 0;
     int b = 0, tiles_b;
@@ -420,6 +421,14 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             idx_row = p.idx + ((long long)b * p.Hi + hi_idx) * p.budget;
         }
         int* pool = pooled ? p.tile_ctr + ((long long)b * IY + y) * p.ctr_stride : nullptr;
+        // Optional deviation from Algorithm 1: the newest token is attended even if it was not selected.
+        // The reserved last slot of the list stands for it unless the (ascending) list already ends with it.
+        int newest_pos = -1;
+        if (MODE == MODE_SPARSE && NEWEST) {
+            const int cnt = total - 1;
+            const int last = cnt > 0 ? __ldg(idx_row + cnt - 1) : -1;
+            if (N > 0 && last != N - 1) newest_pos = N - 1;
+        }
 
         float* score_row0 = nullptr;
         float* score_row1 = nullptr;
@@ -486,6 +495,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         auto load_pos = [&](int tile) -> int {
             if (MODE != MODE_SPARSE || tile < 0) return -1;
             const int e = tile * TILE + c16;
+            if (NEWEST && e == total - 1) return newest_pos;
             return (e < total) ? __ldg(idx_row + e) : -1;
         };
         long long offA = 0;

@@ -49,6 +49,7 @@ struct tidal_ctx {
     int state_rows = 0;                         // capacity in (sequence, head) rows
     int* status = nullptr;                      // device word, sticky
     int out_bf16 = 0;                           // outputs are written as bf16 instead of fp32
+    int attend_newest = 0;                      // sparse layers also attend the newest token (not in the paper)
     int cursor_set = 0;                         // which of the two sets of pool cursors the last attention launch used
     int64_t launches = 0;
     // Whole steps are recorded once as CUDA graphs (programmatic dependent launches included) and
@@ -249,7 +250,7 @@ constexpr size_t attn_smem() {
     return (size_t)NW * STAGES * STAGE_BYTES + (MODE == MODE_SELECT ? HIST_SMEM : 0) + 1024;   // + alignment slack
 }
 
-template <int MODE, int NW, int STAGES>
+template <int MODE, int NW, int STAGES, bool NEWEST = false>
 tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, cudaStream_t st) {
     // Programmatic dependent launch: the kernel may begin while its predecessor in the stream
     // drains; it waits (griddepcontrol.wait) before touching anything that predecessor wrote.
@@ -268,7 +269,7 @@ tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, cudaStream_t
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     ctx->launches++;
-    return cudaLaunchKernelEx(&cfg, attn_kernel<MODE, NW, STAGES>, a) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, attn_kernel<MODE, NW, STAGES, NEWEST>, a) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }
 
 // How a selection layer produces its ranking scores. Per query head: one row per head, histogram
@@ -376,6 +377,7 @@ tidal_status_t run_sparse(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, c
     if (const int S = pooled_splits(kv, kv->batch * per_batch, grid)) {
         a.splits_per_item = S;
     }
+    if (ctx->attend_newest) return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES, true>(ctx, a, grid, st);
     return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(ctx, a, grid, st);
 }
 
@@ -403,7 +405,7 @@ struct KeyBuilder {
 void step_key(KeyBuilder& kb, const tidal_ctx* ctx, int tag, int32_t num_layers, const uint8_t* schedule,
                      const tidal_kv_t* kvs, int32_t k, int32_t granularity, int host_layers) {
     kb.add(tag); kb.add(num_layers); kb.add(k); kb.add(granularity); kb.add(host_layers);
-    kb.add(ctx->ws); kb.add(ctx->state); kb.add(ctx->out_bf16);
+    kb.add(ctx->ws); kb.add(ctx->state); kb.add(ctx->out_bf16); kb.add(ctx->attend_newest);
     kb.add_raw(schedule, (size_t)num_layers);
     for (int i = 0; i < num_layers; ++i) {
         // field by field: the struct has padding whose bytes are not the caller's to define
@@ -493,9 +495,10 @@ tidal_status_t tidal_create(tidal_ctx_t** out, int device, size_t workspace_byte
     const int d0 = resident_ctas(attn_kernel<MODE_FULL, DENSE_NW, DENSE_STAGES>, DENSE_NW * 32, attn_smem<MODE_FULL, DENSE_NW, DENSE_STAGES>(), ctx->sm_count);
     const int d1 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW, DENSE_STAGES>, DENSE_NW * 32, attn_smem<MODE_SELECT, DENSE_NW, DENSE_STAGES>(), ctx->sm_count);
     const int s0 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>, SPARSE_NW * 32, attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(), ctx->sm_count);
+    const int s1 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES, true>, SPARSE_NW * 32, attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(), ctx->sm_count);
     const size_t topk_smem = 2 * (size_t)(MAX_CTX / 32) * sizeof(unsigned) + 8192 * sizeof(uint2);
     const bool topk_ok = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topk_smem) == cudaSuccess;
-    if (d0 <= 0 || d1 <= 0 || s0 <= 0 || !topk_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
+    if (d0 <= 0 || d1 <= 0 || s0 <= 0 || s1 < s0 || !topk_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
     ctx->dense_slots = std::min(d0, d1);
     ctx->sparse_slots = s0;
     if (cudaMalloc((void**)&ctx->status, 256) != cudaSuccess || cudaMemset(ctx->status, 0, 256) != cudaSuccess) {
@@ -598,6 +601,7 @@ tidal_status_t tidal_sparse_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const v
     if (k <= 0) return TIDAL_ERR_INVALID;
     const int Hi = num_index_heads;
     if (Hi != kv->num_q_heads && Hi != kv->num_kv_heads && Hi != 1) return TIDAL_ERR_INVALID;
+    if (ctx->attend_newest && !idx_count) return TIDAL_ERR_INVALID;   // the end of each list must be known
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
     const WsLayout w = layout_ws(kv, k, 0);
     if ((rc = ensure_all(ctx, kv, w.total)) != TIDAL_OK) return rc;
@@ -708,6 +712,12 @@ tidal_status_t tidal_decode_step(tidal_ctx_t* ctx, int32_t num_layers, const uin
         return decode_step_enqueue(ctx, num_layers, schedule, kv_per_layer, q_per_layer, out_per_layer, k, granularity,
                                    idx, idx_count, 0, st);
     });
+}
+
+tidal_status_t tidal_set_attend_newest(tidal_ctx_t* ctx, int32_t enabled) {
+    if (!ctx) return TIDAL_ERR_INVALID;
+    ctx->attend_newest = enabled != 0;
+    return TIDAL_OK;
 }
 
 tidal_status_t tidal_set_output_dtype(tidal_ctx_t* ctx, int32_t dtype) {

@@ -653,3 +653,42 @@ def test_two_contexts_on_two_streams_do_not_interfere(td):
         assert other.device_status() == binding.OK
     finally:
         other.close()
+
+
+@pytest.mark.parametrize("layout", ["hnd_interleaved", "paged"])
+def test_sparse_layers_can_always_attend_the_newest_token(td, layout):
+    """The optional variant (not in the paper): every list is extended by the newest position unless it
+    already ends with it; compared with the oracle on lists extended the same way, alone and in a step."""
+    sched = [1, 2, 2]
+    w = wl(3, 8, 2, 900, 48, ragged=True, ctx_min=100, seed=41, layers=len(sched))
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    if layout == "paged":
+        pt, total = synth.make_page_table(w, extra_pages=2)
+        layers = [synth.make_layer(w, i, DEV, layout="paged", q=qs[i], page_table=pt, num_pages=total) for i in range(len(sched))]
+    else:
+        layers = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(len(sched))]
+    lens = layers[0].ctx_lens.cpu().numpy()
+    _, idx, cnt = td.select_attn(layers[0], qs[0], w.k)
+    idx_h, cnt_h = idx.cpu().numpy().copy(), cnt.cpu().numpy().copy()
+    idx_h[0, 0, w.k - 1] = lens[0] - 1                    # one list that already ends with the newest token
+    idx_h[0, 0, : w.k - 1] = np.arange(w.k - 1)
+    idx_d = torch.from_numpy(idx_h).to(DEV)
+    td.set_attend_newest(True)
+    try:
+        sp = td.sparse_attn(layers[1], qs[1], idx_d, cnt)
+        outs, idx2, cnt2 = td.decode_step(sched, layers, qs, w.k)
+        with pytest.raises(binding.TidalError):
+            td.sparse_attn(layers[1], qs[1], idx_d)       # the end of the lists must be known
+        torch.cuda.synchronize()
+    finally:
+        td.set_attend_newest(False)
+    okv1, okv2 = util.oracle_kv(layers[1]), util.oracle_kv(layers[2])
+    aug, cnt_aug = oracle.with_newest(okv1, idx_h, cnt_h)
+    util.check_out(sp.cpu().numpy(), oracle.sparse_attn(okv1, synth.bits(qs[1]), aug, cnt_aug), "newest.sparse")
+    plain = td.sparse_attn(layers[1], qs[1], idx_d, cnt)
+    assert not torch.allclose(plain, sp, atol=1e-6)      # the extra token changes the result ...
+    assert torch.allclose(plain[0, 0], sp[0, 0], atol=5e-4)   # ... except where the list had it already
+    aug2, cnt_aug2 = oracle.with_newest(okv1, idx2.cpu().numpy(), cnt2.cpu().numpy())
+    util.check_out(outs[1].cpu().numpy(), oracle.sparse_attn(okv1, synth.bits(qs[1]), aug2, cnt_aug2), "newest.step1")
+    util.check_out(outs[2].cpu().numpy(), oracle.sparse_attn(okv2, synth.bits(qs[2]), aug2, cnt_aug2), "newest.step2")
+    assert td.device_status() == binding.OK

@@ -444,3 +444,21 @@ def test_append_through_a_page_table_equals_contiguous_append():
     for b in range(B):
         pos = lens[b] - 1
         assert np.array_equal(pkv.k.reshape(pool_k.shape)[perm[b, pos // PS], pos % PS], kn[b])
+
+
+# ---- optional variant: sparse layers always attend the newest token ----------------------------
+def test_newest_token_variant_closed_forms():
+    """A dominant newest key returns the newest value row although rho excludes it; a list that already
+    ends with the newest position is left alone (no double count)."""
+    B, Hq, Hkv, N = 1, 2, 1, 60
+    q, k, v, kv = make(B, Hq, Hkv, N, 53)
+    qv = bf16_val(q)
+    k[0, N - 1, 0] = bf16_bits(40.0 * (qv[0, 0] + qv[0, 1]))
+    idx = np.array([[[3, 10, 20], [5, 6, N - 1]]], np.int32)
+    cnt = np.array([3], np.int32)
+    plain = oracle.sparse_attn(kv, q, idx, cnt)
+    aug, cnt2 = oracle.with_newest(kv, idx, cnt)
+    assert aug[0, 0].tolist() == [3, 10, 20, N - 1] and aug[0, 1].tolist() == [5, 6, N - 1, -1] and cnt2.tolist() == [4]
+    out = oracle.sparse_attn(kv, q, aug, cnt2)
+    assert np.allclose(out[0, 0], bf16_val(v)[0, N - 1, 0], atol=1e-6)      # head 0 now sees the dominant key
+    assert np.array_equal(out[0, 1], plain[0, 1])                            # head 1 had it already
