@@ -51,9 +51,10 @@ enum {
     TIDAL_ERR_UNSUPPORTED = -2,   /* valid request outside what is built (head_dim != 128, ...) */
     TIDAL_ERR_NOMEM = -3,         /* workspace allocation failed */
     TIDAL_ERR_CUDA = -4,          /* a CUDA runtime call failed */
-    TIDAL_ERR_TIMEOUT = -5,       /* reserved: a bounded device-side wait expired */
+    TIDAL_ERR_TIMEOUT = -5,       /* reserved: a bounded device-side wait expired (no kernel waits on another) */
     TIDAL_ERR_INDEX = -6,         /* device saw a token index or page id out of range */
-    TIDAL_ERR_TOO_LARGE = -7      /* tidal_sparse_attn_noalloc only: problem exceeds its fixed scratch */
+    TIDAL_ERR_TOO_LARGE = -7,     /* tidal_sparse_attn_noalloc only: problem exceeds its fixed scratch */
+    TIDAL_ERR_INTERNAL = -8       /* a kernel found the host's launch plan inconsistent: a bug, results invalid */
 };
 
 enum { TIDAL_KV_CONTIG = 0, TIDAL_KV_PAGED = 1 };
@@ -176,6 +177,16 @@ tidal_status_t tidal_set_output_dtype(tidal_ctx_t *ctx, int32_t dtype);
  * off and frees the recordings. */
 tidal_status_t tidal_set_graphs(tidal_ctx_t *ctx, int32_t enabled);
 
+/* Overlap between the layers of a step (on by default). tidal_decode_step receives every layer's
+ * query, lengths, page table and cache up front, so all of them are complete, in stream order, before
+ * the call. With enabled != 0 a full-attention or sparse layer therefore streams its whole input while
+ * the layer before it is still finishing and waits for that layer only before it writes scratch memory
+ * and its output (a sparse layer right after a selection layer always waits first: the top-k writes its
+ * index list). With enabled = 0 a layer only prefetches cache rows ahead of the previous layer's end and
+ * reads its query afterwards, as a caller would need whose queries are produced between the layers.
+ * The single-layer calls always wait for all earlier work in the stream before reading anything. */
+tidal_status_t tidal_set_layer_overlap(tidal_ctx_t *ctx, int32_t enabled);
+
 /* The step of Algorithm 1 including its cache update: layer i's new key and value rows
  * (k_new_per_layer[i], v_new_per_layer[i]: device bf16 [batch, Hkv, head_dim], as for
  * tidal_kv_append) are written at position ctx_lens[b] - 1 of layer i's cache, then the layers
@@ -223,8 +234,8 @@ tidal_status_t tidal_sparse_attn_noalloc(const tidal_kv_t *kv, const void *q, co
                                          const int32_t *idx_count, int32_t k, int32_t num_index_heads,
                                          float *out, void *stream);
 
-/* Waits for `stream`, then returns and clears the sticky device status word:
- * TIDAL_OK, TIDAL_ERR_INDEX, or TIDAL_ERR_CUDA if the stream reports an error. */
+/* Waits for `stream`, then returns and clears the sticky device status word: TIDAL_OK,
+ * TIDAL_ERR_INDEX, TIDAL_ERR_INTERNAL, or TIDAL_ERR_CUDA if the stream reports an error. */
 tidal_status_t tidal_device_status(tidal_ctx_t *ctx, void *stream);
 
 /* Kernels launched through this context since it was created. */

@@ -17,7 +17,7 @@ from . import build as _build
 
 OK = 0
 ERR_INVALID, ERR_UNSUPPORTED, ERR_NOMEM, ERR_CUDA, ERR_TIMEOUT, ERR_INDEX = -1, -2, -3, -4, -5, -6
-ERR_TOO_LARGE = -7
+ERR_TOO_LARGE, ERR_INTERNAL = -7, -8
 KV_CONTIG, KV_PAGED = 0, 1
 SEL_PER_QHEAD, SEL_PER_KVHEAD, SEL_SHARED = 0, 1, 2
 LAYER_FULL, LAYER_SELECT, LAYER_SPARSE = 0, 1, 2
@@ -27,6 +27,7 @@ EXPORTS = [
     "tidal_sparse_attn", "tidal_decode_step", "tidal_decode_step_host", "tidal_device_status",
     "tidal_launch_count", "tidal_strerror", "tidal_sparse_attn_noalloc", "tidal_kv_append",
     "tidal_decode_step_append", "tidal_set_graphs", "tidal_set_output_dtype", "tidal_set_attend_newest",
+    "tidal_set_layer_overlap",
 ]
 
 
@@ -61,9 +62,9 @@ def load() -> C.CDLL:
     if not os.path.exists(path) or _build.is_stale():
         try:
             _build.build()
-        except Exception as exc:  # no silent fallback: the product needs its CUDA library
-            if not os.path.exists(path):
-                raise ImportError(f"libtidal.so is missing and could not be built: {exc}") from exc
+        except Exception as exc:  # no silent fallback: neither to another implementation nor to an outdated library
+            what = "is older than its sources" if os.path.exists(path) else "is missing"
+            raise ImportError(f"libtidal.so {what} and could not be rebuilt: {exc}") from exc
     L = C.CDLL(path)
     P, I32, I64 = C.c_void_p, C.c_int32, C.c_int64
     KVP = C.POINTER(tidal_kv_t)
@@ -79,6 +80,8 @@ def load() -> C.CDLL:
     L.tidal_set_attend_newest.restype = I32
     L.tidal_set_output_dtype.argtypes = [P, I32]
     L.tidal_set_output_dtype.restype = I32
+    L.tidal_set_layer_overlap.argtypes = [P, I32]
+    L.tidal_set_layer_overlap.restype = I32
     L.tidal_set_graphs.argtypes = [P, I32]
     L.tidal_set_graphs.restype = I32
     L.tidal_kv_append.argtypes = [P, KVP, P, P, P]
@@ -296,6 +299,10 @@ class Tidal:
     def set_graphs(self, enabled: bool) -> None:
         """Record whole steps as CUDA graphs and replay them (on by default; needs a non-default stream)."""
         _check(self.lib.tidal_set_graphs(self.ctx, 1 if enabled else 0), "tidal_set_graphs")
+
+    def set_layer_overlap(self, enabled: bool) -> None:
+        """Layers of a step may stream their inputs while the layer before them finishes (on by default)."""
+        _check(self.lib.tidal_set_layer_overlap(self.ctx, 1 if enabled else 0), "tidal_set_layer_overlap")
 
     def device_status(self) -> int:
         return self.lib.tidal_device_status(self.ctx, _stream())

@@ -31,16 +31,11 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-// Development hook: a tracing build (never the shipped library) defines this to record a
-// timestamp per warp at the numbered point; normally it expands to nothing.
-#ifndef TIDAL_TRACE
-#define TIDAL_TRACE(point)
-#endif
-
 namespace tidal {
 
 enum { MODE_FULL = 0, MODE_SELECT = 1, MODE_SPARSE = 2 };
-enum { STATUS_BAD_INDEX = 1, STATUS_BAD_PAGE = 2 };
+// Bits of the sticky device status word.
+enum { STATUS_BAD_INDEX = 1, STATUS_BAD_PAGE = 2, STATUS_SPLIT_OVERFLOW = 4 };
 
 constexpr int HEAD_DIM = 128;
 constexpr int TILE = 16;                 // positions per tile == page size
@@ -83,6 +78,11 @@ struct AttnParams {
     int ctr_stride;            // ints between the cursors of consecutive items (32: one 128-byte line each)
     int pdl;                   // launched with programmatic stream serialization: see pdl_wait()
     int wait_first;            // the preceding kernel may have written ctx_lens / idx: wait before reading anything
+    int wait_late;             // every input (query, lengths, index list, cache rows) was complete before the
+                               // preceding kernel started: stream the whole item first and wait for that kernel
+                               // only before the first write to memory shared with it (partial results, counters)
+    int trigger_early;         // with wait_late: let the next kernel's CTAs take the slots of ours as they retire,
+                               // without first waiting for the kernel before us (see the host's launch rule)
     int* status;
 };
 
@@ -335,13 +335,13 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = lane >> 2, tig = lane & 3;
-    TIDAL_TRACE(0);
     constexpr int RING_BYTES = NW * STAGES * STAGE_BYTES;
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem + RING_BYTES);   // MODE_SELECT: [columns][bins] counters
     const bool hist_on = (MODE == MODE_SELECT) && p.hist != nullptr;
 
     bool waited = !p.pdl;
     if (p.pdl && p.wait_first) { pdl_wait(); pdl_trigger(); waited = true; }
+    else if (p.pdl && p.wait_late && p.trigger_early) pdl_trigger();
 
     // ---- this CTA's share of the flattened (sequence, item, tile) space ---------------------------
     const bool per_qhead = (MODE == MODE_SPARSE) && (p.Hi == p.Hq);
@@ -600,7 +600,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         // By the time the fixed chunk runs out the answer is there; asked for only after the wait, the
         // forty-odd warps of an item queue up on one address and stall at that point.
         if (pooled) grab();
-        if (!waited) {
+        if (!waited && !p.wait_late) {
             while (commits < STAGES && tA >= 0 && tA < tiles_b - 1) {
                 issue(issued % STAGES);
                 ++issued;
@@ -611,7 +611,6 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             pdl_trigger();
             waited = true;
         }
-        TIDAL_TRACE(1);
 
         // Q^T fragments: column gid is head head0+gid; this lane holds the 16-byte
         // pieces 4j+tig (j = 0..3) of that head's query row.
@@ -636,7 +635,6 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             cp_async_commit();
             ++commits;
         }
-        TIDAL_TRACE(2);
         for (int it = 0; it < issued; ++it) {
             if (it == 0 && ring_full) {
                 cp_async_wait<STAGES - 1>();
@@ -647,7 +645,6 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                 if (tA >= 0) { issue((it + STAGES - 1) % STAGES); ++issued; }
                 cp_async_commit();
             }
-            if (it == 0) { TIDAL_TRACE(3); }
             const int stage = it % STAGES;
             const uint32_t ks = wbase_u32 + stage * STAGE_BYTES;
             consume_tile<MODE>(p, ks, ks + TILE_BYTES, qf, acc, s_vmask[warp][stage], gid, tig,
@@ -655,7 +652,13 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         }
         cp_async_wait<0>();
         __syncwarp();
-        TIDAL_TRACE(4);
+        // All of this item's tiles are in the accumulators. With a late wait the grid dependency is
+        // resolved only now: everything below writes memory that the preceding kernel may still use.
+        if (!waited) {
+            pdl_wait();
+            if (!p.trigger_early) pdl_trigger();
+            waited = true;
+        }
 
         if (hist_on) {                        // add this segment's histogram to the global one
             __syncthreads();
@@ -728,10 +731,11 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                 const long long pr = (row0 + col) * p.max_splits + split;
                 p.part_o[pr * HEAD_DIM + c] = O;
                 if (c == 0) p.part_ml[pr] = make_float2(M, L);
+            } else if (e == 0) {
+                atomicOr(p.status, STATUS_SPLIT_OVERFLOW);    // the host's bound on splits per row was wrong: say so
             }
         }
-        TIDAL_TRACE(5);
-        if (nsplits == 1 && pooled && threadIdx.x == 0) *pool = 0;
+        if (nsplits == 1 && pooled && threadIdx.x == 0) { *pool = 0; __threadfence(); }
         if (nsplits > 1) {
             // ---- the last CTA of this item to arrive combines the splits ---------------------------------
             __syncthreads();
@@ -797,11 +801,13 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                     for (; s < ns; ++s) O += __ldcg(po + (long long)s * HEAD_DIM) * fs[s];
                     store_out(p, (row0 + col) * HEAD_DIM + c, O * linv[col]);
                 }
-                if (threadIdx.x == 0) { *ctr = 0; if (pooled) *pool = 0; }   // ready for the next launch
+                // Ready for the next launch. The fence makes the cleared cursor visible device-wide before
+                // this CTA retires: a later launch may request tiles from it without waiting for this grid
+                // (see the host's rule for early triggers), and cannot start before this CTA is gone.
+                if (threadIdx.x == 0) { *ctr = 0; if (pooled) { *pool = 0; __threadfence(); } }
             }
         }
         __syncthreads();                          // shared memory is reused by the next segment
-        TIDAL_TRACE(6);
 
         // ---- advance to the next segment -----------------------------------------------------------------
         if (pooled) break;

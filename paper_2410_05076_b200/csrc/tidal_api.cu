@@ -50,7 +50,8 @@ struct tidal_ctx {
     int* status = nullptr;                      // device word, sticky
     int out_bf16 = 0;                           // outputs are written as bf16 instead of fp32
     int attend_newest = 0;                      // sparse layers also attend the newest token (not in the paper)
-    int cursor_set = 0;                         // which of the two sets of pool cursors the last attention launch used
+    int cursor_set = 0;                         // which of the sets of pool cursors the last attention launch used
+    int layer_overlap = 1;                      // layers of a step may stream their inputs while the layer before them finishes
     int64_t launches = 0;
     // Whole steps are recorded once as CUDA graphs (programmatic dependent launches included) and
     // replayed while every host-visible argument stays the same: one launch per step instead of one
@@ -184,17 +185,18 @@ tidal_status_t ensure_ws(tidal_ctx* ctx, size_t bytes) {
     return TIDAL_OK;
 }
 
-// State layout for a capacity of R rows: counters | cursor | done | tile_ctr set 0 | tile_ctr set 1, each
-// [R][CTR_STRIDE], then hist[R][TK_BINS]. Consecutive attention launches alternate between the two sets of
-// pool cursors, so that a launch may use its set before its predecessor has finished with the other.
+// State layout for a capacity of R rows: counters | cursor | done | tile_ctr sets 0..2, each
+// [R][CTR_STRIDE], then hist[R][TK_BINS]. Consecutive attention launches rotate through the sets of
+// pool cursors, so that a launch may use its set before its predecessor has finished with another.
 // Every counter has a 128-byte line of its own: hundreds of warps hit them at once, and atomics to one
 // line are served one after the other.
 constexpr int CTR_STRIDE = 32;
+constexpr int CURSOR_SETS = 6;
 inline int* state_counters(const tidal_ctx* c) { return (int*)c->state; }
 inline int* state_cursor(const tidal_ctx* c) { return (int*)c->state + (size_t)CTR_STRIDE * c->state_rows; }
 inline int* state_done(const tidal_ctx* c) { return (int*)c->state + 2 * (size_t)CTR_STRIDE * c->state_rows; }
 inline int* state_tile_ctr(const tidal_ctx* c) { return (int*)c->state + 3 * (size_t)CTR_STRIDE * c->state_rows; }
-inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + 5 * (size_t)CTR_STRIDE * c->state_rows; }
+inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + (3 + CURSOR_SETS) * (size_t)CTR_STRIDE * c->state_rows; }
 
 tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     if (ctx->state_rows >= rows) return TIDAL_OK;
@@ -202,7 +204,7 @@ tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     drop_graphs(ctx);
     if (ctx->state) { cudaDeviceSynchronize(); cudaFree(ctx->state); ctx->state = nullptr; ctx->state_rows = 0; }
     const int cap = (int)align_up((size_t)rows, 64);
-    const size_t bytes = (size_t)cap * (5 * CTR_STRIDE + TK_BINS) * sizeof(int);
+    const size_t bytes = (size_t)cap * ((3 + CURSOR_SETS) * CTR_STRIDE + TK_BINS) * sizeof(int);
     void* p = nullptr;
     if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TIDAL_ERR_NOMEM; }
     if (cudaMemset(p, 0, bytes) != cudaSuccess) { cudaFree(p); return TIDAL_ERR_CUDA; }
@@ -247,16 +249,28 @@ void fill_common(AttnParams& a, const tidal_ctx* ctx, const tidal_kv_t* kv, cons
 
 template <int MODE, int NW, int STAGES>
 constexpr size_t attn_smem() {
-    return (size_t)NW * STAGES * STAGE_BYTES + (MODE == MODE_SELECT ? HIST_SMEM : 0) + 1024;   // + alignment slack
+    return (size_t)NW * STAGES * STAGE_BYTES +
+           (MODE == MODE_SELECT ? HIST_SMEM : 0) + 1024;   // + alignment slack
 }
 
 template <int MODE, int NW, int STAGES, bool NEWEST = false>
-tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, cudaStream_t st) {
+tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, int full_grid, cudaStream_t st) {
     // Programmatic dependent launch: the kernel may begin while its predecessor in the stream
     // drains; it waits (griddepcontrol.wait) before touching anything that predecessor wrote.
     a.pdl = 1;
-    ctx->cursor_set ^= 1;
+    ctx->cursor_set = (ctx->cursor_set + 1) % CURSOR_SETS;
     a.tile_ctr = state_tile_ctr(ctx) + (size_t)ctx->cursor_set * CTR_STRIDE * ctx->state_rows;
+    // A kernel that waits late triggers its successor at once, before it has itself waited for its
+    // predecessor, so several consecutive launches can be resident together. The one thing a kernel
+    // touches before its own wait is its set of pool cursors, last used CURSOR_SETS launches ago by a
+    // kernel that must have finished with it. It has: the launches in between either waited before they
+    // triggered (then stream order guarantees it), or each of them holds all its CTAs until its own
+    // predecessor is complete and (CURSOR_SETS - 1) of them fill every resident slot of the GPU, so this
+    // launch cannot have started while a CTA of that old kernel was still resident. Hence the rule:
+    // early trigger only for pooled launches (every CTA stays until the wait) whose grid is at least
+    // 1 / (CURSOR_SETS - 1) of the resident slots for this kernel's CTA size.
+    a.trigger_early = a.wait_late && a.splits_per_item > 0 && (long long)(CURSOR_SETS - 1) * grid >= full_grid;
+    if (!a.trigger_early) a.wait_late = 0;      // without the early trigger the late wait only delays the successor
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(grid, 1, 1);
@@ -286,12 +300,16 @@ SelectPlan select_plan(const tidal_kv_t* kv, int Hi, bool caller_scores) {
 }
 
 // hist != nullptr: the kernel also accumulates the per-head histogram the top-k needs.
+// How a layer's kernel treats the kernel before it in the stream (see AttnParams::wait_first / wait_late).
+enum Dep { DEP_FIRST, DEP_PREFETCH, DEP_LATE };
+
 tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, float* out, float* scores,
-                         long long score_stride, bool fuse_hist, bool wait_first, const WsLayout& w, cudaStream_t st,
+                         long long score_stride, bool fuse_hist, Dep dep, const WsLayout& w, cudaStream_t st,
                          bool agg = false) {
     AttnParams a;
     fill_common(a, ctx, kv, q, out, w);
-    a.wait_first = wait_first;
+    a.wait_first = dep == DEP_FIRST;
+    a.wait_late = dep == DEP_LATE && scores == nullptr;   // a selection layer writes scores while it streams
     const long long tiles = (long long)kv->batch * kv->num_kv_heads * ((kv->max_ctx_len + TILE - 1) / TILE);
     int grid = grid_for(tiles, ctx->dense_slots);
     if (const int S = pooled_splits(kv, kv->batch * kv->num_kv_heads, grid)) {
@@ -301,8 +319,8 @@ tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, fl
     a.score_stride = score_stride;
     a.agg = agg ? 1 : 0;
     a.hist = fuse_hist ? state_hist(ctx) : nullptr;
-    if (scores) return launch_attn<MODE_SELECT, DENSE_NW, DENSE_STAGES>(ctx, a, grid, st);
-    return launch_attn<MODE_FULL, DENSE_NW, DENSE_STAGES>(ctx, a, grid, st);
+    if (scores) return launch_attn<MODE_SELECT, DENSE_NW, DENSE_STAGES>(ctx, a, grid, std::min(ctx->dense_slots, GRID_MAX), st);
+    return launch_attn<MODE_FULL, DENSE_NW, DENSE_STAGES>(ctx, a, grid, std::min(ctx->dense_slots, GRID_MAX), st);
 }
 
 // `rows`: score rows per sequence (query heads, or KV heads when the attention kernel stored group sums).
@@ -365,20 +383,32 @@ tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* score
 }
 
 tidal_status_t run_sparse(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, const int* idx,
-                          const int* idx_count, int k, int Hi, float* out, bool wait_first, const WsLayout& w,
+                          const int* idx_count, int k, int Hi, float* out, Dep dep, bool chain, const WsLayout& w,
                           cudaStream_t st) {
     AttnParams a;
     fill_common(a, ctx, kv, q, out, w);
-    a.wait_first = wait_first;
+    a.wait_first = dep == DEP_FIRST;
+    a.wait_late = dep == DEP_LATE;
     const int per_batch = (Hi == kv->num_q_heads) ? kv->num_q_heads : kv->num_kv_heads;
     const long long tiles = (long long)kv->batch * per_batch * ((k + TILE - 1) / TILE);
+    const int full = std::min(ctx->sparse_slots, GRID_MAX);
     int grid = grid_for(tiles, ctx->sparse_slots);
     a.idx = idx; a.idx_count = idx_count; a.budget = k; a.Hi = Hi;
-    if (const int S = pooled_splits(kv, kv->batch * per_batch, grid)) {
+    // In a chain of sparse layers that overlap (late wait, early trigger) a launch takes about a third
+    // of the resident slots, so that about three layers are in flight at any time, one behind the
+    // other: while the CTAs of one layer start up (lengths, index entries, first rows: a chain of
+    // dependent loads) or merge their results, the others keep the memory system busy. Every item gets
+    // the same number of CTAs.
+    const int items = kv->batch * per_batch;
+    if (chain && kv->batch == 1) {
+        const int S = std::max(1, (full + 3 * items / 2) / (3 * items));
+        grid = std::min(grid, S * items);
+    }
+    if (const int S = pooled_splits(kv, items, grid)) {
         a.splits_per_item = S;
     }
-    if (ctx->attend_newest) return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES, true>(ctx, a, grid, st);
-    return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(ctx, a, grid, st);
+    if (ctx->attend_newest) return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES, true>(ctx, a, grid, std::min(ctx->sparse_slots, GRID_MAX), st);
+    return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(ctx, a, grid, std::min(ctx->sparse_slots, GRID_MAX), st);
 }
 
 template <typename K>
@@ -405,7 +435,7 @@ struct KeyBuilder {
 void step_key(KeyBuilder& kb, const tidal_ctx* ctx, int tag, int32_t num_layers, const uint8_t* schedule,
                      const tidal_kv_t* kvs, int32_t k, int32_t granularity, int host_layers) {
     kb.add(tag); kb.add(num_layers); kb.add(k); kb.add(granularity); kb.add(host_layers);
-    kb.add(ctx->ws); kb.add(ctx->state); kb.add(ctx->out_bf16); kb.add(ctx->attend_newest);
+    kb.add(ctx->ws); kb.add(ctx->state); kb.add(ctx->out_bf16); kb.add(ctx->attend_newest); kb.add(ctx->layer_overlap);
     kb.add_raw(schedule, (size_t)num_layers);
     for (int i = 0; i < num_layers; ++i) {
         // field by field: the struct has padding whose bytes are not the caller's to define
@@ -569,7 +599,7 @@ tidal_status_t tidal_full_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const voi
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
     const WsLayout w = layout_ws(kv, 1, 0);
     if ((rc = ensure_all(ctx, kv, w.total)) != TIDAL_OK) return rc;
-    return run_dense(ctx, kv, q, out, nullptr, 0, false, true, w, (cudaStream_t)stream);
+    return run_dense(ctx, kv, q, out, nullptr, 0, false, DEP_FIRST, w, (cudaStream_t)stream);
 }
 
 tidal_status_t tidal_select_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const void* q, int32_t k,
@@ -588,7 +618,7 @@ tidal_status_t tidal_select_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const v
     const long long stride = scores_opt ? (long long)kv->max_ctx_len : w.score_stride;
     cudaStream_t st = (cudaStream_t)stream;
     const SelectPlan sp = select_plan(kv, Hi, scores_opt != nullptr);
-    if ((rc = run_dense(ctx, kv, q, out, scores, stride, sp.fuse, true, w, st, sp.agg)) != TIDAL_OK) return rc;
+    if ((rc = run_dense(ctx, kv, q, out, scores, stride, sp.fuse, DEP_FIRST, w, st, sp.agg)) != TIDAL_OK) return rc;
     return run_topk(ctx, kv, scores, stride, k, sp.rows, Hi, sp.fuse, idx, idx_count, w, st);
 }
 
@@ -605,7 +635,7 @@ tidal_status_t tidal_sparse_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const v
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
     const WsLayout w = layout_ws(kv, k, 0);
     if ((rc = ensure_all(ctx, kv, w.total)) != TIDAL_OK) return rc;
-    return run_sparse(ctx, kv, q, idx, idx_count, k, Hi, out, true, w, (cudaStream_t)stream);
+    return run_sparse(ctx, kv, q, idx, idx_count, k, Hi, out, DEP_FIRST, false, w, (cudaStream_t)stream);
 }
 
 // Validates a step and sizes the workspace for it (may allocate and synchronise).
@@ -645,16 +675,24 @@ static tidal_status_t decode_step_enqueue(tidal_ctx_t* ctx, int32_t num_layers, 
     for (int i = 0; i < num_layers; ++i) {
         const tidal_kv_t* kv = &kvs[i];
         const WsLayout w = layout_ws(kv, k, host_layers);
+        // Every query, length, page table and cache row of the step was complete before the call, so a
+        // layer may read all of them while the layer before it is still running and needs that layer to
+        // have finished only before it writes scratch memory (DEP_LATE). The exceptions: the first
+        // kernel of the step (whatever ran before it in the stream may have produced its inputs), and a
+        // sparse layer right after a selection layer, whose index list is written by the top-k.
+        const Dep dep = i == 0 ? DEP_FIRST : (ctx->layer_overlap ? DEP_LATE : DEP_PREFETCH);
         if (schedule[i] == TIDAL_LAYER_FULL) {
-            rc = run_dense(ctx, kv, qs[i], outs[i], nullptr, 0, false, i == 0, w, st);
+            rc = run_dense(ctx, kv, qs[i], outs[i], nullptr, 0, false, dep, w, st);
         } else if (schedule[i] == TIDAL_LAYER_SELECT) {
             float* scores = (float*)((char*)ctx->ws + w.scores);
             const SelectPlan sp = select_plan(kv, Hi, false);
-            rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, sp.fuse, i == 0, w, st, sp.agg);
+            rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, sp.fuse, dep, w, st, sp.agg);
             if (rc == TIDAL_OK) rc = run_topk(ctx, kv, scores, w.score_stride, k, sp.rows, Hi, sp.fuse, idx, idx_count, w, st);
         } else {
-            // the index list is fresh when the previous layer selected it
-            rc = run_sparse(ctx, kv, qs[i], idx, idx_count, k, Hi, outs[i], i == 0 || schedule[i - 1] == TIDAL_LAYER_SELECT, w, st);
+            const bool fresh_idx = i == 0 || schedule[i - 1] == TIDAL_LAYER_SELECT;
+            const bool chain = ctx->layer_overlap && ((i > 0 && schedule[i - 1] == TIDAL_LAYER_SPARSE) ||
+                                                      (i + 1 < num_layers && schedule[i + 1] == TIDAL_LAYER_SPARSE));
+            rc = run_sparse(ctx, kv, qs[i], idx, idx_count, k, Hi, outs[i], fresh_idx ? DEP_FIRST : dep, chain, w, st);
         }
         if (rc != TIDAL_OK) return rc;
     }
@@ -717,6 +755,12 @@ tidal_status_t tidal_decode_step(tidal_ctx_t* ctx, int32_t num_layers, const uin
 tidal_status_t tidal_set_attend_newest(tidal_ctx_t* ctx, int32_t enabled) {
     if (!ctx) return TIDAL_ERR_INVALID;
     ctx->attend_newest = enabled != 0;
+    return TIDAL_OK;
+}
+
+tidal_status_t tidal_set_layer_overlap(tidal_ctx_t* ctx, int32_t enabled) {
+    if (!ctx) return TIDAL_ERR_INVALID;
+    ctx->layer_overlap = enabled != 0;
     return TIDAL_OK;
 }
 
@@ -805,8 +849,10 @@ tidal_status_t tidal_device_status(tidal_ctx_t* ctx, void* stream) {
     int word = 0;
     if (cudaMemcpy(&word, ctx->status, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) return TIDAL_ERR_CUDA;
     if (word != 0 && cudaMemset(ctx->status, 0, sizeof(int)) != cudaSuccess) return TIDAL_ERR_CUDA;
+    if (word & STATUS_SPLIT_OVERFLOW) return TIDAL_ERR_INTERNAL;
     return word ? TIDAL_ERR_INDEX : TIDAL_OK;
 }
+
 
 int64_t tidal_launch_count(const tidal_ctx_t* ctx) { return ctx ? ctx->launches : 0; }
 
@@ -820,6 +866,7 @@ const char* tidal_strerror(tidal_status_t s) {
         case TIDAL_ERR_TIMEOUT: return "device-side wait timed out";
         case TIDAL_ERR_INDEX: return "token index or page id out of range";
         case TIDAL_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of the allocation-free entry point";
+        case TIDAL_ERR_INTERNAL: return "launch plan inconsistency detected on the device (results are invalid)";
         default: return "unknown status";
     }
 }

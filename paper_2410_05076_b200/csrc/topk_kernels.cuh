@@ -24,10 +24,6 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#ifndef TIDAL_TRACE2
-#define TIDAL_TRACE2(point)        // development hook, see attn_kernels.cuh
-#endif
-
 namespace tidal {
 
 constexpr int TK_THREADS = 512;
@@ -223,7 +219,6 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     const int N = max(0, min(p.ctx_lens[b], p.max_ctx));
     const int kk = min(p.k, N);
     int* out = p.idx + (long long)item * p.k;
-    TIDAL_TRACE2(0);
     const int s0 = blockIdx.x * TK_SPAN, s1 = min(N, s0 + TK_SPAN);
     if (blockIdx.x == 0 && hi == 0 && tid == 0 && p.idx_count) p.idx_count[b] = kk;
     unsigned* gh = p.hist + (long long)item * TK_BINS;
@@ -292,10 +287,8 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         reinterpret_cast<uint4*>(sh_hist)[tid] = h4;
     }
     __syncthreads();
-    TIDAL_TRACE2(1);
     int need = kk;
     const int b1 = pick_digit(sh_hist, TK_BINS, warp_sums, bcast, need);
-    TIDAL_TRACE2(2);
     // `need` of the keys in bin b1 are still to be taken; every key in a higher bin is a winner.
     asm volatile("cp.async.wait_group 0;\n" ::: "memory");
     __syncthreads();
@@ -333,7 +326,6 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         word |= __shfl_xor_sync(0xffffffffu, word, 4);
         if ((lane & 7) == 0) bm[bm_base + j * (TK_THREADS / 8) + warp * 4 + (lane >> 3)] = word;
     }
-    TIDAL_TRACE2(10);
 
     // ---- the threshold bin's own keys: append to the candidate list, one cursor bump per CTA -------
     int cta_total;
@@ -363,7 +355,6 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         }
     }
 
-    TIDAL_TRACE2(3);
     // ---- the last CTA of this index head resolves the rest ------------------------------------------
     __syncthreads();
     const int words = (N + 31) >> 5;
@@ -390,7 +381,6 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
             s_last = (old == nparts - 1);
         }
         __syncthreads();
-        TIDAL_TRACE2(4);
         if (!s_last) return;
 
         // One round trip for everything the last CTA needs: the candidate count, the winners' bitmap
@@ -434,7 +424,6 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         __syncthreads();
     }
 
-    TIDAL_TRACE2(5);
     // second digit: the next 11 key bits (every candidate already has first digit b1)
     const int s2 = p.shift - 11;                       // bits left for the third digit (10 or 11)
     for (int i = tid; i < M; i += TK_THREADS) atomicAdd(&sh_hist[(c[i].x >> s2) & 0x7ffu], 1u);
@@ -444,7 +433,6 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     const int in_bin = (int)sh_hist[d2];               // candidates that share both digits with the threshold key
     __syncthreads();                                   // sh_hist is recycled below
 
-    TIDAL_TRACE2(6);
     constexpr int SMALL = 64;
     if (in_bin <= SMALL) {
         // A handful of keys are left: rank them directly. Entry i is taken iff fewer than `need` of the
@@ -482,7 +470,6 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         __syncthreads();
         const int d3 = pick_digit(sh_hist, 1 << s2, warp_sums, bcast, need);
         const uint32_t thr = prefix2 | (uint32_t)d3;   // the k'-th largest key; `need` keys equal to it are taken
-        TIDAL_TRACE2(7);
         // candidates above / equal to the threshold, as position bitmaps
         for (int i = tid; i < M; i += TK_THREADS) {
             const uint2 e = c[i];
@@ -492,7 +479,6 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         __syncthreads();
     }
 
-    TIDAL_TRACE2(8);
     if (need == 0 && (per & 3) == 0 && words == per * TK_THREADS) {
         // No equal-key positions are pending (the usual case) and the words divide evenly: only the
         // winners' bitmap is enumerated, fetched as 16-byte pieces (consecutive threads are `per` words
@@ -505,10 +491,8 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
             const uint4 t = src[j];
             mine += __popc(t.x) + __popc(t.y) + __popc(t.z) + __popc(t.w);
         }
-        TIDAL_TRACE2(11);
         int tot;
         int at = block_scan_incl<int>(mine, warp_sums, tot) - mine;
-        TIDAL_TRACE2(12);
 #pragma unroll 1
         for (int j = 0; j < per; ++j) {
             unsigned bits = cgt[w0 + j];
@@ -524,10 +508,8 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     unsigned long long cnt = 0;
     for (int w = w0; w < w1; ++w)
         cnt += ((unsigned long long)__popc(cgt[w]) << 32) | (unsigned long long)__popc(ceq[w]);
-    TIDAL_TRACE2(11);
     unsigned long long tot;
     const unsigned long long excl = block_scan_incl<unsigned long long>(cnt, warp_sums64, tot) - cnt;
-    TIDAL_TRACE2(12);
     int eq_seen = (int)(excl & 0xffffffffu);
     int at = (int)(excl >> 32) + min(eq_seen, need);
     for (int w = w0; w < w1; ++w) {
@@ -545,10 +527,8 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
         }
     }
     }
-    TIDAL_TRACE2(13);
     for (int i = kk + tid; i < p.k; i += TK_THREADS) out[i] = -1;
 
-    TIDAL_TRACE2(9);
     // leave the shared state clean for the next call
     for (int i = tid; i < TK_BINS; i += TK_THREADS) gh[i] = 0;
     if (tid == 0 && !solo) { p.cursor[(size_t)item * p.ctr_stride] = 0; p.done[(size_t)item * p.ctr_stride] = 0; }
