@@ -90,11 +90,19 @@ typedef struct {
     float sm_scale;                 /* 0 => 1/sqrt(head_dim), the scale of Eq. 1 */
 } tidal_kv_t;
 
-/* Create a context on CUDA device `device`. workspace_bytes = 0 lets the
- * workspace grow on demand (a call may then allocate, so size it up front with
- * tidal_workspace_bytes() before capturing calls into a CUDA graph). */
+/* Create a context on CUDA device `device`. workspace_bytes preallocates that much scratch
+ * (0 = none). Whatever a later call needs beyond what the context holds is allocated inside that
+ * call (which then also synchronises the device): use tidal_reserve() to do all of it up front. */
 tidal_status_t tidal_create(tidal_ctx_t **ctx, int device, size_t workspace_bytes);
 tidal_status_t tidal_destroy(tidal_ctx_t *ctx);
+
+/* Allocates, now, everything later calls with this cache shape (batch, heads, max_ctx_len) and a
+ * budget up to k will need: the scratch workspace and the small block of counters and histograms
+ * that scale with batch * num_q_heads. num_layers_host is the layer count of later
+ * tidal_decode_step_host calls (0 if that call is not used). After it, calls with shapes no larger
+ * allocate nothing and do not synchronise, so they can be captured into a CUDA graph from the first
+ * one on. May allocate and synchronise itself; call it outside any capture. */
+tidal_status_t tidal_reserve(tidal_ctx_t *ctx, const tidal_kv_t *kv, int32_t k, int32_t num_layers_host);
 
 /* Workspace a call with this cache shape and budget k needs (split-context
  * partial results, the score buffer of a selection layer, top-k histograms). */
@@ -219,7 +227,7 @@ tidal_status_t tidal_decode_step_host(tidal_ctx_t *ctx, int32_t num_layers, cons
  *
  * This one takes no context and never calls cudaMalloc, cudaFree or any allocating routine: its
  * scratch (split partial results, arrival counters, pool cursors) is one static device array of
- * about 2.07 MiB (4096 partial rows) that every GPU loading the library holds until the process
+ * about 2.06 MiB (4096 partial rows) that every GPU loading the library holds until the process
  * exits. It runs on the CURRENT device. Arguments and results are those of tidal_sparse_attn,
  * with these differences:
  *   - batch * num_q_heads must not exceed 4096, otherwise TIDAL_ERR_TOO_LARGE (nothing enqueued);

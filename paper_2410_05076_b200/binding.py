@@ -27,7 +27,7 @@ EXPORTS = [
     "tidal_sparse_attn", "tidal_decode_step", "tidal_decode_step_host", "tidal_device_status",
     "tidal_launch_count", "tidal_strerror", "tidal_sparse_attn_noalloc", "tidal_kv_append",
     "tidal_decode_step_append", "tidal_set_graphs", "tidal_set_output_dtype", "tidal_set_attend_newest",
-    "tidal_set_layer_overlap",
+    "tidal_set_layer_overlap", "tidal_reserve",
 ]
 
 
@@ -82,6 +82,8 @@ def load() -> C.CDLL:
     L.tidal_set_output_dtype.restype = I32
     L.tidal_set_layer_overlap.argtypes = [P, I32]
     L.tidal_set_layer_overlap.restype = I32
+    L.tidal_reserve.argtypes = [P, KVP, I32, I32]
+    L.tidal_reserve.restype = I32
     L.tidal_set_graphs.argtypes = [P, I32]
     L.tidal_set_graphs.restype = I32
     L.tidal_kv_append.argtypes = [P, KVP, P, P, P]
@@ -183,6 +185,11 @@ class Tidal:
     def workspace_bytes(layer, k: int) -> int:
         s = kv_struct(layer)
         return load().tidal_workspace_bytes(C.byref(s), k)
+
+    def reserve(self, layer, k: int, num_layers_host: int = 0) -> None:
+        """Allocate everything later calls with this cache shape and budget need (then they can be captured)."""
+        s = kv_struct(layer)
+        _check(self.lib.tidal_reserve(self.ctx, C.byref(s), k, num_layers_host), "tidal_reserve")
 
     def kv_append(self, layer, k_new: torch.Tensor, v_new: torch.Tensor) -> None:
         """Write the new token's rows (bf16 [B, Hkv, d]) at position ctx_lens[b] - 1 of the layer's cache."""

@@ -207,7 +207,12 @@ tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     const size_t bytes = (size_t)cap * ((3 + CURSOR_SETS) * CTR_STRIDE + TK_BINS) * sizeof(int);
     void* p = nullptr;
     if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TIDAL_ERR_NOMEM; }
-    if (cudaMemset(p, 0, bytes) != cudaSuccess) { cudaFree(p); return TIDAL_ERR_CUDA; }
+    // on a stream of its own, so that nothing here is the legacy stream's business, and waited for
+    cudaStream_t zs = nullptr;
+    bool zeroed = cudaStreamCreateWithFlags(&zs, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaMemsetAsync(p, 0, bytes, zs) == cudaSuccess && cudaStreamSynchronize(zs) == cudaSuccess;
+    if (zs) cudaStreamDestroy(zs);
+    if (!zeroed) { cudaGetLastError(); cudaFree(p); return TIDAL_ERR_CUDA; }
     ctx->state = p;
     ctx->state_rows = cap;
     return TIDAL_OK;
@@ -559,6 +564,14 @@ size_t tidal_workspace_bytes(const tidal_kv_t* kv, int32_t k) {
     return ws_bytes_for(kv, k, 0);
 }
 
+tidal_status_t tidal_reserve(tidal_ctx_t* ctx, const tidal_kv_t* kv, int32_t k, int32_t num_layers_host) {
+    if (!ctx || k <= 0 || num_layers_host < 0 || num_layers_host > 1024) return TIDAL_ERR_INVALID;
+    const tidal_status_t rc = check_kv(kv);
+    if (rc != TIDAL_OK) return rc;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    return ensure_all(ctx, kv, ws_bytes_for(kv, k, num_layers_host));
+}
+
 static void fill_append(AppendParams& a, const tidal_ctx* ctx, const tidal_kv_t* kv, const void* k_new,
                         const void* v_new);
 
@@ -716,6 +729,11 @@ tidal_status_t tidal_decode_step_append(tidal_ctx_t* ctx, int32_t num_layers, co
             return TIDAL_ERR_INVALID;
     }
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    // The whole step is validated (and its workspace sized) before the first row is written: an
+    // argument error must leave the caches as they were.
+    const tidal_status_t ok = decode_step_prepare(ctx, num_layers, schedule, kv_per_layer, q_per_layer, out_per_layer,
+                                                  k, granularity, 0);
+    if (ok != TIDAL_OK) return ok;
     const int pairs = kv_per_layer[0].batch * kv_per_layer[0].num_kv_heads;
     for (int l0 = 0; l0 < num_layers; l0 += APPEND_MAX_LAYERS) {
         const int n = std::min(APPEND_MAX_LAYERS, num_layers - l0);
@@ -886,7 +904,7 @@ constexpr int NOALLOC_MAX_ROWS = 4096;      // (sequence, query head) rows; also
 constexpr size_t NOALLOC_PART_O = (size_t)NOALLOC_MAX_ROWS * HEAD_DIM * sizeof(float);   // 2 MiB
 constexpr size_t NOALLOC_PART_ML = (size_t)NOALLOC_MAX_ROWS * sizeof(float2);           // 32 KiB
 constexpr size_t NOALLOC_WORDS = 2 * (size_t)NOALLOC_MAX_ROWS * sizeof(int) + 256;      // counters, cursors, status
-constexpr size_t NOALLOC_BYTES = NOALLOC_PART_O + NOALLOC_PART_ML + NOALLOC_WORDS;      // about 2.07 MiB
+constexpr size_t NOALLOC_BYTES = NOALLOC_PART_O + NOALLOC_PART_ML + NOALLOC_WORDS;      // 2 MiB + 64 KiB + 256 B, about 2.06 MiB
 
 // Held by every GPU that loads the library until the process exits. In host code this name is
 // only a handle for cudaGetSymbolAddress, never a device address.

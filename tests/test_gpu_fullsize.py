@@ -43,13 +43,24 @@ def select_then_sparse(td, w, sel_layer, sp_layer, max_band_members_per_head=64)
         for h in range(w.num_q_heads):
             inside = util.check_idx_row(idx_h[b, h], sc[b, h], w.k, int(lens[b]), f"{w.name}.idx[{b},{h}]")
             assert inside <= max_band_members_per_head
+    # Heavy hitters are selected: always when the oracle scores them clear of the k'-th score, and nearly
+    # all of them anyway (their logits are about 5.7 +- 1; only at the smallest k / N of the sweep does
+    # the k'-th score, about 2.9 there, reach into that distribution's tail).
     planted = synth.planted_positions(w, sel_layer, [int(n) for n in lens])
+    found = planted_total = 0
     for b in range(w.batch):
         if w.k >= lens[b]:
             continue
+        n = int(lens[b])
         for g in range(w.num_kv_heads):
             for i, pos in enumerate(planted[b, g].tolist()):
-                assert pos in idx_h[b, g * w.group + i % w.group]      # heavy hitters are selected
+                h = g * w.group + i % w.group
+                kth = np.partition(sc[b, h, :n], n - w.k)[n - w.k]
+                hit = pos in idx_h[b, h]
+                assert hit or sc[b, h, pos] <= kth + util.TIE_BAND
+                found += hit
+                planted_total += 1
+    assert found >= 0.97 * planted_total
     del okv, lay
     torch.cuda.empty_cache()
     lay2 = mk(sp_layer)
@@ -106,8 +117,10 @@ def test_sixty_four_layer_variant_group_of_eight(td):
     select_then_sparse(td, w, 31, 32)
 
 
-@pytest.mark.parametrize("ctx,k", [(262144, 8192), (65536, 512), (4096, 8192), (16384, 1024)])
+@pytest.mark.parametrize("ctx", synth.SWEEP_CTX)
+@pytest.mark.parametrize("k", synth.SWEEP_K)
 def test_config5_sweep_points(td, ctx, k):
+    """All 25 points of the context x budget sweep that bench.py times."""
     w = synth.sweep_point(ctx, min(k, ctx))      # the API takes k <= max_ctx_len; k' = min(k, N)
     select_then_sparse(td, w, 0, 1)
 

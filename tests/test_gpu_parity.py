@@ -692,3 +692,179 @@ def test_sparse_layers_can_always_attend_the_newest_token(td, layout):
     util.check_out(outs[1].cpu().numpy(), oracle.sparse_attn(okv1, synth.bits(qs[1]), aug2, cnt_aug2), "newest.step1")
     util.check_out(outs[2].cpu().numpy(), oracle.sparse_attn(okv2, synth.bits(qs[2]), aug2, cnt_aug2), "newest.step2")
     assert td.device_status() == binding.OK
+
+
+@pytest.mark.parametrize("layout", ["hnd_interleaved", "paged"])
+@pytest.mark.parametrize("B,Hq,Hkv,N,k,ragged", [(1, 8, 2, 300, 40, False), (3, 16, 2, 777, 100, True), (1, 4, 4, 4097, 256, False)])
+def test_no_call_writes_outside_its_output_buffers(td, layout, B, Hq, Hkv, N, k, ragged):
+    """Every caller-owned output (out, idx, idx_count, scores) sits between guard zones of a fixed pattern,
+    which must be intact after each call: full, selection (scores in the caller's buffer and in the
+    workspace), sparse, a whole step, and the step with bf16 outputs (half the bytes in the same buffer)."""
+    w = wl(B, Hq, Hkv, N, k, planted=min(8, N), ragged=ragged, ctx_min=max(1, N // 3), seed=43, layers=3)
+    qs = [synth.make_q(w, i, DEV) for i in range(3)]
+    if layout == "paged":
+        pt, total = synth.make_page_table(w, extra_pages=3)
+        lays = [synth.make_layer(w, i, DEV, layout="paged", q=qs[i], page_table=pt, num_pages=total) for i in range(3)]
+    else:
+        lays = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(3)]
+    okv, qb = util.oracle_kv(lays[0]), synth.bits(qs[0])
+    out = util.Guarded((B, Hq, 128), torch.float32, DEV, fill=float("nan"))
+    idx = util.Guarded((B, Hq, k), torch.int32, DEV, fill=-7)
+    cnt = util.Guarded((B,), torch.int32, DEV, fill=-7)
+    sc = util.Guarded((B, Hq, N), torch.float32, DEV, fill=float("nan"))
+    guards = {"out": out, "idx": idx, "idx_count": cnt, "scores": sc}
+
+    def check_all(what):
+        for name, g in guards.items():
+            g.check(f"{what}: {name}")
+
+    td.full_attn(lays[0], qs[0], out=out.t)
+    check_all("full")
+    ref_out, ref_sc = oracle.full_attn(okv, qb, want_scores=True)
+    util.check_out(out.t.cpu().numpy(), ref_out, "full")
+    out.t.fill_(float("nan"))
+    td.select_attn(lays[0], qs[0], k, out=out.t, idx=idx.t, idx_count=cnt.t, scores=sc.t)
+    check_all("select with caller scores")
+    util.check_out(out.t.cpu().numpy(), ref_out, "select")
+    lens = lays[0].ctx_lens.cpu().numpy()
+    for b in range(B):
+        for h in range(Hq):
+            util.check_idx_row(idx.t[b, h].cpu().numpy(), ref_sc[b, h], k, int(lens[b]), "select.idx")
+    idx.t.fill_(-7)
+    td.select_attn(lays[0], qs[0], k, out=out.t, idx=idx.t, idx_count=cnt.t)
+    check_all("select with workspace scores")
+    out.t.fill_(float("nan"))
+    td.sparse_attn(lays[1], qs[1], idx.t, cnt.t, out=out.t)
+    check_all("sparse")
+    util.check_out(out.t.cpu().numpy(), oracle.sparse_attn(util.oracle_kv(lays[1]), synth.bits(qs[1]),
+                                                           idx.t.cpu().numpy(), cnt.t.cpu().numpy()), "sparse")
+    # a whole step writing three guarded outputs and the guarded index list
+    outs = [util.Guarded((B, Hq, 128), torch.float32, DEV, fill=float("nan")) for _ in range(3)]
+    for i, g in enumerate(outs):
+        guards[f"out{i}"] = g
+    step = td.make_step([0, 1, 2], lays, qs, [g.t for g in outs], k)
+    # make_step owns its idx / idx_count; run it, then the same schedule by hand into the guarded ones
+    step()
+    check_all("step")
+    td.set_output_bf16(True)
+    try:
+        bouts = [util.Guarded((B, Hq, 128), torch.bfloat16, DEV) for _ in range(3)]
+        for i, g in enumerate(bouts):
+            guards[f"bf16 out{i}"] = g
+        td.make_step([0, 1, 2], lays, qs, [g.t for g in bouts], k)()
+        check_all("bf16 step")
+    finally:
+        td.set_output_bf16(False)
+    assert td.device_status() == binding.OK
+
+
+def test_bf16_outputs_match_the_oracle(td):
+    """Outputs rounded to bf16 against the oracle: the usual bounds widened by one bf16 step of the value
+    (2^-8 relative: the rounding of a correctly computed fp32 result moves it by at most half a step, the
+    fp32 result itself may sit on the other side of a rounding boundary)."""
+    sched = [0, 1, 2]
+    w = wl(2, 8, 2, 700, 64, ragged=True, ctx_min=300, seed=31, layers=len(sched))
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    layers = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(len(sched))]
+    td.set_output_bf16(True)
+    try:
+        outs, idx, cnt = td.decode_step(sched, layers, qs, w.k)
+        sel, idx2, cnt2 = td.select_attn(layers[1], qs[1], w.k)
+        sp = td.sparse_attn(layers[2], qs[2], idx2, cnt2)
+        torch.cuda.synchronize()
+    finally:
+        td.set_output_bf16(False)
+    idx_h, cnt_h = idx.cpu().numpy(), cnt.cpu().numpy()
+    refs = [oracle.full_attn(util.oracle_kv(layers[0]), synth.bits(qs[0])),
+            oracle.full_attn(util.oracle_kv(layers[1]), synth.bits(qs[1])),
+            oracle.sparse_attn(util.oracle_kv(layers[2]), synth.bits(qs[2]), idx_h, cnt_h)]
+
+    def check_bf16(got, ref, what):
+        got = got.float().cpu().numpy().astype(np.float64)
+        assert np.isfinite(got).all()
+        err = np.abs(got - ref)
+        assert (err <= util.MAX_ABS_TOL + np.abs(ref) * 2.0 ** -8).all(), f"{what}: max abs err {err.max():.3e}"
+        assert err.mean() <= util.MEAN_ABS_TOL + np.abs(ref).mean() * 2.0 ** -8, f"{what}: mean abs err {err.mean():.3e}"
+        # and in fact the error is the rounding alone
+        assert (err <= 1e-3 + np.abs(ref) * 2.0 ** -8).all(), what
+
+    for i in range(3):
+        assert outs[i].dtype == torch.bfloat16
+        check_bf16(outs[i], refs[i], f"bf16 step layer {i}")
+    check_bf16(sel, refs[1], "bf16 select")
+    assert torch.equal(idx2, idx)
+    check_bf16(sp, refs[2], "bf16 sparse")
+    assert td.device_status() == binding.OK
+
+
+def test_an_invalid_step_leaves_the_caches_untouched(td):
+    """tidal_decode_step_append validates the whole step before it writes a single row: a schedule with a
+    sparse layer ahead of any selection layer is refused and every cache byte is as before."""
+    sched = [0, 2, 1]
+    w = wl(2, 8, 2, 300, 16, ragged=True, ctx_min=50, seed=47, layers=3)
+    qs = [synth.make_q(w, i, DEV) for i in range(3)]
+    layers = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(3)]
+    before = [l.keep[0].clone() for l in layers]
+    kn = [torch.ones(w.batch, w.num_kv_heads, 128, dtype=torch.bfloat16, device=DEV) for _ in sched]
+    with pytest.raises(binding.TidalError) as e:
+        td.decode_step_append(sched, layers, qs, kn, kn, w.k)
+    assert e.value.status == binding.ERR_INVALID
+    torch.cuda.synchronize()
+    for l, b in zip(layers, before):
+        assert torch.equal(l.keep[0], b)
+    # k larger than a selection layer's max_ctx_len is refused the same way
+    with pytest.raises(binding.TidalError):
+        td.decode_step_append([0, 1, 2], layers, qs, kn, kn, 301)
+    torch.cuda.synchronize()
+    for l, b in zip(layers, before):
+        assert torch.equal(l.keep[0], b)
+
+
+def test_reserve_then_capture_the_first_call(td):
+    """tidal_reserve sizes workspace and counters, so that the very first call of a fresh context can be
+    recorded into a CUDA graph (nothing allocates, nothing touches the legacy stream)."""
+    sched = [0, 1, 2, 2]
+    w = wl(2, 8, 2, 1500, 64, ragged=True, ctx_min=400, seed=53, layers=len(sched))
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    layers = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(len(sched))]
+    ref_outs, ref_idx, _ = td.decode_step(sched, layers, qs, w.k)
+    torch.cuda.synchronize()
+    fresh = binding.Tidal(0)
+    try:
+        fresh.reserve(layers[0], w.k)
+        outs = [torch.zeros_like(o) for o in ref_outs]
+        step = fresh.make_step(sched, layers, qs, outs, w.k)
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                step()                                    # the context's first call ever
+        graph.replay()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(step.idx, ref_idx)
+        for o, r in zip(outs, ref_outs):
+            assert torch.allclose(o, r, rtol=0, atol=5e-4)
+        assert fresh.device_status() == binding.OK
+    finally:
+        fresh.close()
+
+
+def test_extreme_ragged_batches_stay_within_the_split_bound(td):
+    """One long sequence among many one-token ones, and the reverse: the number of CTAs that share a row
+    is bounded on the host; a kernel that found the bound too small would set the status word."""
+    for lens in ([4000] + [1] * 60, [1] * 60 + [4000], [4000, 3999] + [17] * 30, [16] * 64):
+        B = len(lens)
+        w = wl(B, 4, 2, max(lens), min(32, max(lens)), planted=1, seed=59)
+        q, lay = build(w, "paged")
+        lay.ctx_lens = torch.tensor(lens, dtype=torch.int32, device=DEV)
+        okv, qb = util.oracle_kv(lay), synth.bits(q)
+        out, idx, cnt = td.select_attn(lay, q, w.k)
+        ref, sc = oracle.full_attn(okv, qb, want_scores=True)
+        util.check_out(out.cpu().numpy(), ref, "ragged.select")
+        for b in (0, B - 1):
+            for h in range(4):
+                util.check_idx_row(idx.cpu().numpy()[b, h], sc[b, h], w.k, lens[b], "ragged.idx")
+        sp = td.sparse_attn(lay, q, idx, cnt)
+        util.check_out(sp.cpu().numpy(), oracle.sparse_attn(okv, qb, idx.cpu().numpy(), cnt.cpu().numpy()), "ragged.sparse")
+        assert td.device_status() == binding.OK

@@ -52,3 +52,31 @@ def check_idx_row(got_row, ref_scores, k, n, what=""):
     assert (s[sel] >= kth - TIE_BAND).all(), f"{what}: member below the tie band"
     ref_sel = oracle.topk(s, k)[:kk]
     return int(kk - np.intersect1d(sel, ref_sel).size)   # differences inside the band
+
+
+CANARY_BYTES = 512      # guard zone on each side of a guarded buffer
+
+
+class Guarded:
+    """A device tensor with CANARY_BYTES of a fixed pattern directly before and after it in memory.
+    compute-sanitizer is not available where these tests run; the guard zones catch stores that
+    stray past either end of an output buffer. `t` is the tensor to hand to the library."""
+
+    def __init__(self, shape, dtype, device, fill=None):
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        body = (n + 255) // 256 * 256                      # keeps the alignment of whatever follows
+        self.raw = torch.empty(CANARY_BYTES + body + CANARY_BYTES, dtype=torch.uint8, device=device)
+        self.pattern = (torch.arange(CANARY_BYTES, device=device) * 37 + 11).to(torch.uint8)
+        self.raw[:CANARY_BYTES] = self.pattern
+        self.raw[CANARY_BYTES + n:] = 0xA5
+        self.raw[CANARY_BYTES + body:] = self.pattern
+        self.n, self.body = n, body
+        self.t = self.raw[CANARY_BYTES:CANARY_BYTES + n].view(dtype).view(*shape)
+        if fill is not None:
+            self.t.fill_(fill)
+
+    def check(self, what=""):
+        torch.cuda.synchronize()
+        assert torch.equal(self.raw[:CANARY_BYTES], self.pattern), f"{what}: store before the buffer"
+        assert (self.raw[CANARY_BYTES + self.n:CANARY_BYTES + self.body] == 0xA5).all(), f"{what}: store just past the buffer"
+        assert torch.equal(self.raw[CANARY_BYTES + self.body:], self.pattern), f"{what}: store after the buffer"
