@@ -185,6 +185,19 @@ tidal_status_t tidal_set_output_dtype(tidal_ctx_t *ctx, int32_t dtype);
  * off and frees the recordings. */
 tidal_status_t tidal_set_graphs(tidal_ctx_t *ctx, int32_t enabled);
 
+/* Optional candidate compaction inside a selection layer's attention kernel (off by default: on B200
+ * it measured slower than ranking all scores from the fused histogram, see the design notes; it is
+ * kept as a tested alternative). Applies to one sequence, one token set per query head, groups of at
+ * most four and k <= max_ctx_len / 6; other cases always rank all scores. With margin > 0, every CTA
+ * of the attention kernel estimates, from the first few hundred scores it sees, a provisional
+ * threshold that about margin * k / N of a head's scores should reach, and lists the scores at or
+ * above it; the top-k then runs on that list alone. The result is exact whatever the margin: the list
+ * is used only if it provably contains the k best (its k-th best score is not below the largest
+ * threshold any CTA used); otherwise all scores are ranked by the same kernel, which is slower.
+ * margin: 0 = off (default); 3 is a sensible value; values below 1 make the shortcut fail on purpose
+ * (that is how the tests reach the exact fallback). */
+tidal_status_t tidal_set_select_margin(tidal_ctx_t *ctx, float margin);
+
 /* Overlap between the layers of a step (on by default). tidal_decode_step receives every layer's
  * query, lengths, page table and cache up front, so all of them are complete, in stream order, before
  * the call. With enabled != 0 a full-attention or sparse layer therefore streams its whole input while

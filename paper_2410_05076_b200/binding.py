@@ -27,7 +27,7 @@ EXPORTS = [
     "tidal_sparse_attn", "tidal_decode_step", "tidal_decode_step_host", "tidal_device_status",
     "tidal_launch_count", "tidal_strerror", "tidal_sparse_attn_noalloc", "tidal_kv_append",
     "tidal_decode_step_append", "tidal_set_graphs", "tidal_set_output_dtype", "tidal_set_attend_newest",
-    "tidal_set_layer_overlap", "tidal_reserve",
+    "tidal_set_layer_overlap", "tidal_reserve", "tidal_set_select_margin",
 ]
 
 
@@ -82,6 +82,8 @@ def load() -> C.CDLL:
     L.tidal_set_output_dtype.restype = I32
     L.tidal_set_layer_overlap.argtypes = [P, I32]
     L.tidal_set_layer_overlap.restype = I32
+    L.tidal_set_select_margin.argtypes = [P, C.c_float]
+    L.tidal_set_select_margin.restype = I32
     L.tidal_reserve.argtypes = [P, KVP, I32, I32]
     L.tidal_reserve.restype = I32
     L.tidal_set_graphs.argtypes = [P, I32]
@@ -306,6 +308,10 @@ class Tidal:
     def set_graphs(self, enabled: bool) -> None:
         """Record whole steps as CUDA graphs and replay them (on by default; needs a non-default stream)."""
         _check(self.lib.tidal_set_graphs(self.ctx, 1 if enabled else 0), "tidal_set_graphs")
+
+    def set_select_margin(self, margin: float) -> None:
+        """Safety factor of the selection layers' provisional thresholds (default 3; 0: rank all scores)."""
+        _check(self.lib.tidal_set_select_margin(self.ctx, margin), "tidal_set_select_margin")
 
     def set_layer_overlap(self, enabled: bool) -> None:
         """Layers of a step may stream their inputs while the layer before them finishes (on by default)."""

@@ -43,6 +43,11 @@ constexpr int TILE_BYTES = TILE * HEAD_DIM * 2;   // 4 KB of K, same of V
 constexpr int STAGE_BYTES = 2 * TILE_BYTES;
 constexpr int HIST_BINS = 2048;          // global histogram row: up to 11 top bits of the score key
 constexpr int HIST_SMEM_WORDS = 8192;    // shared histogram: columns x bins <= 8192 counters (32 KB)
+// Candidate compaction in the selection layer's kernel (layout of the 32 KB behind the rings):
+constexpr int CAL_TILES = 3;             // tiles per warp whose scores are staged to estimate the threshold (one ring fill)
+constexpr int CAND_COLS = 4;             // query heads per KV head it supports
+constexpr int CAND_BUF = 64;             // per (warp, head) buffer of candidates in shared memory ...
+constexpr int CAND_FLUSH = 32;           // ... written out once it holds this many (two more tiles add at most 32)
 constexpr int GRAB_TILES = 4;            // tiles a warp takes from its item's pool at a time afterwards (gather kernel)
 constexpr int GRAB_TILES_DENSE = 2;      // the same for the streaming kernels, whose items hold thousands of tiles
 
@@ -72,6 +77,16 @@ struct AttnParams {
     float2* part_ml;           // [B*Hq, max_splits] (running max in base 2, sum)
     int* counters;             // one per (sequence, item), zero between launches
     int max_splits;            // partial slots per (sequence, head) row
+    // MODE_SELECT, optional (one sequence, one token set per query head, groups of at most four): instead
+    // of the histogram, every CTA estimates a threshold per head from its first tiles and appends the
+    // (key, position) of every score at or above it to that head's candidate list; the largest threshold
+    // any CTA used is recorded, so that the top-k can tell whether the list is complete down to the k-th score.
+    int compact;
+    uint2* cand;               // [B*Hq][cand_stride]
+    long long cand_stride;
+    int* cand_cursor;          // [B*Hq][ctr_stride] entries in the list, zero between launches
+    unsigned* thr_max;         // [B*Hq][ctr_stride] largest threshold key used, zero between launches
+    float margin;              // the threshold aims at this multiple of k' / N of the scores
     unsigned* hist;            // MODE_SELECT, optional: [B*Hq][HIST_BINS] += histogram of the top key bits
     int hist_shift;            // bin = key >> hist_shift (21: 2048 bins, 22: 1024 bins for groups above 4)
     int* tile_ctr;             // splits_per_item > 0: per-item pool cursor, zero between launches
@@ -184,6 +199,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
 __device__ __forceinline__ uint32_t score_key_bits(float s) {
     uint32_t u = __float_as_uint(s);
     if (u == 0x80000000u) u = 0u;
+    if ((u & 0x7fffffffu) > 0x7f800000u) return 0u;      // not a number: below every number
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
@@ -198,11 +214,19 @@ struct WarpAcc {
 // Consume one staged tile: 16 K rows at ks, 16 V rows at vs (swizzled, see
 // the issue code), `vmask` bit r set when row r is a real cached token,
 // pos_base + r its position (only used to store scores).
+// What one warp needs to compact candidates while it consumes a tile (selection layers only).
+struct CandWarp {
+    uint32_t* stage;           // calibration: where this tile's keys go, [16 rows][CAND_COLS]; null afterwards
+    float thr0, thr1;          // thresholds of this lane's two heads
+    uint2* buf;                // this warp's candidate buffers [CAND_COLS][CAND_BUF]
+    int* cnt;                  // ... and their fill counts [CAND_COLS]
+};
+
 template <int MODE>
 __device__ __forceinline__ void consume_tile(const AttnParams& p, uint32_t ks, uint32_t vs,
                                              const uint32_t (&qf)[4][4], WarpAcc& acc, uint32_t vmask,
                                              int gid, int tig, float* score_row0, float* score_row1,
-                                             int pos_base, uint32_t* hist) {
+                                             int pos_base, uint32_t* hist, const CandWarp* cw = nullptr) {
     // ---- S^T = K . Q^T ------------------------------------------------------
     // Two independent accumulator chains (even / odd 32-element blocks of the head dimension).
     float s[4] = {0.f, 0.f, 0.f, 0.f};
@@ -253,6 +277,42 @@ __device__ __forceinline__ void consume_tile(const AttnParams& p, uint32_t ks, u
         if (score_row1) {
             if (v0) st_keep(score_row1 + pos_base + gid, f1, keep);
             if (v1) st_keep(score_row1 + pos_base + gid + 8, f3, keep);
+        }
+        if (cw) {
+            if (cw->stage) {
+                // calibration tiles: keep the keys (0 where there is no token) for the threshold estimate
+                if (score_row0) {
+                    cw->stage[gid * CAND_COLS + 2 * tig] = v0 ? score_key_bits(f0) : 0u;
+                    cw->stage[(gid + 8) * CAND_COLS + 2 * tig] = v1 ? score_key_bits(f2) : 0u;
+                }
+                if (score_row1) {
+                    cw->stage[gid * CAND_COLS + 2 * tig + 1] = v0 ? score_key_bits(f1) : 0u;
+                    cw->stage[(gid + 8) * CAND_COLS + 2 * tig + 1] = v1 ? score_key_bits(f3) : 0u;
+                }
+            } else {
+                // Slots in the warp's per-head buffers come from ballots, not from atomics that return a
+                // value (their round trips would stall the warp four times per tile): the lanes that share
+                // a tig hold the scores of the same two heads.
+                const bool c0 = score_row0 && v0 && f0 >= cw->thr0, c2 = score_row0 && v1 && f2 >= cw->thr0;
+                const bool c1 = score_row1 && v0 && f1 >= cw->thr1, c3 = score_row1 && v1 && f3 >= cw->thr1;
+                const unsigned m0 = __ballot_sync(0xffffffffu, c0), m2 = __ballot_sync(0xffffffffu, c2);
+                const unsigned m1 = __ballot_sync(0xffffffffu, c1), m3 = __ballot_sync(0xffffffffu, c3);
+                if (m0 | m1 | m2 | m3) {
+                    const unsigned grp = 0x11111111u << tig, below = (1u << (gid * 4 + tig)) - 1u;
+                    const int h0 = 2 * tig, h1 = h0 + 1;
+                    const int base0 = score_row0 ? cw->cnt[h0] : 0, base1 = score_row1 ? cw->cnt[h1] : 0;
+                    const int n00 = __popc(m0 & grp), n01 = __popc(m2 & grp), n10 = __popc(m1 & grp), n11 = __popc(m3 & grp);
+                    if (c0) cw->buf[h0 * CAND_BUF + base0 + __popc(m0 & grp & below)] = make_uint2(score_key_bits(f0), pos_base + gid);
+                    if (c2) cw->buf[h0 * CAND_BUF + base0 + n00 + __popc(m2 & grp & below)] = make_uint2(score_key_bits(f2), pos_base + gid + 8);
+                    if (c1) cw->buf[h1 * CAND_BUF + base1 + __popc(m1 & grp & below)] = make_uint2(score_key_bits(f1), pos_base + gid);
+                    if (c3) cw->buf[h1 * CAND_BUF + base1 + n10 + __popc(m3 & grp & below)] = make_uint2(score_key_bits(f3), pos_base + gid + 8);
+                    __syncwarp();                     // every lane has read the counts it needs
+                    if (gid == 0) {
+                        if (score_row0 && (n00 | n01)) cw->cnt[h0] = base0 + n00 + n01;
+                        if (score_row1 && (n10 | n11)) cw->cnt[h1] = base1 + n10 + n11;
+                    }
+                }
+            }
         }
         if (hist) {      // histogram of the top key bits of every stored score, per head
             const int nb = 1 << (32 - p.hist_shift);
@@ -390,6 +450,26 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
     if (hist_on) {
         for (int i = threadIdx.x; i < HIST_SMEM_WORDS; i += NW * 32) hist[i] = 0;
         __syncthreads();
+    }
+    // Candidate compaction (pooled launches only: a CTA serves one item). The 32 KB behind the rings hold
+    //   stage    [NW][CAL_TILES][16][CAND_COLS] keys of the calibration tiles
+    //   st_pos   [NW][CAL_TILES] first position of each staged tile (-1: none), st_vm: its valid rows
+    //   thr_key  [CAND_COLS] the thresholds as keys, thr_val as values
+    //   cbuf     [NW][CAND_COLS][CAND_BUF] candidates waiting to be written out, ccnt [NW][CAND_COLS] fill counts
+    const bool compact = (MODE == MODE_SELECT) && p.compact && p.splits_per_item > 0;
+    uint32_t* stage_all = hist;
+    int* st_pos = reinterpret_cast<int*>(stage_all + NW * CAL_TILES * 16 * CAND_COLS);
+    uint32_t* st_vm = reinterpret_cast<uint32_t*>(st_pos + NW * CAL_TILES);
+    uint32_t* thr_key = st_vm + NW * CAL_TILES;
+    float* thr_val = reinterpret_cast<float*>(thr_key + CAND_COLS);
+    int* ccnt_all = reinterpret_cast<int*>(thr_val + CAND_COLS);
+    uint2* cbuf_all = reinterpret_cast<uint2*>(ccnt_all + NW * CAND_COLS);        // 8-byte aligned: all counts above are even
+    static_assert((NW * CAL_TILES * 16 * CAND_COLS + 2 * NW * CAL_TILES + 2 * CAND_COLS + NW * CAND_COLS) * 4 +
+                  NW * CAND_COLS * CAND_BUF * 8 <= HIST_SMEM_WORDS * 4 || MODE != MODE_SELECT, "compaction scratch exceeds the histogram area");
+    if (compact) {
+        if (lane < CAL_TILES) st_pos[warp * CAL_TILES + lane] = -1;
+        if (lane < CAND_COLS) ccnt_all[warp * CAND_COLS + lane] = 0;
+        __syncwarp();
     }
 
     uint8_t* wbase = smem + (size_t)warp * STAGES * STAGE_BYTES;
@@ -635,6 +715,100 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             cp_async_commit();
             ++commits;
         }
+        // ---- candidate compaction: helpers of this warp ---------------------------------------------------
+        CandWarp cw;
+        cw.stage = nullptr;
+        cw.thr0 = cw.thr1 = INFINITY;
+        cw.buf = cbuf_all + warp * CAND_COLS * CAND_BUF;
+        cw.cnt = ccnt_all + warp * CAND_COLS;
+        bool calibrated = false;
+        // Write out the buffers of this warp that hold at least `least` candidates: one cursor bump per buffer.
+        auto cand_flush = [&](int least) {
+            __syncwarp();
+            const int c = (lane < ncols) ? cw.cnt[lane] : 0;
+            unsigned m = __ballot_sync(0xffffffffu, c >= least && c > 0);
+            while (m) {
+                const int col = __ffs(m) - 1;
+                m &= m - 1;
+                const int n = __shfl_sync(0xffffffffu, c, col);
+                const long long row = (long long)b * p.Hq + head0 + col;
+                int base = 0;
+                if (lane == 0) base = atomicAdd(p.cand_cursor + row * p.ctr_stride, n);
+                base = __shfl_sync(0xffffffffu, base, 0);
+                uint2* dst = p.cand + row * p.cand_stride;
+                for (int i = lane; i < n; i += 32)
+                    if (base + i < p.cand_stride) dst[base + i] = cw.buf[col * CAND_BUF + i];
+                if (lane == 0) cw.cnt[col] = 0;
+            }
+            __syncwarp();
+        };
+        // Once per CTA, by all warps together: thresholds from the staged scores of every warp's first tiles
+        // (the r-th largest staged key of a head, r = margin * k' / N of the sample), then every warp
+        // compacts its own staged tiles with them.
+        auto calibrate = [&]() {
+            __syncthreads();
+            if (warp < ncols) {
+                const int col = warp;
+                constexpr int PER_LANE = (NW * CAL_TILES * 16 + 31) / 32;
+                uint32_t keys[PER_LANE];
+                int nvalid = 0;
+#pragma unroll
+                for (int u = 0; u < PER_LANE; ++u) {
+                    const int e = lane + 32 * u, wt = e >> 4, r = e & 15;        // wt = warp * CAL_TILES + tile
+                    const bool ok = wt < NW * CAL_TILES && st_pos[wt] >= 0 && ((st_vm[wt] >> r) & 1u);
+                    keys[u] = ok ? stage_all[(wt * 16 + r) * CAND_COLS + col] : 0u;
+                    nvalid += ok;
+                }
+#pragma unroll
+                for (int sh = 16; sh >= 1; sh >>= 1) nvalid += __shfl_xor_sync(0xffffffffu, nvalid, sh);
+                const int kk = min(p.budget, N);
+                const float frac = p.margin * (float)kk / (float)max(N, 1);
+                const int rank = (int)ceilf(frac * (float)nvalid) + 2;
+                uint32_t tk = 0;                                            // 0: everything is a candidate
+                if (nvalid >= 64 && rank < nvalid) {
+                    // the rank-th largest staged key: the largest value that at least `rank` keys reach
+                    for (int bit = 31; bit >= 12; --bit) {           // 20 bits: the threshold need not be finer
+                        const uint32_t trial = tk | (1u << bit);
+                        int cnt = 0;
+#pragma unroll
+                        for (int u = 0; u < PER_LANE; ++u) cnt += keys[u] >= trial;
+#pragma unroll
+                        for (int sh = 16; sh >= 1; sh >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, sh);
+                        if (cnt >= rank) tk = trial;
+                    }
+                }
+                if (lane == 0) {
+                    thr_key[col] = tk;
+                    // the value whose key is tk (key 0 belongs to no number: everything passes)
+                    thr_val[col] = tk == 0 ? -INFINITY : __uint_as_float((tk & 0x80000000u) ? (tk & 0x7fffffffu) : ~tk);
+                    atomicMax(p.thr_max + ((long long)b * p.Hq + head0 + col) * p.ctr_stride, tk);
+                }
+            }
+            __syncthreads();
+            cw.thr0 = (2 * tig < ncols) ? thr_val[2 * tig] : INFINITY;
+            cw.thr1 = (2 * tig + 1 < ncols) ? thr_val[2 * tig + 1] : INFINITY;
+            for (int t = 0; t < CAL_TILES; ++t) {
+                const int wt = warp * CAL_TILES + t, pos0 = st_pos[wt];
+                if (pos0 < 0) break;
+                const uint32_t vm = st_vm[wt];
+                static_assert(CAND_COLS == 4, "a lane's column below is its tig");
+#pragma unroll
+                for (int u = 0; u < 16 * CAND_COLS / 32; ++u) {
+                    const int e = lane + 32 * u, r = e / CAND_COLS, col = tig;        // e % CAND_COLS == lane & 3
+                    const uint32_t key = stage_all[(wt * 16 + r) * CAND_COLS + col];
+                    const bool take = col < ncols && ((vm >> r) & 1u) && key >= thr_key[col];
+                    const unsigned m = __ballot_sync(0xffffffffu, take) & (0x11111111u << tig);
+                    const int base = (col < ncols) ? cw.cnt[col] : 0;
+                    if (take) cw.buf[col * CAND_BUF + base + __popc(m & ((1u << lane) - 1u))] = make_uint2(key, (unsigned)(pos0 + r));
+                    __syncwarp();
+                    if (gid == 0 && m) cw.cnt[col] = base + __popc(m);
+                    __syncwarp();
+                }
+                cand_flush(CAND_FLUSH);
+            }
+            calibrated = true;
+        };
+
         for (int it = 0; it < issued; ++it) {
             if (it == 0 && ring_full) {
                 cp_async_wait<STAGES - 1>();
@@ -647,11 +821,56 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             }
             const int stage = it % STAGES;
             const uint32_t ks = wbase_u32 + stage * STAGE_BYTES;
-            consume_tile<MODE>(p, ks, ks + TILE_BYTES, qf, acc, s_vmask[warp][stage], gid, tig,
-                               score_row0, score_row1, s_posbase[warp][stage], hist_on ? hist : nullptr);
+            if (MODE == MODE_SELECT && compact) {
+                if (!calibrated && it == CAL_TILES) calibrate();
+                cw.stage = nullptr;
+                if (!calibrated) {
+                    const int wt = warp * CAL_TILES + it;
+                    cw.stage = stage_all + wt * 16 * CAND_COLS;
+                    if (lane == 0) { st_pos[wt] = s_posbase[warp][stage]; st_vm[wt] = s_vmask[warp][stage]; }
+                }
+                // A buffer that has reached CAND_FLUSH entries reserves its place in the head's list now (lane
+                // `col` asks for buffer `col`) and is written out after the tile, when the answer has arrived;
+                // what the tile itself adds stays behind as the start of the next batch.
+                int pend_n = 0, pend_base = 0;
+                __syncwarp();                                         // the counts as the previous tile left them
+                if (calibrated && lane < ncols) {
+                    const int c = cw.cnt[lane];
+                    if (c >= CAND_FLUSH) {
+                        pend_n = c;
+                        pend_base = atomicAdd(p.cand_cursor + ((long long)b * p.Hq + head0 + lane) * p.ctr_stride, c);
+                    }
+                }
+                consume_tile<MODE>(p, ks, ks + TILE_BYTES, qf, acc, s_vmask[warp][stage], gid, tig,
+                                   score_row0, score_row1, s_posbase[warp][stage], nullptr, &cw);
+                __syncwarp();
+                unsigned pend = __ballot_sync(0xffffffffu, pend_n > 0);
+                while (pend) {
+                    const int col = __ffs(pend) - 1;
+                    pend &= pend - 1;
+                    const int n = __shfl_sync(0xffffffffu, pend_n, col), base = __shfl_sync(0xffffffffu, pend_base, col);
+                    uint2* dst = p.cand + ((long long)b * p.Hq + head0 + col) * p.cand_stride;
+                    uint2* src = cw.buf + col * CAND_BUF;
+                    const int total = cw.cnt[col];                    // n plus what this tile added (at most 16)
+                    for (int i = lane; i < n; i += 32)
+                        if (base + i < p.cand_stride) dst[base + i] = src[i];
+                    const uint2 moved = (lane < total - n) ? src[n + lane] : make_uint2(0u, 0u);
+                    __syncwarp();
+                    if (lane < total - n) src[lane] = moved;
+                    if (lane == 0) cw.cnt[col] = total - n;
+                    __syncwarp();
+                }
+            } else {
+                consume_tile<MODE>(p, ks, ks + TILE_BYTES, qf, acc, s_vmask[warp][stage], gid, tig,
+                                   score_row0, score_row1, s_posbase[warp][stage], hist_on ? hist : nullptr);
+            }
         }
         cp_async_wait<0>();
         __syncwarp();
+        if (MODE == MODE_SELECT && compact) {
+            if (!calibrated) calibrate();         // fewer tiles than the calibration takes: every warp still meets here
+            cand_flush(1);
+        }
         // All of this item's tiles are in the accumulators. With a late wait the grid dependency is
         // resolved only now: everything below writes memory that the preceding kernel may still use.
         if (!waited) {

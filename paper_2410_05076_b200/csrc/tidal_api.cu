@@ -51,6 +51,7 @@ struct tidal_ctx {
     int out_bf16 = 0;                           // outputs are written as bf16 instead of fp32
     int attend_newest = 0;                      // sparse layers also attend the newest token (not in the paper)
     int cursor_set = 0;                         // which of the sets of pool cursors the last attention launch used
+    float select_margin = 0.f;                  // > 0: selection layers compact candidates above a provisional threshold aimed at this multiple of k'/N
     int layer_overlap = 1;                      // layers of a step may stream their inputs while the layer before them finishes
     int64_t launches = 0;
     // Whole steps are recorded once as CUDA graphs (programmatic dependent launches included) and
@@ -185,7 +186,7 @@ tidal_status_t ensure_ws(tidal_ctx* ctx, size_t bytes) {
     return TIDAL_OK;
 }
 
-// State layout for a capacity of R rows: counters | cursor | done | tile_ctr sets 0..2, each
+// State layout for a capacity of R rows: counters | cursor | done | thr_max | tile_ctr sets, each
 // [R][CTR_STRIDE], then hist[R][TK_BINS]. Consecutive attention launches rotate through the sets of
 // pool cursors, so that a launch may use its set before its predecessor has finished with another.
 // Every counter has a 128-byte line of its own: hundreds of warps hit them at once, and atomics to one
@@ -195,8 +196,9 @@ constexpr int CURSOR_SETS = 6;
 inline int* state_counters(const tidal_ctx* c) { return (int*)c->state; }
 inline int* state_cursor(const tidal_ctx* c) { return (int*)c->state + (size_t)CTR_STRIDE * c->state_rows; }
 inline int* state_done(const tidal_ctx* c) { return (int*)c->state + 2 * (size_t)CTR_STRIDE * c->state_rows; }
-inline int* state_tile_ctr(const tidal_ctx* c) { return (int*)c->state + 3 * (size_t)CTR_STRIDE * c->state_rows; }
-inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + (3 + CURSOR_SETS) * (size_t)CTR_STRIDE * c->state_rows; }
+inline unsigned* state_thr_max(const tidal_ctx* c) { return (unsigned*)c->state + 3 * (size_t)CTR_STRIDE * c->state_rows; }
+inline int* state_tile_ctr(const tidal_ctx* c) { return (int*)c->state + 4 * (size_t)CTR_STRIDE * c->state_rows; }
+inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + (4 + CURSOR_SETS) * (size_t)CTR_STRIDE * c->state_rows; }
 
 tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     if (ctx->state_rows >= rows) return TIDAL_OK;
@@ -204,7 +206,7 @@ tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     drop_graphs(ctx);
     if (ctx->state) { cudaDeviceSynchronize(); cudaFree(ctx->state); ctx->state = nullptr; ctx->state_rows = 0; }
     const int cap = (int)align_up((size_t)rows, 64);
-    const size_t bytes = (size_t)cap * ((3 + CURSOR_SETS) * CTR_STRIDE + TK_BINS) * sizeof(int);
+    const size_t bytes = (size_t)cap * ((4 + CURSOR_SETS) * CTR_STRIDE + TK_BINS) * sizeof(int);
     void* p = nullptr;
     if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TIDAL_ERR_NOMEM; }
     // on a stream of its own, so that nothing here is the legacy stream's business, and waited for
@@ -295,12 +297,25 @@ tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, int full_gri
 // fused. Fewer index heads than query heads: the ranking score is the sum of the member heads'
 // scaled logits; unless the caller wants the per-head scores, the attention kernel stores the
 // group sums directly (one row per KV head; histogram fused when a set belongs to one KV head).
-struct SelectPlan { bool agg, fuse; int rows; };
-SelectPlan select_plan(const tidal_kv_t* kv, int Hi, bool caller_scores) {
+// With one sequence, one set per query head and enough scores per set, the attention kernel compacts
+// candidates instead (no histogram) and a single CTA per head finishes the selection on them.
+struct SelectPlan { bool agg, fuse, compact; int rows; };
+constexpr int COMPACT_LIST_SMEM = 12288;      // candidates the compacting top-k keeps in shared memory
+
+int dense_grid(const tidal_ctx* ctx, const tidal_kv_t* kv) {
+    const long long tiles = (long long)kv->batch * kv->num_kv_heads * ((kv->max_ctx_len + TILE - 1) / TILE);
+    return grid_for(tiles, ctx->dense_slots);
+}
+
+SelectPlan select_plan(const tidal_ctx* ctx, const tidal_kv_t* kv, int Hi, int k, bool caller_scores) {
     SelectPlan s;
     s.agg = Hi != kv->num_q_heads && !caller_scores;
     s.rows = s.agg ? kv->num_kv_heads : kv->num_q_heads;
     s.fuse = Hi == s.rows;
+    s.compact = ctx->select_margin > 0.f && Hi == kv->num_q_heads && kv->batch == 1 &&
+                kv->num_q_heads / kv->num_kv_heads <= CAND_COLS && 6LL * k <= kv->max_ctx_len &&
+                pooled_splits(kv, kv->num_kv_heads, dense_grid(ctx, kv)) > 0;
+    if (s.compact) s.fuse = false;
     return s;
 }
 
@@ -310,13 +325,21 @@ enum Dep { DEP_FIRST, DEP_PREFETCH, DEP_LATE };
 
 tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, float* out, float* scores,
                          long long score_stride, bool fuse_hist, Dep dep, const WsLayout& w, cudaStream_t st,
-                         bool agg = false) {
+                         bool agg = false, int compact_k = 0) {
     AttnParams a;
     fill_common(a, ctx, kv, q, out, w);
     a.wait_first = dep == DEP_FIRST;
     a.wait_late = dep == DEP_LATE && scores == nullptr;   // a selection layer writes scores while it streams
-    const long long tiles = (long long)kv->batch * kv->num_kv_heads * ((kv->max_ctx_len + TILE - 1) / TILE);
-    int grid = grid_for(tiles, ctx->dense_slots);
+    int grid = dense_grid(ctx, kv);
+    if (compact_k > 0) {
+        a.compact = 1;
+        a.cand = (uint2*)((char*)ctx->ws + w.cand);
+        a.cand_stride = w.cand_stride;
+        a.cand_cursor = state_cursor(ctx);
+        a.thr_max = state_thr_max(ctx);
+        a.margin = ctx->select_margin;
+        a.budget = compact_k;
+    }
     if (const int S = pooled_splits(kv, kv->batch * kv->num_kv_heads, grid)) {
         a.splits_per_item = S;        // the grid keeps its size: some items get one CTA more than others
     }
@@ -331,7 +354,7 @@ tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, fl
 // `rows`: score rows per sequence (query heads, or KV heads when the attention kernel stored group sums).
 tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* scores, long long score_stride,
                         int k, int rows, int Hi, bool hist_done, int* idx, int* idx_count, const WsLayout& w,
-                        cudaStream_t st) {
+                        cudaStream_t st, bool compact = false) {
     TopkParams t;
     std::memset(&t, 0, sizeof t);
     t.scores = scores; t.score_stride = score_stride;
@@ -374,6 +397,15 @@ tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* score
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (compact) {
+        t.thr_max = state_thr_max(ctx);
+        t.list_smem = COMPACT_LIST_SMEM;
+        const size_t bm_words = (size_t)(kv->max_ctx_len + 31) / 32;
+        cfg.gridDim = dim3(items, 1, 1);
+        cfg.dynamicSmemBytes = 2 * (bm_words + 1) * sizeof(unsigned) + (size_t)COMPACT_LIST_SMEM * sizeof(uint2);
+        ctx->launches++;
+        return cudaLaunchKernelEx(&cfg, topk_compact_kernel, t) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+    }
     if (!hist_done) {
         cfg.gridDim = dim3(parts, items, 1);
         cfg.dynamicSmemBytes = 0;
@@ -440,7 +472,7 @@ struct KeyBuilder {
 void step_key(KeyBuilder& kb, const tidal_ctx* ctx, int tag, int32_t num_layers, const uint8_t* schedule,
                      const tidal_kv_t* kvs, int32_t k, int32_t granularity, int host_layers) {
     kb.add(tag); kb.add(num_layers); kb.add(k); kb.add(granularity); kb.add(host_layers);
-    kb.add(ctx->ws); kb.add(ctx->state); kb.add(ctx->out_bf16); kb.add(ctx->attend_newest); kb.add(ctx->layer_overlap);
+    kb.add(ctx->ws); kb.add(ctx->state); kb.add(ctx->out_bf16); kb.add(ctx->attend_newest); kb.add(ctx->layer_overlap); kb.add(ctx->select_margin);
     kb.add_raw(schedule, (size_t)num_layers);
     for (int i = 0; i < num_layers; ++i) {
         // field by field: the struct has padding whose bytes are not the caller's to define
@@ -533,7 +565,9 @@ tidal_status_t tidal_create(tidal_ctx_t** out, int device, size_t workspace_byte
     const int s1 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES, true>, SPARSE_NW * 32, attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(), ctx->sm_count);
     const size_t topk_smem = 2 * (size_t)(MAX_CTX / 32) * sizeof(unsigned) + 8192 * sizeof(uint2);
     const bool topk_ok = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topk_smem) == cudaSuccess;
-    if (d0 <= 0 || d1 <= 0 || s0 <= 0 || s1 < s0 || !topk_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
+    const size_t compact_smem = 2 * ((size_t)(MAX_CTX / 32) + 1) * sizeof(unsigned) + (size_t)COMPACT_LIST_SMEM * sizeof(uint2);
+    const bool compact_ok = cudaFuncSetAttribute(topk_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)compact_smem) == cudaSuccess;
+    if (d0 <= 0 || d1 <= 0 || s0 <= 0 || s1 < s0 || !topk_ok || !compact_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
     ctx->dense_slots = std::min(d0, d1);
     ctx->sparse_slots = s0;
     if (cudaMalloc((void**)&ctx->status, 256) != cudaSuccess || cudaMemset(ctx->status, 0, 256) != cudaSuccess) {
@@ -630,9 +664,9 @@ tidal_status_t tidal_select_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const v
     float* scores = scores_opt ? scores_opt : (float*)((char*)ctx->ws + w.scores);
     const long long stride = scores_opt ? (long long)kv->max_ctx_len : w.score_stride;
     cudaStream_t st = (cudaStream_t)stream;
-    const SelectPlan sp = select_plan(kv, Hi, scores_opt != nullptr);
-    if ((rc = run_dense(ctx, kv, q, out, scores, stride, sp.fuse, DEP_FIRST, w, st, sp.agg)) != TIDAL_OK) return rc;
-    return run_topk(ctx, kv, scores, stride, k, sp.rows, Hi, sp.fuse, idx, idx_count, w, st);
+    const SelectPlan sp = select_plan(ctx, kv, Hi, k, scores_opt != nullptr);
+    if ((rc = run_dense(ctx, kv, q, out, scores, stride, sp.fuse, DEP_FIRST, w, st, sp.agg, sp.compact ? k : 0)) != TIDAL_OK) return rc;
+    return run_topk(ctx, kv, scores, stride, k, sp.rows, Hi, sp.fuse, idx, idx_count, w, st, sp.compact);
 }
 
 tidal_status_t tidal_sparse_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const void* q, const int32_t* idx,
@@ -698,9 +732,9 @@ static tidal_status_t decode_step_enqueue(tidal_ctx_t* ctx, int32_t num_layers, 
             rc = run_dense(ctx, kv, qs[i], outs[i], nullptr, 0, false, dep, w, st);
         } else if (schedule[i] == TIDAL_LAYER_SELECT) {
             float* scores = (float*)((char*)ctx->ws + w.scores);
-            const SelectPlan sp = select_plan(kv, Hi, false);
-            rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, sp.fuse, dep, w, st, sp.agg);
-            if (rc == TIDAL_OK) rc = run_topk(ctx, kv, scores, w.score_stride, k, sp.rows, Hi, sp.fuse, idx, idx_count, w, st);
+            const SelectPlan sp = select_plan(ctx, kv, Hi, k, false);
+            rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, sp.fuse, dep, w, st, sp.agg, sp.compact ? k : 0);
+            if (rc == TIDAL_OK) rc = run_topk(ctx, kv, scores, w.score_stride, k, sp.rows, Hi, sp.fuse, idx, idx_count, w, st, sp.compact);
         } else {
             const bool fresh_idx = i == 0 || schedule[i - 1] == TIDAL_LAYER_SELECT;
             const bool chain = ctx->layer_overlap && ((i > 0 && schedule[i - 1] == TIDAL_LAYER_SPARSE) ||
@@ -773,6 +807,12 @@ tidal_status_t tidal_decode_step(tidal_ctx_t* ctx, int32_t num_layers, const uin
 tidal_status_t tidal_set_attend_newest(tidal_ctx_t* ctx, int32_t enabled) {
     if (!ctx) return TIDAL_ERR_INVALID;
     ctx->attend_newest = enabled != 0;
+    return TIDAL_OK;
+}
+
+tidal_status_t tidal_set_select_margin(tidal_ctx_t* ctx, float margin) {
+    if (!ctx || !(margin >= 0.f) || margin > 64.f) return TIDAL_ERR_INVALID;
+    ctx->select_margin = margin;
     return TIDAL_OK;
 }
 

@@ -57,14 +57,33 @@ struct TopkParams {
     int vec_ok;                // score rows are 16-byte aligned: float4 loads allowed
     int shift;                 // first digit = key >> shift (21 or 22); the rest is split 11 + (shift-11) bits
     int pdl;                   // launched with programmatic stream serialization: wait for the producer of the scores
+    unsigned* thr_max;         // topk_compact_kernel: [items][ctr_stride] largest provisional threshold key, zero between calls
+    int list_smem;             // topk_compact_kernel: candidates its shared memory holds
 };
 
 // Larger float <=> larger key; -0 and +0 map to the same key.
+// A score that is not a number gets key 0, below every number (the float comparisons used elsewhere
+// in the selection are false for it as well, so it is never ranked above anything).
 __device__ __forceinline__ uint32_t score_key(float s) {
     uint32_t u = __float_as_uint(s);
     if (u == 0x80000000u) u = 0u;
+    if ((u & 0x7fffffffu) > 0x7f800000u) return 0u;
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
+
+// Keys of (key, position) pairs or of a row of scores, behind one interface, so that the exact
+// selection below can run on a compacted candidate list or, when that list turns out to be
+// incomplete, on all scores of the row.
+struct PairSource {
+    const uint2* c;
+    int n;
+    __device__ __forceinline__ uint2 get(int i) const { return c[i]; }
+};
+struct ScoreSource {
+    const float* s;
+    int n;
+    __device__ __forceinline__ uint2 get(int i) const { return make_uint2(score_key(__ldcg(s + i)), (unsigned)i); }
+};
 
 // The value whose key is `key` (inverse of score_key; -0 never occurs as a key).
 __device__ __forceinline__ float key_score(uint32_t key) {
@@ -503,6 +522,8 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
                 bits &= bits - 1;
             }
         }
+        // (scores that are not numbers are counted but never taken: the list may then come out short)
+        for (int i = min(tot, kk) + tid; i < kk; i += TK_THREADS) out[i] = -1;
     } else {
     // ordered enumeration: (winner count, equal count) scanned together in one 64-bit value
     unsigned long long cnt = 0;
@@ -526,12 +547,223 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
             bits &= bits - 1;
         }
     }
+    const int taken = (int)(tot >> 32) + min((int)(tot & 0xffffffffu), need);
+    for (int i = min(taken, kk) + tid; i < kk; i += TK_THREADS) out[i] = -1;
     }
     for (int i = kk + tid; i < p.k; i += TK_THREADS) out[i] = -1;
 
     // leave the shared state clean for the next call
     for (int i = tid; i < TK_BINS; i += TK_THREADS) gh[i] = 0;
     if (tid == 0 && !solo) { p.cursor[(size_t)item * p.ctr_stride] = 0; p.done[(size_t)item * p.ctr_stride] = 0; }
+}
+
+// The k'-th largest key of a source by three digit passes (most significant first); on return `need`
+// is how many keys equal to it are to be taken. Every thread gets the same result.
+template <typename Src>
+__device__ __noinline__ uint32_t kth_largest_key(const Src src, int shift, int& need, unsigned* sh_hist,
+                                                 int* warp_sums, int* bcast) {
+    const int tid = threadIdx.x;
+    const int s2 = shift - 11;
+    for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
+    __syncthreads();
+    for (int i = tid; i < src.n; i += TK_THREADS) atomicAdd(&sh_hist[src.get(i).x >> shift], 1u);
+    __syncthreads();
+    const int b1 = pick_digit(sh_hist, TK_BINS, warp_sums, bcast, need);
+    for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
+    __syncthreads();
+    for (int i = tid; i < src.n; i += TK_THREADS) {
+        const uint32_t k32 = src.get(i).x;
+        if ((int)(k32 >> shift) == b1) atomicAdd(&sh_hist[(k32 >> s2) & 0x7ffu], 1u);
+    }
+    __syncthreads();
+    const int d2 = pick_digit(sh_hist, TK_BINS, warp_sums, bcast, need);
+    const uint32_t prefix2 = ((uint32_t)b1 << shift) | ((uint32_t)d2 << s2);
+    for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
+    __syncthreads();
+    for (int i = tid; i < src.n; i += TK_THREADS) {
+        const uint32_t k32 = src.get(i).x;
+        if ((k32 >> s2) == (prefix2 >> s2)) atomicAdd(&sh_hist[k32 & ((1u << s2) - 1u)], 1u);
+    }
+    __syncthreads();
+    const int d3 = pick_digit(sh_hist, 1 << s2, warp_sums, bcast, need);
+    return prefix2 | (uint32_t)d3;
+}
+
+// Positions of a source whose key exceeds `thr` into the bitmap cgt, those equal to it into ceq.
+template <typename Src>
+__device__ __noinline__ void mark_winners(const Src src, uint32_t thr, unsigned* cgt, unsigned* ceq) {
+    for (int i = threadIdx.x; i < src.n; i += TK_THREADS) {
+        const uint2 e = src.get(i);
+        if (e.x > thr) atomicOr(&cgt[e.y >> 5], 1u << (e.y & 31));
+        else if (e.x == thr) atomicOr(&ceq[e.y >> 5], 1u << (e.y & 31));
+    }
+}
+
+// argTopK on the candidate lists that the selection layer's attention kernel compacted: one CTA per
+// (sequence, head). The list holds every score at or above a provisional threshold chosen by each CTA
+// of that kernel; thr_max is the largest threshold any of them used, so the list is complete for all
+// keys >= thr_max. If the k'-th largest key of the list is at least thr_max it is the k'-th largest of
+// the row and the list decides everything; otherwise (a threshold was too optimistic, or the list
+// outgrew its buffer) the same exact selection runs on the row's scores instead: slower, same result.
+__global__ void __launch_bounds__(TK_THREADS) topk_compact_kernel(const TopkParams p) {
+    extern __shared__ __align__(16) uint8_t tk_smem[];
+    __shared__ __align__(16) unsigned sh_hist[TK_BINS];
+    __shared__ int warp_sums[TK_THREADS / 32];
+    __shared__ unsigned long long warp_sums64[TK_THREADS / 32];
+    __shared__ int bcast[2];
+
+    const int item = blockIdx.x, b = item / p.Hi, tid = threadIdx.x;
+    if (p.pdl) {
+        asm volatile("griddepcontrol.wait;\n" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+    }
+    const int N = max(0, min(p.ctx_lens[b], p.max_ctx));
+    const int kk = min(p.k, N);
+    int* out = p.idx + (long long)item * p.k;
+    if (item % p.Hi == 0 && tid == 0 && p.idx_count) p.idx_count[b] = kk;
+    int* cursor = p.cursor + (size_t)item * p.ctr_stride;
+    unsigned* tmax = p.thr_max + (size_t)item * p.ctr_stride;
+    const int M_raw = __ldcg(cursor);
+    const uint32_t t_max = __ldcg(tmax);
+    __syncthreads();                                   // everybody has read them: they can be cleared for the next call
+    if (tid == 0) { *cursor = 0; *tmax = 0; }
+    if (kk == N) {                                     // everything is kept
+        for (int i = tid; i < N; i += TK_THREADS) out[i] = i;
+        for (int i = N + tid; i < p.k; i += TK_THREADS) out[i] = -1;
+        return;
+    }
+    const int words = (N + 31) >> 5;
+    unsigned* cgt = reinterpret_cast<unsigned*>(tk_smem);
+    unsigned* ceq = cgt + words;
+    uint2* slist = reinterpret_cast<uint2*>(ceq + words);                  // 8 * words bytes in: 8-byte aligned
+    for (int i = tid; i < 2 * words; i += TK_THREADS) cgt[i] = 0;
+
+    const float* srow = p.scores + (long long)item * p.score_stride;
+    const uint2* glist = p.cand + (long long)item * p.cand_stride;
+    bool from_list = M_raw >= kk && M_raw <= p.cand_stride;
+    int need = kk;
+    if (from_list) {
+        // ---- the list: into shared memory if it fits, its smallest and largest key on the way ----------
+        PairSource src{glist, M_raw};
+        const bool in_smem = M_raw <= p.list_smem;
+        uint32_t kmin = 0xffffffffu, kmax = 0u;
+        constexpr int LD = 8;                          // loads in flight per thread
+        for (int i0 = 0; i0 < M_raw; i0 += LD * TK_THREADS) {
+            uint2 r[LD];
+#pragma unroll
+            for (int u = 0; u < LD; ++u) {
+                const int i = i0 + u * TK_THREADS + tid;
+                r[u] = (i < M_raw) ? __ldcg(glist + i) : make_uint2(0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < LD; ++u) {
+                const int i = i0 + u * TK_THREADS + tid;
+                if (i < M_raw) {
+                    if (in_smem) slist[i] = r[u];
+                    kmin = min(kmin, r[u].x);
+                    kmax = max(kmax, r[u].x);
+                }
+            }
+        }
+        if (in_smem) src.c = slist;
+#pragma unroll
+        for (int sh = 16; sh >= 1; sh >>= 1) {
+            kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, sh));
+            kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, sh));
+        }
+        unsigned* red = reinterpret_cast<unsigned*>(warp_sums64);     // [32] words
+        if ((tid & 31) == 0) { red[tid >> 5] = kmin; red[16 + (tid >> 5)] = kmax; }
+        for (int i = tid; i < TK_BINS; i += TK_THREADS) sh_hist[i] = 0;
+        __syncthreads();
+#pragma unroll
+        for (int w = 0; w < TK_THREADS / 32; ++w) { kmin = min(kmin, red[w]); kmax = max(kmax, red[16 + w]); }
+        // ---- one digit of 11 bits over the list's own key range (the candidates of a head share their
+        // top key bits, so the usual most-significant digit would put them all into a few bins) --------
+        const uint32_t range = kmax - kmin;
+        const int dsh = max(0, 21 - __clz(range | 1u));               // (range >> dsh) < 2048
+        for (int i = tid; i < M_raw; i += TK_THREADS) atomicAdd(&sh_hist[(src.get(i).x - kmin) >> dsh], 1u);
+        __syncthreads();
+        const int b1 = pick_digit(sh_hist, TK_BINS, warp_sums, bcast, need);
+        const int in_bin = (int)sh_hist[b1];
+        __syncthreads();                               // sh_hist is recycled below
+        constexpr int FEW = TK_BINS / 2;               // (key, position) pairs that fit the histogram's memory
+        uint32_t thr = 0;
+        if (in_bin <= FEW) {
+            // everything above the threshold bin wins; the bin's own entries are ranked directly
+            uint2* few = reinterpret_cast<uint2*>(sh_hist);
+            if (tid == 0) { bcast[0] = 0; bcast[1] = (int)0xffffffffu; }
+            __syncthreads();
+            for (int i = tid; i < M_raw; i += TK_THREADS) {
+                const uint2 e = src.get(i);
+                const int d = (int)((e.x - kmin) >> dsh);
+                if (d > b1) atomicOr(&cgt[e.y >> 5], 1u << (e.y & 31));
+                else if (d == b1) few[atomicAdd(&bcast[0], 1)] = e;
+            }
+            __syncthreads();
+            const int n = bcast[0];
+            for (int t = tid; t < n; t += TK_THREADS) {
+                const uint2 me = few[t];
+                int beaten_by = 0;
+                for (int j = 0; j < n; ++j) {
+                    const uint2 o = few[j];
+                    beaten_by += (o.x > me.x) || (o.x == me.x && o.y < me.y);
+                }
+                if (beaten_by < need) {
+                    atomicOr(&cgt[me.y >> 5], 1u << (me.y & 31));
+                    atomicMin(reinterpret_cast<unsigned*>(&bcast[1]), me.x);      // the smallest key taken is the k'-th largest
+                }
+            }
+            __syncthreads();
+            thr = (uint32_t)bcast[1];
+            need = 0;                                  // equal keys were resolved by the ranking
+            __syncthreads();
+        } else {
+            // many equal or nearly equal keys: the general digit-by-digit selection
+            need = kk;
+            thr = kth_largest_key(src, p.shift, need, sh_hist, warp_sums, bcast);
+            mark_winners(src, thr, cgt, ceq);
+        }
+        from_list = thr >= t_max;                      // complete down to the k'-th key?
+    }
+    if (!from_list) {
+        ScoreSource src{srow, N};
+        __syncthreads();
+        for (int i = tid; i < 2 * words; i += TK_THREADS) cgt[i] = 0;
+        need = kk;
+        __syncthreads();
+        const uint32_t thr = kth_largest_key(src, p.shift, need, sh_hist, warp_sums, bcast);
+        mark_winners(src, thr, cgt, ceq);
+    }
+    __syncthreads();
+
+    // ordered enumeration: (winner count, equal count) scanned together in one 64-bit value; of the
+    // positions whose key equals the threshold the lowest `need` are taken
+    const int per = (words + TK_THREADS - 1) / TK_THREADS;
+    const int w0 = min(words, tid * per), w1 = min(words, w0 + per);
+    unsigned long long cnt = 0;
+    for (int w = w0; w < w1; ++w)
+        cnt += ((unsigned long long)__popc(cgt[w]) << 32) | (unsigned long long)__popc(ceq[w]);
+    unsigned long long tot;
+    const unsigned long long excl = block_scan_incl<unsigned long long>(cnt, warp_sums64, tot) - cnt;
+    int eq_seen = (int)(excl & 0xffffffffu);
+    int at = (int)(excl >> 32) + min(eq_seen, need);
+    for (int w = w0; w < w1; ++w) {
+        unsigned e = ceq[w];
+        const int ne = __popc(e);
+        const int keep = min(max(need - eq_seen, 0), ne);
+        eq_seen += ne;
+        while (__popc(e) > keep) e &= ~(0x80000000u >> __clz(e));
+        unsigned bits = cgt[w] | e;
+        while (bits) {
+            const int pbit = __ffs(bits) - 1;
+            if (at < p.k) out[at] = (w << 5) + pbit;
+            ++at;
+            bits &= bits - 1;
+        }
+    }
+    // scores that are not numbers rank below everything and may leave the list short: pad, never stale
+    const int taken = (int)(tot >> 32) + min((int)(tot & 0xffffffffu), need);
+    for (int i = min(taken, kk) + tid; i < p.k; i += TK_THREADS) out[i] = -1;
 }
 
 }  // namespace tidal

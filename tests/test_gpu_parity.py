@@ -868,3 +868,81 @@ def test_extreme_ragged_batches_stay_within_the_split_bound(td):
         sp = td.sparse_attn(lay, q, idx, cnt)
         util.check_out(sp.cpu().numpy(), oracle.sparse_attn(okv, qb, idx.cpu().numpy(), cnt.cpu().numpy()), "ragged.sparse")
         assert td.device_status() == binding.OK
+
+
+@pytest.mark.parametrize("N,k,Hq,Hkv", [(8200, 300, 8, 2), (40000, 2000, 4, 4), (131072, 4096, 8, 2)])
+def test_candidate_compaction_is_exact_with_and_without_its_fallback(td, N, k, Hq, Hkv):
+    """The optional compaction of top-k candidates inside the selection kernel: with a generous margin the
+    list decides, with a margin below 1 the provisional thresholds are too high and the kernel must notice
+    and rank all scores instead; either way the sets are the ones the oracle's full sort gives, twice in a
+    row (the lists' cursors and thresholds must be left clean)."""
+    w = wl(1, Hq, Hkv, N, k, planted=16, seed=61)
+    q, lay = build(w, "hnd_interleaved")
+    ref, sc = oracle.full_attn(util.oracle_kv(lay), synth.bits(q), want_scores=True)
+    _, base_idx, _ = td.select_attn(lay, q, k)                 # compaction off
+    try:
+        for margin in (3.0, 1.0, 0.3):
+            td.set_select_margin(margin)
+            for _ in range(2):
+                out, idx, cnt = td.select_attn(lay, q, k)
+                util.check_out(out.cpu().numpy(), ref, f"margin {margin}")
+                assert cnt.item() == k
+                for h in range(Hq):
+                    util.check_idx_row(idx.cpu().numpy()[0, h], sc[0, h], k, N, f"margin {margin} head {h}")
+                assert torch.equal(idx, base_idx)               # the tie rule is the same on every path
+    finally:
+        td.set_select_margin(0.0)
+    assert td.device_status() == binding.OK
+
+
+def test_candidate_compaction_on_scores_that_drift_along_the_context(td):
+    """Provisional thresholds come from the first tiles each CTA sees. Here the keys of the second half
+    of the context are scaled up, so CTAs disagree widely about the threshold: the result must still be
+    exact (through the list where it is complete, through the fallback where it is not), also inside a
+    decode step followed by a sparse layer."""
+    N, k = 65536, 1024
+    w = wl(1, 8, 2, N, k, planted=16, seed=67, layers=2)
+    qs = [synth.make_q(w, i, DEV) for i in range(2)]
+    lays = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(2)]
+    buf = lays[0].keep[0]                                         # [B][Hkv][N][K|V][d]
+    buf[:, :, N // 2:, 0, :] *= 3.0
+    buf[:, :, : N // 8, 0, :] *= 0.25
+    ref, sc = oracle.full_attn(util.oracle_kv(lays[0]), synth.bits(qs[0]), want_scores=True)
+    try:
+        for margin in (3.0, 1.5):
+            td.set_select_margin(margin)
+            outs, idx, cnt = td.decode_step([1, 2], lays, qs, k)
+            util.check_out(outs[0].cpu().numpy(), ref, "drift.select")
+            idx_h = idx.cpu().numpy()
+            for h in range(8):
+                util.check_idx_row(idx_h[0, h], sc[0, h], k, N, f"drift head {h}")
+            util.check_out(outs[1].cpu().numpy(), oracle.sparse_attn(util.oracle_kv(lays[1]), synth.bits(qs[1]), idx_h,
+                                                                     cnt.cpu().numpy()), "drift.sparse")
+    finally:
+        td.set_select_margin(0.0)
+    assert td.device_status() == binding.OK
+
+
+def test_scores_that_are_not_numbers_never_leave_stale_indices(td):
+    """Keys holding NaN (and infinities) make some scores NaN: what is selected among them is unspecified,
+    but every entry of the list must be a valid position or -1, in every top-k path."""
+    N, k = 20000, 1500
+    w = wl(1, 4, 2, N, k, planted=4, seed=71)
+    q, lay = build(w, "hnd_interleaved")
+    buf = lay.keep[0]
+    buf[0, :, 100:19000:7, 0, 5] = float("nan")
+    buf[0, :, 3, 0, 0] = float("inf")
+    idx = torch.full((1, 4, k), 123456789, dtype=torch.int32, device=DEV)
+    try:
+        for margin in (0.0, 3.0, 0.3):
+            td.set_select_margin(margin)
+            idx.fill_(123456789)
+            td.select_attn(lay, q, k, idx=idx)
+            got = idx.cpu().numpy()
+            assert ((got >= -1) & (got < N)).all(), margin
+            for h in range(4):
+                sel = got[0, h][got[0, h] >= 0]
+                assert len(np.unique(sel)) == len(sel) and (np.diff(sel) > 0).all()
+    finally:
+        td.set_select_margin(0.0)
+    td.device_status()
