@@ -31,9 +31,23 @@ from paper_2410_05076_b200 import synth  # noqa: E402
 
 METRIC = "us_per_decode_step_attention_all_layers"
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes (read + write) of one full-attention launch at the cfg3 shape, from the ncu
-# capture summarised in profiles/attn_topk_kernels_cfg3_ncu_full.md (dram__bytes_read.sum + dram__bytes_write.sum).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg3": 536.94e6 + 3.86e6}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_dram_traffic.txt")
+
+
+def ncu_traffic(workload: str) -> dict:
+    """DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of each kernel, as
+    `python -m paper_2410_05076_b200.ncu_summary` extracted them from an ncu capture. Lines read
+    `<workload> <kernel> <bytes>`; a missing file or workload gives an empty dict (traffic: null)."""
+    out = {}
+    try:
+        with open(TRAFFIC_FILE) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) == 3 and parts[0] == workload:
+                    out[parts[1]] = float(parts[2])
+    except OSError:
+        pass
+    return out
 
 
 def describe(w: synth.Workload) -> str:
@@ -133,9 +147,10 @@ def physical_gpu_index(local: int) -> int:
     return local
 
 
-def oracle_sample(w: synth.Workload, qs, layers, host_cache=None, index_heads=None):
-    """Time the CPU oracle, as it stands, on one layer of each type and scale by the layer mix.
-    Only the oracle calls are timed; the host copies of the sampled layers may be cached by the caller."""
+def oracle_sample(w: synth.Workload, qs, layers, host_cache=None, index_heads=None, repeats: int = 3):
+    """Time the CPU oracle, as it stands, on one layer of each type (median of `repeats` runs each)
+    and scale by the layer mix. Only the oracle calls are timed; the host copies of the sampled layers
+    may be cached by the caller."""
     import oracle
     from oracle import adapter
 
@@ -149,23 +164,25 @@ def oracle_sample(w: synth.Workload, qs, layers, host_cache=None, index_heads=No
             okv, qb = adapter.kv_from_layer(layers[i]), adapter.bits(qs[i])
             if host_cache is not None:
                 host_cache[i] = (okv, qb)
-        t0 = time.perf_counter()
-        if t == 0:
-            oracle.full_attn(okv, qb)
-        elif t == 1:
+        if t == 2 and rho is None:
             _, idx, cnt = oracle.select_attn(okv, qb, w.k, index_heads)
             rho = (idx, cnt)
-        else:
-            if rho is None:
+        samples = []
+        for _ in range(repeats):
+            t0 = time.perf_counter()
+            if t == 0:
+                oracle.full_attn(okv, qb)
+            elif t == 1:
                 _, idx, cnt = oracle.select_attn(okv, qb, w.k, index_heads)
                 rho = (idx, cnt)
-                t0 = time.perf_counter()
-            oracle.sparse_attn(okv, qb, rho[0], rho[1])
-        times[t] = time.perf_counter() - t0
+            else:
+                oracle.sparse_attn(okv, qb, rho[0], rho[1])
+            samples.append(time.perf_counter() - t0)
+        times[t] = statistics.median(samples)
         del okv
     total = sum(times[t] * w.sched.count(t) for t in times)
-    sample = ("one layer of each type timed once (layers " + ",".join(str(first[t]) for t in sorted(first)) +
-              f"), scaled by the {w.sched.count(0)}+{w.sched.count(1)}+{w.sched.count(2)} layer mix")
+    sample = (f"one layer of each type (layers " + ",".join(str(first[t]) for t in sorted(first)) +
+              f"), median of {repeats} runs each, scaled by the {w.sched.count(0)}+{w.sched.count(1)}+{w.sched.count(2)} layer mix")
     return total * 1e6, oracle.num_threads(), sample, {int(t): times[t] * 1e6 for t in times}
 
 
@@ -266,10 +283,84 @@ def sweep(td, dev, reps):
         del sel_layers, sp_layers
         torch.cuda.empty_cache()
     assert td.device_status() == 0
-    print(json.dumps({"sweep": "cfg5: B1 32q/8kv d128; per-layer cost of a selection layer (attention + top-k) and "
-                      "of a sparse layer, from chains of layers run through tidal_decode_step over distinct "
-                      "KV copies (cold in L2), CUDA events", "reps": reps, "points": points}),
-          flush=True)
+    return {"sweep": "cfg5: B1 32q/8kv d128; per-layer cost of a selection layer (attention + top-k) and "
+                     "of a sparse layer, from chains of layers run through tidal_decode_step over distinct "
+                     "KV copies (cold in L2), CUDA events", "reps": reps, "points": points}
+
+
+def time_schedule(td, kinds, layers, qs, outs, k, gran, nrep):
+    """One sub-schedule run through tidal_decode_step nrep times (no host gaps between its launches, the
+    library's step graph and the overlap between layers active): CUDA events, microseconds per run."""
+    st = td.make_step(list(kinds), list(layers), list(qs), list(outs), k, gran)
+    for _ in range(3):
+        st()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(nrep):
+        st()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) * 1e3 / nrep
+
+
+def layers_in_step(td, w, layers, qs, outs, gran, nrep):
+    """Per-layer-type cost inside a step, from differences of sub-schedule times over the workload's own
+    layer caches (every launch finds its cache cold in L2):
+      full    a chain of full-attention layers over distinct caches, per layer;
+      sparse  (selection layer + all sparse layers) minus (that selection layer alone), per sparse layer;
+      select  the workload's schedule from its first selection layer on, minus the same schedule with the
+              second selection layer run as a sparse layer, plus one sparse layer: a selection layer
+              (attention + top-k) in its real surroundings, including what it costs the sparse layer after
+              it, which must wait for the new index list."""
+    ts = lambda ids, kinds: time_schedule(td, kinds, [layers[i] for i in ids], [qs[i] for i in ids],
+                                          [outs[i] for i in ids], w.k, gran, nrep)
+    F, S, P = synth.LAYER_FULL, synth.LAYER_SELECT, synth.LAYER_SPARSE
+    out = {}
+    nchain = min(8, w.num_layers)
+    if nchain >= 2:
+        out["full_us"] = ts(range(nchain), [F] * nchain) / nchain
+        out["full_bytes"] = sum(layers[i].kv_bytes() for i in range(nchain)) / nchain
+    sel_ids = [i for i, tk in enumerate(w.sched) if tk == S]
+    sp_ids = [i for i, tk in enumerate(w.sched) if tk == P]
+    if sel_ids and len(sp_ids) >= 2:
+        t_sel = ts(sel_ids[:1], [S])
+        t_chain = ts(sel_ids[:1] + sp_ids, [S] + [P] * len(sp_ids))
+        out["sparse_us"] = (t_chain - t_sel) / len(sp_ids)
+        out["select_alone_us"] = t_sel
+        if len(sel_ids) >= 2:
+            tail = list(range(sel_ids[0], w.num_layers))
+            kinds = [w.sched[i] for i in tail]
+            kinds_one = [P if (i == sel_ids[1]) else w.sched[i] for i in tail]
+            out["select_us"] = ts(tail, kinds) - ts(tail, kinds_one) + out["sparse_us"]
+            out["select_bytes"] = layers[sel_ids[1]].kv_bytes()
+        else:
+            out["select_us"] = t_sel
+            out["select_bytes"] = layers[sel_ids[0]].kv_bytes()
+    return out
+
+
+def quick_workload(td, name, dev, gran, nrep):
+    """Step time and per-layer-type times of another configuration (compact: for the line's other_workloads)."""
+    w = synth.workload(name)
+    qs, layers = build_workload(w, dev)
+    outs = [torch.empty(w.batch, w.num_q_heads, w.head_dim, dtype=torch.float32, device=dev) for _ in layers]
+    step_us = time_schedule(td, w.sched, layers, qs, outs, w.k, gran, nrep)
+    lt = layers_in_step(td, w, layers, qs, outs, gran, max(3, nrep // 2))
+    sparse_bytes = sum(min(w.k, n) for n in w.ctx_lens()) * w.num_q_heads * 516
+    res = {"workload": describe(w), "step_us": round(step_us, 2)}
+    if "full_us" in lt:
+        res["full_us"] = round(lt["full_us"], 2)
+        res["full_frac_of_8TBs"] = round(lt["full_bytes"] / lt["full_us"] / 1e3 / NOMINAL_HBM_GBS, 3)
+    if "select_us" in lt:
+        res["select_us_incl_topk"] = round(lt["select_us"], 2)
+        res["select_frac_of_8TBs"] = round(lt["select_bytes"] / lt["select_us"] / 1e3 / NOMINAL_HBM_GBS, 3)
+    if "sparse_us" in lt:
+        res["sparse_us"] = round(lt["sparse_us"], 2)
+        res["sparse_frac_of_8TBs"] = round(sparse_bytes / lt["sparse_us"] / 1e3 / NOMINAL_HBM_GBS, 3)
+    assert td.device_status() == 0
+    del qs, layers, outs
+    torch.cuda.empty_cache()
+    return res
 
 
 def main():
@@ -280,6 +371,8 @@ def main():
     ap.add_argument("--impl", default="tidal", choices=["tidal", "reference"])
     ap.add_argument("--workload", default="cfg3")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="skip the compact figures for cfg1, cfg2, cfg64, cfg4 and the cfg5 sweep")
     ap.add_argument("--granularity", default="qhead", choices=["qhead", "kvhead", "shared"],
                     help="one token set per query head (default), per KV head, or shared by all heads "
                          "(the latter two rank by the sum of the member heads' scaled logits)")
@@ -326,7 +419,7 @@ def main():
         profile_case(td, w, dev, args.steps)
         return
     if args.sweep:
-        sweep(td, dev, max(3, min(args.steps, 30)))
+        print(json.dumps(sweep(td, dev, max(3, min(args.steps, 30)))), flush=True)
         return
     qs, layers = build_workload(w, dev)
     outs = [torch.empty(w.batch, w.num_q_heads, w.head_dim, dtype=torch.float32, device=dev) for _ in layers]
@@ -358,91 +451,62 @@ def main():
     if status != binding.OK:
         raise SystemExit(f"device status {status} after the timed region")
 
-    # ---- per-layer events: the dominant kernel's own duration, live ------------------------------
-    # The same launches as a step, issued layer by layer through the C-ABI with an event between
-    # layers. Layers of type FULL are exactly one launch of the streaming attention kernel.
+    # ---- the layers in situ: the dominant kernel's own duration, live -------------------------------
     nrep = max(3, min(args.steps, 20))
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(w.num_layers + 1)] for _ in range(nrep)]
-    idx, cnt = step.idx, step.idx_count
-    for r in range(nrep):
-        evs[r][0].record()
-        for i, tkind in enumerate(w.sched):
-            if tkind == synth.LAYER_FULL:
-                td.full_attn(layers[i], qs[i], out=outs[i])
-            elif tkind == synth.LAYER_SELECT:
-                td.select_attn(layers[i], qs[i], w.k, gran, out=outs[i], idx=idx, idx_count=cnt)
-            else:
-                td.sparse_attn(layers[i], qs[i], idx, cnt, out=outs[i])
-            evs[r][i + 1].record()
-    torch.cuda.synchronize()
-    per_type = {0: [], 1: [], 2: []}
-    for r in range(nrep):
-        for i, tkind in enumerate(w.sched):
-            per_type[tkind].append(evs[r][i].elapsed_time(evs[r][i + 1]) * 1e3)
-    layer_us = {k: (sum(v) / len(v) if v else None) for k, v in per_type.items()}
-    full_layers = [i for i, tk in enumerate(w.sched) if tk == synth.LAYER_FULL]
-    dense_bytes = sum(kv_bytes[i] for i in full_layers) / max(1, len(full_layers)) if full_layers else kv_bytes[0]
-    dense_us = layer_us[0] if layer_us[0] else layer_us[1]
     peak, peak_kind = measured_peak_gbs()
-    achieved = dense_bytes / (dense_us * 1e-6) / 1e9
-    sparse_bytes = w.batch * gather_lists * min(w.k, w.ctx) * 512 + w.batch * index_heads * min(w.k, w.ctx) * 4
-    roofline = {"bound": "hbm", "kernel": "attn_kernel<FULL> (full-attention layers; the selection layers run the same loop)",
-                "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(w.name), "bytes_per_launch": dense_bytes,
-                "us_per_launch": dense_us}
-    layers_report = {
-        "note": "full_us / select_us_incl_topk / sparse_us: one C-ABI call per layer from Python with an event "
-                "between calls (includes host gaps); *_in_step: the same kernels back to back inside tidal_decode_step",
-        "full_us": layer_us[0], "select_us_incl_topk": layer_us[1], "sparse_us": layer_us[2],
-        "select_frac_of_8TBs": (dense_bytes / (layer_us[1] * 1e-6) / 1e9 / NOMINAL_HBM_GBS) if layer_us[1] else None,
-        "sparse_GBs": (sparse_bytes / (layer_us[2] * 1e-6) / 1e9) if layer_us[2] else None,
-        "sparse_frac_of_8TBs": (sparse_bytes / (layer_us[2] * 1e-6) / 1e9 / NOMINAL_HBM_GBS) if layer_us[2] else None,
-    }
+    lt = layers_in_step(td, w, layers, qs, outs, gran, nrep)
+    k_eff = [min(w.k, n) for n in w.ctx_lens()]
+    sparse_bytes = sum(k_eff) * (gather_lists * 512 + index_heads * 4)
+    traffic = ncu_traffic(w.name)
+
+    def kernel_entry(kernel, bytes_per_launch, us, traffic_key, launches_per_step, note=None):
+        if not us:
+            return None
+        ach = bytes_per_launch / us / 1e3
+        e = {"kernel": kernel, "achieved": ach, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+             "frac": ach / peak, "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
+             "traffic": traffic.get(traffic_key), "bytes_per_launch": bytes_per_launch, "us_per_launch": us,
+             "launches_per_step": launches_per_step, "share_of_step": launches_per_step * us / (ms_step * 1e3)}
+        if note:
+            e["note"] = note
+        return e
+
+    n_full, n_sel, n_sp = w.sched.count(0), w.sched.count(1), w.sched.count(2)
+    sparse_entry = kernel_entry("attn_kernel<SPARSE> (sparse layers: gather of the selected K/V rows)", sparse_bytes,
+                                lt.get("sparse_us"), "sparse", n_sp)
+    full_entry = kernel_entry("attn_kernel<FULL> (full-attention layers)", lt.get("full_bytes", 0), lt.get("full_us"),
+                              "full", n_full)
+    select_entry = kernel_entry("attn_kernel<SELECT> + top-k (selection layers)", lt.get("select_bytes", 0),
+                                lt.get("select_us"), "select", n_sel,
+                                "bytes_per_launch counts the KV cache only; the scores (4 B per position and query "
+                                "head, written once and read back from L2) are not in the denominator")
+    if select_entry and traffic.get("topk") is not None and select_entry["traffic"] is not None:
+        select_entry["traffic"] += traffic["topk"]
+    # the kernel with the largest share of the step leads; the others follow as siblings
+    entries = [e for e in (sparse_entry, full_entry, select_entry) if e]
+    entries.sort(key=lambda e: -e["share_of_step"])
+    roofline = {"bound": "hbm"}
+    roofline.update(entries[0])
+    roofline["measured"] = ("per-launch time = difference of sub-schedule times run through tidal_decode_step over the "
+                            "workload's own layer caches (cold in L2), CUDA events on the launching stream; traffic = "
+                            "dram__bytes_read.sum + dram__bytes_write.sum of one launch from the ncu capture summarised "
+                            "under profiles/ (null if not captured for this workload)")
+    roofline["target"] = "north star: selection and sparse layers at >= 0.70 of 8 TB/s (frac_of_nominal_8TBs)"
+    roofline["siblings"] = entries[1:]
     step_bytes = sum(kv_bytes[i] if tk != synth.LAYER_SPARSE else sparse_bytes for i, tk in enumerate(w.sched))
-
-    # ---- the same layers in situ: sub-schedules run through tidal_decode_step (no host gaps between
-    # launches, programmatic dependent launch active), differences of CUDA-event times ------------------
-    def time_schedule(ids, kinds):
-        st = td.make_step(kinds, [layers[i] for i in ids], [qs[i] for i in ids], [outs[i] for i in ids], w.k, gran)
-        for _ in range(3):
-            st()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for _ in range(nrep):
-            st()
-        b.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) * 1e3 / nrep
-
-    # The streaming kernel back to back over distinct layer caches (any layer's cache can be run as a
-    # full or as a selection layer): the dominant kernel's own duration without host gaps.
-    nchain = min(8, w.num_layers)
-    if nchain >= 2:
-        chain_ids = list(range(nchain))
-        full_chain_us = time_schedule(chain_ids, [synth.LAYER_FULL] * nchain) / nchain
-        sel_chain_us = time_schedule(chain_ids, [synth.LAYER_SELECT] * nchain) / nchain
-        chain_bytes = sum(kv_bytes[i] for i in chain_ids) / nchain
-        achieved = chain_bytes / (full_chain_us * 1e-6) / 1e9
-        roofline.update({"achieved": achieved, "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                         "bytes_per_launch": chain_bytes, "us_per_launch": full_chain_us,
-                         "measured": f"{nchain} launches of the full-attention kernel over {nchain} distinct layer caches "
-                                     "through tidal_decode_step, CUDA events on the launching stream, average per launch"})
-        layers_report.update({"full_us_in_step": full_chain_us, "select_us_incl_topk_in_step": sel_chain_us,
-                              "select_in_step_frac_of_8TBs": chain_bytes / sel_chain_us / 1e3 / NOMINAL_HBM_GBS})
-
-    sel_ids = [i for i, tk in enumerate(w.sched) if tk == synth.LAYER_SELECT]
-    sp_ids = [i for i, tk in enumerate(w.sched) if tk == synth.LAYER_SPARSE]
-    if sel_ids and len(sp_ids) >= 2:
-        t_sel = time_schedule(sel_ids[:1], [synth.LAYER_SELECT])
-        t_chain = time_schedule(sel_ids[:1] + sp_ids, [synth.LAYER_SELECT] + [synth.LAYER_SPARSE] * len(sp_ids))
-        sp_in = (t_chain - t_sel) / len(sp_ids)
-        layers_report.update({
-            "select_us_alone_in_decode_step_call": t_sel,
-            "sparse_us_in_step": sp_in,
-            "sparse_in_step_GBs": sparse_bytes / sp_in / 1e3,
-            "sparse_in_step_frac_of_8TBs": sparse_bytes / sp_in / 1e3 / NOMINAL_HBM_GBS,
-        })
+    layers_report = {
+        "note": "microseconds per layer inside tidal_decode_step (see roofline.measured); sum_check = "
+                "full*n_full + select*n_select + sparse*n_sparse, to be compared with value",
+        "full_us_in_step": lt.get("full_us"), "select_us_incl_topk_in_step": lt.get("select_us"),
+        "sparse_us_in_step": lt.get("sparse_us"), "select_us_alone_in_decode_step_call": lt.get("select_alone_us"),
+        "sum_check_us": sum((lt.get(kx) or 0) * n for kx, n in (("full_us", n_full), ("select_us", n_sel), ("sparse_us", n_sp))),
+    }
+    # the same step with the overlap between layers switched off: every layer reads its query only after
+    # the layer before it has finished, as a model with projections between the layers would need it
+    td.set_layer_overlap(False)
+    no_overlap_us = time_schedule(td, w.sched, layers, qs, outs, w.k, gran, nrep)
+    td.set_layer_overlap(True)
+    layers_report["step_us_without_layer_overlap"] = no_overlap_us
 
     # ---- end to end through the host-buffer entry point ----------------------------------------------
     q_host = torch.stack([q.cpu() for q in qs]).contiguous().pin_memory()
@@ -459,11 +523,26 @@ def main():
     e2e_us = max_over_ranks(e2e_s, dist, dev) / args.steps * 1e6
     if not torch.allclose(out_host[0].to(dev), outs[0], rtol=0, atol=1e-3):
         raise SystemExit("host-buffer step and device step disagree")
+    h2d_bytes, d2h_bytes = q_host.numel() * 2, out_host.numel() * 4
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         us, cores, sample, _ = oracle_sample(w, qs, layers, index_heads=index_heads)
         cpu = {"value": us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample}
+
+    # ---- the other configurations, compactly (one GPU, default run only) ------------------------------
+    other = None
+    if rank == 0 and world == 1 and not args.no_other_workloads and args.workload == "cfg3":
+        del step, step_host, qs, layers, outs
+        torch.cuda.empty_cache()
+        other = {"note": "step_us: the whole schedule through tidal_decode_step, CUDA events; per-layer figures as "
+                         "in `layers`; fractions are algorithmic bytes / time / 8 TB/s (cfg1 is latency-bound: 5 MB per step)"}
+        for name in ("cfg1", "cfg2", "cfg64", "cfg4"):
+            other[name] = quick_workload(td, name, dev, gran, max(3, min(args.steps, 10)))
+        sw = sweep(td, dev, 3)
+        other["cfg5_sweep"] = {"what": sw["sweep"], "columns": ["ctx", "k", "select_us_incl_topk", "sparse_us"],
+                               "points": [[p["ctx"], p["k"], round(p["select_us_incl_topk"], 1), round(p["sparse_us"], 2)]
+                                          for p in sw["points"]]}
 
     if rank == 0:
         line = {
@@ -480,9 +559,9 @@ def main():
                        "step_bytes": step_bytes,
                        "step_frac_of_8TBs": step_bytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
             "clocks": clocks, "gpu_launches": launches,
-            "e2e": {"value": e2e_us / world, "unit": "us", "h2d_bytes_per_step": q_host.numel() * 2,
-                    "d2h_bytes_per_step": out_host.numel() * 4},
-            "roofline": roofline, "layers": layers_report, "cpu_baseline": cpu,
+            "e2e": {"value": e2e_us / world, "unit": "us", "h2d_bytes_per_step": h2d_bytes,
+                    "d2h_bytes_per_step": d2h_bytes},
+            "roofline": roofline, "layers": layers_report, "cpu_baseline": cpu, "other_workloads": other,
         }
         print(json.dumps(line), flush=True)
     if dist is not None:

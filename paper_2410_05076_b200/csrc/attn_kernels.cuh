@@ -384,7 +384,9 @@ __device__ __forceinline__ void consume_tile(const AttnParams& p, uint32_t ks, u
 __device__ __forceinline__ int item_tiles(int total) { return max(1, (total + TILE - 1) / TILE); }
 
 // NEWEST (gather kernel only): every list has one more slot that stands for the newest token.
-template <int MODE, int NW, int STAGES, bool NEWEST = false>
+// COMPACT (selection kernel only): the instantiation that compacts top-k candidates; the default
+// selection kernel carries none of that code.
+template <int MODE, int NW, int STAGES, bool NEWEST = false, bool COMPACT = false>
 __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     // Ring slots must be 256-byte aligned (the V fragment addressing XORs bits 5-7).
@@ -456,7 +458,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
     //   st_pos   [NW][CAL_TILES] first position of each staged tile (-1: none), st_vm: its valid rows
     //   thr_key  [CAND_COLS] the thresholds as keys, thr_val as values
     //   cbuf     [NW][CAND_COLS][CAND_BUF] candidates waiting to be written out, ccnt [NW][CAND_COLS] fill counts
-    const bool compact = (MODE == MODE_SELECT) && p.compact && p.splits_per_item > 0;
+    constexpr bool compact = (MODE == MODE_SELECT) && COMPACT;      // the host launches it for pooled grids only
     uint32_t* stage_all = hist;
     int* st_pos = reinterpret_cast<int*>(stage_all + NW * CAL_TILES * 16 * CAND_COLS);
     uint32_t* st_vm = reinterpret_cast<uint32_t*>(st_pos + NW * CAL_TILES);
@@ -821,7 +823,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             }
             const int stage = it % STAGES;
             const uint32_t ks = wbase_u32 + stage * STAGE_BYTES;
-            if (MODE == MODE_SELECT && compact) {
+            if constexpr (compact) {
                 if (!calibrated && it == CAL_TILES) calibrate();
                 cw.stage = nullptr;
                 if (!calibrated) {
@@ -867,7 +869,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         }
         cp_async_wait<0>();
         __syncwarp();
-        if (MODE == MODE_SELECT && compact) {
+        if constexpr (compact) {
             if (!calibrated) calibrate();         // fewer tiles than the calibration takes: every warp still meets here
             cand_flush(1);
         }
@@ -981,6 +983,12 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                 float v0[CB];
 #pragma unroll
                 for (int u = 0; u < CB; ++u) v0[u] = (has0 && u < ns) ? __ldcg(po0 + (long long)u * HEAD_DIM) : 0.f;
+                // The item's pool cursor is cleared for a later launch now, behind this thread's loads (the
+                // fence then costs nothing extra: it returns when they do). The fence makes the cleared
+                // cursor visible device-wide before this CTA can retire: a later launch may request tiles
+                // from it without waiting for this grid (see the host's rule for early triggers), and cannot
+                // start before this CTA is gone.
+                if (pooled && threadIdx.x == NW * 32 - 1) { *pool = 0; __threadfence(); }
                 for (int col = warp; col < ncols; col += NW) {
                     const long long pr = (row0 + col) * p.max_splits;
                     float M = -INFINITY;
@@ -1020,10 +1028,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                     for (; s < ns; ++s) O += __ldcg(po + (long long)s * HEAD_DIM) * fs[s];
                     store_out(p, (row0 + col) * HEAD_DIM + c, O * linv[col]);
                 }
-                // Ready for the next launch. The fence makes the cleared cursor visible device-wide before
-                // this CTA retires: a later launch may request tiles from it without waiting for this grid
-                // (see the host's rule for early triggers), and cannot start before this CTA is gone.
-                if (threadIdx.x == 0) { *ctr = 0; if (pooled) { *pool = 0; __threadfence(); } }
+                if (threadIdx.x == 0) *ctr = 0;       // ready for the next launch
             }
         }
         __syncthreads();                          // shared memory is reused by the next segment

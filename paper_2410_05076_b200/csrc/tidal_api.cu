@@ -260,7 +260,7 @@ constexpr size_t attn_smem() {
            (MODE == MODE_SELECT ? HIST_SMEM : 0) + 1024;   // + alignment slack
 }
 
-template <int MODE, int NW, int STAGES, bool NEWEST = false>
+template <int MODE, int NW, int STAGES, bool NEWEST = false, bool COMPACT = false>
 tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, int full_grid, cudaStream_t st) {
     // Programmatic dependent launch: the kernel may begin while its predecessor in the stream
     // drains; it waits (griddepcontrol.wait) before touching anything that predecessor wrote.
@@ -290,7 +290,7 @@ tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, int full_gri
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     ctx->launches++;
-    return cudaLaunchKernelEx(&cfg, attn_kernel<MODE, NW, STAGES, NEWEST>, a) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, attn_kernel<MODE, NW, STAGES, NEWEST, COMPACT>, a) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }
 
 // How a selection layer produces its ranking scores. Per query head: one row per head, histogram
@@ -325,11 +325,13 @@ enum Dep { DEP_FIRST, DEP_PREFETCH, DEP_LATE };
 
 tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, float* out, float* scores,
                          long long score_stride, bool fuse_hist, Dep dep, const WsLayout& w, cudaStream_t st,
-                         bool agg = false, int compact_k = 0) {
+                         bool agg = false, int compact_k = 0, bool private_scores = false) {
     AttnParams a;
     fill_common(a, ctx, kv, q, out, w);
     a.wait_first = dep == DEP_FIRST;
-    a.wait_late = dep == DEP_LATE && scores == nullptr;   // a selection layer writes scores while it streams
+    // A selection layer writes scores while it streams: it may do so ahead of its wait only when no earlier
+    // kernel can still be reading the score buffer (the step driver knows), and not with candidate lists.
+    a.wait_late = dep == DEP_LATE && (scores == nullptr || (private_scores && compact_k == 0));
     int grid = dense_grid(ctx, kv);
     if (compact_k > 0) {
         a.compact = 1;
@@ -347,6 +349,10 @@ tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, fl
     a.score_stride = score_stride;
     a.agg = agg ? 1 : 0;
     a.hist = fuse_hist ? state_hist(ctx) : nullptr;
+    if (scores && a.compact) {
+        if (a.splits_per_item <= 0) return TIDAL_ERR_INTERNAL;      // select_plan admits pooled grids only
+        return launch_attn<MODE_SELECT, DENSE_NW, DENSE_STAGES, false, true>(ctx, a, grid, std::min(ctx->dense_slots, GRID_MAX), st);
+    }
     if (scores) return launch_attn<MODE_SELECT, DENSE_NW, DENSE_STAGES>(ctx, a, grid, std::min(ctx->dense_slots, GRID_MAX), st);
     return launch_attn<MODE_FULL, DENSE_NW, DENSE_STAGES>(ctx, a, grid, std::min(ctx->dense_slots, GRID_MAX), st);
 }
@@ -561,13 +567,14 @@ tidal_status_t tidal_create(tidal_ctx_t** out, int device, size_t workspace_byte
     ctx->sm_count = prop.multiProcessorCount;
     const int d0 = resident_ctas(attn_kernel<MODE_FULL, DENSE_NW, DENSE_STAGES>, DENSE_NW * 32, attn_smem<MODE_FULL, DENSE_NW, DENSE_STAGES>(), ctx->sm_count);
     const int d1 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW, DENSE_STAGES>, DENSE_NW * 32, attn_smem<MODE_SELECT, DENSE_NW, DENSE_STAGES>(), ctx->sm_count);
+    const int d2 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW, DENSE_STAGES, false, true>, DENSE_NW * 32, attn_smem<MODE_SELECT, DENSE_NW, DENSE_STAGES>(), ctx->sm_count);
     const int s0 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>, SPARSE_NW * 32, attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(), ctx->sm_count);
     const int s1 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES, true>, SPARSE_NW * 32, attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(), ctx->sm_count);
     const size_t topk_smem = 2 * (size_t)(MAX_CTX / 32) * sizeof(unsigned) + 8192 * sizeof(uint2);
     const bool topk_ok = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topk_smem) == cudaSuccess;
     const size_t compact_smem = 2 * ((size_t)(MAX_CTX / 32) + 1) * sizeof(unsigned) + (size_t)COMPACT_LIST_SMEM * sizeof(uint2);
     const bool compact_ok = cudaFuncSetAttribute(topk_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)compact_smem) == cudaSuccess;
-    if (d0 <= 0 || d1 <= 0 || s0 <= 0 || s1 < s0 || !topk_ok || !compact_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
+    if (d0 <= 0 || d1 <= 0 || d2 < d1 || s0 <= 0 || s1 < s0 || !topk_ok || !compact_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
     ctx->dense_slots = std::min(d0, d1);
     ctx->sparse_slots = s0;
     if (cudaMalloc((void**)&ctx->status, 256) != cudaSuccess || cudaMemset(ctx->status, 0, 256) != cudaSuccess) {
@@ -733,7 +740,11 @@ static tidal_status_t decode_step_enqueue(tidal_ctx_t* ctx, int32_t num_layers, 
         } else if (schedule[i] == TIDAL_LAYER_SELECT) {
             float* scores = (float*)((char*)ctx->ws + w.scores);
             const SelectPlan sp = select_plan(ctx, kv, Hi, k, false);
-            rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, sp.fuse, dep, w, st, sp.agg, sp.compact ? k : 0);
+            // The score buffer's last reader is the top-k of the selection layer before this one. If a
+            // sparse layer ran in between, its first kernel waited for that top-k before it let anything
+            // else start, so nobody reads the buffer any more; right after another selection layer, wait.
+            const bool scores_free = i > 0 && schedule[i - 1] != TIDAL_LAYER_SELECT;
+            rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, sp.fuse, dep, w, st, sp.agg, sp.compact ? k : 0, scores_free);
             if (rc == TIDAL_OK) rc = run_topk(ctx, kv, scores, w.score_stride, k, sp.rows, Hi, sp.fuse, idx, idx_count, w, st, sp.compact);
         } else {
             const bool fresh_idx = i == 0 || schedule[i - 1] == TIDAL_LAYER_SELECT;

@@ -261,14 +261,19 @@ __global__ void __launch_bounds__(TK_THREADS) topk_select_kernel(const TopkParam
     const float* srow = p.scores + ((long long)b * p.Hq + (long long)hi * members) * p.score_stride;
     float* raw = reinterpret_cast<float*>(tk_smem);                // [TK_SPAN]
     if (p.vec_ok && members == 1) {
+        // The attention kernel asked L2 to keep the scores (evict-last) until they were read back: this is
+        // that read, and it hands the lines back (evict-first), so that they do not crowd the caller's
+        // next kernels out of the cache.
+        uint64_t done_with;
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(done_with));
 #pragma unroll
         for (int j = 0; j < TK_BATCHES * TK_VEC; ++j) {
             const int off = 4 * (j * TK_THREADS + tid);
             const int pos = s0 + off;
             const int nbytes = max(0, min(4, N - pos)) * 4;        // zero-fill past the end of the cache
             const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(raw + off));
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n"
-                         ::"r"(dst), "l"(nbytes ? srow + pos : srow), "r"(nbytes) : "memory");
+            asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;\n"
+                         ::"r"(dst), "l"(nbytes ? srow + pos : srow), "r"(nbytes), "l"(done_with) : "memory");
         }
         asm volatile("cp.async.commit_group;\n" ::: "memory");
     } else if (p.vec_ok) {
