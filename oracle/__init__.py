@@ -24,6 +24,7 @@ _HDR = os.path.join(_HERE, "tidal_oracle.h")
 _LIB = os.path.join(_HERE, "libtidal_oracle.so")
 
 LAYER_FULL, LAYER_SELECT, LAYER_SPARSE = 0, 1, 2
+KV_BF16, KV_FP8_E4M3 = 0, 1
 
 
 def build(force: bool = False) -> str:
@@ -47,6 +48,7 @@ class _KV(C.Structure):
         ("stride_page", C.c_int64),
         ("page_table", C.c_void_p), ("page_size", C.c_int32), ("max_pages_per_seq", C.c_int32),
         ("ctx_lens", C.c_void_p), ("sm_scale", C.c_float),
+        ("kv_dtype", C.c_int32), ("k_scale", C.c_void_p), ("v_scale", C.c_void_p),
     ]
 
 
@@ -77,6 +79,8 @@ def lib():
         L.oracle_schedule.argtypes = [I, I, P]
         L.oracle_schedule.restype = None
         L.oracle_num_threads.restype = I
+        L.oracle_e4m3_decode.argtypes = [C.c_uint8]
+        L.oracle_e4m3_decode.restype = C.c_float
         _lib = L
     return _lib
 
@@ -102,16 +106,28 @@ class KV:
     sm_scale: float = 0.0
     k_offset: int = 0   # element offsets of K and V inside their arrays
     v_offset: int = 0
+    kv_dtype: int = 0   # 0: bf16 bits in uint16 arrays; 1: OCP FP8 E4M3 codes in uint8 arrays
+    k_scale: Optional[np.ndarray] = None   # fp8: float32 [num_kv_heads], None = 1
+    v_scale: Optional[np.ndarray] = None
 
     def c_struct(self) -> _KV:
-        assert self.k.dtype == np.uint16 and self.v.dtype == np.uint16
+        want = np.uint8 if self.kv_dtype == KV_FP8_E4M3 else np.uint16
+        assert self.k.dtype == want and self.v.dtype == want
+        esz = 1 if self.kv_dtype == KV_FP8_E4M3 else 2
         self.ctx_lens = np.ascontiguousarray(self.ctx_lens, dtype=np.int32)
         s = _KV()
         s.batch, s.num_q_heads, s.num_kv_heads, s.head_dim = (
             self.batch, self.num_q_heads, self.num_kv_heads, self.head_dim)
         s.paged = 1 if self.page_table is not None else 0
-        s.k = self.k.ctypes.data + 2 * self.k_offset
-        s.v = self.v.ctypes.data + 2 * self.v_offset
+        s.k = self.k.ctypes.data + esz * self.k_offset
+        s.v = self.v.ctypes.data + esz * self.v_offset
+        s.kv_dtype = self.kv_dtype
+        if self.k_scale is not None:
+            self.k_scale = np.ascontiguousarray(self.k_scale, dtype=np.float32)
+            s.k_scale = self.k_scale.ctypes.data
+        if self.v_scale is not None:
+            self.v_scale = np.ascontiguousarray(self.v_scale, dtype=np.float32)
+            s.v_scale = self.v_scale.ctypes.data
         s.stride_b, s.stride_pos, s.stride_head, s.stride_page = (
             self.stride_b, self.stride_pos, self.stride_head, self.stride_page)
         if self.page_table is not None:
@@ -220,9 +236,18 @@ def with_newest(kv: KV, idx: np.ndarray, idx_count: np.ndarray):
 
 def kv_append(kv: KV, k_new: np.ndarray, v_new: np.ndarray) -> None:
     """C.append(k, v): writes the rows [B, Hkv, d] at position ctx_lens[b] - 1 of kv's arrays, in place."""
-    k_new, v_new = _q(k_new), _q(v_new)
+    want = np.uint8 if kv.kv_dtype == KV_FP8_E4M3 else np.uint16
+    assert k_new.dtype == want and v_new.dtype == want
+    k_new, v_new = np.ascontiguousarray(k_new), np.ascontiguousarray(v_new)
     st = kv.c_struct()
     lib().oracle_kv_append(C.byref(st), k_new.ctypes.data, v_new.ctypes.data)
+
+
+def e4m3_decode(codes) -> np.ndarray:
+    """Values of OCP FP8 E4M3 codes (any array of uint8), one call of the C decoder per element."""
+    codes = np.asarray(codes, dtype=np.uint8)
+    f = lib().oracle_e4m3_decode
+    return np.array([f(int(c)) for c in codes.reshape(-1)], dtype=np.float32).reshape(codes.shape)
 
 
 def schedule(num_layers: int, reselect_layer: int) -> np.ndarray:

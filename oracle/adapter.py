@@ -12,7 +12,9 @@ from . import KV
 
 
 def bits(t: torch.Tensor) -> np.ndarray:
-    """bf16 tensor -> numpy uint16 array with the same bits (host copy)."""
+    """bf16 tensor -> numpy uint16 array with the same bits; 8-bit tensors (fp8 codes) -> uint8 (host copy)."""
+    if t.element_size() == 1:
+        return t.detach().contiguous().view(torch.uint8).cpu().numpy()
     return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
@@ -37,4 +39,6 @@ def kv_from_layer(layer) -> KV:
         stride_page=layer.stride_page,
         page_table=None if layer.page_table is None else layer.page_table.cpu().numpy(),
         page_size=layer.page_size, max_pages_per_seq=layer.max_pages_per_seq,
-        sm_scale=layer.sm_scale)
+        sm_scale=layer.sm_scale, kv_dtype=getattr(layer, "kv_dtype", 0),
+        k_scale=None if getattr(layer, "k_scale", None) is None else layer.k_scale.cpu().numpy(),
+        v_scale=None if getattr(layer, "v_scale", None) is None else layer.v_scale.cpu().numpy())

@@ -20,14 +20,35 @@ static float bf16_to_float(uint16_t bits) {
     return f;
 }
 
-/* Row (b, pos, g) of K or V: C[pos] of Algorithm 1 for one KV head. */
-static const uint16_t *kv_row(const oracle_kv_t *kv, const uint16_t *base, int b, int pos, int g) {
+float oracle_e4m3_decode(uint8_t code) {
+    int sign = code >> 7, e = (code >> 3) & 15, m = code & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;                        /* the only non-number; no infinities */
+    if (e == 0) v = ldexp((double)m / 8.0, -6);               /* subnormal */
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return (float)(sign ? -v : v);
+}
+
+/* Element offset of row (b, pos, g) of K or V: C[pos] of Algorithm 1 for one KV head. */
+static int64_t kv_row(const oracle_kv_t *kv, int b, int pos, int g) {
     if (kv->paged) {
         int64_t page = kv->page_table[(int64_t)b * kv->max_pages_per_seq + pos / kv->page_size];
         int64_t slot = pos % kv->page_size;
-        return base + page * kv->stride_page + slot * kv->stride_pos + (int64_t)g * kv->stride_head;
+        return page * kv->stride_page + slot * kv->stride_pos + (int64_t)g * kv->stride_head;
     }
-    return base + (int64_t)b * kv->stride_b + (int64_t)pos * kv->stride_pos + (int64_t)g * kv->stride_head;
+    return (int64_t)b * kv->stride_b + (int64_t)pos * kv->stride_pos + (int64_t)g * kv->stride_head;
+}
+
+/* The number stored at element `at` of K (which = 0) or V (which = 1) for KV head g: a bf16 widened
+ * exactly, or an fp8 code decoded and multiplied by the head's scale. */
+static double kv_value(const oracle_kv_t *kv, int which, int64_t at, int g) {
+    const uint16_t *base = which ? kv->v : kv->k;
+    if (kv->kv_dtype == ORACLE_KV_FP8_E4M3) {
+        const float *scale = which ? kv->v_scale : kv->k_scale;
+        double s = scale ? (double)scale[g] : 1.0;
+        return (double)oracle_e4m3_decode(((const uint8_t *)base)[at]) * s;
+    }
+    return (double)bf16_to_float(base[at]);
 }
 
 static double scale_of(const oracle_kv_t *kv) {
@@ -40,9 +61,9 @@ static float logit_at(const oracle_kv_t *kv, const uint16_t *q, int b, int h, in
     int d = kv->head_dim;
     int g = h / (kv->num_q_heads / kv->num_kv_heads);
     const uint16_t *qh = q + ((int64_t)b * kv->num_q_heads + h) * d;
-    const uint16_t *kr = kv_row(kv, kv->k, b, pos, g);
+    int64_t kr = kv_row(kv, b, pos, g);
     double dot = 0.0;
-    for (int c = 0; c < d; ++c) dot += (double)bf16_to_float(qh[c]) * (double)bf16_to_float(kr[c]);
+    for (int c = 0; c < d; ++c) dot += (double)bf16_to_float(qh[c]) * kv_value(kv, 0, kr + c, g);
     return (float)(dot * scale_of(kv));
 }
 
@@ -70,8 +91,8 @@ static void weighted_values(const oracle_kv_t *kv, int b, int g, const int32_t *
     for (int j = 0; j < n; ++j) {
         double p = exp((double)s[j] - (double)m);
         l += p;
-        const uint16_t *vr = kv_row(kv, kv->v, b, pos ? pos[j] : j, g);
-        for (int c = 0; c < d; ++c) acc[c] += p * (double)bf16_to_float(vr[c]);
+        int64_t vr = kv_row(kv, b, pos ? pos[j] : j, g);
+        for (int c = 0; c < d; ++c) acc[c] += p * kv_value(kv, 1, vr + c, g);
     }
     for (int c = 0; c < d; ++c) o[c] = (n > 0) ? (float)(acc[c] / l) : 0.0f;
     free(acc);
@@ -214,11 +235,15 @@ void oracle_kv_append(const oracle_kv_t *kv, const uint16_t *k_new, const uint16
         int pos = kv->ctx_lens[b] - 1;
         if (pos < 0) continue;
         for (int g = 0; g < kv->num_kv_heads; ++g) {
-            uint16_t *kr = (uint16_t *)kv_row(kv, kv->k, b, pos, g);
-            uint16_t *vr = (uint16_t *)kv_row(kv, kv->v, b, pos, g);
-            const uint16_t *ks = k_new + ((int64_t)b * kv->num_kv_heads + g) * d;
-            const uint16_t *vs = v_new + ((int64_t)b * kv->num_kv_heads + g) * d;
-            for (int c = 0; c < d; ++c) { kr[c] = ks[c]; vr[c] = vs[c]; }
+            int64_t at = kv_row(kv, b, pos, g);
+            int64_t from = ((int64_t)b * kv->num_kv_heads + g) * d;
+            if (kv->kv_dtype == ORACLE_KV_FP8_E4M3) {
+                uint8_t *kr = (uint8_t *)kv->k + at, *vr = (uint8_t *)kv->v + at;
+                for (int c = 0; c < d; ++c) { kr[c] = ((const uint8_t *)k_new)[from + c]; vr[c] = ((const uint8_t *)v_new)[from + c]; }
+            } else {
+                uint16_t *kr = (uint16_t *)kv->k + at, *vr = (uint16_t *)kv->v + at;
+                for (int c = 0; c < d; ++c) { kr[c] = k_new[from + c]; vr[c] = v_new[from + c]; }
+            }
         }
     }
 }

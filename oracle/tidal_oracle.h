@@ -32,6 +32,14 @@
  * equals contiguous; the 2+2+28 / 2+2+60 layer mix of Section 4.3.
  * Parity unpinned: absolute attention outputs of the paper's trained models
  * on its datasets (the paper prints no numeric attention output).
+ *
+ * 8-bit caches (not in the paper, which assumes half precision; a reading of this
+ * build): K and V may be stored as OCP FP8 E4M3 bytes with one float scale per KV
+ * head for K and one for V. The oracle's definition is "dequantise, then Eq. 1":
+ * every element is decode(byte) * scale[g], taken in double, and everything else
+ * is unchanged. Pins: the decoder against torch.float8_e4m3fn for all 256 codes;
+ * with power-of-two scales and values that bf16 also represents, every result
+ * equals the bf16 path's on the dequantised cache bit for bit; scale linearity.
  */
 #ifndef TIDAL_ORACLE_H
 #define TIDAL_ORACLE_H
@@ -58,7 +66,17 @@ typedef struct {
     int32_t page_size, max_pages_per_seq;
     const int32_t *ctx_lens;   /* [batch]; the cache already holds the new token (Algorithm 1) */
     float sm_scale;            /* 0 => 1/sqrt(head_dim) */
+    int32_t kv_dtype;          /* ORACLE_KV_BF16: k, v point to uint16 bf16 bits (as declared);
+                                  ORACLE_KV_FP8_E4M3: they point to bytes, strides still count elements */
+    const float *k_scale, *v_scale;   /* fp8 only: [num_kv_heads] each, NULL = 1 */
 } oracle_kv_t;
+
+enum { ORACLE_KV_BF16 = 0, ORACLE_KV_FP8_E4M3 = 1 };
+
+/* Value of one OCP FP8 E4M3 code: sign, 4 exponent bits (bias 7), 3 mantissa bits; exponent 0 is
+ * subnormal (m/8 * 2^-6); there are no infinities and S.1111.111 is NaN, so the largest finite
+ * value is 448. */
+float oracle_e4m3_decode(uint8_t code);
 
 enum { ORACLE_LAYER_FULL = 0, ORACLE_LAYER_SELECT = 1, ORACLE_LAYER_SPARSE = 2 };
 
@@ -105,7 +123,8 @@ int oracle_decode_step(int num_layers, const uint8_t *schedule, const oracle_kv_
                        int k, int num_index_heads, int32_t *idx, int32_t *idx_count);
 
 /* C.append(k, v) of Algorithm 1 for one layer: the new token's key and value rows (bf16
- * [B, Hkv, d]) are written at position ctx_lens[b] - 1, the slot the lengths already count.
+ * [B, Hkv, d]; for an fp8 cache already-quantised bytes [B, Hkv, d]) are written at position
+ * ctx_lens[b] - 1, the slot the lengths already count.
  * The cache arrays are written through the descriptor's (const) base pointers. */
 void oracle_kv_append(const oracle_kv_t *kv, const uint16_t *k_new, const uint16_t *v_new);
 

@@ -121,6 +121,9 @@ class LayerKV:
     max_pages_per_seq: int = 0
     sm_scale: float = 0.0
     keep: list = field(default_factory=list)    # owning buffers
+    kv_dtype: int = 0                           # 0: bf16; 1: OCP FP8 E4M3 codes with per-KV-head scales
+    k_scale: Optional[torch.Tensor] = None      # float32 [Hkv] on the device (fp8 only)
+    v_scale: Optional[torch.Tensor] = None
 
     @property
     def paged(self) -> bool:
@@ -128,7 +131,7 @@ class LayerKV:
 
     def kv_bytes(self) -> int:
         """Bytes of K and V that a full pass over the cache must read."""
-        return int(self.ctx_lens.sum().item()) * self.num_kv_heads * self.head_dim * 2 * 2
+        return int(self.ctx_lens.sum().item()) * self.num_kv_heads * self.head_dim * 2 * (1 if self.kv_dtype else 2)
 
 
 def _gen(device, seed: int) -> torch.Generator:
@@ -234,6 +237,43 @@ def make_layer(w: Workload, layer: int, device, layout: str = "hnd_interleaved",
     raise ValueError(layout)
 
 
+KV_BF16, KV_FP8_E4M3 = 0, 1
+
+
+def to_fp8(layer: LayerKV, k_scale: Optional[torch.Tensor] = None, v_scale: Optional[torch.Tensor] = None) -> LayerKV:
+    """The same cache stored as OCP FP8 E4M3 codes (torch's float8_e4m3fn cast: round to nearest even,
+    saturating) with one scale per KV head for K and one for V: code = cast(value / scale). The default
+    scales map each KV head's largest magnitude to 240, a little over half of the format's range. The
+    buffer keeps its layout; element strides stay what they were, rows are half as long in bytes.
+    Data preparation only (a storage format), no arithmetic of the method."""
+    assert layer.kv_dtype == KV_BF16 and len(layer.keep) == 1, "needs a cache held in one buffer"
+    buf = layer.keep[0]
+    Hkv, dev = layer.num_kv_heads, buf.device
+    paged = layer.page_table is not None
+    hdim = 1                                       # [B][Hkv][N][2][d] and [page][Hkv][16][2][d]: heads are dim 1
+    kview, vview = buf.select(-2, 0), buf.select(-2, 1)
+    red = [i for i in range(kview.dim()) if i != hdim]
+    if k_scale is None:
+        k_scale = (kview.float().abs().amax(dim=red) / 240.0).clamp_min(2.0 ** -20)
+    if v_scale is None:
+        v_scale = (vview.float().abs().amax(dim=red) / 240.0).clamp_min(2.0 ** -20)
+    k_scale, v_scale = k_scale.to(dev, torch.float32), v_scale.to(dev, torch.float32)
+    shape = [1] * buf.dim()
+    shape[hdim] = Hkv
+    q8 = torch.empty(buf.shape, dtype=torch.float8_e4m3fn, device=dev)
+    q8.select(-2, 0).copy_((kview.float() / k_scale.view(shape[:-1])).to(torch.float8_e4m3fn))
+    q8.select(-2, 1).copy_((vview.float() / v_scale.view(shape[:-1])).to(torch.float8_e4m3fn))
+    out = LayerKV(k=q8.select(-2, 0), v=q8.select(-2, 1), batch=layer.batch, num_q_heads=layer.num_q_heads,
+                  num_kv_heads=Hkv, head_dim=layer.head_dim, ctx_lens=layer.ctx_lens, max_ctx_len=layer.max_ctx_len,
+                  stride_b=layer.stride_b, stride_pos=layer.stride_pos, stride_head=layer.stride_head,
+                  stride_page=layer.stride_page, page_table=layer.page_table, page_size=layer.page_size,
+                  max_pages_per_seq=layer.max_pages_per_seq, sm_scale=layer.sm_scale, keep=[q8],
+                  kv_dtype=KV_FP8_E4M3, k_scale=k_scale, v_scale=v_scale)
+    if paged:
+        out.num_pages = getattr(layer, "num_pages", 0) or buf.shape[0]
+    return out
+
+
 def make_page_table(w: Workload, extra_pages: int = 0):
     """One page table shared by all layers: each sequence's logical pages are a
     slice of one seeded shuffle of all physical pages. Returns (int32 [B, max_pages]
@@ -252,5 +292,7 @@ def make_page_table(w: Workload, extra_pages: int = 0):
 
 
 def bits(t: torch.Tensor):
-    """bf16 tensor -> numpy uint16 array holding the same bits (host copy)."""
+    """bf16 tensor -> numpy uint16 array holding the same bits; fp8 tensor -> uint8 codes (host copy)."""
+    if t.element_size() == 1:
+        return t.detach().contiguous().view(torch.uint8).cpu().numpy()
     return t.detach().contiguous().view(torch.int16).cpu().numpy().view("uint16")

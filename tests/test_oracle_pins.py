@@ -462,3 +462,100 @@ def test_newest_token_variant_closed_forms():
     out = oracle.sparse_attn(kv, q, aug, cnt2)
     assert np.allclose(out[0, 0], bf16_val(v)[0, N - 1, 0], atol=1e-6)      # head 0 now sees the dominant key
     assert np.array_equal(out[0, 1], plain[0, 1])                            # head 1 had it already
+
+
+# ---- 8-bit (FP8 E4M3) caches: dequantise, then Eq. 1 ------------------------------------------------
+def make_fp8(B, Hq, Hkv, N, seed, k_scale=None, v_scale=None, lens=None):
+    """NHD cache of E4M3 codes drawn from torch's cast of N(0,1) draws, plus the values they stand for."""
+    r = np.random.default_rng(seed)
+    q = bf16_bits(r.standard_normal((B, Hq, D)))
+    kt = torch.from_numpy(r.standard_normal((B, N, Hkv, D)).astype(np.float32)).to(torch.float8_e4m3fn)
+    vt = torch.from_numpy(r.standard_normal((B, N, Hkv, D)).astype(np.float32)).to(torch.float8_e4m3fn)
+    kc, vc = kt.view(torch.uint8).numpy().copy(), vt.view(torch.uint8).numpy().copy()
+    lens = np.full(B, N, np.int32) if lens is None else np.asarray(lens, np.int32)
+    kv = oracle.KV(k=kc.reshape(-1), v=vc.reshape(-1), batch=B, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D,
+                   ctx_lens=lens, stride_b=N * Hkv * D, stride_pos=Hkv * D, stride_head=D,
+                   kv_dtype=oracle.KV_FP8_E4M3, k_scale=k_scale, v_scale=v_scale)
+    return q, kt.float().numpy(), vt.float().numpy(), kv      # torch's own decoding of the codes
+
+
+def test_e4m3_decoder_matches_torch_and_the_format_definition():
+    """All 256 codes against torch.float8_e4m3fn (an independent implementation), plus the landmarks of
+    the format: largest finite value 448, smallest subnormal 2^-9, no infinities, two NaN codes."""
+    codes = np.arange(256, dtype=np.uint8)
+    mine = oracle.e4m3_decode(codes)
+    ref = torch.from_numpy(codes).view(torch.float8_e4m3fn).float().numpy()
+    assert np.array_equal(np.isnan(mine), np.isnan(ref)) and np.isnan(mine).sum() == 2
+    assert np.array_equal(mine[~np.isnan(mine)], ref[~np.isnan(ref)])
+    assert mine[0x7e] == 448.0 and mine[0xfe] == -448.0 and mine[0x01] == 2.0 ** -9 and mine[0x08] == 2.0 ** -6
+    assert mine[0x38] == 1.0 and mine[0x00] == 0.0 and np.isfinite(mine[~np.isnan(mine)]).all()
+
+
+def test_fp8_cache_with_unit_scales_equals_the_bf16_path_on_the_same_values():
+    """Every E4M3 value is also a bf16 value, so a cache of codes with scale 1 and a bf16 cache holding the
+    decoded values must give identical logits, outputs, token sets and sparse outputs, bit for bit."""
+    B, Hq, Hkv, N, k = 2, 4, 2, 150, 20
+    q, kf, vf, kv8 = make_fp8(B, Hq, Hkv, N, seed=5, lens=[150, 97])
+    kv16 = oracle.KV(k=bf16_bits(kf).reshape(-1), v=bf16_bits(vf).reshape(-1), batch=B, num_q_heads=Hq,
+                     num_kv_heads=Hkv, head_dim=D, ctx_lens=kv8.ctx_lens, stride_b=N * Hkv * D,
+                     stride_pos=Hkv * D, stride_head=D)
+    assert np.array_equal(bf16_val(bf16_bits(kf)), kf.astype(np.float64))          # representable indeed
+    o8, i8, c8, s8 = oracle.select_attn(kv8, q, k, want_scores=True)
+    o16, i16, c16, s16 = oracle.select_attn(kv16, q, k, want_scores=True)
+    assert np.array_equal(s8, s16) and np.array_equal(o8, o16) and np.array_equal(i8, i16) and np.array_equal(c8, c16)
+    assert np.array_equal(oracle.sparse_attn(kv8, q, i8, c8), oracle.sparse_attn(kv16, q, i16, c16))
+
+
+def test_fp8_scales_are_per_kv_head_and_match_a_bf16_cache_of_the_scaled_values():
+    """Power-of-two scales keep the dequantised values representable in bf16: the result must equal the
+    bf16 path on those values bit for bit (each head with its own scale), and equal Eq. 1 in numpy."""
+    B, Hq, Hkv, N = 1, 4, 2, 120
+    ks, vs = np.array([0.5, 4.0], np.float32), np.array([2.0, 0.25], np.float32)
+    q, kf, vf, kv8 = make_fp8(B, Hq, Hkv, N, seed=7, k_scale=ks, v_scale=vs)
+    kd, vd = kf * ks[None, None, :, None], vf * vs[None, None, :, None]
+    kv16 = oracle.KV(k=bf16_bits(kd).reshape(-1), v=bf16_bits(vd).reshape(-1), batch=B, num_q_heads=Hq,
+                     num_kv_heads=Hkv, head_dim=D, ctx_lens=kv8.ctx_lens, stride_b=N * Hkv * D,
+                     stride_pos=Hkv * D, stride_head=D)
+    o8, s8 = oracle.full_attn(kv8, q, want_scores=True)
+    o16, s16 = oracle.full_attn(kv16, q, want_scores=True)
+    assert np.array_equal(s8, s16) and np.array_equal(o8, o16)
+    ref = eq1_numpy(q, bf16_bits(kd), bf16_bits(vd), kv8.ctx_lens)
+    assert np.abs(o8 - ref).max() < 1e-6
+    # scales that are not powers of two: against numpy in float64 on decode * scale
+    ks2, vs2 = np.array([0.3, 1.7], np.float32), np.array([0.9, 1.1], np.float32)
+    kv8.k_scale, kv8.v_scale = ks2, vs2
+    qf = bf16_val(q)
+    o = oracle.full_attn(kv8, q)
+    for h in range(Hq):
+        g = h // 2
+        a = (kf[0, :, g].astype(np.float64) * float(ks2[g])) @ qf[0, h] / np.sqrt(D)
+        p = np.exp(a - a.max())
+        want = (p / p.sum()) @ (vf[0, :, g].astype(np.float64) * float(vs2[g]))
+        assert np.abs(o[0, h] - want).max() < 1e-6
+
+
+def test_fp8_value_scale_is_linear_and_key_scale_acts_like_the_softmax_scale():
+    B, Hq, Hkv, N = 1, 2, 1, 90
+    q, kf, vf, kv = make_fp8(B, Hq, Hkv, N, seed=9)
+    base, sc = oracle.full_attn(kv, q, want_scores=True)
+    kv.v_scale = np.array([8.0], np.float32)
+    assert np.array_equal(oracle.full_attn(kv, q), base * 8.0)
+    kv.v_scale = None
+    kv.k_scale = np.array([0.5], np.float32)
+    half, sc_half = oracle.full_attn(kv, q, want_scores=True)
+    assert np.array_equal(sc_half, sc * 0.5)
+    kv.k_scale = None
+    kv.sm_scale = 0.5 / np.sqrt(D)
+    assert np.abs(oracle.full_attn(kv, q) - half).max() < 1e-6
+
+
+def test_fp8_append_copies_codes_to_the_last_counted_row():
+    B, Hq, Hkv, N = 2, 2, 2, 40
+    q, kf, vf, kv = make_fp8(B, Hq, Hkv, N, seed=11, lens=[40, 13])
+    before_k, before_v = kv.k.copy(), kv.v.copy()
+    kn = np.arange(B * Hkv * D, dtype=np.uint8).reshape(B, Hkv, D) % 120
+    vn = (kn + 3).astype(np.uint8)
+    oracle.kv_append(kv, kn, vn)
+    want_k, want_v = before_k.reshape(B, N, Hkv, D).copy(), before_v.reshape(B, N, Hkv, D).copy()
+    want_k[0, 39], want_v[0, 39], want_k[1, 12], want_v[1, 12] = kn[0], vn[0], kn[1], vn[1]
+    assert np.array_equal(kv.k.reshape(B, N, Hkv, D), want_k) and np.array_equal(kv.v.reshape(B, N, Hkv, D), want_v)
