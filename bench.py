@@ -66,15 +66,23 @@ def measured_peak_gbs():
         return 6650.0, "fallback"
 
 
-def build_workload(w: synth.Workload, device):
+def build_workload(w: synth.Workload, device, kv_dtype: str = "bf16"):
+    """Queries and per-layer caches; with kv_dtype 'fp8' every cache is stored as E4M3 codes with
+    per-KV-head scales (the bf16 original of a layer is dropped as soon as it has been converted)."""
     qs = [synth.make_q(w, i, device) for i in range(w.num_layers)]
+    conv = synth.to_fp8 if kv_dtype == "fp8" else (lambda l: l)
     if w.paged:
         pt, total = synth.make_page_table(w)
-        layers = [synth.make_layer(w, i, device, layout="paged", q=qs[i], page_table=pt, num_pages=total)
+        layers = [conv(synth.make_layer(w, i, device, layout="paged", q=qs[i], page_table=pt, num_pages=total))
                   for i in range(w.num_layers)]
     else:
-        layers = [synth.make_layer(w, i, device, q=qs[i]) for i in range(w.num_layers)]
+        layers = [conv(synth.make_layer(w, i, device, q=qs[i])) for i in range(w.num_layers)]
     return qs, layers
+
+
+def row_bytes(kv_dtype: str) -> int:
+    """Bytes of one gathered position of one KV head: a key row and a value row."""
+    return 256 if kv_dtype == "fp8" else 512
 
 
 class ClockSampler(threading.Thread):
@@ -339,15 +347,15 @@ def layers_in_step(td, w, layers, qs, outs, gran, nrep):
     return out
 
 
-def quick_workload(td, name, dev, gran, nrep):
+def quick_workload(td, name, dev, gran, nrep, kv_dtype: str = "bf16"):
     """Step time and per-layer-type times of another configuration (compact: for the line's other_workloads)."""
     w = synth.workload(name)
-    qs, layers = build_workload(w, dev)
+    qs, layers = build_workload(w, dev, kv_dtype)
     outs = [torch.empty(w.batch, w.num_q_heads, w.head_dim, dtype=torch.float32, device=dev) for _ in layers]
     step_us = time_schedule(td, w.sched, layers, qs, outs, w.k, gran, nrep)
     lt = layers_in_step(td, w, layers, qs, outs, gran, max(3, nrep // 2))
-    sparse_bytes = sum(min(w.k, n) for n in w.ctx_lens()) * w.num_q_heads * 516
-    res = {"workload": describe(w), "step_us": round(step_us, 2)}
+    sparse_bytes = sum(min(w.k, n) for n in w.ctx_lens()) * w.num_q_heads * (row_bytes(kv_dtype) + 4)
+    res = {"workload": describe(w) + (" [KV as FP8 E4M3 codes]" if kv_dtype == "fp8" else ""), "step_us": round(step_us, 2)}
     if "full_us" in lt:
         res["full_us"] = round(lt["full_us"], 2)
         res["full_frac_of_8TBs"] = round(lt["full_bytes"] / lt["full_us"] / 1e3 / NOMINAL_HBM_GBS, 3)
@@ -371,6 +379,9 @@ def main():
     ap.add_argument("--impl", default="tidal", choices=["tidal", "reference"])
     ap.add_argument("--workload", default="cfg3")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kv-dtype", default="bf16", choices=["bf16", "fp8"],
+                    help="element type of the KV cache: bf16 (the metric's configuration) or fp8 (E4M3 codes with "
+                         "per-KV-head scales; reported as a variant, never as the headline)")
     ap.add_argument("--no-other-workloads", action="store_true",
                     help="skip the compact figures for cfg1, cfg2, cfg64, cfg4 and the cfg5 sweep")
     ap.add_argument("--granularity", default="qhead", choices=["qhead", "kvhead", "shared"],
@@ -421,7 +432,7 @@ def main():
     if args.sweep:
         print(json.dumps(sweep(td, dev, max(3, min(args.steps, 30)))), flush=True)
         return
-    qs, layers = build_workload(w, dev)
+    qs, layers = build_workload(w, dev, args.kv_dtype)
     outs = [torch.empty(w.batch, w.num_q_heads, w.head_dim, dtype=torch.float32, device=dev) for _ in layers]
     gran = {"qhead": binding.SEL_PER_QHEAD, "kvhead": binding.SEL_PER_KVHEAD, "shared": binding.SEL_SHARED}[args.granularity]
     index_heads = {"qhead": w.num_q_heads, "kvhead": w.num_kv_heads, "shared": 1}[args.granularity]
@@ -456,7 +467,7 @@ def main():
     peak, peak_kind = measured_peak_gbs()
     lt = layers_in_step(td, w, layers, qs, outs, gran, nrep)
     k_eff = [min(w.k, n) for n in w.ctx_lens()]
-    sparse_bytes = sum(k_eff) * (gather_lists * 512 + index_heads * 4)
+    sparse_bytes = sum(k_eff) * (gather_lists * row_bytes(args.kv_dtype) + index_heads * 4)
     traffic = ncu_traffic(w.name)
 
     def kernel_entry(kernel, bytes_per_launch, us, traffic_key, launches_per_step, note=None):
@@ -532,13 +543,15 @@ def main():
 
     # ---- the other configurations, compactly (one GPU, default run only) ------------------------------
     other = None
-    if rank == 0 and world == 1 and not args.no_other_workloads and args.workload == "cfg3":
+    if rank == 0 and world == 1 and not args.no_other_workloads and args.workload == "cfg3" and args.kv_dtype == "bf16":
         del step, step_host, qs, layers, outs
         torch.cuda.empty_cache()
         other = {"note": "step_us: the whole schedule through tidal_decode_step, CUDA events; per-layer figures as "
                          "in `layers`; fractions are algorithmic bytes / time / 8 TB/s (cfg1 is latency-bound: 5 MB per step)"}
         for name in ("cfg1", "cfg2", "cfg64", "cfg4"):
             other[name] = quick_workload(td, name, dev, gran, max(3, min(args.steps, 10)))
+        # the headline workload with an 8-bit cache: half the bytes per layer (fractions are of those bytes)
+        other["cfg3_kv_fp8"] = quick_workload(td, "cfg3", dev, gran, max(3, min(args.steps, 10)), "fp8")
         sw = sweep(td, dev, 3)
         other["cfg5_sweep"] = {"what": sw["sweep"], "columns": ["ctx", "k", "select_us_incl_topk", "sparse_us"],
                                "points": [[p["ctx"], p["k"], round(p["select_us_incl_topk"], 1), round(p["sparse_us"], 2)]
@@ -548,8 +561,11 @@ def main():
         line = {
             "metric": METRIC, "value": whole_job_us_per_step(ms_step, world), "unit": "us", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": describe(w), "replicas": world, "granularity": args.granularity,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if args.kv_dtype == "bf16" else "fp8_e4m3 cache, fp16 products, fp32 accumulation",
+            "data": "synthetic",
+            "config": {"workload": describe(w) + ("" if args.kv_dtype == "bf16" else " [KV as FP8 E4M3 codes: a variant, not the metric's configuration]"),
+                       "replicas": world, "granularity": args.granularity,
                        "launch": "tidal_decode_step on a non-default stream: the step's kernels are recorded once as a "
                                  "CUDA graph by the library and replayed (gpu_launches counts the kernels, not the graphs)",
                        "l2": ("every layer has its own KV cache: %.2f GiB are streamed or gathered from per step, %s the "

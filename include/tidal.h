@@ -88,7 +88,18 @@ typedef struct {
     const int32_t *ctx_lens;        /* device int32 [batch] */
     int32_t max_ctx_len;            /* host upper bound of ctx_lens; 1 .. 262144 */
     float sm_scale;                 /* 0 => 1/sqrt(head_dim), the scale of Eq. 1 */
+    int32_t kv_dtype;               /* TIDAL_KV_BF16 (0) or TIDAL_KV_FP8_E4M3 */
+    const float *k_scale, *v_scale; /* FP8 only: device float [num_kv_heads] each, NULL = 1 */
 } tidal_kv_t;
+
+/* Element type of the cache. The paper assumes half precision; TIDAL_KV_FP8_E4M3 is this library's
+ * 8-bit variant: k and v hold OCP FP8 E4M3 codes (no infinities, largest value 448) and element
+ * (b, pos, g, c) stands for decode(code) * k_scale[g] (v_scale[g] for V); attention is Eq. 1 on those
+ * values. Strides still count elements, i.e. bytes, and must be multiples of 16; a row is 128
+ * contiguous bytes. The query stays bf16 (it is converted to fp16 inside the kernels, exactly for
+ * magnitudes between 6.1e-5 and 65504). Not available: tidal_set_attend_newest,
+ * tidal_sparse_attn_noalloc, tidal_set_select_margin (ignored). */
+enum { TIDAL_KV_BF16 = 0, TIDAL_KV_FP8_E4M3 = 1 };
 
 /* Create a context on CUDA device `device`. workspace_bytes preallocates that much scratch
  * (0 = none). Whatever a later call needs beyond what the context holds is allocated inside that
@@ -109,7 +120,8 @@ tidal_status_t tidal_reserve(tidal_ctx_t *ctx, const tidal_kv_t *kv, int32_t k, 
 size_t tidal_workspace_bytes(const tidal_kv_t *kv, int32_t k);
 
 /* C.append(k, v) of Algorithm 1 for one layer: writes the new token's key and value rows
- * (k_new, v_new: device bf16 [batch, num_kv_heads, head_dim], contiguous, 16-byte aligned) into
+ * (k_new, v_new: device bf16 [batch, num_kv_heads, head_dim], contiguous, 16-byte aligned; for an
+ * FP8 cache the rows are E4M3 codes already, quantised by the caller with the cache's scales) into
  * the cache at position ctx_lens[b] - 1, the slot that the lengths already count, through the
  * layout described by `kv` (contiguous or paged). The cache memory behind kv->k / kv->v is
  * WRITTEN by this call although the descriptor declares it const. Sequences with

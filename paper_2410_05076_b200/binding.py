@@ -19,6 +19,7 @@ OK = 0
 ERR_INVALID, ERR_UNSUPPORTED, ERR_NOMEM, ERR_CUDA, ERR_TIMEOUT, ERR_INDEX = -1, -2, -3, -4, -5, -6
 ERR_TOO_LARGE, ERR_INTERNAL = -7, -8
 KV_CONTIG, KV_PAGED = 0, 1
+KV_BF16, KV_FP8_E4M3 = 0, 1
 SEL_PER_QHEAD, SEL_PER_KVHEAD, SEL_SHARED = 0, 1, 2
 LAYER_FULL, LAYER_SELECT, LAYER_SPARSE = 0, 1, 2
 
@@ -41,6 +42,7 @@ class tidal_kv_t(C.Structure):
         ("page_table", C.c_void_p), ("page_size", C.c_int32), ("max_pages_per_seq", C.c_int32),
         ("num_pages", C.c_int32),
         ("ctx_lens", C.c_void_p), ("max_ctx_len", C.c_int32), ("sm_scale", C.c_float),
+        ("kv_dtype", C.c_int32), ("k_scale", C.c_void_p), ("v_scale", C.c_void_p),
     ]
 
 
@@ -134,6 +136,10 @@ def kv_struct(layer) -> tidal_kv_t:
     s.ctx_lens = layer.ctx_lens.data_ptr()
     s.max_ctx_len = layer.max_ctx_len
     s.sm_scale = layer.sm_scale
+    s.kv_dtype = getattr(layer, "kv_dtype", 0)
+    if s.kv_dtype:
+        s.k_scale = layer.k_scale.data_ptr() if layer.k_scale is not None else None
+        s.v_scale = layer.v_scale.data_ptr() if layer.v_scale is not None else None
     return s
 
 

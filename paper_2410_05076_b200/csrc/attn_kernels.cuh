@@ -41,6 +41,10 @@ constexpr int HEAD_DIM = 128;
 constexpr int TILE = 16;                 // positions per tile == page size
 constexpr int TILE_BYTES = TILE * HEAD_DIM * 2;   // 4 KB of K, same of V
 constexpr int STAGE_BYTES = 2 * TILE_BYTES;
+// 8-bit caches (FP8 E4M3 codes): rows are 128 bytes, a 16-position tile is 2 KB of K and 2 KB of V.
+constexpr int ROW_BYTES8 = HEAD_DIM;
+constexpr int TILE_BYTES8 = TILE * ROW_BYTES8;
+constexpr int STAGE_BYTES8 = 2 * TILE_BYTES8;
 constexpr int HIST_BINS = 2048;          // global histogram row: up to 11 top bits of the score key
 constexpr int HIST_SMEM_WORDS = 8192;    // shared histogram: columns x bins <= 8192 counters (32 KB)
 // Candidate compaction in the selection layer's kernel (layout of the 32 KB behind the rings):
@@ -64,6 +68,8 @@ struct AttnParams {
     int max_ctx;               // host bound of ctx_lens; larger device values are clamped to it
     int Hq, Hkv, G;
     float scale, scale_log2;
+    const float* k_scale;      // 8-bit caches: per-KV-head dequantisation scales [Hkv] (null: 1)
+    const float* v_scale;
     int batch;
     int splits_per_item;       // > 0: pooled mode, CTA c works on item c % items; an item is served by every CTA
                                // of the grid that maps to it (this many, or one more); 0: static flat split
@@ -379,6 +385,158 @@ __device__ __forceinline__ void consume_tile(const AttnParams& p, uint32_t ks, u
     }
 }
 
+__device__ __forceinline__ void mma_f16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                              uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// Four E4M3 codes in one word -> two fp16 pairs (exact: every E4M3 value is an fp16 value).
+__device__ __forceinline__ void e4m3x4_to_f16x2x2(uint32_t w, uint32_t& lo, uint32_t& hi) {
+    asm("{\n.reg .b16 l, h;\nmov.b32 {l, h}, %2;\ncvt.rn.f16x2.e4m3x2 %0, l;\ncvt.rn.f16x2.e4m3x2 %1, h;\n}\n"
+        : "=r"(lo), "=r"(hi) : "r"(w));
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;\n" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+// Two bf16 in one word -> the same two numbers as fp16 (exact inside fp16's range).
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) {
+    return pack_f16(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+
+// The same step for a tile of an 8-bit cache: 16 key rows of 128 bytes at ks, 16 value rows at vs, both
+// holding E4M3 codes (16-byte piece c of row r at piece c ^ ((r&1)<<2) for K, c ^ (r&7) for V). Codes
+// are converted to fp16 in registers and both products run as fp16 MMAs; qf holds the query as fp16:
+// qf[s][2i], qf[s][2i+1] are head-dim elements 16c + 4i .. 16c + 4i + 3 for this lane's piece c = tig + 4s.
+// `scale` / `scale_log2` already contain the head's key scale. The O^T fragments come out with a
+// different row order than in the 16-bit kernel: o[t][0..1] is d = 16t + 2gid, o[t][2..3] is d = 16t + 2gid + 1.
+template <int MODE>
+__device__ __forceinline__ void consume_tile8(const AttnParams& p, float scale, float scale_log2, uint32_t ks,
+                                              uint32_t vs, const uint32_t (&qf)[2][8], WarpAcc& acc, uint32_t vmask,
+                                              int gid, int tig, float* score_row0, float* score_row1,
+                                              int pos_base, uint32_t* hist) {
+    float s[4] = {0.f, 0.f, 0.f, 0.f};
+    float s2[4] = {0.f, 0.f, 0.f, 0.f};
+    const uint32_t krow = ks + gid * ROW_BYTES8;
+    const uint32_t kswz = (gid & 1) << 2;
+#pragma unroll
+    for (int sl = 0; sl < 2; ++sl) {
+        uint32_t ka[4], kb[4];
+        const uint32_t off = ((uint32_t)((tig + 4 * sl) ^ kswz)) << 4;
+        lds128(krow + off, ka);                        // row gid, 16 codes
+        lds128(krow + 8 * ROW_BYTES8 + off, kb);       // row gid + 8
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint32_t a0, a2, a1, a3;
+            e4m3x4_to_f16x2x2(ka[i], a0, a2);
+            e4m3x4_to_f16x2x2(kb[i], a1, a3);
+            if (i & 1) mma_f16_16816(s2, a0, a1, a2, a3, qf[sl][2 * i], qf[sl][2 * i + 1]);
+            else mma_f16_16816(s, a0, a1, a2, a3, qf[sl][2 * i], qf[sl][2 * i + 1]);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) s[i] += s2[i];
+    const bool v0 = (vmask >> gid) & 1u, v1 = (vmask >> (gid + 8)) & 1u;
+    if (MODE == MODE_SELECT) {
+        const float f0 = s[0] * scale, f1 = s[1] * scale, f2 = s[2] * scale, f3 = s[3] * scale;
+        const uint64_t keep = l2_evict_last_policy();
+        if (p.agg) {
+            float a0 = f0 + f1, a1 = f2 + f3;
+            a0 += __shfl_xor_sync(0xffffffffu, a0, 1);
+            a1 += __shfl_xor_sync(0xffffffffu, a1, 1);
+            a0 += __shfl_xor_sync(0xffffffffu, a0, 2);
+            a1 += __shfl_xor_sync(0xffffffffu, a1, 2);
+            if (tig == 0) {
+                if (v0) st_keep(score_row0 + pos_base + gid, a0, keep);
+                if (v1) st_keep(score_row0 + pos_base + gid + 8, a1, keep);
+                if (hist) {
+                    if (v0) atomicAdd(hist + (score_key_bits(a0) >> p.hist_shift), 1u);
+                    if (v1) atomicAdd(hist + (score_key_bits(a1) >> p.hist_shift), 1u);
+                }
+            }
+        } else {
+            if (score_row0) {
+                if (v0) st_keep(score_row0 + pos_base + gid, f0, keep);
+                if (v1) st_keep(score_row0 + pos_base + gid + 8, f2, keep);
+            }
+            if (score_row1) {
+                if (v0) st_keep(score_row1 + pos_base + gid, f1, keep);
+                if (v1) st_keep(score_row1 + pos_base + gid + 8, f3, keep);
+            }
+            if (hist) {
+                const int nb = 1 << (32 - p.hist_shift);
+                uint32_t* h0 = hist + (2 * tig) * nb;
+                uint32_t* h1 = h0 + nb;
+                if (score_row0) {
+                    if (v0) atomicAdd(h0 + (score_key_bits(f0) >> p.hist_shift), 1u);
+                    if (v1) atomicAdd(h0 + (score_key_bits(f2) >> p.hist_shift), 1u);
+                }
+                if (score_row1) {
+                    if (v0) atomicAdd(h1 + (score_key_bits(f1) >> p.hist_shift), 1u);
+                    if (v1) atomicAdd(h1 + (score_key_bits(f3) >> p.hist_shift), 1u);
+                }
+            }
+        }
+    }
+    // ---- running softmax (base 2), as in the 16-bit kernel ------------------------------------------
+    const float NEG_INF = -INFINITY;
+    float t0 = v0 ? s[0] * scale_log2 : NEG_INF, t1 = v0 ? s[1] * scale_log2 : NEG_INF;
+    float t2 = v1 ? s[2] * scale_log2 : NEG_INF, t3 = v1 ? s[3] * scale_log2 : NEG_INF;
+    float mx0 = fmaxf(t0, t2), mx1 = fmaxf(t1, t3);
+    if (__any_sync(0xffffffffu, (mx0 > acc.m[0]) || (mx1 > acc.m[1]))) {
+#pragma unroll
+        for (int sh = 4; sh <= 16; sh <<= 1) {
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, sh));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
+        }
+        const float g0 = fmaxf(acc.m[0], mx0), g1 = fmaxf(acc.m[1], mx1);
+        const float a0 = (g0 == NEG_INF) ? 1.f : fast_exp2(acc.m[0] - g0);
+        const float a1 = (g1 == NEG_INF) ? 1.f : fast_exp2(acc.m[1] - g1);
+        acc.l[0] *= a0;
+        acc.l[1] *= a1;
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            acc.o[t][0] *= a0; acc.o[t][1] *= a1; acc.o[t][2] *= a0; acc.o[t][3] *= a1;
+        }
+        acc.m[0] = g0;
+        acc.m[1] = g1;
+    }
+    const float mn0 = acc.m[0], mn1 = acc.m[1];
+    const float ms0 = (mn0 == NEG_INF) ? 0.f : mn0, ms1 = (mn1 == NEG_INF) ? 0.f : mn1;
+    const float p0 = fast_exp2(t0 - ms0), p1 = fast_exp2(t1 - ms1);
+    const float p2 = fast_exp2(t2 - ms0), p3 = fast_exp2(t3 - ms1);
+    acc.l[0] += p0 + p2;
+    acc.l[1] += p1 + p3;
+    const uint32_t pb0 = movmatrix_trans(pack_f16(p0, p1));
+    const uint32_t pb1 = movmatrix_trans(pack_f16(p2, p3));
+    // ---- O^T += V^T . P^T ------------------------------------------------------------------------------
+    // ldmatrix.trans moves 16-bit units, i.e. pairs of codes (d, d+1) of one position. Matrix (pos half
+    // hp, piece c) hands lane (gid, tig) the word [V[p][d0], V[p][d1], V[p+1][d0], V[p+1][d1]] with
+    // p = 8hp + 2tig, d0 = 16c + 2gid, d1 = d0 + 1. A byte permute regroups it into (V[p][d0], V[p+1][d0])
+    // and (V[p][d1], V[p+1][d1]): the A fragments of rows d0 (MMA row gid) and d1 (MMA row gid + 8).
+    const int lane = gid * 4 + tig;
+    const int rr = lane & 7, mi = lane >> 3;
+    const int vrow = rr + ((mi >> 1) << 3);
+    const uint32_t vbase = vs + vrow * ROW_BYTES8;
+    const uint32_t vswz = rr;                          // vrow & 7
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        uint32_t m[4];
+        ldmatrix_x4_trans(vbase + ((uint32_t)((2 * u + (mi & 1)) ^ vswz) << 4), m);
+        uint32_t x0, y0, x2, y2, x1, y1, x3, y3;
+        e4m3x4_to_f16x2x2(__byte_perm(m[0], 0, 0x3120), x0, y0);      // piece 2u, positions 0-7
+        e4m3x4_to_f16x2x2(__byte_perm(m[2], 0, 0x3120), x2, y2);      // piece 2u, positions 8-15
+        mma_f16_16816(acc.o[2 * u], x0, y0, x2, y2, pb0, pb1);
+        e4m3x4_to_f16x2x2(__byte_perm(m[1], 0, 0x3120), x1, y1);      // piece 2u + 1
+        e4m3x4_to_f16x2x2(__byte_perm(m[3], 0, 0x3120), x3, y3);
+        mma_f16_16816(acc.o[2 * u + 1], x1, y1, x3, y3, pb0, pb1);
+    }
+}
+
 // Tiles of one (sequence, head group) item: at least one, so that an empty item still
 // produces its (all-zero) output row.
 __device__ __forceinline__ int item_tiles(int total) { return max(1, (total + TILE - 1) / TILE); }
@@ -386,8 +544,13 @@ __device__ __forceinline__ int item_tiles(int total) { return max(1, (total + TI
 // NEWEST (gather kernel only): every list has one more slot that stands for the newest token.
 // COMPACT (selection kernel only): the instantiation that compacts top-k candidates; the default
 // selection kernel carries none of that code.
-template <int MODE, int NW, int STAGES, bool NEWEST = false, bool COMPACT = false>
+// KV8: the cache holds FP8 E4M3 codes (128-byte rows, per-KV-head scales); same kernel, half-size ring
+// slots, conversion to fp16 in front of the MMAs (consume_tile8).
+template <int MODE, int NW, int STAGES, bool NEWEST = false, bool COMPACT = false, bool KV8 = false>
 __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
+    static_assert(!(COMPACT && KV8), "candidate compaction is built for 16-bit caches only");
+    constexpr int SLOT_BYTES = KV8 ? STAGE_BYTES8 : STAGE_BYTES;
+    constexpr int KPART_BYTES = KV8 ? TILE_BYTES8 : TILE_BYTES;       // the value rows of a slot start here
     extern __shared__ __align__(128) uint8_t smem_raw[];
     // Ring slots must be 256-byte aligned (the V fragment addressing XORs bits 5-7).
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -397,7 +560,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = lane >> 2, tig = lane & 3;
-    constexpr int RING_BYTES = NW * STAGES * STAGE_BYTES;
+    constexpr int RING_BYTES = NW * STAGES * SLOT_BYTES;
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem + RING_BYTES);   // MODE_SELECT: [columns][bins] counters
     const bool hist_on = (MODE == MODE_SELECT) && p.hist != nullptr;
 
@@ -474,7 +637,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         __syncwarp();
     }
 
-    uint8_t* wbase = smem + (size_t)warp * STAGES * STAGE_BYTES;
+    uint8_t* wbase = smem + (size_t)warp * STAGES * SLOT_BYTES;
     const uint32_t wbase_u32 = smem_u32(wbase);
     const int c16 = lane & 15, rhalf = lane >> 4;
     const long long lane_src = (long long)rhalf * p.stride_pos + c16 * 8;
@@ -484,6 +647,16 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
     const uint32_t kdst = rhalf * 256 + ((c16 ^ (rhalf << 2)) << 4);
     const uint32_t vdst = rhalf * 256;
     const uint32_t vc = c16 ^ rhalf;
+    // 8-bit caches: lane l copies piece l&7 of rows (l>>3) + 4i, i = 0..3 (one instruction moves four
+    // whole 128-byte rows); K piece c of row r goes to c ^ ((r&1)<<2), V piece c to c ^ (r&7).
+    const int piece8 = lane & 7, row8 = lane >> 3;
+    const long long lane_src8 = (long long)row8 * p.stride_pos + piece8 * 16;
+    const long long four_rows = 4 * p.stride_pos;
+    const uint32_t kdst8 = row8 * ROW_BYTES8 + ((piece8 ^ ((row8 & 1) << 2)) << 4);
+    const uint32_t vdst8 = row8 * ROW_BYTES8;
+    const uint32_t vc8 = piece8 ^ row8;                                // row & 7 == row8 ^ ((i&1)<<2)
+    const uint8_t* kbytes = reinterpret_cast<const uint8_t*>(p.k);
+    const uint8_t* vbytes = reinterpret_cast<const uint8_t*>(p.v);
     const bool pooled = p.splits_per_item > 0;
     const uint64_t kv_policy = l2_evict_first_policy();
 
@@ -614,7 +787,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         // l&15 of rows (l>>4) + 2i, i = 0..7: one instruction moves two whole rows.
         auto issue = [&](int stage) {
             const int tile = tA;
-            const uint32_t ks = wbase_u32 + stage * STAGE_BYTES, vs = ks + TILE_BYTES;
+            const uint32_t ks = wbase_u32 + stage * SLOT_BYTES, vs = ks + KPART_BYTES;
             uint32_t vmask;
             if (MODE != MODE_SPARSE) {
                 tA = tB;
@@ -632,6 +805,18 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                 }
                 const int nvalid = ok ? max(0, min(TILE, total - pos0)) : 0;
                 vmask = (1u << nvalid) - 1u;
+                if constexpr (KV8) {
+                    const long long off8 = off - lane_src + lane_src8;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const bool rv = row8 + 4 * i < nvalid;
+                        const long long eo = rv ? off8 + i * four_rows : 0;
+                        cp_async16_hint(ks + kdst8 + i * 512, kbytes + eo, rv ? 16 : 0, kv_policy);
+                        cp_async16_hint(vs + vdst8 + i * 512 + ((vc8 ^ ((i & 1) << 2)) << 4), vbytes + eo, rv ? 16 : 0, kv_policy);
+                    }
+                    if (lane == 0) { s_vmask[warp][stage] = vmask; s_posbase[warp][stage] = pos0; }
+                    return;
+                }
                 const __nv_bfloat16* ksrc = p.k + off;
                 const __nv_bfloat16* vsrc = p.v + off;
                 if (nvalid == TILE) {
@@ -657,6 +842,19 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                 tB = (tA >= 0) ? next_tile() : -1;
                 posB = load_pos(tB);
                 vmask = __ballot_sync(0xffffffffu, valid) & 0xffffu;
+                if constexpr (KV8) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int r = row8 + 4 * i;
+                        const long long ro = __shfl_sync(0xffffffffu, off, r);
+                        const bool rv = (vmask >> r) & 1u;
+                        const long long eo = rv ? ro + piece8 * 16 : 0;
+                        cp_async16_hint(ks + kdst8 + i * 512, kbytes + eo, rv ? 16 : 0, kv_policy);
+                        cp_async16_hint(vs + vdst8 + i * 512 + ((vc8 ^ ((i & 1) << 2)) << 4), vbytes + eo, rv ? 16 : 0, kv_policy);
+                    }
+                    if (lane == 0) { s_vmask[warp][stage] = vmask; s_posbase[warp][stage] = 0; }
+                    return;
+                }
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const int r = rhalf + 2 * i;
@@ -697,16 +895,33 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         // Q^T fragments: column gid is head head0+gid; this lane holds the 16-byte
         // pieces 4j+tig (j = 0..3) of that head's query row.
         uint32_t qf[4][4];
+        uint32_t qf8[2][8];                             // 8-bit caches: the query as fp16, see consume_tile8
         {
             const uint4* qp = reinterpret_cast<const uint4*>(
                 p.q + ((long long)b * p.Hq + head0 + min(gid, ncols - 1)) * HEAD_DIM);
             const bool on = gid < ncols;
+            if constexpr (KV8) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint4 t = __ldg(qp + 4 * j + tig);
-                qf[j][0] = on ? t.x : 0u; qf[j][1] = on ? t.y : 0u; qf[j][2] = on ? t.z : 0u; qf[j][3] = on ? t.w : 0u;
+                for (int sl = 0; sl < 2; ++sl) {
+                    const int c = tig + 4 * sl;         // this lane's 16-code piece of a key row = 32 bytes of the query row
+                    const uint4 t0 = __ldg(qp + 2 * c), t1 = __ldg(qp + 2 * c + 1);
+                    const uint32_t w[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) qf8[sl][i] = on ? bf16x2_to_f16x2(w[i]) : 0u;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint4 t = __ldg(qp + 4 * j + tig);
+                    qf[j][0] = on ? t.x : 0u; qf[j][1] = on ? t.y : 0u; qf[j][2] = on ? t.z : 0u; qf[j][3] = on ? t.w : 0u;
+                }
             }
         }
+        // 8-bit caches: the key scale of this KV head goes into the logit scale, the value scale is applied
+        // to the accumulators once, at the end
+        const float kscale = (KV8 && p.k_scale) ? __ldg(p.k_scale + g) : 1.f;
+        const float vscale = (KV8 && p.v_scale) ? __ldg(p.v_scale + g) : 1.f;
+        const float seg_scale = p.scale * kscale, seg_scale_log2 = p.scale_log2 * kscale;
 
 
         // Before the grid dependency was resolved the whole ring may have been filled (one slot more
@@ -822,8 +1037,11 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
                 cp_async_commit();
             }
             const int stage = it % STAGES;
-            const uint32_t ks = wbase_u32 + stage * STAGE_BYTES;
-            if constexpr (compact) {
+            const uint32_t ks = wbase_u32 + stage * SLOT_BYTES;
+            if constexpr (KV8) {
+                consume_tile8<MODE>(p, seg_scale, seg_scale_log2, ks, ks + KPART_BYTES, qf8, acc, s_vmask[warp][stage],
+                                    gid, tig, score_row0, score_row1, s_posbase[warp][stage], hist_on ? hist : nullptr);
+            } else if constexpr (compact) {
                 if (!calibrated && it == CAL_TILES) calibrate();
                 cw.stage = nullptr;
                 if (!calibrated) {
@@ -908,10 +1126,17 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
         for (int t = 0; t < 8; ++t) {
             float* w0 = mo + ((warp * 8 + 2 * tig) * HEAD_DIM);
             float* w1 = w0 + HEAD_DIM;
-            w0[16 * t + gid] = acc.o[t][0];
-            w1[16 * t + gid] = acc.o[t][1];
-            w0[16 * t + 8 + gid] = acc.o[t][2];
-            w1[16 * t + 8 + gid] = acc.o[t][3];
+            if constexpr (KV8) {                      // rows of the O^T fragments are d = 16t + 2gid and + 1 here
+                w0[16 * t + 2 * gid] = acc.o[t][0] * vscale;
+                w1[16 * t + 2 * gid] = acc.o[t][1] * vscale;
+                w0[16 * t + 2 * gid + 1] = acc.o[t][2] * vscale;
+                w1[16 * t + 2 * gid + 1] = acc.o[t][3] * vscale;
+            } else {
+                w0[16 * t + gid] = acc.o[t][0];
+                w1[16 * t + gid] = acc.o[t][1];
+                w0[16 * t + 8 + gid] = acc.o[t][2];
+                w1[16 * t + 8 + gid] = acc.o[t][3];
+            }
         }
         if (gid == 0) {
             mml[warp * 8 + 2 * tig] = make_float2(acc.m[0], acc.l[0]);
@@ -1056,6 +1281,7 @@ struct AppendParams {
     int max_pages, num_pages, paged;
     const int* ctx_lens;
     int max_ctx, batch, Hkv;
+    int elem_bytes;            // 2: bf16 rows of 256 bytes; 1: rows of 128 bytes of E4M3 codes
     int* status;
 };
 
@@ -1074,10 +1300,12 @@ __device__ __forceinline__ void kv_append_rows(const AppendParams& p) {
         off = (long long)b * p.stride_b + (long long)pos * p.stride_pos + (long long)g * p.stride_head;
     }
     const long long src = (long long)pair * HEAD_DIM;
-    // lanes 0-15 move the key row, lanes 16-31 the value row, 16 bytes each
-    const uint4* from = reinterpret_cast<const uint4*>((lane < 16 ? p.k_new : p.v_new) + src) + (lane & 15);
-    uint4* to = reinterpret_cast<uint4*>((lane < 16 ? p.k : p.v) + off) + (lane & 15);
-    *to = __ldg(from);
+    // lanes 0-15 move the key row, lanes 16-31 the value row, 16 bytes each (an 8-bit row takes 8 lanes)
+    const int piece = lane & 15;
+    if (piece * 16 >= HEAD_DIM * p.elem_bytes) return;
+    const char* from = reinterpret_cast<const char*>(lane < 16 ? p.k_new : p.v_new) + src * p.elem_bytes + piece * 16;
+    char* to = reinterpret_cast<char*>(lane < 16 ? p.k : p.v) + off * p.elem_bytes + piece * 16;
+    *reinterpret_cast<uint4*>(to) = __ldg(reinterpret_cast<const uint4*>(from));
 }
 
 __global__ void __launch_bounds__(128) kv_append_kernel(const AppendParams p) { kv_append_rows(p); }

@@ -29,6 +29,8 @@ constexpr int MAX_GROUP = 8;            // query heads per KV head that fit the 
 // Streaming (full / selection) and gather (sparse) launch shapes.
 constexpr int DENSE_NW = 8, DENSE_STAGES = 3;
 constexpr int SPARSE_NW = 4, SPARSE_STAGES = 3;
+// 8-bit caches: ring slots are half as large, so twice as many keep the same bytes in flight.
+constexpr int DENSE_STAGES8 = 6, SPARSE_STAGES8 = 6;
 constexpr size_t HIST_SMEM = HIST_SMEM_WORDS * sizeof(uint32_t);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -123,6 +125,11 @@ tidal_status_t check_kv(const tidal_kv_t* kv) {
     if (kv->batch > 65535 || kv->num_q_heads > 65535) return TIDAL_ERR_UNSUPPORTED;
     if ((long long)kv->batch * kv->num_q_heads > 262144) return TIDAL_ERR_UNSUPPORTED;   // split counters fit the zeroed head of the workspace
     if (((uintptr_t)kv->k | (uintptr_t)kv->v) & 15) return TIDAL_ERR_INVALID;
+    if (kv->kv_dtype != TIDAL_KV_BF16 && kv->kv_dtype != TIDAL_KV_FP8_E4M3) return TIDAL_ERR_INVALID;
+    // rows must start on 16-byte boundaries: 8 elements of 16 bits, 16 of 8 bits
+    const int64_t align_mask = kv->kv_dtype == TIDAL_KV_FP8_E4M3 ? 15 : 7;
+    if ((kv->stride_pos | kv->stride_head | kv->stride_b | kv->stride_page) & align_mask) return TIDAL_ERR_INVALID;
+    if (kv->kv_dtype == TIDAL_KV_FP8_E4M3 && ((((uintptr_t)kv->k_scale | (uintptr_t)kv->v_scale) & 3) != 0)) return TIDAL_ERR_INVALID;
     if ((kv->stride_pos | kv->stride_head) & 7) return TIDAL_ERR_INVALID;
     if (kv->stride_pos < 0 || kv->stride_head < 0 || kv->stride_b < 0 || kv->stride_page < 0) return TIDAL_ERR_INVALID;
     if (!(kv->sm_scale >= 0.f) || std::isinf(kv->sm_scale)) return TIDAL_ERR_INVALID;
@@ -242,6 +249,7 @@ void fill_common(AttnParams& a, const tidal_ctx* ctx, const tidal_kv_t* kv, cons
     a.Hq = kv->num_q_heads; a.Hkv = kv->num_kv_heads; a.G = a.Hq / a.Hkv;
     a.scale = kv->sm_scale > 0.f ? kv->sm_scale : 1.0f / std::sqrt((float)kv->head_dim);
     a.scale_log2 = a.scale * 1.4426950408889634f;
+    if (kv->kv_dtype == TIDAL_KV_FP8_E4M3) { a.k_scale = kv->k_scale; a.v_scale = kv->v_scale; }
     char* ws = (char*)ctx->ws;
     a.counters = state_counters(ctx);
     a.part_ml = (float2*)(ws + w.part_ml);
@@ -254,13 +262,13 @@ void fill_common(AttnParams& a, const tidal_ctx* ctx, const tidal_kv_t* kv, cons
     a.status = ctx->status;
 }
 
-template <int MODE, int NW, int STAGES>
+template <int MODE, int NW, int STAGES, bool KV8 = false>
 constexpr size_t attn_smem() {
-    return (size_t)NW * STAGES * STAGE_BYTES +
+    return (size_t)NW * STAGES * (KV8 ? STAGE_BYTES8 : STAGE_BYTES) +
            (MODE == MODE_SELECT ? HIST_SMEM : 0) + 1024;   // + alignment slack
 }
 
-template <int MODE, int NW, int STAGES, bool NEWEST = false, bool COMPACT = false>
+template <int MODE, int NW, int STAGES, bool NEWEST = false, bool COMPACT = false, bool KV8 = false>
 tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, int full_grid, cudaStream_t st) {
     // Programmatic dependent launch: the kernel may begin while its predecessor in the stream
     // drains; it waits (griddepcontrol.wait) before touching anything that predecessor wrote.
@@ -282,7 +290,7 @@ tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, int full_gri
     std::memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(grid, 1, 1);
     cfg.blockDim = dim3(NW * 32, 1, 1);
-    cfg.dynamicSmemBytes = attn_smem<MODE, NW, STAGES>();
+    cfg.dynamicSmemBytes = attn_smem<MODE, NW, STAGES, KV8>();
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -290,7 +298,7 @@ tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, int full_gri
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     ctx->launches++;
-    return cudaLaunchKernelEx(&cfg, attn_kernel<MODE, NW, STAGES, NEWEST, COMPACT>, a) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, attn_kernel<MODE, NW, STAGES, NEWEST, COMPACT, KV8>, a) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }
 
 // How a selection layer produces its ranking scores. Per query head: one row per head, histogram
@@ -312,7 +320,7 @@ SelectPlan select_plan(const tidal_ctx* ctx, const tidal_kv_t* kv, int Hi, int k
     s.agg = Hi != kv->num_q_heads && !caller_scores;
     s.rows = s.agg ? kv->num_kv_heads : kv->num_q_heads;
     s.fuse = Hi == s.rows;
-    s.compact = ctx->select_margin > 0.f && Hi == kv->num_q_heads && kv->batch == 1 &&
+    s.compact = ctx->select_margin > 0.f && kv->kv_dtype == TIDAL_KV_BF16 && Hi == kv->num_q_heads && kv->batch == 1 &&
                 kv->num_q_heads / kv->num_kv_heads <= CAND_COLS && 6LL * k <= kv->max_ctx_len &&
                 pooled_splits(kv, kv->num_kv_heads, dense_grid(ctx, kv)) > 0;
     if (s.compact) s.fuse = false;
@@ -349,6 +357,11 @@ tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, fl
     a.score_stride = score_stride;
     a.agg = agg ? 1 : 0;
     a.hist = fuse_hist ? state_hist(ctx) : nullptr;
+    if (kv->kv_dtype == TIDAL_KV_FP8_E4M3) {
+        const int full8 = std::min(ctx->dense_slots, GRID_MAX);
+        if (scores) return launch_attn<MODE_SELECT, DENSE_NW, DENSE_STAGES8, false, false, true>(ctx, a, grid, full8, st);
+        return launch_attn<MODE_FULL, DENSE_NW, DENSE_STAGES8, false, false, true>(ctx, a, grid, full8, st);
+    }
     if (scores && a.compact) {
         if (a.splits_per_item <= 0) return TIDAL_ERR_INTERNAL;      // select_plan admits pooled grids only
         return launch_attn<MODE_SELECT, DENSE_NW, DENSE_STAGES, false, true>(ctx, a, grid, std::min(ctx->dense_slots, GRID_MAX), st);
@@ -450,6 +463,10 @@ tidal_status_t run_sparse(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, c
     if (const int S = pooled_splits(kv, items, grid)) {
         a.splits_per_item = S;
     }
+    if (kv->kv_dtype == TIDAL_KV_FP8_E4M3) {
+        if (ctx->attend_newest) return TIDAL_ERR_UNSUPPORTED;
+        return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES8, false, false, true>(ctx, a, grid, std::min(ctx->sparse_slots, GRID_MAX), st);
+    }
     if (ctx->attend_newest) return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES, true>(ctx, a, grid, std::min(ctx->sparse_slots, GRID_MAX), st);
     return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(ctx, a, grid, std::min(ctx->sparse_slots, GRID_MAX), st);
 }
@@ -486,7 +503,7 @@ void step_key(KeyBuilder& kb, const tidal_ctx* ctx, int tag, int32_t num_layers,
         kb.add(v.batch); kb.add(v.num_q_heads); kb.add(v.num_kv_heads); kb.add(v.head_dim); kb.add(v.kv_layout);
         kb.add(v.k); kb.add(v.v); kb.add(v.stride_b); kb.add(v.stride_pos); kb.add(v.stride_head); kb.add(v.stride_page);
         kb.add(v.page_table); kb.add(v.page_size); kb.add(v.max_pages_per_seq); kb.add(v.num_pages);
-        kb.add(v.ctx_lens); kb.add(v.max_ctx_len); kb.add(v.sm_scale);
+        kb.add(v.ctx_lens); kb.add(v.max_ctx_len); kb.add(v.sm_scale); kb.add(v.kv_dtype); kb.add(v.k_scale); kb.add(v.v_scale);
     }
 }
 
@@ -570,11 +587,14 @@ tidal_status_t tidal_create(tidal_ctx_t** out, int device, size_t workspace_byte
     const int d2 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW, DENSE_STAGES, false, true>, DENSE_NW * 32, attn_smem<MODE_SELECT, DENSE_NW, DENSE_STAGES>(), ctx->sm_count);
     const int s0 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>, SPARSE_NW * 32, attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(), ctx->sm_count);
     const int s1 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES, true>, SPARSE_NW * 32, attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(), ctx->sm_count);
+    const int e0 = resident_ctas(attn_kernel<MODE_FULL, DENSE_NW, DENSE_STAGES8, false, false, true>, DENSE_NW * 32, attn_smem<MODE_FULL, DENSE_NW, DENSE_STAGES8, true>(), ctx->sm_count);
+    const int e1 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW, DENSE_STAGES8, false, false, true>, DENSE_NW * 32, attn_smem<MODE_SELECT, DENSE_NW, DENSE_STAGES8, true>(), ctx->sm_count);
+    const int e2 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES8, false, false, true>, SPARSE_NW * 32, attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES8, true>(), ctx->sm_count);
     const size_t topk_smem = 2 * (size_t)(MAX_CTX / 32) * sizeof(unsigned) + 8192 * sizeof(uint2);
     const bool topk_ok = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topk_smem) == cudaSuccess;
     const size_t compact_smem = 2 * ((size_t)(MAX_CTX / 32) + 1) * sizeof(unsigned) + (size_t)COMPACT_LIST_SMEM * sizeof(uint2);
     const bool compact_ok = cudaFuncSetAttribute(topk_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)compact_smem) == cudaSuccess;
-    if (d0 <= 0 || d1 <= 0 || d2 < d1 || s0 <= 0 || s1 < s0 || !topk_ok || !compact_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
+    if (d0 <= 0 || d1 <= 0 || d2 < d1 || s0 <= 0 || s1 < s0 || e0 < d0 || e1 < d1 || e2 < s0 || !topk_ok || !compact_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
     ctx->dense_slots = std::min(d0, d1);
     ctx->sparse_slots = s0;
     if (cudaMalloc((void**)&ctx->status, 256) != cudaSuccess || cudaMemset(ctx->status, 0, 256) != cudaSuccess) {
@@ -643,6 +663,7 @@ static void fill_append(AppendParams& a, const tidal_ctx* ctx, const tidal_kv_t*
     a.paged = kv->kv_layout == TIDAL_KV_PAGED;
     a.ctx_lens = kv->ctx_lens; a.max_ctx = kv->max_ctx_len;
     a.batch = kv->batch; a.Hkv = kv->num_kv_heads;
+    a.elem_bytes = kv->kv_dtype == TIDAL_KV_FP8_E4M3 ? 1 : 2;
     a.status = ctx->status;
 }
 
@@ -1005,6 +1026,7 @@ extern "C" tidal_status_t tidal_sparse_attn_noalloc(const tidal_kv_t* kv, const 
     if (k <= 0) return TIDAL_ERR_INVALID;
     const int Hi = num_index_heads;
     if (Hi != kv->num_q_heads && Hi != kv->num_kv_heads && Hi != 1) return TIDAL_ERR_INVALID;
+    if (kv->kv_dtype != TIDAL_KV_BF16) return TIDAL_ERR_UNSUPPORTED;
     const long long rows = (long long)kv->batch * kv->num_q_heads;
     if (rows > NOALLOC_MAX_ROWS) return TIDAL_ERR_TOO_LARGE;
     int device = -1;

@@ -946,3 +946,106 @@ def test_scores_that_are_not_numbers_never_leave_stale_indices(td):
     finally:
         td.set_select_margin(0.0)
     td.device_status()
+
+
+# ---- 8-bit (FP8 E4M3) caches ------------------------------------------------------------------------
+FP8_CASES = [
+    # batch, Hq, Hkv, ctx, k, ragged
+    (1, 8, 2, 300, 40, False),
+    (2, 8, 2, 1000, 64, True),
+    (1, 4, 4, 4097, 256, False),       # MHA, ragged tail of one position
+    (3, 16, 2, 777, 100, True),        # group 8
+    (1, 2, 1, 2500, 17, False),
+    (1, 8, 2, 17, 17, False),
+    (1, 4, 2, 1, 1, False),
+    (1, 32, 8, 20000, 1024, False),    # pooled grid, several CTAs per head
+]
+
+
+@pytest.mark.parametrize("layout", ["hnd_interleaved", "paged"])
+@pytest.mark.parametrize("B,Hq,Hkv,N,k,ragged", FP8_CASES)
+def test_fp8_cache_layers_match_the_oracle(td, layout, B, Hq, Hkv, N, k, ragged):
+    """Full, selection and sparse layers over a cache of E4M3 codes with per-KV-head scales, against the
+    oracle's dequantise-then-Eq. 1 on the same codes and scales."""
+    w = wl(B, Hq, Hkv, N, k, planted=min(8, N), ragged=ragged, ctx_min=max(1, N // 3), seed=73)
+    q, lay16 = build(w, layout)
+    lay = synth.to_fp8(lay16)
+    assert lay.kv_dtype == synth.KV_FP8_E4M3 and lay.k.element_size() == 1
+    okv, qb = util.oracle_kv(lay), synth.bits(q)
+    lens = lay.ctx_lens.cpu().numpy()
+    ref_out, ref_sc = oracle.full_attn(okv, qb, want_scores=True)
+    util.check_out(td.full_attn(lay, q).cpu().numpy(), ref_out, "fp8.full")
+    scores = torch.full((B, Hq, N), float("nan"), dtype=torch.float32, device=DEV)
+    out, idx, cnt = td.select_attn(lay, q, k, scores=scores)
+    util.check_out(out.cpu().numpy(), ref_out, "fp8.select")
+    assert cnt.cpu().numpy().tolist() == [min(k, int(n)) for n in lens]
+    sc, idx_h = scores.cpu().numpy(), idx.cpu().numpy()
+    for b in range(B):
+        n = int(lens[b])
+        assert np.abs(sc[b, :, :n] - ref_sc[b, :, :n]).max() <= 1e-4
+        for h in range(Hq):
+            util.check_idx_row(idx_h[b, h], ref_sc[b, h], k, n, f"fp8.idx[{b},{h}]")
+    _, ref_idx, ref_cnt = oracle.select_attn(okv, qb, k)
+    sp = td.sparse_attn(lay, q, torch.from_numpy(ref_idx).to(DEV), torch.from_numpy(ref_cnt).to(DEV))
+    util.check_out(sp.cpu().numpy(), oracle.sparse_attn(okv, qb, ref_idx, ref_cnt), "fp8.sparse")
+    # quantisation is visible: the 8-bit result is close to, but not the same as, the 16-bit one
+    if N > 16:
+        assert not torch.equal(td.full_attn(lay16, q), td.full_attn(lay, q))
+    assert td.device_status() == binding.OK
+
+
+def test_fp8_decode_step_with_aggregated_sets_and_append(td):
+    """A whole step (F, S, sp, S, sp) over E4M3 caches with the cache update (codes are copied), one token
+    set per KV head, against the oracle stepping over host copies."""
+    sched = [0, 1, 2, 1, 2]
+    w = wl(2, 8, 2, 900, 64, ragged=True, ctx_min=200, seed=79, layers=len(sched))
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    layers = [synth.to_fp8(synth.make_layer(w, i, DEV, q=qs[i])) for i in range(len(sched))]
+    g = torch.Generator(device="cpu").manual_seed(3)
+    k_new = [torch.randn(w.batch, w.num_kv_heads, 128, generator=g).to(torch.float8_e4m3fn) for _ in sched]
+    v_new = [torch.randn(w.batch, w.num_kv_heads, 128, generator=g).to(torch.float8_e4m3fn) for _ in sched]
+    okvs = [util.oracle_kv(l) for l in layers]
+    for okv, kn, vn in zip(okvs, k_new, v_new):
+        oracle.kv_append(okv, synth.bits(kn), synth.bits(vn))
+    outs, idx, cnt = td.decode_step_append(sched, layers, qs, [t.to(DEV) for t in k_new], [t.to(DEV) for t in v_new],
+                                           w.k, granularity=binding.SEL_PER_KVHEAD)
+    torch.cuda.synchronize()
+    for l, okv in zip(layers, okvs):
+        after = util.oracle_kv(l)
+        assert np.array_equal(after.k, okv.k) and np.array_equal(after.v, okv.v)
+    lens = layers[0].ctx_lens.cpu().numpy()
+    cur = None
+    for i, t in enumerate(sched):
+        qb, got = synth.bits(qs[i]), outs[i].cpu().numpy()
+        if t in (0, 1):
+            ref, sc = oracle.full_attn(okvs[i], qb, want_scores=True)
+            util.check_out(got, ref, f"fp8.step.layer{i}")
+            if t == 1:
+                _, gi, gc = td.select_attn(layers[i], qs[i], w.k, granularity=binding.SEL_PER_KVHEAD)
+                cur = (gi.cpu().numpy(), gc.cpu().numpy())
+                for b in range(w.batch):
+                    for g_ in range(w.num_kv_heads):
+                        agg = sc[b, 4 * g_: 4 * g_ + 4, : lens[b]].astype(np.float64).sum(0).astype(np.float32)
+                        util.check_idx_row(cur[0][b, g_], agg, w.k, int(lens[b]), f"fp8.step.idx{i}")
+        else:
+            util.check_out(got, oracle.sparse_attn(okvs[i], qb, cur[0], cur[1]), f"fp8.step.layer{i}")
+    assert np.array_equal(idx.cpu().numpy(), cur[0])
+    assert td.device_status() == binding.OK
+
+
+def test_fp8_argument_rules(td):
+    w = wl(1, 8, 2, 64, 8, seed=83)
+    q, lay16 = build(w, "hnd_interleaved")
+    lay = synth.to_fp8(lay16)
+    import ctypes as C
+    out = torch.empty(1, 8, 128, dtype=torch.float32, device=DEV)
+    s = binding.kv_struct(lay)
+    assert td.lib.tidal_full_attn(td.ctx, C.byref(s), q.data_ptr(), out.data_ptr(), None) == binding.OK
+    s.stride_pos = 264                                    # not a multiple of 16 bytes
+    assert td.lib.tidal_full_attn(td.ctx, C.byref(s), q.data_ptr(), out.data_ptr(), None) == binding.ERR_INVALID
+    s = binding.kv_struct(lay); s.kv_dtype = 7
+    assert td.lib.tidal_full_attn(td.ctx, C.byref(s), q.data_ptr(), out.data_ptr(), None) == binding.ERR_INVALID
+    idx = torch.zeros(1, 8, 8, dtype=torch.int32, device=DEV)
+    s = binding.kv_struct(lay)
+    assert td.lib.tidal_sparse_attn_noalloc(C.byref(s), q.data_ptr(), idx.data_ptr(), None, 8, 8, out.data_ptr(), None) == binding.ERR_UNSUPPORTED
+    torch.cuda.synchronize()
