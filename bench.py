@@ -222,16 +222,17 @@ def run_reference(args, w, rank):
     print(json.dumps(line), flush=True)
 
 
-def profile_case(td, w, dev, steps):
+def profile_case(td, w, dev, steps, kv_dtype="bf16"):
     """One layer of each type (about 1.5 GiB at cfg3), run in the order full, select, sparse."""
     need = [w.sched.index(t) if t in w.sched else 0 for t in (0, 1, 2)]
     qs = {i: synth.make_q(w, i, dev) for i in set(need)}
+    conv = synth.to_fp8 if kv_dtype == "fp8" else (lambda l: l)
     if w.paged:
         pt, total = synth.make_page_table(w)
-        layers = {i: synth.make_layer(w, i, dev, layout="paged", q=qs[i], page_table=pt, num_pages=total)
+        layers = {i: conv(synth.make_layer(w, i, dev, layout="paged", q=qs[i], page_table=pt, num_pages=total))
                   for i in set(need)}
     else:
-        layers = {i: synth.make_layer(w, i, dev, q=qs[i]) for i in set(need)}
+        layers = {i: conv(synth.make_layer(w, i, dev, q=qs[i])) for i in set(need)}
     torch.cuda.synchronize()
     idx = cnt = None
     for _ in range(steps):
@@ -427,7 +428,7 @@ def main():
 
     td = binding.Tidal(local)
     if args.profile_case:
-        profile_case(td, w, dev, args.steps)
+        profile_case(td, w, dev, args.steps, args.kv_dtype)
         return
     if args.sweep:
         print(json.dumps(sweep(td, dev, max(3, min(args.steps, 30)))), flush=True)
