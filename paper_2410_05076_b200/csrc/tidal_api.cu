@@ -330,6 +330,8 @@ SelectPlan select_plan(const tidal_ctx* ctx, const tidal_kv_t* kv, int Hi, int k
 // hist != nullptr: the kernel also accumulates the per-head histogram the top-k needs.
 // How a layer's kernel treats the kernel before it in the stream (see AttnParams::wait_first / wait_late).
 enum Dep { DEP_FIRST, DEP_PREFETCH, DEP_LATE };
+// Where a sparse layer sits in a run of consecutive sparse layers of a step (see run_sparse).
+enum Chain { CHAIN_NONE, CHAIN_FIRST, CHAIN_MIDDLE, CHAIN_LAST };
 
 tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, float* out, float* scores,
                          long long score_stride, bool fuse_hist, Dep dep, const WsLayout& w, cudaStream_t st,
@@ -439,7 +441,7 @@ tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* score
 }
 
 tidal_status_t run_sparse(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, const int* idx,
-                          const int* idx_count, int k, int Hi, float* out, Dep dep, bool chain, const WsLayout& w,
+                          const int* idx_count, int k, int Hi, float* out, Dep dep, Chain chain, const WsLayout& w,
                           cudaStream_t st) {
     AttnParams a;
     fill_common(a, ctx, kv, q, out, w);
@@ -455,9 +457,14 @@ tidal_status_t run_sparse(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, c
     // other: while the CTAs of one layer start up (lengths, index entries, first rows: a chain of
     // dependent loads) or merge their results, the others keep the memory system busy. Every item gets
     // the same number of CTAs.
+    // The first layer of a chain runs alone until its successors have joined it and gets about half
+    // the slots; the last one, which nothing follows into the slots it frees, gets one CTA per item
+    // more than a third (measured at cfg3: step 658 -> 645 us against a third everywhere).
     const int items = kv->batch * per_batch;
-    if (chain && kv->batch == 1) {
-        const int S = std::max(1, (full + 3 * items / 2) / (3 * items));
+    if (chain != CHAIN_NONE && kv->batch == 1) {
+        const int third = std::max(1, (full + 3 * items / 2) / (3 * items));
+        const int S = chain == CHAIN_FIRST ? std::max(third, (full + items) / (2 * items))
+                      : chain == CHAIN_LAST ? third + 1 : third;
         grid = std::min(grid, S * items);
     }
     if (const int S = pooled_splits(kv, items, grid)) {
@@ -710,7 +717,7 @@ tidal_status_t tidal_sparse_attn(tidal_ctx_t* ctx, const tidal_kv_t* kv, const v
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
     const WsLayout w = layout_ws(kv, k, 0);
     if ((rc = ensure_all(ctx, kv, w.total)) != TIDAL_OK) return rc;
-    return run_sparse(ctx, kv, q, idx, idx_count, k, Hi, out, DEP_FIRST, false, w, (cudaStream_t)stream);
+    return run_sparse(ctx, kv, q, idx, idx_count, k, Hi, out, DEP_FIRST, CHAIN_NONE, w, (cudaStream_t)stream);
 }
 
 // Validates a step and sizes the workspace for it (may allocate and synchronise).
@@ -769,8 +776,10 @@ static tidal_status_t decode_step_enqueue(tidal_ctx_t* ctx, int32_t num_layers, 
             if (rc == TIDAL_OK) rc = run_topk(ctx, kv, scores, w.score_stride, k, sp.rows, Hi, sp.fuse, idx, idx_count, w, st, sp.compact);
         } else {
             const bool fresh_idx = i == 0 || schedule[i - 1] == TIDAL_LAYER_SELECT;
-            const bool chain = ctx->layer_overlap && ((i > 0 && schedule[i - 1] == TIDAL_LAYER_SPARSE) ||
-                                                      (i + 1 < num_layers && schedule[i + 1] == TIDAL_LAYER_SPARSE));
+            const bool has_prev = i > 0 && schedule[i - 1] == TIDAL_LAYER_SPARSE;
+            const bool has_next = i + 1 < num_layers && schedule[i + 1] == TIDAL_LAYER_SPARSE;
+            const Chain chain = !ctx->layer_overlap || (!has_prev && !has_next) ? CHAIN_NONE
+                                : !has_prev ? CHAIN_FIRST : !has_next ? CHAIN_LAST : CHAIN_MIDDLE;
             rc = run_sparse(ctx, kv, qs[i], idx, idx_count, k, Hi, outs[i], fresh_idx ? DEP_FIRST : dep, chain, w, st);
         }
         if (rc != TIDAL_OK) return rc;
