@@ -611,7 +611,12 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
             }
         }
     }
-    if (lo >= hi && p.splits_per_item == 0) return;
+    if (lo >= hi && p.splits_per_item == 0) {
+        // No work for this CTA. A late-waiting launch promises that none of its CTAs retires before the
+        // kernel before it is complete (the host's early-trigger rule counts on it), so it waits too.
+        if (!waited) pdl_wait();
+        return;
+    }
     if (hist_on) {
         for (int i = threadIdx.x; i < HIST_SMEM_WORDS; i += NW * 32) hist[i] = 0;
         __syncthreads();

@@ -284,7 +284,7 @@ tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, int full_gri
     // launch cannot have started while a CTA of that old kernel was still resident. Hence the rule:
     // early trigger only for pooled launches (every CTA stays until the wait) whose grid is at least
     // 1 / (CURSOR_SETS - 1) of the resident slots for this kernel's CTA size.
-    a.trigger_early = a.wait_late && a.splits_per_item > 0 && (long long)(CURSOR_SETS - 1) * grid >= full_grid;
+    a.trigger_early = a.wait_late && (long long)(CURSOR_SETS - 1) * grid >= full_grid;
     if (!a.trigger_early) a.wait_late = 0;      // without the early trigger the late wait only delays the successor
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
@@ -461,7 +461,7 @@ tidal_status_t run_sparse(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, c
     // the slots; the last one, which nothing follows into the slots it frees, gets one CTA per item
     // more than a third (measured at cfg3: step 658 -> 645 us against a third everywhere).
     const int items = kv->batch * per_batch;
-    if (chain != CHAIN_NONE && kv->batch == 1) {
+    if (chain != CHAIN_NONE) {
         const int third = std::max(1, (full + 3 * items / 2) / (3 * items));
         const int S = chain == CHAIN_FIRST ? std::max(third, (full + items) / (2 * items))
                       : chain == CHAIN_LAST ? third + 1 : third;
