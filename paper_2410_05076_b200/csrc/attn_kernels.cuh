@@ -547,7 +547,7 @@ __device__ __forceinline__ int item_tiles(int total) { return max(1, (total + TI
 // KV8: the cache holds FP8 E4M3 codes (128-byte rows, per-KV-head scales); same kernel, half-size ring
 // slots, conversion to fp16 in front of the MMAs (consume_tile8).
 template <int MODE, int NW, int STAGES, bool NEWEST = false, bool COMPACT = false, bool KV8 = false>
-__global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(NW * 32, (MODE == MODE_SPARSE && KV8) ? 2 : 1) attn_kernel(const AttnParams p) {
     static_assert(!(COMPACT && KV8), "candidate compaction is built for 16-bit caches only");
     constexpr int SLOT_BYTES = KV8 ? STAGE_BYTES8 : STAGE_BYTES;
     constexpr int KPART_BYTES = KV8 ? TILE_BYTES8 : TILE_BYTES;       // the value rows of a slot start here
@@ -635,7 +635,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attn_kernel(const AttnParams p) {
     int* ccnt_all = reinterpret_cast<int*>(thr_val + CAND_COLS);
     uint2* cbuf_all = reinterpret_cast<uint2*>(ccnt_all + NW * CAND_COLS);        // 8-byte aligned: all counts above are even
     static_assert((NW * CAL_TILES * 16 * CAND_COLS + 2 * NW * CAL_TILES + 2 * CAND_COLS + NW * CAND_COLS) * 4 +
-                  NW * CAND_COLS * CAND_BUF * 8 <= HIST_SMEM_WORDS * 4 || MODE != MODE_SELECT, "compaction scratch exceeds the histogram area");
+                  NW * CAND_COLS * CAND_BUF * 8 <= HIST_SMEM_WORDS * 4 || !COMPACT, "compaction scratch exceeds the histogram area");
     if (compact) {
         if (lane < CAL_TILES) st_pos[warp * CAL_TILES + lane] = -1;
         if (lane < CAND_COLS) ccnt_all[warp * CAND_COLS + lane] = 0;

@@ -30,7 +30,9 @@ constexpr int MAX_GROUP = 8;            // query heads per KV head that fit the 
 constexpr int DENSE_NW = 8, DENSE_STAGES = 3;
 constexpr int SPARSE_NW = 4, SPARSE_STAGES = 3;
 // 8-bit caches: ring slots are half as large, so twice as many keep the same bytes in flight.
-constexpr int DENSE_STAGES8 = 6, SPARSE_STAGES8 = 6;
+constexpr int DENSE_STAGES8 = 4, SPARSE_STAGES8 = 4;
+constexpr int SPARSE_NW8 = 6;
+constexpr int DENSE_NW8 = 12;
 constexpr size_t HIST_SMEM = HIST_SMEM_WORDS * sizeof(uint32_t);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -361,8 +363,8 @@ tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, fl
     a.hist = fuse_hist ? state_hist(ctx) : nullptr;
     if (kv->kv_dtype == TIDAL_KV_FP8_E4M3) {
         const int full8 = std::min(ctx->dense_slots, GRID_MAX);
-        if (scores) return launch_attn<MODE_SELECT, DENSE_NW, DENSE_STAGES8, false, false, true>(ctx, a, grid, full8, st);
-        return launch_attn<MODE_FULL, DENSE_NW, DENSE_STAGES8, false, false, true>(ctx, a, grid, full8, st);
+        if (scores) return launch_attn<MODE_SELECT, DENSE_NW8, DENSE_STAGES8, false, false, true>(ctx, a, grid, full8, st);
+        return launch_attn<MODE_FULL, DENSE_NW8, DENSE_STAGES8, false, false, true>(ctx, a, grid, full8, st);
     }
     if (scores && a.compact) {
         if (a.splits_per_item <= 0) return TIDAL_ERR_INTERNAL;      // select_plan admits pooled grids only
@@ -472,7 +474,7 @@ tidal_status_t run_sparse(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, c
     }
     if (kv->kv_dtype == TIDAL_KV_FP8_E4M3) {
         if (ctx->attend_newest) return TIDAL_ERR_UNSUPPORTED;
-        return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES8, false, false, true>(ctx, a, grid, std::min(ctx->sparse_slots, GRID_MAX), st);
+        return launch_attn<MODE_SPARSE, SPARSE_NW8, SPARSE_STAGES8, false, false, true>(ctx, a, grid, std::min(ctx->sparse_slots, GRID_MAX), st);
     }
     if (ctx->attend_newest) return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES, true>(ctx, a, grid, std::min(ctx->sparse_slots, GRID_MAX), st);
     return launch_attn<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(ctx, a, grid, std::min(ctx->sparse_slots, GRID_MAX), st);
@@ -594,9 +596,9 @@ tidal_status_t tidal_create(tidal_ctx_t** out, int device, size_t workspace_byte
     const int d2 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW, DENSE_STAGES, false, true>, DENSE_NW * 32, attn_smem<MODE_SELECT, DENSE_NW, DENSE_STAGES>(), ctx->sm_count);
     const int s0 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>, SPARSE_NW * 32, attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(), ctx->sm_count);
     const int s1 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES, true>, SPARSE_NW * 32, attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES>(), ctx->sm_count);
-    const int e0 = resident_ctas(attn_kernel<MODE_FULL, DENSE_NW, DENSE_STAGES8, false, false, true>, DENSE_NW * 32, attn_smem<MODE_FULL, DENSE_NW, DENSE_STAGES8, true>(), ctx->sm_count);
-    const int e1 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW, DENSE_STAGES8, false, false, true>, DENSE_NW * 32, attn_smem<MODE_SELECT, DENSE_NW, DENSE_STAGES8, true>(), ctx->sm_count);
-    const int e2 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES8, false, false, true>, SPARSE_NW * 32, attn_smem<MODE_SPARSE, SPARSE_NW, SPARSE_STAGES8, true>(), ctx->sm_count);
+    const int e0 = resident_ctas(attn_kernel<MODE_FULL, DENSE_NW8, DENSE_STAGES8, false, false, true>, DENSE_NW8 * 32, attn_smem<MODE_FULL, DENSE_NW8, DENSE_STAGES8, true>(), ctx->sm_count);
+    const int e1 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW8, DENSE_STAGES8, false, false, true>, DENSE_NW8 * 32, attn_smem<MODE_SELECT, DENSE_NW8, DENSE_STAGES8, true>(), ctx->sm_count);
+    const int e2 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW8, SPARSE_STAGES8, false, false, true>, SPARSE_NW8 * 32, attn_smem<MODE_SPARSE, SPARSE_NW8, SPARSE_STAGES8, true>(), ctx->sm_count);
     const size_t topk_smem = 2 * (size_t)(MAX_CTX / 32) * sizeof(unsigned) + 8192 * sizeof(uint2);
     const bool topk_ok = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topk_smem) == cudaSuccess;
     const size_t compact_smem = 2 * ((size_t)(MAX_CTX / 32) + 1) * sizeof(unsigned) + (size_t)COMPACT_LIST_SMEM * sizeof(uint2);
