@@ -235,9 +235,11 @@ tidal_status_t tidal_decode_step_append(tidal_ctx_t *ctx, int32_t num_layers, co
 
 /* The same step for a caller whose queries and outputs live in HOST memory
  * (pinned for full speed): q_host is bf16 [num_layers, batch, Hq, head_dim],
- * out_host fp32 of the same shape. Copies q to the device, runs
- * tidal_decode_step with idx/idx_count in the workspace, copies the outputs
- * back and WAITS for the stream. The KV cache stays resident on the device. */
+ * out_host fp32 of the same shape. Runs tidal_decode_step with idx/idx_count in
+ * the workspace and WAITS for the stream. Page-locked buffers are read and written
+ * by the kernels directly over the bus (q_host 16-byte aligned); pageable ones are
+ * copied to and from a staging area on the device. The KV cache stays resident on
+ * the device. */
 tidal_status_t tidal_decode_step_host(tidal_ctx_t *ctx, int32_t num_layers, const uint8_t *schedule,
                                       const tidal_kv_t *kv_per_layer, const void *q_host,
                                       float *out_host, int32_t k, int32_t granularity, void *stream);

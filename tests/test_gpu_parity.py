@@ -199,6 +199,24 @@ def test_decode_step_host_buffers(td):
     # beyond rounding) may differ between two runs
     for i in range(len(sched)):
         assert torch.allclose(out_host[i], outs[i].cpu(), rtol=0, atol=5e-4)
+    # pageable host buffers take the staging path (copies) instead of being accessed by the kernels
+    q_page = torch.stack([q.cpu() for q in qs]).contiguous()
+    out_page = torch.zeros(len(sched), 1, 8, 128, dtype=torch.float32)
+    assert not q_page.is_pinned() and not out_page.is_pinned()
+    td.make_step_host(sched, layers, q_page, out_page, w.k)()
+    for i in range(len(sched)):
+        assert torch.allclose(out_page[i], outs[i].cpu(), rtol=0, atol=5e-4)
+    # and every layer against the oracle, through the pinned path
+    cur = None
+    for i, t in enumerate(sched):
+        okv, qb = util.oracle_kv(layers[i]), synth.bits(qs[i])
+        if t != 2:
+            util.check_out(out_host[i].numpy(), oracle.full_attn(okv, qb), f"host.layer{i}")
+            if t == 1:
+                _, gi, gc = td.select_attn(layers[i], qs[i], w.k)
+                cur = (gi.cpu().numpy(), gc.cpu().numpy())
+        else:
+            util.check_out(out_host[i].numpy(), oracle.sparse_attn(okv, qb, cur[0], cur[1]), f"host.layer{i}")
 
 
 @pytest.mark.parametrize("N,k", [(333, 20), (9000, 700), (40000, 5000)])
