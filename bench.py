@@ -331,7 +331,7 @@ def layers_in_step(td, w, layers, qs, outs, gran, nrep):
         out["full_bytes"] = sum(layers[i].kv_bytes() for i in range(nchain)) / nchain
     sel_ids = [i for i, tk in enumerate(w.sched) if tk == S]
     sp_ids = [i for i, tk in enumerate(w.sched) if tk == P]
-    if sel_ids and len(sp_ids) >= 2:
+    if sel_ids and sp_ids:
         t_sel = ts(sel_ids[:1], [S])
         t_chain = ts(sel_ids[:1] + sp_ids, [S] + [P] * len(sp_ids))
         out["sparse_us"] = (t_chain - t_sel) / len(sp_ids)
