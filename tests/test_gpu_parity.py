@@ -1069,7 +1069,8 @@ def test_fp8_argument_rules(td):
     torch.cuda.synchronize()
 
 
-@pytest.mark.parametrize("shape", ["one sequence, chains of sparse layers", "paged ragged batch", "small grids"])
+@pytest.mark.parametrize("shape", ["one sequence, chains of sparse layers", "paged ragged batch", "small grids",
+                                   "full and sparse layers interleaved"])
 def test_overlapping_layers_repeatably_equal_the_non_overlapped_step(td, shape):
     """Layers of a step overlap (late wait, early trigger, several sparse layers in flight, pool cursors
     used ahead of the wait). Run the step hundreds of times back to back, so that consecutive steps overlap
@@ -1081,8 +1082,10 @@ def test_overlapping_layers_repeatably_equal_the_non_overlapped_step(td, shape):
     elif shape == "paged ragged batch":
         w = synth.Workload("ov2", 4, 16, 4, 12, 9000, 512, 8, [0, 1] + [2] * 5 + [0, 1] + [2] * 3, 7,
                            ragged=True, ctx_min=2000, paged=True)
-    else:
+    elif shape == "small grids":
         w = synth.Workload("ov3", 1, 8, 2, 12, 3000, 256, 8, [0, 1] + [2] * 10, 5)
+    else:
+        w = synth.Workload("ov4", 1, 32, 8, 11, 24000, 2048, 8, [1, 2, 0, 2, 0, 0, 2, 1, 1, 2, 0], 8)
     L = len(w.sched)
     qs = [synth.make_q(w, i, DEV) for i in range(L)]
     if w.paged:
@@ -1101,7 +1104,7 @@ def test_overlapping_layers_repeatably_equal_the_non_overlapped_step(td, shape):
         finally:
             td.set_layer_overlap(True)
         ref, ref_idx, ref_cnt = [o.clone() for o in outs], plain.idx.clone(), plain.idx_count.clone()
-        last = L - 1                                           # a sparse layer, fed by the last selection layer
+        last = max(i for i, kind in enumerate(w.sched) if kind == 2)      # a sparse layer, fed by the last selection layer
         want = oracle.sparse_attn(util.oracle_kv(lays[last]), synth.bits(qs[last]), ref_idx.cpu().numpy(), ref_cnt.cpu().numpy())
         util.check_out(ref[last].cpu().numpy(), want, "non-overlapped reference")
         step = td.make_step(w.sched, lays, qs, outs, w.k)
