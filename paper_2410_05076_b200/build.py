@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtidal.so")
 SOURCES = ["tidal_api.cu"]
-DEPS = ["tidal_api.cu", "attn_kernels.cuh", "topk_kernels.cuh", os.path.join("..", "..", "include", "tidal.h")]
+DEPS = ["tidal_api.cu", "attn_kernels.cuh", "split_select_kernels.cuh", "topk_kernels.cuh", os.path.join("..", "..", "include", "tidal.h")]
 
 
 def nvcc_path() -> str:

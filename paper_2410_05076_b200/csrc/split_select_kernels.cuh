@@ -1,0 +1,457 @@
+// A token selection layer in two passes over the cache (one sequence, bf16, one set per query head).
+//
+// Algorithm 1's selection layer needs the scaled logits of every cached token twice: for the softmax
+// of its own output and for argTopK. The fused kernel (attn_kernel<MODE_SELECT>) streams K and V
+// together and the top-k can only start when all of it is done; the sparse layers after it then wait
+// for the top-k, and for those 20 microseconds the memory system idles. Here the layer is split:
+//
+//   score_pass_kernel  streams the KEY rows only: logits, their histogram (for the top-k), and the
+//                      softmax statistics (max M and sum L per head); the last CTA of a KV head publishes
+//                      (M, L) and clears the layer's output rows.
+//   value_pass_kernel  streams the VALUE rows only: softmax weights come from the stored logits and the
+//                      final M, so every partial result has the same scale and CTAs simply add their
+//                      part of sum_j p_j v_j / L to the output with atomics: no partial buffers, no combine.
+//
+// The step driver launches the value pass on a second stream, so that it runs beside the top-k and the
+// first sparse layers that follow: the top-k's latency chain and the ramp of the sparse chain are filled
+// with value rows streaming. Key and value rows interleave in memory at 256-byte granularity; reading every
+// other 256-byte row costs HBM nothing (measured: the same useful bandwidth as the dense stream).
+#pragma once
+
+#include "attn_kernels.cuh"
+
+namespace tidal {
+
+constexpr float LOG2E = 1.4426950408889634f;
+
+// Tile sequence of one warp of a pooled launch (see attn_kernel): a fixed first chunk, then GRAB
+// tiles at a time from the item's cursor, requested one chunk ahead.
+struct PoolWalk {
+    int cur, cur_end, grab_raw, tiles, pool_base, lane;
+    int* pool;
+    template <int GRAB>
+    __device__ __forceinline__ void start(int* cursor, int tiles_, int item_warps, int my_warp, int first_tiles_max, int lane_) {
+        pool = cursor; tiles = tiles_; lane = lane_; grab_raw = 0;
+        const int first = (tiles <= item_warps * first_tiles_max) ? max(1, (tiles + item_warps - 1) / max(item_warps, 1))
+                                                                  : first_tiles_max;
+        pool_base = item_warps * first;
+        cur = my_warp * first;
+        cur_end = min(tiles, cur + first);
+        if (lane == 0) grab_raw = pool_base + atomicAdd(pool, GRAB);
+    }
+    template <int GRAB>
+    __device__ __forceinline__ int next() {
+        if (cur >= cur_end) {
+            if (cur_end >= tiles || pool_base >= tiles) return -1;
+            cur = __shfl_sync(0xffffffffu, grab_raw, 0);
+            if (cur >= tiles) { cur_end = tiles; return -1; }
+            cur_end = min(tiles, cur + GRAB);
+            if (lane == 0) grab_raw = pool_base + atomicAdd(pool, GRAB);
+        }
+        return cur++;
+    }
+};
+
+// ---- pass 1: logits, histogram, softmax statistics -------------------------------------------------------
+// Uses of AttnParams: q, k, strides, page table, ctx_lens, scale(s), scores / score_stride, hist / hist_shift,
+// part_ml / max_splits / counters / tile_ctr / ctr_stride (the main stream's scratch), ml_final, out (cleared),
+// pdl / wait_first / wait_late / trigger_early, status. batch must be 1, splits_per_item > 0.
+template <int NW, int STAGES>
+__global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams p) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    __shared__ uint32_t s_vmask[NW][STAGES];
+    __shared__ int s_posbase[NW][STAGES];
+    __shared__ float2 s_ml[NW][8];
+    __shared__ int s_is_last;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int gid = lane >> 2, tig = lane & 3;
+    constexpr int RING_BYTES = NW * STAGES * TILE_BYTES;
+    uint32_t* hist = reinterpret_cast<uint32_t*>(smem + RING_BYTES);
+    const bool hist_on = p.hist != nullptr;
+
+    bool waited = !p.pdl;
+    if (p.pdl && p.wait_first) { pdl_wait(); pdl_trigger(); waited = true; }
+    else if (p.pdl && p.wait_late && p.trigger_early) pdl_trigger();
+
+    const int n_items = p.Hkv;                               // one sequence
+    const int g = blockIdx.x % n_items, part = blockIdx.x / n_items;
+    const int item_ctas = ((int)gridDim.x - g + n_items - 1) / n_items;
+    const int N = max(min(p.ctx_lens[0], p.max_ctx), 0);
+    const int tiles = item_tiles(N);
+    const int head0 = g * p.G, ncols = p.G;
+    if (hist_on) {
+        for (int i = threadIdx.x; i < HIST_SMEM_WORDS; i += NW * 32) hist[i] = 0;
+        __syncthreads();
+    }
+    float* score_row0 = (2 * tig < ncols) ? p.scores + (long long)(head0 + 2 * tig) * p.score_stride : nullptr;
+    float* score_row1 = (2 * tig + 1 < ncols) ? p.scores + (long long)(head0 + 2 * tig + 1) * p.score_stride : nullptr;
+
+    const uint32_t wbase = smem_u32(smem + (size_t)warp * STAGES * TILE_BYTES);
+    const int c16 = lane & 15, rhalf = lane >> 4;
+    const long long lane_src = (long long)rhalf * p.stride_pos + c16 * 8;
+    const long long two_rows = 2 * p.stride_pos;
+    const uint32_t kdst = rhalf * 256 + ((c16 ^ (rhalf << 2)) << 4);
+    const long long item_off = (long long)g * p.stride_head;
+    const uint64_t kv_policy = l2_evict_first_policy();
+    const uint64_t keep = l2_evict_last_policy();
+
+    int* pool = p.tile_ctr + (long long)g * p.ctr_stride;
+    PoolWalk walk;
+    constexpr int GRAB = GRAB_TILES_DENSE;
+    walk.template start<GRAB>(pool, tiles, item_ctas * NW, part * NW + warp, STAGES + 2, lane);
+    int tA = walk.template next<GRAB>();
+    int tB = (tA >= 0) ? walk.template next<GRAB>() : -1;
+
+    auto issue = [&](int stage) {
+        const int tile = tA;
+        tA = tB;
+        tB = (tA >= 0) ? walk.template next<GRAB>() : -1;
+        const uint32_t ks = wbase + stage * TILE_BYTES;
+        const int pos0 = tile * TILE;
+        long long off;
+        bool ok = true;
+        if (p.paged) {
+            const int page = __ldg(p.page_table + tile);
+            ok = (unsigned)page < (unsigned)p.num_pages;
+            if (!ok && lane == 0) atomicOr(p.status, STATUS_BAD_PAGE);
+            off = (ok ? (long long)page * p.stride_page : 0) + item_off + lane_src;
+        } else {
+            off = item_off + (long long)pos0 * p.stride_pos + lane_src;
+        }
+        const int nvalid = ok ? max(0, min(TILE, N - pos0)) : 0;
+        const __nv_bfloat16* ksrc = p.k + off;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const bool rv = rhalf + 2 * i < nvalid;
+            cp_async16_hint(ks + kdst + i * 512, rv ? ksrc + i * two_rows : p.k, rv ? 16 : 0, kv_policy);
+        }
+        if (lane == 0) { s_vmask[warp][stage] = (1u << nvalid) - 1u; s_posbase[warp][stage] = pos0; }
+    };
+
+    int issued = 0, commits = 0;
+    if (!waited && !p.wait_late) {
+        while (commits < STAGES && tA >= 0 && tA < tiles - 1) { issue(issued % STAGES); ++issued; cp_async_commit(); ++commits; }
+        pdl_wait();
+        pdl_trigger();
+        waited = true;
+    }
+    // a selection layer that waits late writes its scores ahead of the wait: the host allows that only
+    // when nothing can still be reading the score buffer
+    uint32_t qf[4][4];
+    {
+        const uint4* qp = reinterpret_cast<const uint4*>(p.q + (long long)(head0 + min(gid, ncols - 1)) * HEAD_DIM);
+        const bool on = gid < ncols;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint4 t = __ldg(qp + 4 * j + tig);
+            qf[j][0] = on ? t.x : 0u; qf[j][1] = on ? t.y : 0u; qf[j][2] = on ? t.z : 0u; qf[j][3] = on ? t.w : 0u;
+        }
+    }
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;      // heads 2tig, 2tig+1: max (all lanes of a tig agree), this lane's sum
+    const bool ring_full = commits == STAGES;
+    while (commits < STAGES - 1) {
+        if (tA >= 0) { issue(issued % STAGES); ++issued; }
+        cp_async_commit();
+        ++commits;
+    }
+    for (int it = 0; it < issued; ++it) {
+        if (it == 0 && ring_full) {
+            cp_async_wait<STAGES - 1>();
+            __syncwarp();
+        } else {
+            cp_async_wait<STAGES - 2>();
+            __syncwarp();
+            if (tA >= 0) { issue((it + STAGES - 1) % STAGES); ++issued; }
+            cp_async_commit();
+        }
+        const int stage = it % STAGES;
+        const uint32_t ks = wbase + stage * TILE_BYTES;
+        const uint32_t vmask = s_vmask[warp][stage];
+        const int pos_base = s_posbase[warp][stage];
+        // S^T = K . Q^T, as in consume_tile
+        float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
+        const uint32_t krow = ks + gid * 256;
+        const uint32_t kswz = (gid & 1) << 2;
+#pragma unroll
+        for (int j = 0; j < 4; j += 2) {
+            uint32_t ka[4], kb[4], kc[4], kd[4];
+            const uint32_t off0 = (((4 * j + tig) ^ kswz) << 4), off1 = (((4 * j + 4 + tig) ^ kswz) << 4);
+            lds128(krow + off0, ka);
+            lds128(krow + 8 * 256 + off0, kb);
+            lds128(krow + off1, kc);
+            lds128(krow + 8 * 256 + off1, kd);
+            mma_bf16_16816(s, ka[0], kb[0], ka[1], kb[1], qf[j][0], qf[j][1]);
+            mma_bf16_16816(s2, kc[0], kd[0], kc[1], kd[1], qf[j + 1][0], qf[j + 1][1]);
+            mma_bf16_16816(s, ka[2], kb[2], ka[3], kb[3], qf[j][2], qf[j][3]);
+            mma_bf16_16816(s2, kc[2], kd[2], kc[3], kd[3], qf[j + 1][2], qf[j + 1][3]);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) s[i] += s2[i];
+        const bool v0 = (vmask >> gid) & 1u, v1 = (vmask >> (gid + 8)) & 1u;
+        const float f0 = s[0] * p.scale, f1 = s[1] * p.scale, f2 = s[2] * p.scale, f3 = s[3] * p.scale;
+        if (score_row0) {
+            if (v0) st_keep(score_row0 + pos_base + gid, f0, keep);
+            if (v1) st_keep(score_row0 + pos_base + gid + 8, f2, keep);
+        }
+        if (score_row1) {
+            if (v0) st_keep(score_row1 + pos_base + gid, f1, keep);
+            if (v1) st_keep(score_row1 + pos_base + gid + 8, f3, keep);
+        }
+        if (hist_on) {
+            const int nb = 1 << (32 - p.hist_shift);
+            uint32_t* h0 = hist + (2 * tig) * nb;
+            uint32_t* h1 = h0 + nb;
+            if (score_row0) {
+                if (v0) atomicAdd(h0 + (score_key_bits(f0) >> p.hist_shift), 1u);
+                if (v1) atomicAdd(h0 + (score_key_bits(f2) >> p.hist_shift), 1u);
+            }
+            if (score_row1) {
+                if (v0) atomicAdd(h1 + (score_key_bits(f1) >> p.hist_shift), 1u);
+                if (v1) atomicAdd(h1 + (score_key_bits(f3) >> p.hist_shift), 1u);
+            }
+        }
+        // softmax statistics in base 2. The value pass recomputes the weights from the STORED logits
+        // (f * log2 e), so the statistics are taken from exactly those numbers.
+        const float t0 = v0 ? f0 * LOG2E : -INFINITY, t1 = v0 ? f1 * LOG2E : -INFINITY;
+        const float t2 = v1 ? f2 * LOG2E : -INFINITY, t3 = v1 ? f3 * LOG2E : -INFINITY;
+        float mx0 = fmaxf(t0, t2), mx1 = fmaxf(t1, t3);
+        if (__any_sync(0xffffffffu, (mx0 > m0) || (mx1 > m1))) {
+#pragma unroll
+            for (int sh = 4; sh <= 16; sh <<= 1) {
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, sh));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
+            }
+            const float g0 = fmaxf(m0, mx0), g1 = fmaxf(m1, mx1);
+            l0 *= (g0 == -INFINITY) ? 1.f : fast_exp2(m0 - g0);
+            l1 *= (g1 == -INFINITY) ? 1.f : fast_exp2(m1 - g1);
+            m0 = g0;
+            m1 = g1;
+        }
+        const float ms0 = (m0 == -INFINITY) ? 0.f : m0, ms1 = (m1 == -INFINITY) ? 0.f : m1;
+        l0 += fast_exp2(t0 - ms0) + fast_exp2(t2 - ms0);
+        l1 += fast_exp2(t1 - ms1) + fast_exp2(t3 - ms1);
+    }
+    cp_async_wait<0>();
+    __syncwarp();
+    if (!waited) {
+        pdl_wait();
+        if (!p.trigger_early) pdl_trigger();
+        waited = true;
+    }
+    if (hist_on) {
+        __syncthreads();
+        const int nb = 1 << (32 - p.hist_shift);
+        for (int i = threadIdx.x; i < ncols * nb; i += NW * 32) {
+            const uint32_t w = hist[i];
+            if (w) atomicAdd(p.hist + (long long)(head0 + i / nb) * HIST_BINS + (i % nb), w);
+        }
+    }
+    // ---- (max, sum) of this CTA, then of the KV head --------------------------------------------------------
+#pragma unroll
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+        l0 += __shfl_xor_sync(0xffffffffu, l0, sh);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, sh);
+    }
+    if (gid == 0) {
+        s_ml[warp][2 * tig] = make_float2(m0, l0);
+        s_ml[warp][2 * tig + 1] = make_float2(m1, l1);
+    }
+    __syncthreads();
+    const int nsplits = item_ctas;
+    if (threadIdx.x < ncols) {
+        const int col = threadIdx.x;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) M = fmaxf(M, s_ml[w][col].x);
+        float L = 0.f;
+        if (M != -INFINITY)
+#pragma unroll
+            for (int w = 0; w < NW; ++w) {
+                const float2 ml = s_ml[w][col];
+                L += ml.y * ((ml.x == -INFINITY) ? 0.f : fast_exp2(ml.x - M));
+            }
+        if (part < p.max_splits) p.part_ml[(long long)(head0 + col) * p.max_splits + part] = make_float2(M, L);
+        else atomicOr(p.status, STATUS_SPLIT_OVERFLOW);
+    }
+    __syncthreads();
+    int* ctr = p.counters + (long long)g * p.ctr_stride;
+    if (threadIdx.x == 0) {
+        int old;
+        asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;\n" : "=r"(old) : "l"(ctr) : "memory");
+        s_is_last = (old == nsplits - 1);
+    }
+    __syncthreads();
+    if (s_is_last) {
+        const int ns = min(nsplits, p.max_splits);
+        if (warp < ncols) {
+            const int col = warp;
+            const long long pr = (long long)(head0 + col) * p.max_splits;
+            float M = -INFINITY;
+            for (int sidx = lane; sidx < ns; sidx += 32) M = fmaxf(M, __ldcg(&p.part_ml[pr + sidx].x));
+#pragma unroll
+            for (int sh = 16; sh >= 1; sh >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sh));
+            float L = 0.f;
+            for (int sidx = lane; sidx < ns; sidx += 32) {
+                const float2 ml = __ldcg(&p.part_ml[pr + sidx]);
+                L += ml.y * ((ml.x == -INFINITY || M == -INFINITY) ? 0.f : fast_exp2(ml.x - M));
+            }
+#pragma unroll
+            for (int sh = 16; sh >= 1; sh >>= 1) L += __shfl_xor_sync(0xffffffffu, L, sh);
+            if (lane == 0) p.ml_final[head0 + col] = make_float2(M, L);
+        }
+        // the value pass adds its parts to the output rows: they start at zero
+        for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) p.out[(long long)head0 * HEAD_DIM + e] = 0.f;
+        if (threadIdx.x == NW * 32 - 1) { *pool = 0; __threadfence(); }
+        if (threadIdx.x == 0) *ctr = 0;
+    }
+}
+
+// ---- pass 2: sum_j softmax_j v_j from the stored logits ------------------------------------------------------
+// Uses of AttnParams: v, strides, page table, ctx_lens, scores / score_stride, ml_final, out (+= with atomics),
+// tile_ctr / ctr_stride (a cursor set of its own: it runs beside the main stream's kernels), status.
+template <int NW, int STAGES>
+__global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams p) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    constexpr int SLOT = TILE_BYTES + 512;                   // 16 value rows, then 16 logits of up to 8 heads
+    __shared__ uint32_t s_vmask[NW][STAGES];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int gid = lane >> 2, tig = lane & 3;
+    const int n_items = p.Hkv;
+    const int g = blockIdx.x % n_items, part = blockIdx.x / n_items;
+    const int item_ctas = ((int)gridDim.x - g + n_items - 1) / n_items;
+    const int N = max(min(p.ctx_lens[0], p.max_ctx), 0);
+    const int tiles = item_tiles(N);
+    const int head0 = g * p.G, ncols = p.G;
+
+    const uint32_t wbase = smem_u32(smem + (size_t)warp * STAGES * SLOT);
+    const int c16 = lane & 15, rhalf = lane >> 4;
+    const long long lane_src = (long long)rhalf * p.stride_pos + c16 * 8;
+    const long long two_rows = 2 * p.stride_pos;
+    const uint32_t vdst = rhalf * 256;
+    const uint32_t vc = c16 ^ rhalf;
+    const long long item_off = (long long)g * p.stride_head;
+    const uint64_t kv_policy = l2_evict_first_policy();
+    // lane l < 4 * ncols fetches 16 bytes (four positions) of head l >> 2's logits
+    const bool score_lane = lane < 4 * ncols;
+    const float* score_src = p.scores + (long long)(head0 + (lane >> 2)) * p.score_stride + 4 * (lane & 3);
+
+    int* pool = p.tile_ctr + (long long)g * p.ctr_stride;
+    PoolWalk walk;
+    constexpr int GRAB = GRAB_TILES_DENSE;
+    walk.template start<GRAB>(pool, tiles, item_ctas * NW, part * NW + warp, STAGES + 2, lane);
+    int tA = walk.template next<GRAB>();
+    int tB = (tA >= 0) ? walk.template next<GRAB>() : -1;
+
+    auto issue = [&](int stage) {
+        const int tile = tA;
+        tA = tB;
+        tB = (tA >= 0) ? walk.template next<GRAB>() : -1;
+        const uint32_t vs = wbase + stage * SLOT;
+        const int pos0 = tile * TILE;
+        long long off;
+        bool ok = true;
+        if (p.paged) {
+            const int page = __ldg(p.page_table + tile);
+            ok = (unsigned)page < (unsigned)p.num_pages;
+            if (!ok && lane == 0) atomicOr(p.status, STATUS_BAD_PAGE);
+            off = (ok ? (long long)page * p.stride_page : 0) + item_off + lane_src;
+        } else {
+            off = item_off + (long long)pos0 * p.stride_pos + lane_src;
+        }
+        const int nvalid = ok ? max(0, min(TILE, N - pos0)) : 0;
+        const __nv_bfloat16* vsrc = p.v + off;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const bool rv = rhalf + 2 * i < nvalid;
+            cp_async16_hint(vs + vdst + i * 512 + ((vc ^ ((i & 3) << 1)) << 4), rv ? vsrc + i * two_rows : p.v, rv ? 16 : 0, kv_policy);
+        }
+        // (logits past the end of the sequence are never used: their rows are masked)
+        if (score_lane) cp_async16(vs + TILE_BYTES + lane * 16, score_src + pos0, 16);
+        if (lane == 0) s_vmask[warp][stage] = (1u << nvalid) - 1u;
+    };
+
+    // the final statistics of this lane's two heads
+    float M0 = -INFINITY, M1 = -INFINITY;
+    if (2 * tig < ncols) M0 = __ldg(&p.ml_final[head0 + 2 * tig].x);
+    if (2 * tig + 1 < ncols) M1 = __ldg(&p.ml_final[head0 + 2 * tig + 1].x);
+    float o[8][4];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) { o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f; }
+
+    int issued = 0, commits = 0;
+    while (commits < STAGES - 1) {
+        if (tA >= 0) { issue(issued % STAGES); ++issued; }
+        cp_async_commit();
+        ++commits;
+    }
+    for (int it = 0; it < issued; ++it) {
+        cp_async_wait<STAGES - 2>();
+        __syncwarp();
+        if (tA >= 0) { issue((it + STAGES - 1) % STAGES); ++issued; }
+        cp_async_commit();
+        const int stage = it % STAGES;
+        const uint32_t vs = wbase + stage * SLOT;
+        const uint32_t vmask = s_vmask[warp][stage];
+        const bool v0 = (vmask >> gid) & 1u, v1 = (vmask >> (gid + 8)) & 1u;
+        // logits of (position gid | gid + 8, heads 2tig | 2tig + 1): head h's 16 floats start at 64 * h
+        const uint32_t sbase = vs + TILE_BYTES;
+        float f0 = 0.f, f1 = 0.f, f2 = 0.f, f3 = 0.f;
+        if (2 * tig < ncols) {
+            asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f0) : "r"(sbase + (2 * tig) * 64 + gid * 4));
+            asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f2) : "r"(sbase + (2 * tig) * 64 + (gid + 8) * 4));
+        }
+        if (2 * tig + 1 < ncols) {
+            asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f1) : "r"(sbase + (2 * tig + 1) * 64 + gid * 4));
+            asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f3) : "r"(sbase + (2 * tig + 1) * 64 + (gid + 8) * 4));
+        }
+        const bool h0 = 2 * tig < ncols && M0 != -INFINITY, h1 = 2 * tig + 1 < ncols && M1 != -INFINITY;
+        const float p0 = (v0 && h0) ? fast_exp2(f0 * LOG2E - M0) : 0.f, p1 = (v0 && h1) ? fast_exp2(f1 * LOG2E - M1) : 0.f;
+        const float p2 = (v1 && h0) ? fast_exp2(f2 * LOG2E - M0) : 0.f, p3 = (v1 && h1) ? fast_exp2(f3 * LOG2E - M1) : 0.f;
+        const uint32_t pb0 = movmatrix_trans(pack_bf16(p0, p1));
+        const uint32_t pb1 = movmatrix_trans(pack_bf16(p2, p3));
+        const int rr = lane & 7, mb = (lane >> 3) & 1;
+        const uint32_t vlane = vs + (rr + ((lane >> 4) << 3)) * 256 + ((rr ^ mb) << 4);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            uint32_t a[4];
+            ldmatrix_x4_trans(vlane ^ (t << 5), a);
+            mma_bf16_16816(o[t], a[0], a[1], a[2], a[3], pb0, pb1);
+        }
+    }
+    cp_async_wait<0>();
+    __syncthreads();                                   // all rings drained; reuse the shared memory
+    // ---- sum the warps of this CTA, then add the CTA's part, divided by the head's sum, to the output ---
+    float* mo = reinterpret_cast<float*>(smem);       // [NW][8][128]
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+        float* w0 = mo + ((warp * 8 + 2 * tig) * HEAD_DIM);
+        float* w1 = w0 + HEAD_DIM;
+        w0[16 * t + gid] = o[t][0];
+        w1[16 * t + gid] = o[t][1];
+        w0[16 * t + 8 + gid] = o[t][2];
+        w1[16 * t + 8 + gid] = o[t][3];
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) {
+        const int col = e >> 7, c = e & 127;
+        float O = 0.f;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) O += mo[(w * 8 + col) * HEAD_DIM + c];
+        const float L = __ldg(&p.ml_final[head0 + col].y);
+        if (L > 0.f && O != 0.f) atomicAdd(p.out + (long long)(head0 + col) * HEAD_DIM + c, O / L);
+    }
+    // the last CTA of this KV head to finish clears the cursor for the next value pass
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int* ctr = p.counters + (long long)g * p.ctr_stride;
+        int old;
+        asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;\n" : "=r"(old) : "l"(ctr) : "memory");
+        if (old == item_ctas - 1) { *ctr = 0; *pool = 0; }
+    }
+}
+
+}  // namespace tidal

@@ -15,6 +15,7 @@
 #include <new>
 
 #include "attn_kernels.cuh"
+#include "split_select_kernels.cuh"
 #include "topk_kernels.cuh"
 
 using namespace tidal;
@@ -56,6 +57,11 @@ struct tidal_ctx {
     int attend_newest = 0;                      // sparse layers also attend the newest token (not in the paper)
     int cursor_set = 0;                         // which of the sets of pool cursors the last attention launch used
     float select_margin = 0.f;                  // > 0: selection layers compact candidates above a provisional threshold aimed at this multiple of k'/N
+    // Split selection layers run their value pass on a stream of the context's own, beside the top-k and
+    // the sparse layers that follow on the caller's stream; two events fork and join the streams.
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    int split_select = 1;
     int layer_overlap = 1;                      // layers of a step may stream their inputs while the layer before them finishes
     int64_t launches = 0;
     // Whole steps are recorded once as CUDA graphs (programmatic dependent launches included) and
@@ -75,7 +81,7 @@ struct tidal_ctx {
 namespace {
 
 struct WsLayout {
-    size_t part_ml, part_o, scores, cand, bitmap, idx, idx_count, q_stage, out_stage, total;
+    size_t part_ml, part_o, ml_final, scores, cand, bitmap, idx, idx_count, q_stage, out_stage, total;
     long long cand_stride, bitmap_stride;
     long long score_stride;
     int max_splits;
@@ -158,6 +164,7 @@ WsLayout layout_ws(const tidal_kv_t* kv, int k, int num_layers_host) {
     w.max_splits = max_splits_for(kv);
     w.part_ml = at;   at += align_up(rows * w.max_splits * sizeof(float2), 256);
     w.part_o = at;    at += align_up(rows * w.max_splits * HEAD_DIM * sizeof(float), 256);
+    w.ml_final = at;  at += align_up(rows * sizeof(float2), 256);
     w.score_stride = (long long)align_up((size_t)kv->max_ctx_len, 16);
     w.scores = at;    at += align_up(rows * (size_t)w.score_stride * sizeof(float), 256);
     w.cand_stride = w.score_stride;
@@ -195,7 +202,8 @@ tidal_status_t ensure_ws(tidal_ctx* ctx, size_t bytes) {
     return TIDAL_OK;
 }
 
-// State layout for a capacity of R rows: counters | cursor | done | thr_max | tile_ctr sets, each
+// State layout for a capacity of R rows: counters | cursor | done | thr_max | side counters | side cursors |
+// tile_ctr sets, each
 // [R][CTR_STRIDE], then hist[R][TK_BINS]. Consecutive attention launches rotate through the sets of
 // pool cursors, so that a launch may use its set before its predecessor has finished with another.
 // Every counter has a 128-byte line of its own: hundreds of warps hit them at once, and atomics to one
@@ -206,8 +214,10 @@ inline int* state_counters(const tidal_ctx* c) { return (int*)c->state; }
 inline int* state_cursor(const tidal_ctx* c) { return (int*)c->state + (size_t)CTR_STRIDE * c->state_rows; }
 inline int* state_done(const tidal_ctx* c) { return (int*)c->state + 2 * (size_t)CTR_STRIDE * c->state_rows; }
 inline unsigned* state_thr_max(const tidal_ctx* c) { return (unsigned*)c->state + 3 * (size_t)CTR_STRIDE * c->state_rows; }
-inline int* state_tile_ctr(const tidal_ctx* c) { return (int*)c->state + 4 * (size_t)CTR_STRIDE * c->state_rows; }
-inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + (4 + CURSOR_SETS) * (size_t)CTR_STRIDE * c->state_rows; }
+inline int* state_side_counters(const tidal_ctx* c) { return (int*)c->state + 4 * (size_t)CTR_STRIDE * c->state_rows; }
+inline int* state_side_cursors(const tidal_ctx* c) { return (int*)c->state + 5 * (size_t)CTR_STRIDE * c->state_rows; }
+inline int* state_tile_ctr(const tidal_ctx* c) { return (int*)c->state + 6 * (size_t)CTR_STRIDE * c->state_rows; }
+inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + (6 + CURSOR_SETS) * (size_t)CTR_STRIDE * c->state_rows; }
 
 tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     if (ctx->state_rows >= rows) return TIDAL_OK;
@@ -215,7 +225,7 @@ tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     drop_graphs(ctx);
     if (ctx->state) { cudaDeviceSynchronize(); cudaFree(ctx->state); ctx->state = nullptr; ctx->state_rows = 0; }
     const int cap = (int)align_up((size_t)rows, 64);
-    const size_t bytes = (size_t)cap * ((4 + CURSOR_SETS) * CTR_STRIDE + TK_BINS) * sizeof(int);
+    const size_t bytes = (size_t)cap * ((6 + CURSOR_SETS) * CTR_STRIDE + TK_BINS) * sizeof(int);
     void* p = nullptr;
     if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TIDAL_ERR_NOMEM; }
     // on a stream of its own, so that nothing here is the legacy stream's business, and waited for
@@ -309,7 +319,11 @@ tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, int full_gri
 // group sums directly (one row per KV head; histogram fused when a set belongs to one KV head).
 // With one sequence, one set per query head and enough scores per set, the attention kernel compacts
 // candidates instead (no histogram) and a single CTA per head finishes the selection on them.
-struct SelectPlan { bool agg, fuse, compact; int rows; };
+struct SelectPlan { bool agg, fuse, compact, split; int rows; };
+constexpr int SCORE_NW = 16, SCORE_STAGES = 3;     // key rows only: 4 KB per tile, six slots per warp
+constexpr int VALUE_NW = 8, VALUE_STAGES = 3;     // value rows + logits: two CTAs per SM beside the sparse layers'
+constexpr size_t SCORE_SMEM = (size_t)SCORE_NW * SCORE_STAGES * TILE_BYTES + HIST_SMEM + 1024;
+constexpr size_t VALUE_SMEM = (size_t)VALUE_NW * VALUE_STAGES * (TILE_BYTES + 512) + 1024;
 constexpr int COMPACT_LIST_SMEM = 12288;      // candidates the compacting top-k keeps in shared memory
 
 int dense_grid(const tidal_ctx* ctx, const tidal_kv_t* kv) {
@@ -326,7 +340,15 @@ SelectPlan select_plan(const tidal_ctx* ctx, const tidal_kv_t* kv, int Hi, int k
                 kv->num_q_heads / kv->num_kv_heads <= CAND_COLS && 6LL * k <= kv->max_ctx_len &&
                 pooled_splits(kv, kv->num_kv_heads, dense_grid(ctx, kv)) > 0;
     if (s.compact) s.fuse = false;
+    s.split = false;
     return s;
+}
+
+// Inside a step a selection layer can run as two passes (split_select_kernels.cuh) when it has one
+// sequence, per-head scores with the fused histogram, a bf16 cache and fp32 outputs.
+bool can_split(const tidal_ctx* ctx, const tidal_kv_t* kv, const SelectPlan& sp) {
+    return ctx->split_select && ctx->layer_overlap && !ctx->out_bf16 && kv->kv_dtype == TIDAL_KV_BF16 && kv->batch == 1 &&
+           !sp.agg && sp.fuse && !sp.compact && pooled_splits(kv, kv->num_kv_heads, dense_grid(ctx, kv)) > 0;
 }
 
 // hist != nullptr: the kernel also accumulates the per-head histogram the top-k needs.
@@ -372,6 +394,76 @@ tidal_status_t run_dense(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, fl
     }
     if (scores) return launch_attn<MODE_SELECT, DENSE_NW, DENSE_STAGES>(ctx, a, grid, std::min(ctx->dense_slots, GRID_MAX), st);
     return launch_attn<MODE_FULL, DENSE_NW, DENSE_STAGES>(ctx, a, grid, std::min(ctx->dense_slots, GRID_MAX), st);
+}
+
+// The context's second stream and the two events that fork and join it (created on first use).
+tidal_status_t ensure_side_stream(tidal_ctx* ctx) {
+    if (ctx->side) return TIDAL_OK;
+    if (cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        return TIDAL_ERR_CUDA;
+    }
+    return TIDAL_OK;
+}
+
+// Pass 1 of a split selection layer on the caller's stream: logits, histogram, softmax statistics.
+tidal_status_t run_score_pass(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, float* out, float* scores,
+                              long long score_stride, Dep dep, bool scores_free, const WsLayout& w, cudaStream_t st) {
+    AttnParams a;
+    fill_common(a, ctx, kv, q, out, w);
+    const int grid = dense_grid(ctx, kv);
+    a.splits_per_item = pooled_splits(kv, kv->num_kv_heads, grid);
+    a.scores = scores;
+    a.score_stride = score_stride;
+    a.hist = state_hist(ctx);
+    a.ml_final = (float2*)((char*)ctx->ws + w.ml_final);
+    // the kernel writes scores while it streams: ahead of its wait only if nobody can still be reading them
+    a.wait_first = !(dep == DEP_LATE && scores_free);
+    a.wait_late = !a.wait_first;
+    a.pdl = 1;
+    ctx->cursor_set = (ctx->cursor_set + 1) % CURSOR_SETS;
+    a.tile_ctr = state_tile_ctr(ctx) + (size_t)ctx->cursor_set * CTR_STRIDE * ctx->state_rows;
+    a.trigger_early = a.wait_late && (long long)(CURSOR_SETS - 1) * grid >= std::min(ctx->dense_slots, GRID_MAX);
+    if (a.wait_late && !a.trigger_early) { a.wait_late = 0; a.wait_first = 1; }
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(SCORE_NW * 32, 1, 1);
+    cfg.dynamicSmemBytes = SCORE_SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    ctx->launches++;
+    return cudaLaunchKernelEx(&cfg, score_pass_kernel<SCORE_NW, SCORE_STAGES>, a) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+}
+
+// Pass 2 on the context's second stream: it starts when pass 1 is complete and runs beside whatever
+// the caller's stream does next. It owns a cursor and a counter array of its own and no other scratch.
+tidal_status_t run_value_pass(tidal_ctx* ctx, const tidal_kv_t* kv, float* out, const float* scores,
+                              long long score_stride, const WsLayout& w, cudaStream_t st) {
+    AttnParams a;
+    fill_common(a, ctx, kv, nullptr, out, w);
+    a.scores = const_cast<float*>(scores);
+    a.score_stride = score_stride;
+    a.ml_final = (float2*)((char*)ctx->ws + w.ml_final);
+    a.counters = state_side_counters(ctx);
+    a.tile_ctr = state_side_cursors(ctx);
+    a.pdl = 0;
+    // about two thirds of the slots: it shares the GPU with the top-k and the first sparse layers
+    const int per_item = std::max(2, 2 * std::min(ctx->sparse_slots, GRID_MAX) / (3 * kv->num_kv_heads));
+    const int grid = per_item * kv->num_kv_heads;
+    a.splits_per_item = per_item;
+    if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
+        return TIDAL_ERR_CUDA;
+    value_pass_kernel<VALUE_NW, VALUE_STAGES><<<grid, VALUE_NW * 32, VALUE_SMEM, ctx->side>>>(a);
+    ctx->launches++;
+    if (cudaGetLastError() != cudaSuccess) return TIDAL_ERR_CUDA;
+    return cudaEventRecord(ctx->ev_join, ctx->side) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }
 
 // `rows`: score rows per sequence (query heads, or KV heads when the attention kernel stored group sums).
@@ -504,7 +596,7 @@ struct KeyBuilder {
 void step_key(KeyBuilder& kb, const tidal_ctx* ctx, int tag, int32_t num_layers, const uint8_t* schedule,
                      const tidal_kv_t* kvs, int32_t k, int32_t granularity, int host_layers) {
     kb.add(tag); kb.add(num_layers); kb.add(k); kb.add(granularity); kb.add(host_layers);
-    kb.add(ctx->ws); kb.add(ctx->state); kb.add(ctx->out_bf16); kb.add(ctx->attend_newest); kb.add(ctx->layer_overlap); kb.add(ctx->select_margin);
+    kb.add(ctx->ws); kb.add(ctx->state); kb.add(ctx->out_bf16); kb.add(ctx->attend_newest); kb.add(ctx->layer_overlap); kb.add(ctx->select_margin); kb.add(ctx->split_select);
     kb.add_raw(schedule, (size_t)num_layers);
     for (int i = 0; i < num_layers; ++i) {
         // field by field: the struct has padding whose bytes are not the caller's to define
@@ -599,11 +691,14 @@ tidal_status_t tidal_create(tidal_ctx_t** out, int device, size_t workspace_byte
     const int e0 = resident_ctas(attn_kernel<MODE_FULL, DENSE_NW8, DENSE_STAGES8, false, false, true>, DENSE_NW8 * 32, attn_smem<MODE_FULL, DENSE_NW8, DENSE_STAGES8, true>(), ctx->sm_count);
     const int e1 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW8, DENSE_STAGES8, false, false, true>, DENSE_NW8 * 32, attn_smem<MODE_SELECT, DENSE_NW8, DENSE_STAGES8, true>(), ctx->sm_count);
     const int e2 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW8, SPARSE_STAGES8, false, false, true>, SPARSE_NW8 * 32, attn_smem<MODE_SPARSE, SPARSE_NW8, SPARSE_STAGES8, true>(), ctx->sm_count);
+    const bool split_ok =
+        cudaFuncSetAttribute(score_pass_kernel<SCORE_NW, SCORE_STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCORE_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(value_pass_kernel<VALUE_NW, VALUE_STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VALUE_SMEM) == cudaSuccess;
     const size_t topk_smem = 2 * (size_t)(MAX_CTX / 32) * sizeof(unsigned) + 8192 * sizeof(uint2);
     const bool topk_ok = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topk_smem) == cudaSuccess;
     const size_t compact_smem = 2 * ((size_t)(MAX_CTX / 32) + 1) * sizeof(unsigned) + (size_t)COMPACT_LIST_SMEM * sizeof(uint2);
     const bool compact_ok = cudaFuncSetAttribute(topk_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)compact_smem) == cudaSuccess;
-    if (d0 <= 0 || d1 <= 0 || d2 < d1 || s0 <= 0 || s1 < s0 || e0 < d0 || e1 < d1 || e2 < s0 || !topk_ok || !compact_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
+    if (d0 <= 0 || d1 <= 0 || d2 < d1 || s0 <= 0 || s1 < s0 || e0 < d0 || e1 < d1 || e2 < s0 || !topk_ok || !compact_ok || !split_ok) { cudaGetLastError(); delete ctx; return TIDAL_ERR_CUDA; }
     ctx->dense_slots = std::min(d0, d1);
     ctx->sparse_slots = s0;
     if (cudaMalloc((void**)&ctx->status, 256) != cudaSuccess || cudaMemset(ctx->status, 0, 256) != cudaSuccess) {
@@ -622,6 +717,9 @@ tidal_status_t tidal_destroy(tidal_ctx_t* ctx) {
     cudaSetDevice(ctx->device);
     cudaDeviceSynchronize();
     drop_graphs(ctx);
+    if (ctx->side) cudaStreamDestroy(ctx->side);
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     if (ctx->ws) cudaFree(ctx->ws);
     if (ctx->state) cudaFree(ctx->state);
     if (ctx->status) cudaFree(ctx->status);
@@ -756,6 +854,7 @@ static tidal_status_t decode_step_enqueue(tidal_ctx_t* ctx, int32_t num_layers, 
                                           int host_layers, cudaStream_t st) {
     const int Hi = hi_of(&kvs[0], granularity);
     tidal_status_t rc = TIDAL_OK;
+    bool side_pending = false;                  // a value pass is in flight on the second stream
     for (int i = 0; i < num_layers; ++i) {
         const tidal_kv_t* kv = &kvs[i];
         const WsLayout w = layout_ws(kv, k, host_layers);
@@ -774,7 +873,16 @@ static tidal_status_t decode_step_enqueue(tidal_ctx_t* ctx, int32_t num_layers, 
             // sparse layer ran in between, its first kernel waited for that top-k before it let anything
             // else start, so nobody reads the buffer any more; right after another selection layer, wait.
             const bool scores_free = i > 0 && schedule[i - 1] != TIDAL_LAYER_SELECT;
-            rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, sp.fuse, dep, w, st, sp.agg, sp.compact ? k : 0, scores_free);
+            if (can_split(ctx, kv, sp) && ensure_side_stream(ctx) == TIDAL_OK) {
+                // key pass -> (value pass on the second stream) | top-k -> the layers that follow. A value
+                // pass still in flight reads the score buffer and the statistics this key pass overwrites.
+                if (side_pending) { if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return TIDAL_ERR_CUDA; side_pending = false; }
+                rc = run_score_pass(ctx, kv, qs[i], outs[i], scores, w.score_stride, dep, scores_free, w, st);
+                if (rc == TIDAL_OK) rc = run_value_pass(ctx, kv, outs[i], scores, w.score_stride, w, st);
+                side_pending = rc == TIDAL_OK;
+            } else {
+                rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, sp.fuse, dep, w, st, sp.agg, sp.compact ? k : 0, scores_free);
+            }
             if (rc == TIDAL_OK) rc = run_topk(ctx, kv, scores, w.score_stride, k, sp.rows, Hi, sp.fuse, idx, idx_count, w, st, sp.compact);
         } else {
             const bool fresh_idx = i == 0 || schedule[i - 1] == TIDAL_LAYER_SELECT;
@@ -786,6 +894,8 @@ static tidal_status_t decode_step_enqueue(tidal_ctx_t* ctx, int32_t num_layers, 
         }
         if (rc != TIDAL_OK) return rc;
     }
+    // the step is complete on the caller's stream only when the second stream's work is
+    if (side_pending && cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return TIDAL_ERR_CUDA;
     return TIDAL_OK;
 }
 
@@ -922,9 +1032,12 @@ tidal_status_t tidal_decode_step_host(tidal_ctx_t* ctx, int32_t num_layers, cons
     if (q_alias && ((uintptr_t)q_alias & 15)) q_alias = nullptr;      // query rows are read as 16-byte pieces
     const void* qs[1024];
     float* outs[1024];
+    // (a selection layer may run as two passes whose second adds to the output with atomics: its rows
+    // stay in device memory and are copied out afterwards)
     for (int i = 0; i < num_layers; ++i) {
+        const bool direct = out_alias && schedule[i] != TIDAL_LAYER_SELECT;
         qs[i] = (q_alias ? q_alias : qd) + (size_t)i * rows * HEAD_DIM * 2;
-        outs[i] = (float*)((out_alias ? out_alias : (char*)od) + (size_t)i * rows * HEAD_DIM * out_elem);
+        outs[i] = (float*)((direct ? out_alias : (char*)od) + (size_t)i * rows * HEAD_DIM * out_elem);
     }
     if ((rc = decode_step_prepare(ctx, num_layers, schedule, kv_per_layer, qs, outs, k, granularity, num_layers)) != TIDAL_OK)
         return rc;
@@ -936,6 +1049,13 @@ tidal_status_t tidal_decode_step_host(tidal_ctx_t* ctx, int32_t num_layers, cons
         if (r != TIDAL_OK) return r;
         if (!out_alias && cudaMemcpyAsync(out_host, od, (size_t)num_layers * rows * HEAD_DIM * out_elem, cudaMemcpyDeviceToHost, st) != cudaSuccess)
             return TIDAL_ERR_CUDA;
+        if (out_alias) {
+            const size_t layer_bytes = rows * HEAD_DIM * out_elem;
+            for (int i = 0; i < num_layers; ++i)
+                if (schedule[i] == TIDAL_LAYER_SELECT &&
+                    cudaMemcpyAsync((char*)out_host + i * layer_bytes, (char*)od + i * layer_bytes, layer_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+                    return TIDAL_ERR_CUDA;
+        }
         return TIDAL_OK;
     };
     // The copies can be recorded with the layers only when both host buffers are page-locked.
