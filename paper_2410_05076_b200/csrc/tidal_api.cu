@@ -320,8 +320,8 @@ tidal_status_t launch_attn(tidal_ctx* ctx, AttnParams& a, int grid, int full_gri
 // With one sequence, one set per query head and enough scores per set, the attention kernel compacts
 // candidates instead (no histogram) and a single CTA per head finishes the selection on them.
 struct SelectPlan { bool agg, fuse, compact, split; int rows; };
-constexpr int SCORE_NW = 16, SCORE_STAGES = 3;     // key rows only: 4 KB per tile, six slots per warp
-constexpr int VALUE_NW = 8, VALUE_STAGES = 3;     // value rows + logits: two CTAs per SM beside the sparse layers'
+constexpr int SCORE_NW = 16, SCORE_STAGES = 3;     // key rows only, 4 KB per tile: sixteen warps keep enough tiles in flight
+constexpr int VALUE_NW = 8, VALUE_STAGES = 3;      // value rows + logits, 4.5 KB per tile: two CTAs per SM, also beside a sparse layer's CTA
 constexpr size_t SCORE_SMEM = (size_t)SCORE_NW * SCORE_STAGES * TILE_BYTES + HIST_SMEM + 1024;
 constexpr size_t VALUE_SMEM = (size_t)VALUE_NW * VALUE_STAGES * (TILE_BYTES + 512) + 1024;
 constexpr int COMPACT_LIST_SMEM = 12288;      // candidates the compacting top-k keeps in shared memory
@@ -454,8 +454,9 @@ tidal_status_t run_value_pass(tidal_ctx* ctx, const tidal_kv_t* kv, float* out, 
     a.counters = state_side_counters(ctx);
     a.tile_ctr = state_side_cursors(ctx);
     a.pdl = 0;
-    // about two thirds of the slots: it shares the GPU with the top-k and the first sparse layers
-    const int per_item = std::max(2, 2 * std::min(ctx->sparse_slots, GRID_MAX) / (3 * kv->num_kv_heads));
+    // most of the slots (its CTAs are the size of the sparse layers'): it shares the GPU with the top-k and the
+    // first sparse layers; between 25 % and 100 % of the slots the step time moved by less than 2 %
+    const int per_item = std::max(2, 85 * std::min(ctx->sparse_slots, GRID_MAX) / (100 * kv->num_kv_heads));
     const int grid = per_item * kv->num_kv_heads;
     a.splits_per_item = per_item;
     if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)

@@ -1119,3 +1119,39 @@ def test_overlapping_layers_repeatably_equal_the_non_overlapped_step(td, shape):
             for o, r in zip(outs, ref):
                 assert torch.allclose(o, r, rtol=0, atol=2e-3), it
     assert td.device_status() == binding.OK
+
+
+@pytest.mark.parametrize("layout", ["hnd_interleaved", "nhd_separate", "paged"])
+@pytest.mark.parametrize("Hq,Hkv,N,k", [(32, 8, 20011, 1024), (16, 16, 24000, 900), (16, 2, 40001, 3000), (8, 4, 70000, 2048)])
+def test_two_pass_selection_layers_match_the_oracle(td, layout, Hq, Hkv, N, k):
+    """Inside a step (one sequence, per-head sets) a selection layer runs as a key pass and a value pass on
+    two streams. Its output, its token sets and the sparse layers after it against the oracle, for groups of
+    1, 2, 4 and 8, context lengths with a ragged last tile, all layouts; and against the fused kernel that the
+    single-layer call uses. Two selection layers in a row share the score buffer: the second key pass must
+    wait for the first value pass."""
+    sched = [0, 1, 1, 2, 2]
+    w = wl(1, Hq, Hkv, N, k, planted=8, seed=97, layers=len(sched))
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    if layout == "paged":
+        pt, total = synth.make_page_table(w, extra_pages=3)
+        lays = [synth.make_layer(w, i, DEV, layout="paged", q=qs[i], page_table=pt, num_pages=total) for i in range(len(sched))]
+    else:
+        lays = [synth.make_layer(w, i, DEV, layout=layout, q=qs[i]) for i in range(len(sched))]
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        outs, idx, cnt = td.decode_step(sched, lays, qs, w.k)
+        side.synchronize()
+    for i in (1, 2):
+        okv, qb = util.oracle_kv(lays[i]), synth.bits(qs[i])
+        ref, sc = oracle.full_attn(okv, qb, want_scores=True)
+        util.check_out(outs[i].cpu().numpy(), ref, f"two-pass layer {i}")
+        fused, fidx, _ = td.select_attn(lays[i], qs[i], w.k)
+        assert torch.allclose(outs[i], fused, rtol=0, atol=1e-3)
+        if i == 2:
+            assert torch.equal(idx, fidx)                  # same scores, same sets as the fused kernel
+            for h in range(0, Hq, max(1, Hq // 4)):
+                util.check_idx_row(idx.cpu().numpy()[0, h], sc[0, h], w.k, N, f"two-pass idx[{h}]")
+    for i in (3, 4):
+        ref = oracle.sparse_attn(util.oracle_kv(lays[i]), synth.bits(qs[i]), idx.cpu().numpy(), cnt.cpu().numpy())
+        util.check_out(outs[i].cpu().numpy(), ref, f"sparse layer {i} after a two-pass selection")
+    assert td.device_status() == binding.OK
