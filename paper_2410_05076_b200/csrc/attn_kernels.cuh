@@ -79,7 +79,8 @@ struct AttnParams {
     const int* idx;            // MODE_SPARSE: [B, Hi, k]
     const int* idx_count;      // MODE_SPARSE: [B] or null
     int budget, Hi;            // MODE_SPARSE: entries per index row, index heads
-    float2* ml_final;          // split selection layer: [Hq] final (max in base 2, sum) of every head's softmax
+    unsigned* split_max;       // two-pass selection layer: [Hq] key of every head's largest logit (0 between layers)
+    float* split_sum;          // ... and [Hq] the sum of its softmax weights relative to that logit (0 between layers)
     float* part_o;             // [B*Hq, max_splits, 128] un-normalised partial outputs
     float2* part_ml;           // [B*Hq, max_splits] (running max in base 2, sum)
     int* counters;             // one per (sequence, item), zero between launches

@@ -5,12 +5,13 @@
 // together and the top-k can only start when all of it is done; the sparse layers after it then wait
 // for the top-k, and for those 20 microseconds the memory system idles. Here the layer is split:
 //
-//   score_pass_kernel  streams the KEY rows only: logits, their histogram (for the top-k), and the
-//                      softmax statistics (max M and sum L per head); the last CTA of a KV head publishes
-//                      (M, L) and clears the layer's output rows.
-//   value_pass_kernel  streams the VALUE rows only: softmax weights come from the stored logits and the
-//                      final M, so every partial result has the same scale and CTAs simply add their
-//                      part of sum_j p_j v_j / L to the output with atomics: no partial buffers, no combine.
+//   score_pass_kernel  streams the KEY rows only: logits, their histogram (for the top-k) and the largest
+//                      logit M of every head (one atomicMax per CTA and head); the first CTA of a KV head
+//                      clears the layer's output rows. No partial results, no combine.
+//   value_pass_kernel  streams the VALUE rows only: softmax weights exp(s - M) come from the stored logits
+//                      and the final M, so every partial result has the same scale and CTAs simply add
+//                      their part of sum_j p_j v_j and of sum_j p_j to the output row and to the head's sum
+//                      with atomics; the last CTA of a KV head to finish divides the rows by the sums.
 //
 // The step driver launches the value pass on a second stream, so that it runs beside the top-k and the
 // first sparse layers that follow: the top-k's latency chain and the ramp of the sparse chain are filled
@@ -53,17 +54,17 @@ struct PoolWalk {
 };
 
 // ---- pass 1: logits, histogram, softmax statistics -------------------------------------------------------
-// Uses of AttnParams: q, k, strides, page table, ctx_lens, scale(s), scores / score_stride, hist / hist_shift,
-// part_ml / max_splits / counters / tile_ctr / ctr_stride (the main stream's scratch), ml_final, out (cleared),
-// pdl / wait_first / wait_late / trigger_early, status. batch must be 1, splits_per_item > 0.
+// Uses of AttnParams: q, k, strides, page table, ctx_lens, scale, scores / score_stride, hist / hist_shift,
+// tile_ctr / ctr_stride (a cursor set of the main stream's rotation), split_max (per head: the order-preserving
+// key of the largest logit, 0 = none yet), out (cleared), pdl / wait_first / wait_late / trigger_early, status.
+// batch must be 1, splits_per_item > 0.
 template <int NW, int STAGES>
 __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams p) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     __shared__ uint32_t s_vmask[NW][STAGES];
     __shared__ int s_posbase[NW][STAGES];
-    __shared__ float2 s_ml[NW][8];
-    __shared__ int s_is_last;
+    __shared__ float s_max[NW][8];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = lane >> 2, tig = lane & 3;
@@ -122,10 +123,15 @@ __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams
         }
         const int nvalid = ok ? max(0, min(TILE, N - pos0)) : 0;
         const __nv_bfloat16* ksrc = p.k + off;
+        if (nvalid == TILE) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const bool rv = rhalf + 2 * i < nvalid;
-            cp_async16_hint(ks + kdst + i * 512, rv ? ksrc + i * two_rows : p.k, rv ? 16 : 0, kv_policy);
+            for (int i = 0; i < 8; ++i) cp_async16_full_hint(ks + kdst + i * 512, ksrc + i * two_rows, kv_policy);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const bool rv = rhalf + 2 * i < nvalid;
+                cp_async16_hint(ks + kdst + i * 512, rv ? ksrc + i * two_rows : p.k, rv ? 16 : 0, kv_policy);
+            }
         }
         if (lane == 0) { s_vmask[warp][stage] = (1u << nvalid) - 1u; s_posbase[warp][stage] = pos0; }
     };
@@ -149,7 +155,7 @@ __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams
             qf[j][0] = on ? t.x : 0u; qf[j][1] = on ? t.y : 0u; qf[j][2] = on ? t.z : 0u; qf[j][3] = on ? t.w : 0u;
         }
     }
-    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;      // heads 2tig, 2tig+1: max (all lanes of a tig agree), this lane's sum
+    float m0 = -INFINITY, m1 = -INFINITY;              // largest logit this lane has seen of heads 2tig, 2tig+1
     const bool ring_full = commits == STAGES;
     while (commits < STAGES - 1) {
         if (tA >= 0) { issue(issued % STAGES); ++issued; }
@@ -212,26 +218,9 @@ __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams
                 if (v1) atomicAdd(h1 + (score_key_bits(f3) >> p.hist_shift), 1u);
             }
         }
-        // softmax statistics in base 2. The value pass recomputes the weights from the STORED logits
-        // (f * log2 e), so the statistics are taken from exactly those numbers.
-        const float t0 = v0 ? f0 * LOG2E : -INFINITY, t1 = v0 ? f1 * LOG2E : -INFINITY;
-        const float t2 = v1 ? f2 * LOG2E : -INFINITY, t3 = v1 ? f3 * LOG2E : -INFINITY;
-        float mx0 = fmaxf(t0, t2), mx1 = fmaxf(t1, t3);
-        if (__any_sync(0xffffffffu, (mx0 > m0) || (mx1 > m1))) {
-#pragma unroll
-            for (int sh = 4; sh <= 16; sh <<= 1) {
-                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, sh));
-                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
-            }
-            const float g0 = fmaxf(m0, mx0), g1 = fmaxf(m1, mx1);
-            l0 *= (g0 == -INFINITY) ? 1.f : fast_exp2(m0 - g0);
-            l1 *= (g1 == -INFINITY) ? 1.f : fast_exp2(m1 - g1);
-            m0 = g0;
-            m1 = g1;
-        }
-        const float ms0 = (m0 == -INFINITY) ? 0.f : m0, ms1 = (m1 == -INFINITY) ? 0.f : m1;
-        l0 += fast_exp2(t0 - ms0) + fast_exp2(t2 - ms0);
-        l1 += fast_exp2(t1 - ms1) + fast_exp2(t3 - ms1);
+        // the largest stored logit of each head: the value pass takes its softmax weights relative to it
+        if (v0) { m0 = fmaxf(m0, f0); m1 = fmaxf(m1, f1); }
+        if (v1) { m0 = fmaxf(m0, f2); m1 = fmaxf(m1, f3); }
     }
     cp_async_wait<0>();
     __syncwarp();
@@ -248,69 +237,36 @@ __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams
             if (w) atomicAdd(p.hist + (long long)(head0 + i / nb) * HIST_BINS + (i % nb), w);
         }
     }
-    // ---- (max, sum) of this CTA, then of the KV head --------------------------------------------------------
+    // ---- the largest logit of this CTA per head, then of the head: one atomicMax on its key -------------
 #pragma unroll
     for (int sh = 4; sh <= 16; sh <<= 1) {
-        l0 += __shfl_xor_sync(0xffffffffu, l0, sh);
-        l1 += __shfl_xor_sync(0xffffffffu, l1, sh);
+        m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, sh));
+        m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, sh));
     }
-    if (gid == 0) {
-        s_ml[warp][2 * tig] = make_float2(m0, l0);
-        s_ml[warp][2 * tig + 1] = make_float2(m1, l1);
-    }
+    if (gid == 0) { s_max[warp][2 * tig] = m0; s_max[warp][2 * tig + 1] = m1; }
     __syncthreads();
-    const int nsplits = item_ctas;
     if (threadIdx.x < ncols) {
-        const int col = threadIdx.x;
         float M = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < NW; ++w) M = fmaxf(M, s_ml[w][col].x);
-        float L = 0.f;
-        if (M != -INFINITY)
-#pragma unroll
-            for (int w = 0; w < NW; ++w) {
-                const float2 ml = s_ml[w][col];
-                L += ml.y * ((ml.x == -INFINITY) ? 0.f : fast_exp2(ml.x - M));
-            }
-        if (part < p.max_splits) p.part_ml[(long long)(head0 + col) * p.max_splits + part] = make_float2(M, L);
-        else atomicOr(p.status, STATUS_SPLIT_OVERFLOW);
+        for (int w = 0; w < NW; ++w) M = fmaxf(M, s_max[w][threadIdx.x]);
+        if (M != -INFINITY) atomicMax(p.split_max + head0 + threadIdx.x, score_key_bits(M));
     }
-    __syncthreads();
-    int* ctr = p.counters + (long long)g * p.ctr_stride;
+    // the value pass adds its parts to the output rows: they start at zero (this pass ends before it starts)
+    if (part == 0)
+        for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) p.out[(long long)head0 * HEAD_DIM + e] = 0.f;
+    // the pool cursor of this launch's set is cleared by the item's last CTA to get here
     if (threadIdx.x == 0) {
+        int* ctr = p.counters + (long long)g * p.ctr_stride;
         int old;
         asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;\n" : "=r"(old) : "l"(ctr) : "memory");
-        s_is_last = (old == nsplits - 1);
-    }
-    __syncthreads();
-    if (s_is_last) {
-        const int ns = min(nsplits, p.max_splits);
-        if (warp < ncols) {
-            const int col = warp;
-            const long long pr = (long long)(head0 + col) * p.max_splits;
-            float M = -INFINITY;
-            for (int sidx = lane; sidx < ns; sidx += 32) M = fmaxf(M, __ldcg(&p.part_ml[pr + sidx].x));
-#pragma unroll
-            for (int sh = 16; sh >= 1; sh >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sh));
-            float L = 0.f;
-            for (int sidx = lane; sidx < ns; sidx += 32) {
-                const float2 ml = __ldcg(&p.part_ml[pr + sidx]);
-                L += ml.y * ((ml.x == -INFINITY || M == -INFINITY) ? 0.f : fast_exp2(ml.x - M));
-            }
-#pragma unroll
-            for (int sh = 16; sh >= 1; sh >>= 1) L += __shfl_xor_sync(0xffffffffu, L, sh);
-            if (lane == 0) p.ml_final[head0 + col] = make_float2(M, L);
-        }
-        // the value pass adds its parts to the output rows: they start at zero
-        for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) p.out[(long long)head0 * HEAD_DIM + e] = 0.f;
-        if (threadIdx.x == NW * 32 - 1) { *pool = 0; __threadfence(); }
-        if (threadIdx.x == 0) *ctr = 0;
+        if (old == item_ctas - 1) { *ctr = 0; *pool = 0; __threadfence(); }
     }
 }
 
 // ---- pass 2: sum_j softmax_j v_j from the stored logits ------------------------------------------------------
-// Uses of AttnParams: v, strides, page table, ctx_lens, scores / score_stride, ml_final, out (+= with atomics),
-// tile_ctr / ctr_stride (a cursor set of its own: it runs beside the main stream's kernels), status.
+// Uses of AttnParams: v, strides, page table, ctx_lens, scores / score_stride, split_max, split_sum (per head,
+// zero between launches), out (+= with atomics, then divided), counters / tile_ctr / ctr_stride (arrays of its
+// own: it runs beside the main stream's kernels), status.
 template <int NW, int STAGES>
 __global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams p) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -374,10 +330,15 @@ __global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams
         if (lane == 0) s_vmask[warp][stage] = (1u << nvalid) - 1u;
     };
 
-    // the final statistics of this lane's two heads
+    // the largest logit of this lane's two heads, in base-2 units (key 0: the head has no token at all)
     float M0 = -INFINITY, M1 = -INFINITY;
-    if (2 * tig < ncols) M0 = __ldg(&p.ml_final[head0 + 2 * tig].x);
-    if (2 * tig + 1 < ncols) M1 = __ldg(&p.ml_final[head0 + 2 * tig + 1].x);
+    {
+        const uint32_t k0 = (2 * tig < ncols) ? __ldcg(p.split_max + head0 + 2 * tig) : 0u;
+        const uint32_t k1 = (2 * tig + 1 < ncols) ? __ldcg(p.split_max + head0 + 2 * tig + 1) : 0u;
+        if (k0) M0 = __uint_as_float((k0 & 0x80000000u) ? (k0 & 0x7fffffffu) : ~k0) * LOG2E;
+        if (k1) M1 = __uint_as_float((k1 & 0x80000000u) ? (k1 & 0x7fffffffu) : ~k1) * LOG2E;
+    }
+    float l0 = 0.f, l1 = 0.f;                          // this lane's share of sum_j p_j
     float o[8][4];
 #pragma unroll
     for (int t = 0; t < 8; ++t) { o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f; }
@@ -411,6 +372,8 @@ __global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams
         const bool h0 = 2 * tig < ncols && M0 != -INFINITY, h1 = 2 * tig + 1 < ncols && M1 != -INFINITY;
         const float p0 = (v0 && h0) ? fast_exp2(f0 * LOG2E - M0) : 0.f, p1 = (v0 && h1) ? fast_exp2(f1 * LOG2E - M1) : 0.f;
         const float p2 = (v1 && h0) ? fast_exp2(f2 * LOG2E - M0) : 0.f, p3 = (v1 && h1) ? fast_exp2(f3 * LOG2E - M1) : 0.f;
+        l0 += p0 + p2;
+        l1 += p1 + p3;
         const uint32_t pb0 = movmatrix_trans(pack_bf16(p0, p1));
         const uint32_t pb1 = movmatrix_trans(pack_bf16(p2, p3));
         const int rr = lane & 7, mb = (lane >> 3) & 1;
@@ -423,9 +386,15 @@ __global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams
         }
     }
     cp_async_wait<0>();
+#pragma unroll
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+        l0 += __shfl_xor_sync(0xffffffffu, l0, sh);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, sh);
+    }
     __syncthreads();                                   // all rings drained; reuse the shared memory
-    // ---- sum the warps of this CTA, then add the CTA's part, divided by the head's sum, to the output ---
+    // ---- sum the warps of this CTA and add the CTA's part to the output rows and to the heads' sums ------
     float* mo = reinterpret_cast<float*>(smem);       // [NW][8][128]
+    float* ml = mo + NW * 8 * HEAD_DIM;               // [NW][8]
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
         float* w0 = mo + ((warp * 8 + 2 * tig) * HEAD_DIM);
@@ -435,22 +404,41 @@ __global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams
         w0[16 * t + 8 + gid] = o[t][2];
         w1[16 * t + 8 + gid] = o[t][3];
     }
+    if (gid == 0) { ml[warp * 8 + 2 * tig] = l0; ml[warp * 8 + 2 * tig + 1] = l1; }
     __syncthreads();
     for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) {
         const int col = e >> 7, c = e & 127;
         float O = 0.f;
 #pragma unroll
         for (int w = 0; w < NW; ++w) O += mo[(w * 8 + col) * HEAD_DIM + c];
-        const float L = __ldg(&p.ml_final[head0 + col].y);
-        if (L > 0.f && O != 0.f) atomicAdd(p.out + (long long)(head0 + col) * HEAD_DIM + c, O / L);
+        if (O != 0.f) atomicAdd(p.out + (long long)(head0 + col) * HEAD_DIM + c, O);
     }
-    // the last CTA of this KV head to finish clears the cursor for the next value pass
+    if (threadIdx.x < ncols) {
+        float L = 0.f;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) L += ml[w * 8 + threadIdx.x];
+        if (L != 0.f) atomicAdd(p.split_sum + head0 + threadIdx.x, L);
+    }
+    // ---- the last CTA of this KV head to arrive divides the rows by the sums and cleans up --------------------
+    __shared__ int s_last;
     __syncthreads();
+    int* ctr = p.counters + (long long)g * p.ctr_stride;
     if (threadIdx.x == 0) {
-        int* ctr = p.counters + (long long)g * p.ctr_stride;
         int old;
         asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;\n" : "=r"(old) : "l"(ctr) : "memory");
-        if (old == item_ctas - 1) { *ctr = 0; *pool = 0; }
+        s_last = (old == item_ctas - 1);
+    }
+    __syncthreads();
+    if (s_last) {
+        for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) {
+            float* dst = p.out + (long long)head0 * HEAD_DIM + e;
+            const float L = __ldcg(p.split_sum + head0 + (e >> 7));
+            const float O = __ldcg(dst);
+            *dst = (L > 0.f) ? O / L : 0.f;
+        }
+        __syncthreads();
+        if (threadIdx.x < ncols) { p.split_sum[head0 + threadIdx.x] = 0.f; p.split_max[head0 + threadIdx.x] = 0u; }
+        if (threadIdx.x == 0) { *ctr = 0; *pool = 0; }
     }
 }
 

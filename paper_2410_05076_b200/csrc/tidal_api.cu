@@ -81,7 +81,7 @@ struct tidal_ctx {
 namespace {
 
 struct WsLayout {
-    size_t part_ml, part_o, ml_final, scores, cand, bitmap, idx, idx_count, q_stage, out_stage, total;
+    size_t part_ml, part_o, scores, cand, bitmap, idx, idx_count, q_stage, out_stage, total;
     long long cand_stride, bitmap_stride;
     long long score_stride;
     int max_splits;
@@ -164,7 +164,6 @@ WsLayout layout_ws(const tidal_kv_t* kv, int k, int num_layers_host) {
     w.max_splits = max_splits_for(kv);
     w.part_ml = at;   at += align_up(rows * w.max_splits * sizeof(float2), 256);
     w.part_o = at;    at += align_up(rows * w.max_splits * HEAD_DIM * sizeof(float), 256);
-    w.ml_final = at;  at += align_up(rows * sizeof(float2), 256);
     w.score_stride = (long long)align_up((size_t)kv->max_ctx_len, 16);
     w.scores = at;    at += align_up(rows * (size_t)w.score_stride * sizeof(float), 256);
     w.cand_stride = w.score_stride;
@@ -203,7 +202,7 @@ tidal_status_t ensure_ws(tidal_ctx* ctx, size_t bytes) {
 }
 
 // State layout for a capacity of R rows: counters | cursor | done | thr_max | side counters | side cursors |
-// tile_ctr sets, each
+// split max | split sum | tile_ctr sets, each
 // [R][CTR_STRIDE], then hist[R][TK_BINS]. Consecutive attention launches rotate through the sets of
 // pool cursors, so that a launch may use its set before its predecessor has finished with another.
 // Every counter has a 128-byte line of its own: hundreds of warps hit them at once, and atomics to one
@@ -216,8 +215,10 @@ inline int* state_done(const tidal_ctx* c) { return (int*)c->state + 2 * (size_t
 inline unsigned* state_thr_max(const tidal_ctx* c) { return (unsigned*)c->state + 3 * (size_t)CTR_STRIDE * c->state_rows; }
 inline int* state_side_counters(const tidal_ctx* c) { return (int*)c->state + 4 * (size_t)CTR_STRIDE * c->state_rows; }
 inline int* state_side_cursors(const tidal_ctx* c) { return (int*)c->state + 5 * (size_t)CTR_STRIDE * c->state_rows; }
-inline int* state_tile_ctr(const tidal_ctx* c) { return (int*)c->state + 6 * (size_t)CTR_STRIDE * c->state_rows; }
-inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + (6 + CURSOR_SETS) * (size_t)CTR_STRIDE * c->state_rows; }
+inline unsigned* state_split_max(const tidal_ctx* c) { return (unsigned*)c->state + 6 * (size_t)CTR_STRIDE * c->state_rows; }
+inline float* state_split_sum(const tidal_ctx* c) { return (float*)c->state + 7 * (size_t)CTR_STRIDE * c->state_rows; }
+inline int* state_tile_ctr(const tidal_ctx* c) { return (int*)c->state + 8 * (size_t)CTR_STRIDE * c->state_rows; }
+inline unsigned* state_hist(const tidal_ctx* c) { return (unsigned*)c->state + (8 + CURSOR_SETS) * (size_t)CTR_STRIDE * c->state_rows; }
 
 tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     if (ctx->state_rows >= rows) return TIDAL_OK;
@@ -225,7 +226,7 @@ tidal_status_t ensure_state(tidal_ctx* ctx, int rows) {
     drop_graphs(ctx);
     if (ctx->state) { cudaDeviceSynchronize(); cudaFree(ctx->state); ctx->state = nullptr; ctx->state_rows = 0; }
     const int cap = (int)align_up((size_t)rows, 64);
-    const size_t bytes = (size_t)cap * ((6 + CURSOR_SETS) * CTR_STRIDE + TK_BINS) * sizeof(int);
+    const size_t bytes = (size_t)cap * ((8 + CURSOR_SETS) * CTR_STRIDE + TK_BINS) * sizeof(int);
     void* p = nullptr;
     if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TIDAL_ERR_NOMEM; }
     // on a stream of its own, so that nothing here is the legacy stream's business, and waited for
@@ -418,7 +419,7 @@ tidal_status_t run_score_pass(tidal_ctx* ctx, const tidal_kv_t* kv, const void* 
     a.scores = scores;
     a.score_stride = score_stride;
     a.hist = state_hist(ctx);
-    a.ml_final = (float2*)((char*)ctx->ws + w.ml_final);
+    a.split_max = state_split_max(ctx);
     // the kernel writes scores while it streams: ahead of its wait only if nobody can still be reading them
     a.wait_first = !(dep == DEP_LATE && scores_free);
     a.wait_late = !a.wait_first;
@@ -450,7 +451,8 @@ tidal_status_t run_value_pass(tidal_ctx* ctx, const tidal_kv_t* kv, float* out, 
     fill_common(a, ctx, kv, nullptr, out, w);
     a.scores = const_cast<float*>(scores);
     a.score_stride = score_stride;
-    a.ml_final = (float2*)((char*)ctx->ws + w.ml_final);
+    a.split_max = state_split_max(ctx);
+    a.split_sum = state_split_sum(ctx);
     a.counters = state_side_counters(ctx);
     a.tile_ctr = state_side_cursors(ctx);
     a.pdl = 0;
