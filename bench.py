@@ -235,10 +235,16 @@ def profile_case(td, w, dev, steps, kv_dtype="bf16"):
         layers = {i: conv(synth.make_layer(w, i, dev, q=qs[i])) for i in set(need)}
     torch.cuda.synchronize()
     idx = cnt = None
+    outs = [torch.empty(w.batch, w.num_q_heads, w.head_dim, dtype=torch.float32, device=dev) for _ in range(3)]
+    step = td.make_step([synth.LAYER_FULL, synth.LAYER_SELECT, synth.LAYER_SPARSE], [layers[i] for i in need],
+                        [qs[i] for i in need], outs, w.k)
     for _ in range(steps):
+        # the single-layer entry points (fused selection kernel) ...
         td.full_attn(layers[need[0]], qs[need[0]])
         _, idx, cnt = td.select_attn(layers[need[1]], qs[need[1]], w.k)
         td.sparse_attn(layers[need[2]], qs[need[2]], idx, cnt)
+        # ... and the same three layers as a step (selection layer in two passes where that applies)
+        step()
     torch.cuda.synchronize()
     print(json.dumps({"profile_case": w.name, "steps": steps, "launches": td.launch_count()}))
 
@@ -492,8 +498,13 @@ def main():
                                 lt.get("select_us"), "select", n_sel,
                                 "bytes_per_launch counts the KV cache only; the scores (4 B per position and query "
                                 "head, written once and read back from L2) are not in the denominator")
-    if select_entry and traffic.get("topk") is not None and select_entry["traffic"] is not None:
-        select_entry["traffic"] += traffic["topk"]
+    if select_entry:
+        # inside a step the selection layer runs as key pass + value pass where that applies, else fused
+        two_pass = args.granularity == "qhead" and w.batch == 1 and args.kv_dtype == "bf16" and traffic.get("score") is not None
+        parts = ("score", "value", "topk") if two_pass else ("select", "topk")
+        select_entry["traffic"] = sum(traffic[k] for k in parts) if all(traffic.get(k) is not None for k in parts) else None
+        select_entry["kernel"] = ("score_pass_kernel + value_pass_kernel + top-k (selection layers, two passes)" if two_pass
+                                  else select_entry["kernel"])
     # the kernel with the largest share of the step leads; the others follow as siblings
     entries = [e for e in (sparse_entry, full_entry, select_entry) if e]
     entries.sort(key=lambda e: -e["share_of_step"])

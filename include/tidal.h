@@ -170,7 +170,10 @@ tidal_status_t tidal_sparse_attn(tidal_ctx_t *ctx, const tidal_kv_t *kv, const v
  * the sparse layers after it. kv_per_layer (host array of descriptors),
  * q_per_layer and out_per_layer (host arrays of device pointers) have
  * num_layers entries. A sparse layer before the first selection layer is
- * TIDAL_ERR_INVALID. Everything is enqueued on `stream` without host waits. */
+ * TIDAL_ERR_INVALID. Everything is enqueued without host waits and is complete, in
+ * stream order, when the work enqueued on `stream` is: a selection layer may run part
+ * of its work (its value pass) on a second stream that the context owns, forked from
+ * and joined back into `stream` with events, also inside a stream capture. */
 tidal_status_t tidal_decode_step(tidal_ctx_t *ctx, int32_t num_layers, const uint8_t *schedule,
                                  const tidal_kv_t *kv_per_layer, const void *const *q_per_layer,
                                  float *const *out_per_layer, int32_t k, int32_t granularity,
@@ -217,6 +220,10 @@ tidal_status_t tidal_set_select_margin(tidal_ctx_t *ctx, float margin);
  * and its output (a sparse layer right after a selection layer always waits first: the top-k writes its
  * index list). With enabled = 0 a layer only prefetches cache rows ahead of the previous layer's end and
  * reads its query afterwards, as a caller would need whose queries are produced between the layers.
+ * With the overlap on, a selection layer over one sequence (per-head sets, bf16 cache, fp32 outputs)
+ * also runs as two passes: keys first (logits, their histogram, the largest logit per head), then the
+ * top-k on `stream` while the values are streamed on the context's second stream beside it and beside
+ * the sparse layers that follow.
  * The single-layer calls always wait for all earlier work in the stream before reading anything. */
 tidal_status_t tidal_set_layer_overlap(tidal_ctx_t *ctx, int32_t enabled);
 

@@ -494,8 +494,18 @@ tidal_status_t run_topk(tidal_ctx* ctx, const tidal_kv_t* kv, const float* score
     const int sel_parts = (kv->max_ctx_len + TK_SPAN - 1) / TK_SPAN;     // select kernel
     t.shift = hist_shift_for(kv);
     t.vec_ok = (((uintptr_t)scores & 15) == 0 && (score_stride & 3) == 0) ? 1 : 0;
-    t.cand_smem = 8192;          // one histogram bin's population; larger lists are read from global memory
+    // Candidates the last CTA of a head can hold in shared memory (a threshold bin's population is about
+    // 2000 of 131072 scores; larger lists are read from global memory). With more CTAs than fit the GPU at
+    // once (batches), the buffer is cut to what fits beside the bitmaps in the 64 KB the score staging needs
+    // anyway, so that three CTAs share an SM instead of two.
     const size_t words = (size_t)(kv->max_ctx_len + 31) / 32;
+    t.cand_smem = 8192;
+    {
+        const long long ctas = (long long)((kv->max_ctx_len + TK_SPAN - 1) / TK_SPAN) * kv->batch * Hi;
+        const size_t staging = (size_t)TK_SPAN * sizeof(float), bitmaps = 2 * words * sizeof(unsigned);
+        if (ctas > 2LL * ctx->sm_count && bitmaps + 2048 * sizeof(uint2) <= staging)
+            t.cand_smem = (int)((staging - bitmaps) / sizeof(uint2));
+    }
     // the last CTA's bitmaps and candidate buffer, or every CTA's score staging area, whichever is larger
     size_t smem = std::max(2 * words * sizeof(unsigned) + (size_t)t.cand_smem * sizeof(uint2),
                            (size_t)TK_SPAN * sizeof(float));

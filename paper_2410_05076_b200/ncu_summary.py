@@ -4,7 +4,8 @@
     python -m paper_2410_05076_b200.ncu_summary cfg3 capture.csv >> profiles/ncu_dram_traffic.txt
 
 Prints one line per kernel, `<workload> <kernel> <bytes>`, where bytes is the mean over the captured
-launches of dram__bytes_read.sum + dram__bytes_write.sum and kernel is one of full, select, sparse, topk.
+launches of dram__bytes_read.sum + dram__bytes_write.sum and kernel is one of full, select (the fused
+selection kernel), score and value (the two passes a selection layer runs as inside a step), topk, sparse.
 bench.py reads these lines for the `traffic` fields of its roofline block.
 """
 from __future__ import annotations
@@ -22,6 +23,10 @@ def kernel_key(name: str):
         return "select"
     if "attn_kernel<2" in name or "attn_kernel<(int)2" in name:
         return "sparse"
+    if "score_pass_kernel" in name:
+        return "score"
+    if "value_pass_kernel" in name:
+        return "value"
     if "topk" in name:
         return "topk"
     return None
@@ -44,7 +49,7 @@ def main(argv):
             continue
         b = float(r[rd]) * UNIT[units[rd]] + float(r[wr]) * UNIT[units[wr]]
         acc.setdefault(key, []).append(b)
-    for key in ("full", "select", "topk", "sparse"):
+    for key in ("full", "select", "score", "value", "topk", "sparse"):
         if key in acc:
             print(f"{workload} {key} {sum(acc[key]) / len(acc[key]):.0f}")
 
