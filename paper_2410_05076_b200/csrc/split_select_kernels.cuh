@@ -57,13 +57,14 @@ struct PoolWalk {
 // Uses of AttnParams: q, k, strides, page table, ctx_lens, scale, scores / score_stride, hist / hist_shift,
 // tile_ctr / ctr_stride (a cursor set of the main stream's rotation), split_max (per head: the order-preserving
 // key of the largest logit, 0 = none yet), out (cleared), pdl / wait_first / wait_late / trigger_early, status.
-// batch must be 1, splits_per_item > 0.
-template <int NW, int STAGES>
+// batch must be 1, splits_per_item > 0. The loop is written for few instructions per tile (a tile is only 4 KB
+// here): constant ring-slot numbers, tile numbers in registers, one unmasked path for whole tiles of eight heads.
+// ROW512: consecutive positions of a head lie 512 bytes apart (K and V rows interleaved, contiguous or paged),
+// so that the sixteen rows of a tile are reached with constant offsets from one pointer.
+template <int NW, int STAGES, bool ROW512>
 __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams p) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    __shared__ uint32_t s_vmask[NW][STAGES];
-    __shared__ int s_posbase[NW][STAGES];
     __shared__ float s_max[NW][8];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -82,19 +83,20 @@ __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams
     const int N = max(min(p.ctx_lens[0], p.max_ctx), 0);
     const int tiles = item_tiles(N);
     const int head0 = g * p.G, ncols = p.G;
-    if (hist_on) {
-        for (int i = threadIdx.x; i < HIST_SMEM_WORDS; i += NW * 32) hist[i] = 0;
-        __syncthreads();
-    }
-    float* score_row0 = (2 * tig < ncols) ? p.scores + (long long)(head0 + 2 * tig) * p.score_stride : nullptr;
-    float* score_row1 = (2 * tig + 1 < ncols) ? p.scores + (long long)(head0 + 2 * tig + 1) * p.score_stride : nullptr;
+    // this lane's two heads (2 tig, 2 tig + 1; clamped to the group, masked where they are used) and its row gid
+    const bool col0 = 2 * tig < ncols, col1 = 2 * tig + 1 < ncols;
+    float* const score_row0 = p.scores + (long long)(head0 + min(2 * tig, ncols - 1)) * p.score_stride + gid;
+    float* const score_row1 = p.scores + (long long)(head0 + min(2 * tig + 1, ncols - 1)) * p.score_stride + gid;
+    const int hshift = p.hist_shift;
+    uint32_t* const h0 = hist + ((2 * tig) << (32 - hshift));
+    uint32_t* const h1 = hist + ((2 * tig + 1) << (32 - hshift));
 
     const uint32_t wbase = smem_u32(smem + (size_t)warp * STAGES * TILE_BYTES);
     const int c16 = lane & 15, rhalf = lane >> 4;
-    const long long lane_src = (long long)rhalf * p.stride_pos + c16 * 8;
     const long long two_rows = 2 * p.stride_pos;
+    const long long tile_step = (long long)TILE * p.stride_pos;
     const uint32_t kdst = rhalf * 256 + ((c16 ^ (rhalf << 2)) << 4);
-    const long long item_off = (long long)g * p.stride_head;
+    const __nv_bfloat16* const kbase = p.k + (long long)g * p.stride_head + (long long)rhalf * p.stride_pos + c16 * 8;
     const uint64_t kv_policy = l2_evict_first_policy();
     const uint64_t keep = l2_evict_last_policy();
 
@@ -102,46 +104,60 @@ __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams
     PoolWalk walk;
     constexpr int GRAB = GRAB_TILES_DENSE;
     walk.template start<GRAB>(pool, tiles, item_ctas * NW, part * NW + warp, STAGES + 2, lane);
-    int tA = walk.template next<GRAB>();
-    int tB = (tA >= 0) ? walk.template next<GRAB>() : -1;
 
-    auto issue = [&](int stage) {
-        const int tile = tA;
-        tA = tB;
-        tB = (tA >= 0) ? walk.template next<GRAB>() : -1;
-        const uint32_t ks = wbase + stage * TILE_BYTES;
-        const int pos0 = tile * TILE;
-        long long off;
-        bool ok = true;
+    // A ring slot's tile number stays in a register (the ring is walked with constant slot numbers); a tile
+    // whose page id is outside the pool is marked and counts as empty.
+    constexpr int BAD_TILE = 1 << 30;
+    auto issue = [&](uint32_t ks, int& tile) {
+        const __nv_bfloat16* src;
         if (p.paged) {
             const int page = __ldg(p.page_table + tile);
-            ok = (unsigned)page < (unsigned)p.num_pages;
-            if (!ok && lane == 0) atomicOr(p.status, STATUS_BAD_PAGE);
-            off = (ok ? (long long)page * p.stride_page : 0) + item_off + lane_src;
+            const bool ok = (unsigned)page < (unsigned)p.num_pages;
+            if (!ok) {
+                if (lane == 0) atomicOr(p.status, STATUS_BAD_PAGE);
+                tile |= BAD_TILE;
+            }
+            src = kbase + (ok ? (long long)page * p.stride_page : 0);
         } else {
-            off = item_off + (long long)pos0 * p.stride_pos + lane_src;
+            src = kbase + tile * tile_step;
         }
-        const int nvalid = ok ? max(0, min(TILE, N - pos0)) : 0;
-        const __nv_bfloat16* ksrc = p.k + off;
+        const int nvalid = (tile & BAD_TILE) ? 0 : max(0, min(TILE, N - tile * TILE));
         if (nvalid == TILE) {
+            if (ROW512) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) cp_async16_full_hint(ks + kdst + i * 512, ksrc + i * two_rows, kv_policy);
+                for (int i = 0; i < 8; ++i) cp_async16_full_hint(ks + kdst + i * 512, src + i * (4 * HEAD_DIM), kv_policy);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) cp_async16_full_hint(ks + kdst + i * 512, src + i * two_rows, kv_policy);
+            }
         } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const bool rv = rhalf + 2 * i < nvalid;
-                cp_async16_hint(ks + kdst + i * 512, rv ? ksrc + i * two_rows : p.k, rv ? 16 : 0, kv_policy);
+                cp_async16_hint(ks + kdst + i * 512, rv ? src + i * two_rows : p.k, rv ? 16 : 0, kv_policy);
             }
         }
-        if (lane == 0) { s_vmask[warp][stage] = (1u << nvalid) - 1u; s_posbase[warp][stage] = pos0; }
     };
 
-    int issued = 0, commits = 0;
-    if (!waited && !p.wait_late) {
-        while (commits < STAGES && tA >= 0 && tA < tiles - 1) { issue(issued % STAGES); ++issued; cp_async_commit(); ++commits; }
-        pdl_wait();
-        pdl_trigger();
-        waited = true;
+    int tl[STAGES];
+#pragma unroll
+    for (int s = 0; s < STAGES; ++s) tl[s] = -1;
+    // fill all but one slot; a kernel that may read ahead of its wait still leaves the last tile (the newest
+    // token's row) for afterwards
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) {
+        int t = walk.template next<GRAB>();
+        if (t >= 0) {
+            if (!waited && !p.wait_late && t == tiles - 1) { pdl_wait(); pdl_trigger(); waited = true; }
+            issue(wbase + s * TILE_BYTES, t);
+        }
+        tl[s] = t;
+        cp_async_commit();
+    }
+    if (!waited && !p.wait_late) { pdl_wait(); pdl_trigger(); waited = true; }
+    if (hist_on) {                                     // (the first tiles are on their way meanwhile)
+        for (int i = threadIdx.x; i < HIST_SMEM_WORDS; i += NW * 32) hist[i] = 0;
+        __syncthreads();
     }
     // a selection layer that waits late writes its scores ahead of the wait: the host allows that only
     // when nothing can still be reading the score buffer
@@ -156,30 +172,15 @@ __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams
         }
     }
     float m0 = -INFINITY, m1 = -INFINITY;              // largest logit this lane has seen of heads 2tig, 2tig+1
-    const bool ring_full = commits == STAGES;
-    while (commits < STAGES - 1) {
-        if (tA >= 0) { issue(issued % STAGES); ++issued; }
-        cp_async_commit();
-        ++commits;
-    }
-    for (int it = 0; it < issued; ++it) {
-        if (it == 0 && ring_full) {
-            cp_async_wait<STAGES - 1>();
-            __syncwarp();
-        } else {
-            cp_async_wait<STAGES - 2>();
-            __syncwarp();
-            if (tA >= 0) { issue((it + STAGES - 1) % STAGES); ++issued; }
-            cp_async_commit();
-        }
-        const int stage = it % STAGES;
-        const uint32_t ks = wbase + stage * TILE_BYTES;
-        const uint32_t vmask = s_vmask[warp][stage];
-        const int pos_base = s_posbase[warp][stage];
+    const uint32_t kswz = (gid & 1) << 2;
+    const uint32_t klane = gid * 256;
+
+    auto consume = [&](uint32_t ks, int tile) {
+        const int pos_base = (tile & ~BAD_TILE) * TILE;
+        const int nvalid = (tile & BAD_TILE) ? 0 : max(0, min(TILE, N - pos_base));
         // S^T = K . Q^T, as in consume_tile
         float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
-        const uint32_t krow = ks + gid * 256;
-        const uint32_t kswz = (gid & 1) << 2;
+        const uint32_t krow = ks + klane;
 #pragma unroll
         for (int j = 0; j < 4; j += 2) {
             uint32_t ka[4], kb[4], kc[4], kd[4];
@@ -195,32 +196,60 @@ __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) s[i] += s2[i];
-        const bool v0 = (vmask >> gid) & 1u, v1 = (vmask >> (gid + 8)) & 1u;
         const float f0 = s[0] * p.scale, f1 = s[1] * p.scale, f2 = s[2] * p.scale, f3 = s[3] * p.scale;
-        if (score_row0) {
-            if (v0) st_keep(score_row0 + pos_base + gid, f0, keep);
-            if (v1) st_keep(score_row0 + pos_base + gid + 8, f2, keep);
-        }
-        if (score_row1) {
-            if (v0) st_keep(score_row1 + pos_base + gid, f1, keep);
-            if (v1) st_keep(score_row1 + pos_base + gid + 8, f3, keep);
-        }
-        if (hist_on) {
-            const int nb = 1 << (32 - p.hist_shift);
-            uint32_t* h0 = hist + (2 * tig) * nb;
-            uint32_t* h1 = h0 + nb;
-            if (score_row0) {
-                if (v0) atomicAdd(h0 + (score_key_bits(f0) >> p.hist_shift), 1u);
-                if (v1) atomicAdd(h0 + (score_key_bits(f2) >> p.hist_shift), 1u);
+        if (nvalid == TILE && ncols == 8) {
+            // the common case: sixteen cached tokens, eight heads, nothing to mask
+            st_keep(score_row0 + pos_base, f0, keep);
+            st_keep(score_row0 + pos_base + 8, f2, keep);
+            st_keep(score_row1 + pos_base, f1, keep);
+            st_keep(score_row1 + pos_base + 8, f3, keep);
+            if (hist_on) {
+                atomicAdd(h0 + (score_key_bits(f0) >> hshift), 1u);
+                atomicAdd(h0 + (score_key_bits(f2) >> hshift), 1u);
+                atomicAdd(h1 + (score_key_bits(f1) >> hshift), 1u);
+                atomicAdd(h1 + (score_key_bits(f3) >> hshift), 1u);
             }
-            if (score_row1) {
-                if (v0) atomicAdd(h1 + (score_key_bits(f1) >> p.hist_shift), 1u);
-                if (v1) atomicAdd(h1 + (score_key_bits(f3) >> p.hist_shift), 1u);
+            // the largest stored logit of each head: the value pass takes its softmax weights relative to it
+            m0 = fmaxf(m0, fmaxf(f0, f2));
+            m1 = fmaxf(m1, fmaxf(f1, f3));
+        } else {
+            const bool v0 = gid < nvalid, v1 = gid + 8 < nvalid;
+            if (col0) {
+                if (v0) st_keep(score_row0 + pos_base, f0, keep);
+                if (v1) st_keep(score_row0 + pos_base + 8, f2, keep);
             }
+            if (col1) {
+                if (v0) st_keep(score_row1 + pos_base, f1, keep);
+                if (v1) st_keep(score_row1 + pos_base + 8, f3, keep);
+            }
+            if (hist_on) {
+                if (col0) {
+                    if (v0) atomicAdd(h0 + (score_key_bits(f0) >> hshift), 1u);
+                    if (v1) atomicAdd(h0 + (score_key_bits(f2) >> hshift), 1u);
+                }
+                if (col1) {
+                    if (v0) atomicAdd(h1 + (score_key_bits(f1) >> hshift), 1u);
+                    if (v1) atomicAdd(h1 + (score_key_bits(f3) >> hshift), 1u);
+                }
+            }
+            if (v0) { m0 = fmaxf(m0, f0); m1 = fmaxf(m1, f1); }
+            if (v1) { m0 = fmaxf(m0, f2); m1 = fmaxf(m1, f3); }
         }
-        // the largest stored logit of each head: the value pass takes its softmax weights relative to it
-        if (v0) { m0 = fmaxf(m0, f0); m1 = fmaxf(m1, f1); }
-        if (v1) { m0 = fmaxf(m0, f2); m1 = fmaxf(m1, f3); }
+    };
+
+    for (bool live = true; live;) {
+#pragma unroll
+        for (int s = 0; s < STAGES; ++s) {
+            if (tl[s] < 0) { live = false; break; }
+            cp_async_wait<STAGES - 2>();
+            __syncwarp();                              // every lane is done with the slot that is refilled next
+            const int sn = (s + STAGES - 1) % STAGES;
+            int t = walk.template next<GRAB>();
+            if (t >= 0) issue(wbase + sn * TILE_BYTES, t);
+            tl[sn] = t;
+            cp_async_commit();
+            consume(wbase + s * TILE_BYTES, tl[s]);
+        }
     }
     cp_async_wait<0>();
     __syncwarp();
@@ -267,12 +296,11 @@ __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams
 // Uses of AttnParams: v, strides, page table, ctx_lens, scores / score_stride, split_max, split_sum (per head,
 // zero between launches), out (+= with atomics, then divided), counters / tile_ctr / ctr_stride (arrays of its
 // own: it runs beside the main stream's kernels), status.
-template <int NW, int STAGES>
+template <int NW, int STAGES, bool ROW512>
 __global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams p) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     constexpr int SLOT = TILE_BYTES + 512;                   // 16 value rows, then 16 logits of up to 8 heads
-    __shared__ uint32_t s_vmask[NW][STAGES];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = lane >> 2, tig = lane & 3;
@@ -285,49 +313,53 @@ __global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams
 
     const uint32_t wbase = smem_u32(smem + (size_t)warp * STAGES * SLOT);
     const int c16 = lane & 15, rhalf = lane >> 4;
-    const long long lane_src = (long long)rhalf * p.stride_pos + c16 * 8;
     const long long two_rows = 2 * p.stride_pos;
-    const uint32_t vdst = rhalf * 256;
+    const long long tile_step = (long long)TILE * p.stride_pos;
     const uint32_t vc = c16 ^ rhalf;
-    const long long item_off = (long long)g * p.stride_head;
+    uint32_t vdst[4];                                        // row pairs i and i + 4 share a swizzle
+#pragma unroll
+    for (int i = 0; i < 4; ++i) vdst[i] = rhalf * 256 + i * 512 + ((vc ^ (i << 1)) << 4);
+    const __nv_bfloat16* const vbase = p.v + (long long)g * p.stride_head + (long long)rhalf * p.stride_pos + c16 * 8;
     const uint64_t kv_policy = l2_evict_first_policy();
     // lane l < 4 * ncols fetches 16 bytes (four positions) of head l >> 2's logits
     const bool score_lane = lane < 4 * ncols;
-    const float* score_src = p.scores + (long long)(head0 + (lane >> 2)) * p.score_stride + 4 * (lane & 3);
+    const float* const score_src = p.scores + (long long)(head0 + min(lane >> 2, ncols - 1)) * p.score_stride + 4 * (lane & 3);
+    const uint32_t score_dst = TILE_BYTES + lane * 16;
 
     int* pool = p.tile_ctr + (long long)g * p.ctr_stride;
     PoolWalk walk;
     constexpr int GRAB = GRAB_TILES_DENSE;
     walk.template start<GRAB>(pool, tiles, item_ctas * NW, part * NW + warp, STAGES + 2, lane);
-    int tA = walk.template next<GRAB>();
-    int tB = (tA >= 0) ? walk.template next<GRAB>() : -1;
 
-    auto issue = [&](int stage) {
-        const int tile = tA;
-        tA = tB;
-        tB = (tA >= 0) ? walk.template next<GRAB>() : -1;
-        const uint32_t vs = wbase + stage * SLOT;
-        const int pos0 = tile * TILE;
-        long long off;
-        bool ok = true;
+    constexpr int BAD_TILE = 1 << 30;
+    auto issue = [&](uint32_t vs, int& tile) {
+        const __nv_bfloat16* src;
         if (p.paged) {
             const int page = __ldg(p.page_table + tile);
-            ok = (unsigned)page < (unsigned)p.num_pages;
-            if (!ok && lane == 0) atomicOr(p.status, STATUS_BAD_PAGE);
-            off = (ok ? (long long)page * p.stride_page : 0) + item_off + lane_src;
+            const bool ok = (unsigned)page < (unsigned)p.num_pages;
+            if (!ok) {
+                if (lane == 0) atomicOr(p.status, STATUS_BAD_PAGE);
+                tile |= BAD_TILE;
+            }
+            src = vbase + (ok ? (long long)page * p.stride_page : 0);
         } else {
-            off = item_off + (long long)pos0 * p.stride_pos + lane_src;
+            src = vbase + tile * tile_step;
         }
-        const int nvalid = ok ? max(0, min(TILE, N - pos0)) : 0;
-        const __nv_bfloat16* vsrc = p.v + off;
+        const int pos0 = (tile & ~BAD_TILE) * TILE;
+        const int nvalid = (tile & BAD_TILE) ? 0 : max(0, min(TILE, N - pos0));
+        if (nvalid == TILE) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const bool rv = rhalf + 2 * i < nvalid;
-            cp_async16_hint(vs + vdst + i * 512 + ((vc ^ ((i & 3) << 1)) << 4), rv ? vsrc + i * two_rows : p.v, rv ? 16 : 0, kv_policy);
+            for (int i = 0; i < 8; ++i)
+                cp_async16_full_hint(vs + vdst[i & 3] + (i >> 2) * 2048, ROW512 ? src + i * (4 * HEAD_DIM) : src + i * two_rows, kv_policy);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const bool rv = rhalf + 2 * i < nvalid;
+                cp_async16_hint(vs + vdst[i & 3] + (i >> 2) * 2048, rv ? src + i * two_rows : p.v, rv ? 16 : 0, kv_policy);
+            }
         }
         // (logits past the end of the sequence are never used: their rows are masked)
-        if (score_lane) cp_async16(vs + TILE_BYTES + lane * 16, score_src + pos0, 16);
-        if (lane == 0) s_vmask[warp][stage] = (1u << nvalid) - 1u;
+        if (score_lane) cp_async16(vs + score_dst, score_src + pos0, 16);
     };
 
     // the largest logit of this lane's two heads, in base-2 units (key 0: the head has no token at all)
@@ -338,51 +370,68 @@ __global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams
         if (k0) M0 = __uint_as_float((k0 & 0x80000000u) ? (k0 & 0x7fffffffu) : ~k0) * LOG2E;
         if (k1) M1 = __uint_as_float((k1 & 0x80000000u) ? (k1 & 0x7fffffffu) : ~k1) * LOG2E;
     }
+    const bool h0 = 2 * tig < ncols && M0 != -INFINITY, h1 = 2 * tig + 1 < ncols && M1 != -INFINITY;
+    const bool plain = ncols == 8 && __all_sync(0xffffffffu, h0 && h1);   // eight heads, each with a finite maximum
     float l0 = 0.f, l1 = 0.f;                          // this lane's share of sum_j p_j
     float o[8][4];
 #pragma unroll
     for (int t = 0; t < 8; ++t) { o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f; }
+    // logits of (position gid | gid + 8, heads 2tig | 2tig + 1): head h's 16 floats start at 64 * h
+    const uint32_t slane = TILE_BYTES + (2 * tig) * 64 + gid * 4;
+    const int rr = lane & 7, mb = (lane >> 3) & 1;
+    const uint32_t vlane = (rr + ((lane >> 4) << 3)) * 256 + ((rr ^ mb) << 4);
 
-    int issued = 0, commits = 0;
-    while (commits < STAGES - 1) {
-        if (tA >= 0) { issue(issued % STAGES); ++issued; }
-        cp_async_commit();
-        ++commits;
-    }
-    for (int it = 0; it < issued; ++it) {
-        cp_async_wait<STAGES - 2>();
-        __syncwarp();
-        if (tA >= 0) { issue((it + STAGES - 1) % STAGES); ++issued; }
-        cp_async_commit();
-        const int stage = it % STAGES;
-        const uint32_t vs = wbase + stage * SLOT;
-        const uint32_t vmask = s_vmask[warp][stage];
-        const bool v0 = (vmask >> gid) & 1u, v1 = (vmask >> (gid + 8)) & 1u;
-        // logits of (position gid | gid + 8, heads 2tig | 2tig + 1): head h's 16 floats start at 64 * h
-        const uint32_t sbase = vs + TILE_BYTES;
-        float f0 = 0.f, f1 = 0.f, f2 = 0.f, f3 = 0.f;
-        if (2 * tig < ncols) {
-            asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f0) : "r"(sbase + (2 * tig) * 64 + gid * 4));
-            asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f2) : "r"(sbase + (2 * tig) * 64 + (gid + 8) * 4));
+    auto consume = [&](uint32_t vs, int tile) {
+        const int nvalid = (tile & BAD_TILE) ? 0 : max(0, min(TILE, N - (tile & ~BAD_TILE) * TILE));
+        float f0, f1, f2, f3;
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f0) : "r"(vs + slane));
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f2) : "r"(vs + slane + 32));
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f1) : "r"(vs + slane + 64));
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f3) : "r"(vs + slane + 96));
+        float p0, p1, p2, p3;
+        if (nvalid == TILE && plain) {
+            p0 = fast_exp2(f0 * LOG2E - M0); p1 = fast_exp2(f1 * LOG2E - M1);
+            p2 = fast_exp2(f2 * LOG2E - M0); p3 = fast_exp2(f3 * LOG2E - M1);
+        } else {
+            const bool v0 = gid < nvalid, v1 = gid + 8 < nvalid;
+            p0 = (v0 && h0) ? fast_exp2(f0 * LOG2E - M0) : 0.f; p1 = (v0 && h1) ? fast_exp2(f1 * LOG2E - M1) : 0.f;
+            p2 = (v1 && h0) ? fast_exp2(f2 * LOG2E - M0) : 0.f; p3 = (v1 && h1) ? fast_exp2(f3 * LOG2E - M1) : 0.f;
         }
-        if (2 * tig + 1 < ncols) {
-            asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f1) : "r"(sbase + (2 * tig + 1) * 64 + gid * 4));
-            asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f3) : "r"(sbase + (2 * tig + 1) * 64 + (gid + 8) * 4));
-        }
-        const bool h0 = 2 * tig < ncols && M0 != -INFINITY, h1 = 2 * tig + 1 < ncols && M1 != -INFINITY;
-        const float p0 = (v0 && h0) ? fast_exp2(f0 * LOG2E - M0) : 0.f, p1 = (v0 && h1) ? fast_exp2(f1 * LOG2E - M1) : 0.f;
-        const float p2 = (v1 && h0) ? fast_exp2(f2 * LOG2E - M0) : 0.f, p3 = (v1 && h1) ? fast_exp2(f3 * LOG2E - M1) : 0.f;
         l0 += p0 + p2;
         l1 += p1 + p3;
         const uint32_t pb0 = movmatrix_trans(pack_bf16(p0, p1));
         const uint32_t pb1 = movmatrix_trans(pack_bf16(p2, p3));
-        const int rr = lane & 7, mb = (lane >> 3) & 1;
-        const uint32_t vlane = vs + (rr + ((lane >> 4) << 3)) * 256 + ((rr ^ mb) << 4);
+        const uint32_t vl = vs + vlane;
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
             uint32_t a[4];
-            ldmatrix_x4_trans(vlane ^ (t << 5), a);
+            ldmatrix_x4_trans(vl ^ (t << 5), a);
             mma_bf16_16816(o[t], a[0], a[1], a[2], a[3], pb0, pb1);
+        }
+    };
+
+    int tl[STAGES];
+#pragma unroll
+    for (int s = 0; s < STAGES; ++s) tl[s] = -1;
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) {
+        int t = walk.template next<GRAB>();
+        if (t >= 0) issue(wbase + s * SLOT, t);
+        tl[s] = t;
+        cp_async_commit();
+    }
+    for (bool live = true; live;) {
+#pragma unroll
+        for (int s = 0; s < STAGES; ++s) {
+            if (tl[s] < 0) { live = false; break; }
+            cp_async_wait<STAGES - 2>();
+            __syncwarp();                              // every lane is done with the slot that is refilled next
+            const int sn = (s + STAGES - 1) % STAGES;
+            int t = walk.template next<GRAB>();
+            if (t >= 0) issue(wbase + sn * SLOT, t);
+            tl[sn] = t;
+            cp_async_commit();
+            consume(wbase + s * SLOT, tl[s]);
         }
     }
     cp_async_wait<0>();

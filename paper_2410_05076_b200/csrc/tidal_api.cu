@@ -440,7 +440,9 @@ tidal_status_t run_score_pass(tidal_ctx* ctx, const tidal_kv_t* kv, const void* 
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     ctx->launches++;
-    return cudaLaunchKernelEx(&cfg, score_pass_kernel<SCORE_NW, SCORE_STAGES>, a) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+    const cudaError_t e = kv->stride_pos == 2 * HEAD_DIM ? cudaLaunchKernelEx(&cfg, score_pass_kernel<SCORE_NW, SCORE_STAGES, true>, a)
+                                                         : cudaLaunchKernelEx(&cfg, score_pass_kernel<SCORE_NW, SCORE_STAGES, false>, a);
+    return e == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }
 
 // Pass 2 on the context's second stream: it starts when pass 1 is complete and runs beside whatever
@@ -463,7 +465,8 @@ tidal_status_t run_value_pass(tidal_ctx* ctx, const tidal_kv_t* kv, float* out, 
     a.splits_per_item = per_item;
     if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
         return TIDAL_ERR_CUDA;
-    value_pass_kernel<VALUE_NW, VALUE_STAGES><<<grid, VALUE_NW * 32, VALUE_SMEM, ctx->side>>>(a);
+    if (kv->stride_pos == 2 * HEAD_DIM) value_pass_kernel<VALUE_NW, VALUE_STAGES, true><<<grid, VALUE_NW * 32, VALUE_SMEM, ctx->side>>>(a);
+    else value_pass_kernel<VALUE_NW, VALUE_STAGES, false><<<grid, VALUE_NW * 32, VALUE_SMEM, ctx->side>>>(a);
     ctx->launches++;
     if (cudaGetLastError() != cudaSuccess) return TIDAL_ERR_CUDA;
     return cudaEventRecord(ctx->ev_join, ctx->side) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
@@ -705,8 +708,10 @@ tidal_status_t tidal_create(tidal_ctx_t** out, int device, size_t workspace_byte
     const int e1 = resident_ctas(attn_kernel<MODE_SELECT, DENSE_NW8, DENSE_STAGES8, false, false, true>, DENSE_NW8 * 32, attn_smem<MODE_SELECT, DENSE_NW8, DENSE_STAGES8, true>(), ctx->sm_count);
     const int e2 = resident_ctas(attn_kernel<MODE_SPARSE, SPARSE_NW8, SPARSE_STAGES8, false, false, true>, SPARSE_NW8 * 32, attn_smem<MODE_SPARSE, SPARSE_NW8, SPARSE_STAGES8, true>(), ctx->sm_count);
     const bool split_ok =
-        cudaFuncSetAttribute(score_pass_kernel<SCORE_NW, SCORE_STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCORE_SMEM) == cudaSuccess &&
-        cudaFuncSetAttribute(value_pass_kernel<VALUE_NW, VALUE_STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VALUE_SMEM) == cudaSuccess;
+        cudaFuncSetAttribute(score_pass_kernel<SCORE_NW, SCORE_STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCORE_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(score_pass_kernel<SCORE_NW, SCORE_STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCORE_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(value_pass_kernel<VALUE_NW, VALUE_STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VALUE_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(value_pass_kernel<VALUE_NW, VALUE_STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VALUE_SMEM) == cudaSuccess;
     const size_t topk_smem = 2 * (size_t)(MAX_CTX / 32) * sizeof(unsigned) + 8192 * sizeof(uint2);
     const bool topk_ok = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topk_smem) == cudaSuccess;
     const size_t compact_smem = 2 * ((size_t)(MAX_CTX / 32) + 1) * sizeof(unsigned) + (size_t)COMPACT_LIST_SMEM * sizeof(uint2);
