@@ -455,12 +455,17 @@ __global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams
     }
     if (gid == 0) { ml[warp * 8 + 2 * tig] = l0; ml[warp * 8 + 2 * tig + 1] = l1; }
     __syncthreads();
-    for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) {
-        const int col = e >> 7, c = e & 127;
-        float O = 0.f;
+    for (int e = threadIdx.x; e < ncols * (HEAD_DIM / 4); e += NW * 32) {      // four output elements per reduction
+        const int col = e >> 5, c = (e & 31) * 4;
+        float4 O = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int w = 0; w < NW; ++w) O += mo[(w * 8 + col) * HEAD_DIM + c];
-        if (O != 0.f) atomicAdd(p.out + (long long)(head0 + col) * HEAD_DIM + c, O);
+        for (int w = 0; w < NW; ++w) {
+            const float4 t = *reinterpret_cast<const float4*>(mo + (w * 8 + col) * HEAD_DIM + c);
+            O.x += t.x; O.y += t.y; O.z += t.z; O.w += t.w;
+        }
+        if (O.x != 0.f || O.y != 0.f || O.z != 0.f || O.w != 0.f)
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};\n" ::"l"(p.out + (long long)(head0 + col) * HEAD_DIM + c),
+                         "f"(O.x), "f"(O.y), "f"(O.z), "f"(O.w) : "memory");
     }
     if (threadIdx.x < ncols) {
         float L = 0.f;

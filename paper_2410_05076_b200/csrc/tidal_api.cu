@@ -891,7 +891,8 @@ static tidal_status_t decode_step_enqueue(tidal_ctx_t* ctx, int32_t num_layers, 
             // sparse layer ran in between, its first kernel waited for that top-k before it let anything
             // else start, so nobody reads the buffer any more; right after another selection layer, wait.
             const bool scores_free = i > 0 && schedule[i - 1] != TIDAL_LAYER_SELECT;
-            if (can_split(ctx, kv, sp) && ensure_side_stream(ctx) == TIDAL_OK) {
+            // (the value pass adds to the output rows four floats at a time)
+            if (can_split(ctx, kv, sp) && ((uintptr_t)outs[i] & 15) == 0 && ensure_side_stream(ctx) == TIDAL_OK) {
                 // key pass -> (value pass on the second stream) | top-k -> the layers that follow. A value
                 // pass still in flight reads the score buffer and the statistics this key pass overwrites.
                 if (side_pending) { if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return TIDAL_ERR_CUDA; side_pending = false; }
