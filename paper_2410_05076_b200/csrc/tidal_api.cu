@@ -755,6 +755,8 @@ tidal_status_t tidal_reserve(tidal_ctx_t* ctx, const tidal_kv_t* kv, int32_t k, 
     const tidal_status_t rc = check_kv(kv);
     if (rc != TIDAL_OK) return rc;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
+    const tidal_status_t rs = ensure_side_stream(ctx);       // a later step's selection layers may use it
+    if (rs != TIDAL_OK) return rs;
     return ensure_all(ctx, kv, ws_bytes_for(kv, k, num_layers_host));
 }
 
