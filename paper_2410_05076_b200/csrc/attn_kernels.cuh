@@ -60,6 +60,7 @@ struct AttnParams {
     const __nv_bfloat16* k;
     const __nv_bfloat16* v;
     float* out;                // [B, Hq, 128]; bf16 instead of fp32 when out_bf16 is set
+    float* out_final;          // value pass of a two-pass selection layer: where the finished rows go (null: out itself)
     int out_bf16;
     long long stride_b, stride_pos, stride_head, stride_page;
     const int* page_table;

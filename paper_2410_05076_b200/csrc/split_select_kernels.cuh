@@ -294,7 +294,8 @@ __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams
 
 // ---- pass 2: sum_j softmax_j v_j from the stored logits ------------------------------------------------------
 // Uses of AttnParams: v, strides, page table, ctx_lens, scores / score_stride, split_max, split_sum (per head,
-// zero between launches), out (+= with atomics, then divided), counters / tile_ctr / ctr_stride (arrays of its
+// zero between launches), out (+= with reductions, then divided, the quotient written to out_final if given),
+// counters / tile_ctr / ctr_stride (arrays of its
 // own: it runs beside the main stream's kernels), status.
 template <int NW, int STAGES, bool ROW512>
 __global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams p) {
@@ -484,11 +485,11 @@ __global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams
     }
     __syncthreads();
     if (s_last) {
+        float* const rows = p.out_final ? p.out_final : p.out;
         for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) {
-            float* dst = p.out + (long long)head0 * HEAD_DIM + e;
             const float L = __ldcg(p.split_sum + head0 + (e >> 7));
-            const float O = __ldcg(dst);
-            *dst = (L > 0.f) ? O / L : 0.f;
+            const float O = __ldcg(p.out + (long long)head0 * HEAD_DIM + e);
+            rows[(long long)head0 * HEAD_DIM + e] = (L > 0.f) ? O / L : 0.f;
         }
         __syncthreads();
         if (threadIdx.x < ncols) { p.split_sum[head0 + threadIdx.x] = 0.f; p.split_max[head0 + threadIdx.x] = 0u; }

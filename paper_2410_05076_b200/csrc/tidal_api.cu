@@ -447,10 +447,11 @@ tidal_status_t run_score_pass(tidal_ctx* ctx, const tidal_kv_t* kv, const void* 
 
 // Pass 2 on the context's second stream: it starts when pass 1 is complete and runs beside whatever
 // the caller's stream does next. It owns a cursor and a counter array of its own and no other scratch.
-tidal_status_t run_value_pass(tidal_ctx* ctx, const tidal_kv_t* kv, float* out, const float* scores,
+tidal_status_t run_value_pass(tidal_ctx* ctx, const tidal_kv_t* kv, float* out, float* out_final, const float* scores,
                               long long score_stride, const WsLayout& w, cudaStream_t st) {
     AttnParams a;
     fill_common(a, ctx, kv, nullptr, out, w);
+    a.out_final = out_final;
     a.scores = const_cast<float*>(scores);
     a.score_stride = score_stride;
     a.split_max = state_split_max(ctx);
@@ -871,7 +872,7 @@ static tidal_status_t decode_step_prepare(tidal_ctx_t* ctx, int32_t num_layers, 
 static tidal_status_t decode_step_enqueue(tidal_ctx_t* ctx, int32_t num_layers, const uint8_t* schedule,
                                           const tidal_kv_t* kvs, const void* const* qs, float* const* outs,
                                           int32_t k, int32_t granularity, int32_t* idx, int32_t* idx_count,
-                                          int host_layers, cudaStream_t st) {
+                                          int host_layers, cudaStream_t st, float* const* acc = nullptr) {
     const int Hi = hi_of(&kvs[0], granularity);
     tidal_status_t rc = TIDAL_OK;
     bool side_pending = false;                  // a value pass is in flight on the second stream
@@ -893,13 +894,15 @@ static tidal_status_t decode_step_enqueue(tidal_ctx_t* ctx, int32_t num_layers, 
             // sparse layer ran in between, its first kernel waited for that top-k before it let anything
             // else start, so nobody reads the buffer any more; right after another selection layer, wait.
             const bool scores_free = i > 0 && schedule[i - 1] != TIDAL_LAYER_SELECT;
-            // (the value pass adds to the output rows four floats at a time)
-            if (can_split(ctx, kv, sp) && ((uintptr_t)outs[i] & 15) == 0 && ensure_side_stream(ctx) == TIDAL_OK) {
+            // The value pass adds to the output rows, four floats at a time: in place, or in the device rows the
+            // caller of this function set aside (outputs in host memory), from where its last CTAs write outs[i].
+            float* const sums = (acc && acc[i]) ? acc[i] : outs[i];
+            if (can_split(ctx, kv, sp) && ((uintptr_t)sums & 15) == 0 && ensure_side_stream(ctx) == TIDAL_OK) {
                 // key pass -> (value pass on the second stream) | top-k -> the layers that follow. A value
                 // pass still in flight reads the score buffer and the statistics this key pass overwrites.
                 if (side_pending) { if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return TIDAL_ERR_CUDA; side_pending = false; }
-                rc = run_score_pass(ctx, kv, qs[i], outs[i], scores, w.score_stride, dep, scores_free, w, st);
-                if (rc == TIDAL_OK) rc = run_value_pass(ctx, kv, outs[i], scores, w.score_stride, w, st);
+                rc = run_score_pass(ctx, kv, qs[i], sums, scores, w.score_stride, dep, scores_free, w, st);
+                if (rc == TIDAL_OK) rc = run_value_pass(ctx, kv, sums, sums == outs[i] ? nullptr : outs[i], scores, w.score_stride, w, st);
                 side_pending = rc == TIDAL_OK;
             } else {
                 rc = run_dense(ctx, kv, qs[i], outs[i], scores, w.score_stride, sp.fuse, dep, w, st, sp.agg, sp.compact ? k : 0, scores_free);
@@ -1053,12 +1056,13 @@ tidal_status_t tidal_decode_step_host(tidal_ctx_t* ctx, int32_t num_layers, cons
     if (q_alias && ((uintptr_t)q_alias & 15)) q_alias = nullptr;      // query rows are read as 16-byte pieces
     const void* qs[1024];
     float* outs[1024];
-    // (a selection layer may run as two passes whose second adds to the output with atomics: its rows
-    // stay in device memory and are copied out afterwards)
+    // (a selection layer may run as two passes whose second adds to the output rows with reductions: those
+    // sums stay in the staging area and the pass's last CTAs write the finished rows to the caller's buffer)
+    float* acc[1024];
     for (int i = 0; i < num_layers; ++i) {
-        const bool direct = out_alias && schedule[i] != TIDAL_LAYER_SELECT;
         qs[i] = (q_alias ? q_alias : qd) + (size_t)i * rows * HEAD_DIM * 2;
-        outs[i] = (float*)((direct ? out_alias : (char*)od) + (size_t)i * rows * HEAD_DIM * out_elem);
+        outs[i] = (float*)((out_alias ? out_alias : (char*)od) + (size_t)i * rows * HEAD_DIM * out_elem);
+        acc[i] = (out_alias && schedule[i] == TIDAL_LAYER_SELECT) ? (float*)((char*)od + (size_t)i * rows * HEAD_DIM * out_elem) : nullptr;
     }
     if ((rc = decode_step_prepare(ctx, num_layers, schedule, kv_per_layer, qs, outs, k, granularity, num_layers)) != TIDAL_OK)
         return rc;
@@ -1066,17 +1070,10 @@ tidal_status_t tidal_decode_step_host(tidal_ctx_t* ctx, int32_t num_layers, cons
         if (!q_alias && cudaMemcpyAsync(qd, q_host, (size_t)num_layers * rows * HEAD_DIM * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
             return TIDAL_ERR_CUDA;
         const tidal_status_t r = decode_step_enqueue(ctx, num_layers, schedule, kv_per_layer, qs, outs, k, granularity,
-                                                     (int*)(ws + w.idx), (int*)(ws + w.idx_count), num_layers, st);
+                                                     (int*)(ws + w.idx), (int*)(ws + w.idx_count), num_layers, st, acc);
         if (r != TIDAL_OK) return r;
         if (!out_alias && cudaMemcpyAsync(out_host, od, (size_t)num_layers * rows * HEAD_DIM * out_elem, cudaMemcpyDeviceToHost, st) != cudaSuccess)
             return TIDAL_ERR_CUDA;
-        if (out_alias) {
-            const size_t layer_bytes = rows * HEAD_DIM * out_elem;
-            for (int i = 0; i < num_layers; ++i)
-                if (schedule[i] == TIDAL_LAYER_SELECT &&
-                    cudaMemcpyAsync((char*)out_host + i * layer_bytes, (char*)od + i * layer_bytes, layer_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-                    return TIDAL_ERR_CUDA;
-        }
         return TIDAL_OK;
     };
     // The copies can be recorded with the layers only when both host buffers are page-locked.
