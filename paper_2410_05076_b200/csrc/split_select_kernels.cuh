@@ -95,7 +95,11 @@ __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams
     const int c16 = lane & 15, rhalf = lane >> 4;
     const long long two_rows = 2 * p.stride_pos;
     const long long tile_step = (long long)TILE * p.stride_pos;
-    const uint32_t kdst = rhalf * 256 + ((c16 ^ (rhalf << 2)) << 4);
+    // key rows in a ring slot: row r at r * 256, its 16-byte piece c at position c ^ (r & 7), so that the eight
+    // rows of an ldmatrix fall into different banks; this lane copies piece c16 of rows rhalf + 2 i
+    uint32_t kdst[4];                                        // rows i and i + 4 share a swizzle
+#pragma unroll
+    for (int i = 0; i < 4; ++i) kdst[i] = (rhalf + 2 * i) * 256 + ((c16 ^ (rhalf + 2 * i)) << 4);
     const __nv_bfloat16* const kbase = p.k + (long long)g * p.stride_head + (long long)rhalf * p.stride_pos + c16 * 8;
     const uint64_t kv_policy = l2_evict_first_policy();
     const uint64_t keep = l2_evict_last_policy();
@@ -125,16 +129,16 @@ __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams
         if (nvalid == TILE) {
             if (ROW512) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) cp_async16_full_hint(ks + kdst + i * 512, src + i * (4 * HEAD_DIM), kv_policy);
+                for (int i = 0; i < 8; ++i) cp_async16_full_hint(ks + kdst[i & 3] + (i >> 2) * 2048, src + i * (4 * HEAD_DIM), kv_policy);
             } else {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) cp_async16_full_hint(ks + kdst + i * 512, src + i * two_rows, kv_policy);
+                for (int i = 0; i < 8; ++i) cp_async16_full_hint(ks + kdst[i & 3] + (i >> 2) * 2048, src + i * two_rows, kv_policy);
             }
         } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const bool rv = rhalf + 2 * i < nvalid;
-                cp_async16_hint(ks + kdst + i * 512, rv ? src + i * two_rows : p.k, rv ? 16 : 0, kv_policy);
+                cp_async16_hint(ks + kdst[i & 3] + (i >> 2) * 2048, rv ? src + i * two_rows : p.k, rv ? 16 : 0, kv_policy);
             }
         }
     };
@@ -161,57 +165,60 @@ __global__ void __launch_bounds__(NW * 32, 1) score_pass_kernel(const AttnParams
     }
     // a selection layer that waits late writes its scores ahead of the wait: the host allows that only
     // when nothing can still be reading the score buffer
-    uint32_t qf[4][4];
+    // B fragments of the eight k-steps: head gid's elements 16 j + 2 tig (+1) and 16 j + 8 + 2 tig (+1)
+    uint32_t qf[8][2];
     {
-        const uint4* qp = reinterpret_cast<const uint4*>(p.q + (long long)(head0 + min(gid, ncols - 1)) * HEAD_DIM);
+        const uint32_t* qw = reinterpret_cast<const uint32_t*>(p.q + (long long)(head0 + min(gid, ncols - 1)) * HEAD_DIM);
         const bool on = gid < ncols;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const uint4 t = __ldg(qp + 4 * j + tig);
-            qf[j][0] = on ? t.x : 0u; qf[j][1] = on ? t.y : 0u; qf[j][2] = on ? t.z : 0u; qf[j][3] = on ? t.w : 0u;
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t w0 = __ldg(qw + 8 * j + tig), w1 = __ldg(qw + 8 * j + 4 + tig);
+            qf[j][0] = on ? w0 : 0u;
+            qf[j][1] = on ? w1 : 0u;
         }
     }
     float m0 = -INFINITY, m1 = -INFINITY;              // largest logit this lane has seen of heads 2tig, 2tig+1
-    const uint32_t kswz = (gid & 1) << 2;
-    const uint32_t klane = gid * 256;
+    // ldmatrix: lane l addresses row (l & 7) + 8 * ((l >> 3) & 1), piece 2 j + (l >> 4) of the tile
+    const int lrow = (lane & 7) + ((lane >> 3) & 1) * 8;
+    const uint32_t klane = lrow * 256 + ((((lane >> 4) & 1) ^ (lane & 7)) << 4);
 
     auto consume = [&](uint32_t ks, int tile) {
         const int pos_base = (tile & ~BAD_TILE) * TILE;
         const int nvalid = (tile & BAD_TILE) ? 0 : max(0, min(TILE, N - pos_base));
-        // S^T = K . Q^T, as in consume_tile
+        // S^T = K . Q^T: positions are the rows of the MMA, the group's heads its columns; two accumulator chains
         float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
-        const uint32_t krow = ks + klane;
+        const uint32_t kl = ks + klane;
 #pragma unroll
-        for (int j = 0; j < 4; j += 2) {
-            uint32_t ka[4], kb[4], kc[4], kd[4];
-            const uint32_t off0 = (((4 * j + tig) ^ kswz) << 4), off1 = (((4 * j + 4 + tig) ^ kswz) << 4);
-            lds128(krow + off0, ka);
-            lds128(krow + 8 * 256 + off0, kb);
-            lds128(krow + off1, kc);
-            lds128(krow + 8 * 256 + off1, kd);
-            mma_bf16_16816(s, ka[0], kb[0], ka[1], kb[1], qf[j][0], qf[j][1]);
-            mma_bf16_16816(s2, kc[0], kd[0], kc[1], kd[1], qf[j + 1][0], qf[j + 1][1]);
-            mma_bf16_16816(s, ka[2], kb[2], ka[3], kb[3], qf[j][2], qf[j][3]);
-            mma_bf16_16816(s2, kc[2], kd[2], kc[3], kd[3], qf[j + 1][2], qf[j + 1][3]);
+        for (int j = 0; j < 8; j += 2) {
+            uint32_t a[4], b[4];
+            ldmatrix_x4(kl ^ (j << 5), a);             // ring slots are 256-byte aligned
+            ldmatrix_x4(kl ^ ((j + 1) << 5), b);
+            mma_bf16_16816(s, a[0], a[1], a[2], a[3], qf[j][0], qf[j][1]);
+            mma_bf16_16816(s2, b[0], b[1], b[2], b[3], qf[j + 1][0], qf[j + 1][1]);
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) s[i] += s2[i];
         const float f0 = s[0] * p.scale, f1 = s[1] * p.scale, f2 = s[2] * p.scale, f3 = s[3] * p.scale;
-        if (nvalid == TILE && ncols == 8) {
-            // the common case: sixteen cached tokens, eight heads, nothing to mask
-            st_keep(score_row0 + pos_base, f0, keep);
-            st_keep(score_row0 + pos_base + 8, f2, keep);
-            st_keep(score_row1 + pos_base, f1, keep);
-            st_keep(score_row1 + pos_base + 8, f3, keep);
-            if (hist_on) {
-                atomicAdd(h0 + (score_key_bits(f0) >> hshift), 1u);
-                atomicAdd(h0 + (score_key_bits(f2) >> hshift), 1u);
-                atomicAdd(h1 + (score_key_bits(f1) >> hshift), 1u);
-                atomicAdd(h1 + (score_key_bits(f3) >> hshift), 1u);
+        if (nvalid == TILE) {
+            // the common case: sixteen cached tokens, no row to mask (lanes beyond the group's heads sit out)
+            if (col0) {
+                st_keep(score_row0 + pos_base, f0, keep);
+                st_keep(score_row0 + pos_base + 8, f2, keep);
+                if (hist_on) {
+                    atomicAdd(h0 + (score_key_bits(f0) >> hshift), 1u);
+                    atomicAdd(h0 + (score_key_bits(f2) >> hshift), 1u);
+                }
+                m0 = fmaxf(m0, fmaxf(f0, f2));
             }
-            // the largest stored logit of each head: the value pass takes its softmax weights relative to it
-            m0 = fmaxf(m0, fmaxf(f0, f2));
-            m1 = fmaxf(m1, fmaxf(f1, f3));
+            if (col1) {
+                st_keep(score_row1 + pos_base, f1, keep);
+                st_keep(score_row1 + pos_base + 8, f3, keep);
+                if (hist_on) {
+                    atomicAdd(h1 + (score_key_bits(f1) >> hshift), 1u);
+                    atomicAdd(h1 + (score_key_bits(f3) >> hshift), 1u);
+                }
+                m1 = fmaxf(m1, fmaxf(f1, f3));
+            }
         } else {
             const bool v0 = gid < nvalid, v1 = gid + 8 < nvalid;
             if (col0) {
@@ -372,7 +379,8 @@ __global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams
         if (k1) M1 = __uint_as_float((k1 & 0x80000000u) ? (k1 & 0x7fffffffu) : ~k1) * LOG2E;
     }
     const bool h0 = 2 * tig < ncols && M0 != -INFINITY, h1 = 2 * tig + 1 < ncols && M1 != -INFINITY;
-    const bool plain = ncols == 8 && __all_sync(0xffffffffu, h0 && h1);   // eight heads, each with a finite maximum
+    const bool col0 = 2 * tig < ncols, col1 = 2 * tig + 1 < ncols;
+    const bool plain = __all_sync(0xffffffffu, (h0 || !col0) && (h1 || !col1));   // every head of the group has a finite maximum
     float l0 = 0.f, l1 = 0.f;                          // this lane's share of sum_j p_j
     float o[8][4];
 #pragma unroll
@@ -391,8 +399,8 @@ __global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams
         asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f3) : "r"(vs + slane + 96));
         float p0, p1, p2, p3;
         if (nvalid == TILE && plain) {
-            p0 = fast_exp2(f0 * LOG2E - M0); p1 = fast_exp2(f1 * LOG2E - M1);
-            p2 = fast_exp2(f2 * LOG2E - M0); p3 = fast_exp2(f3 * LOG2E - M1);
+            p0 = col0 ? fast_exp2(f0 * LOG2E - M0) : 0.f; p1 = col1 ? fast_exp2(f1 * LOG2E - M1) : 0.f;
+            p2 = col0 ? fast_exp2(f2 * LOG2E - M0) : 0.f; p3 = col1 ? fast_exp2(f3 * LOG2E - M1) : 0.f;
         } else {
             const bool v0 = gid < nvalid, v1 = gid + 8 < nvalid;
             p0 = (v0 && h0) ? fast_exp2(f0 * LOG2E - M0) : 0.f; p1 = (v0 && h1) ? fast_exp2(f1 * LOG2E - M1) : 0.f;
