@@ -505,4 +505,462 @@ __global__ void __launch_bounds__(NW * 32, 2) value_pass_kernel(const AttnParams
     }
 }
 
+// ---- the same two passes over an 8-bit cache -------------------------------------------------------------------
+// A 16-position tile of E4M3 codes is 2 KB: half the bytes for the same per-tile cost. Both passes therefore
+// work on units of 32 positions (two tiles, 4 KB per ring slot; with pages, two lookups). Row and fragment
+// layouts, the conversion to fp16 in front of the MMAs and the order of the O^T fragments are those of
+// consume_tile8; the key scale goes into the logit scale, the value scale into the partial sums.
+constexpr int UNIT8_TILES = 2;
+constexpr int UNIT8_BYTES = UNIT8_TILES * TILE_BYTES8;       // 4 KB
+
+// ROWC: consecutive positions of a head lie 256 bytes apart (K and V code rows interleaved).
+template <int NW, int STAGES, bool ROWC>
+__global__ void __launch_bounds__(NW * 32, 1) score_pass8_kernel(const AttnParams p) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    __shared__ float s_max[NW][8];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int gid = lane >> 2, tig = lane & 3;
+    constexpr int RING_BYTES = NW * STAGES * UNIT8_BYTES;
+    uint32_t* hist = reinterpret_cast<uint32_t*>(smem + RING_BYTES);
+    const bool hist_on = p.hist != nullptr;
+
+    bool waited = !p.pdl;
+    if (p.pdl && p.wait_first) { pdl_wait(); pdl_trigger(); waited = true; }
+    else if (p.pdl && p.wait_late && p.trigger_early) pdl_trigger();
+
+    const int n_items = p.Hkv;                               // one sequence
+    const int g = blockIdx.x % n_items, part = blockIdx.x / n_items;
+    const int item_ctas = ((int)gridDim.x - g + n_items - 1) / n_items;
+    const int N = max(min(p.ctx_lens[0], p.max_ctx), 0);
+    const int tiles = item_tiles(N);
+    const int units = (tiles + UNIT8_TILES - 1) / UNIT8_TILES;
+    const int head0 = g * p.G, ncols = p.G;
+    const bool col0 = 2 * tig < ncols, col1 = 2 * tig + 1 < ncols;
+    float* const score_row0 = p.scores + (long long)(head0 + min(2 * tig, ncols - 1)) * p.score_stride + gid;
+    float* const score_row1 = p.scores + (long long)(head0 + min(2 * tig + 1, ncols - 1)) * p.score_stride + gid;
+    const int hshift = p.hist_shift;
+    uint32_t* const h0 = hist + ((2 * tig) << (32 - hshift));
+    uint32_t* const h1 = hist + ((2 * tig + 1) << (32 - hshift));
+
+    const uint32_t wbase = smem_u32(smem + (size_t)warp * STAGES * UNIT8_BYTES);
+    // this lane copies the 16-byte piece piece8 of rows row8 + 4 i of a tile (strides count bytes here)
+    const int piece8 = lane & 7, row8 = lane >> 3;
+    const long long four_rows = 4 * p.stride_pos;
+    const long long tile_step = (long long)TILE * p.stride_pos;
+    const uint32_t kdst8 = row8 * ROW_BYTES8 + ((piece8 ^ ((row8 & 1) << 2)) << 4);
+    const uint8_t* const kbase = reinterpret_cast<const uint8_t*>(p.k) + (long long)g * p.stride_head + (long long)row8 * p.stride_pos + piece8 * 16;
+    const uint64_t kv_policy = l2_evict_first_policy();
+    const uint64_t keep = l2_evict_last_policy();
+
+    int* pool = p.tile_ctr + (long long)g * p.ctr_stride;
+    PoolWalk walk;
+    constexpr int GRAB = GRAB_TILES_DENSE;
+    walk.template start<GRAB>(pool, units, item_ctas * NW, part * NW + warp, STAGES + 2, lane);
+
+    constexpr int BAD_A = 1 << 30, BAD_B = 1 << 29, UNIT_MASK = BAD_B - 1;
+    auto tile_valid = [&](int tile) { return max(0, min(TILE, N - tile * TILE)); };
+    // one tile's sixteen code rows into a ring slot half; returns false for a page id outside the pool
+    auto load_tile = [&](uint32_t dst, int tile) -> bool {
+        const uint8_t* src;
+        bool ok = true;
+        if (p.paged) {
+            const int page = __ldg(p.page_table + tile);
+            ok = (unsigned)page < (unsigned)p.num_pages;
+            if (!ok && lane == 0) atomicOr(p.status, STATUS_BAD_PAGE);
+            src = kbase + (ok ? (long long)page * p.stride_page : 0);
+        } else {
+            src = kbase + tile * tile_step;
+        }
+        const int nvalid = ok ? tile_valid(tile) : 0;
+        if (nvalid == TILE) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                cp_async16_full_hint(dst + kdst8 + i * 512, ROWC ? src + i * (8 * HEAD_DIM) : src + i * four_rows, kv_policy);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const bool rv = row8 + 4 * i < nvalid;
+                cp_async16_hint(dst + kdst8 + i * 512, rv ? src + i * four_rows : reinterpret_cast<const uint8_t*>(p.k), rv ? 16 : 0, kv_policy);
+            }
+        }
+        return ok;
+    };
+    auto issue = [&](uint32_t ks, int& u) {
+        const int ta = UNIT8_TILES * u;
+        int flags = load_tile(ks, ta) ? 0 : BAD_A;
+        if (ta + 1 < tiles && !load_tile(ks + TILE_BYTES8, ta + 1)) flags |= BAD_B;
+        u |= flags;
+    };
+
+    int tl[STAGES];
+#pragma unroll
+    for (int s = 0; s < STAGES; ++s) tl[s] = -1;
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) {
+        int t = walk.template next<GRAB>();
+        if (t >= 0) {
+            if (!waited && !p.wait_late && t == units - 1) { pdl_wait(); pdl_trigger(); waited = true; }
+            issue(wbase + s * UNIT8_BYTES, t);
+        }
+        tl[s] = t;
+        cp_async_commit();
+    }
+    if (!waited && !p.wait_late) { pdl_wait(); pdl_trigger(); waited = true; }
+    if (hist_on) {
+        for (int i = threadIdx.x; i < HIST_SMEM_WORDS; i += NW * 32) hist[i] = 0;
+        __syncthreads();
+    }
+    uint32_t qf8[2][8];                                 // the query as fp16, see consume_tile8
+    {
+        const uint4* qp = reinterpret_cast<const uint4*>(p.q + (long long)(head0 + min(gid, ncols - 1)) * HEAD_DIM);
+        const bool on = gid < ncols;
+#pragma unroll
+        for (int sl = 0; sl < 2; ++sl) {
+            const int c = tig + 4 * sl;
+            const uint4 t0 = __ldg(qp + 2 * c), t1 = __ldg(qp + 2 * c + 1);
+            const uint32_t w[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i) qf8[sl][i] = on ? bf16x2_to_f16x2(w[i]) : 0u;
+        }
+    }
+    const float scale = p.scale * (p.k_scale ? __ldg(p.k_scale + g) : 1.f);
+    float m0 = -INFINITY, m1 = -INFINITY;
+    const uint32_t klane = gid * ROW_BYTES8;
+    const uint32_t kswz = (gid & 1) << 2;
+
+    auto key_part = [&](uint32_t ks, int pos_base, int nvalid) {
+        float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
+        const uint32_t krow = ks + klane;
+#pragma unroll
+        for (int sl = 0; sl < 2; ++sl) {
+            uint32_t ka[4], kb[4];
+            const uint32_t off = ((uint32_t)((tig + 4 * sl) ^ kswz)) << 4;
+            lds128(krow + off, ka);                        // row gid, 16 codes
+            lds128(krow + 8 * ROW_BYTES8 + off, kb);       // row gid + 8
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t a0, a2, a1, a3;
+                e4m3x4_to_f16x2x2(ka[i], a0, a2);
+                e4m3x4_to_f16x2x2(kb[i], a1, a3);
+                if (i & 1) mma_f16_16816(s2, a0, a1, a2, a3, qf8[sl][2 * i], qf8[sl][2 * i + 1]);
+                else mma_f16_16816(s, a0, a1, a2, a3, qf8[sl][2 * i], qf8[sl][2 * i + 1]);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) s[i] += s2[i];
+        const float f0 = s[0] * scale, f1 = s[1] * scale, f2 = s[2] * scale, f3 = s[3] * scale;
+        if (nvalid == TILE) {
+            if (col0) {
+                st_keep(score_row0 + pos_base, f0, keep);
+                st_keep(score_row0 + pos_base + 8, f2, keep);
+                if (hist_on) {
+                    atomicAdd(h0 + (score_key_bits(f0) >> hshift), 1u);
+                    atomicAdd(h0 + (score_key_bits(f2) >> hshift), 1u);
+                }
+                m0 = fmaxf(m0, fmaxf(f0, f2));
+            }
+            if (col1) {
+                st_keep(score_row1 + pos_base, f1, keep);
+                st_keep(score_row1 + pos_base + 8, f3, keep);
+                if (hist_on) {
+                    atomicAdd(h1 + (score_key_bits(f1) >> hshift), 1u);
+                    atomicAdd(h1 + (score_key_bits(f3) >> hshift), 1u);
+                }
+                m1 = fmaxf(m1, fmaxf(f1, f3));
+            }
+        } else {
+            const bool v0 = gid < nvalid, v1 = gid + 8 < nvalid;
+            if (col0) {
+                if (v0) st_keep(score_row0 + pos_base, f0, keep);
+                if (v1) st_keep(score_row0 + pos_base + 8, f2, keep);
+            }
+            if (col1) {
+                if (v0) st_keep(score_row1 + pos_base, f1, keep);
+                if (v1) st_keep(score_row1 + pos_base + 8, f3, keep);
+            }
+            if (hist_on) {
+                if (col0) {
+                    if (v0) atomicAdd(h0 + (score_key_bits(f0) >> hshift), 1u);
+                    if (v1) atomicAdd(h0 + (score_key_bits(f2) >> hshift), 1u);
+                }
+                if (col1) {
+                    if (v0) atomicAdd(h1 + (score_key_bits(f1) >> hshift), 1u);
+                    if (v1) atomicAdd(h1 + (score_key_bits(f3) >> hshift), 1u);
+                }
+            }
+            if (v0) { m0 = fmaxf(m0, f0); m1 = fmaxf(m1, f1); }
+            if (v1) { m0 = fmaxf(m0, f2); m1 = fmaxf(m1, f3); }
+        }
+    };
+    auto consume = [&](uint32_t ks, int uf) {
+        const int ta = UNIT8_TILES * (uf & UNIT_MASK);
+        key_part(ks, ta * TILE, (uf & BAD_A) ? 0 : tile_valid(ta));
+        if (ta + 1 < tiles) key_part(ks + TILE_BYTES8, (ta + 1) * TILE, (uf & BAD_B) ? 0 : tile_valid(ta + 1));
+    };
+
+    for (bool live = true; live;) {
+#pragma unroll
+        for (int s = 0; s < STAGES; ++s) {
+            if (tl[s] < 0) { live = false; break; }
+            cp_async_wait<STAGES - 2>();
+            __syncwarp();
+            const int sn = (s + STAGES - 1) % STAGES;
+            int t = walk.template next<GRAB>();
+            if (t >= 0) issue(wbase + sn * UNIT8_BYTES, t);
+            tl[sn] = t;
+            cp_async_commit();
+            consume(wbase + s * UNIT8_BYTES, tl[s]);
+        }
+    }
+    cp_async_wait<0>();
+    __syncwarp();
+    if (!waited) {
+        pdl_wait();
+        if (!p.trigger_early) pdl_trigger();
+        waited = true;
+    }
+    if (hist_on) {
+        __syncthreads();
+        const int nb = 1 << (32 - p.hist_shift);
+        for (int i = threadIdx.x; i < ncols * nb; i += NW * 32) {
+            const uint32_t w = hist[i];
+            if (w) atomicAdd(p.hist + (long long)(head0 + i / nb) * HIST_BINS + (i % nb), w);
+        }
+    }
+#pragma unroll
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+        m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, sh));
+        m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, sh));
+    }
+    if (gid == 0) { s_max[warp][2 * tig] = m0; s_max[warp][2 * tig + 1] = m1; }
+    __syncthreads();
+    if (threadIdx.x < ncols) {
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) M = fmaxf(M, s_max[w][threadIdx.x]);
+        if (M != -INFINITY) atomicMax(p.split_max + head0 + threadIdx.x, score_key_bits(M));
+    }
+    if (part == 0)
+        for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) p.out[(long long)head0 * HEAD_DIM + e] = 0.f;
+    if (threadIdx.x == 0) {
+        int* ctr = p.counters + (long long)g * p.ctr_stride;
+        int old;
+        asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;\n" : "=r"(old) : "l"(ctr) : "memory");
+        if (old == item_ctas - 1) { *ctr = 0; *pool = 0; __threadfence(); }
+    }
+}
+
+template <int NW, int STAGES, bool ROWC>
+__global__ void __launch_bounds__(NW * 32, 2) value_pass8_kernel(const AttnParams p) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    constexpr int SLOT = UNIT8_BYTES + 1024;                // 32 value rows, then 32 logits of up to 8 heads
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int gid = lane >> 2, tig = lane & 3;
+    const int n_items = p.Hkv;
+    const int g = blockIdx.x % n_items, part = blockIdx.x / n_items;
+    const int item_ctas = ((int)gridDim.x - g + n_items - 1) / n_items;
+    const int N = max(min(p.ctx_lens[0], p.max_ctx), 0);
+    const int tiles = item_tiles(N);
+    const int units = (tiles + UNIT8_TILES - 1) / UNIT8_TILES;
+    const int head0 = g * p.G, ncols = p.G;
+
+    const uint32_t wbase = smem_u32(smem + (size_t)warp * STAGES * SLOT);
+    const int piece8 = lane & 7, row8 = lane >> 3;
+    const long long four_rows = 4 * p.stride_pos;
+    const long long tile_step = (long long)TILE * p.stride_pos;
+    const uint32_t vc8 = piece8 ^ row8;                   // row & 7 == row8 ^ ((i & 1) << 2) for rows row8 + 4 i
+    uint32_t vdst8[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) vdst8[i] = row8 * ROW_BYTES8 + i * 512 + ((vc8 ^ (i << 2)) << 4);
+    const uint8_t* const vbase = reinterpret_cast<const uint8_t*>(p.v) + (long long)g * p.stride_head + (long long)row8 * p.stride_pos + piece8 * 16;
+    const uint64_t kv_policy = l2_evict_first_policy();
+    // lane l < 4 * ncols fetches twice 16 bytes (positions 4 (l & 3) .. + 3 of either tile) of head l >> 2's logits
+    const bool score_lane = lane < 4 * ncols;
+    const float* const score_src = p.scores + (long long)(head0 + min(lane >> 2, ncols - 1)) * p.score_stride + 4 * (lane & 3);
+    const uint32_t score_dst = UNIT8_BYTES + (lane >> 2) * 128 + (lane & 3) * 16;
+
+    int* pool = p.tile_ctr + (long long)g * p.ctr_stride;
+    PoolWalk walk;
+    constexpr int GRAB = GRAB_TILES_DENSE;
+    walk.template start<GRAB>(pool, units, item_ctas * NW, part * NW + warp, STAGES + 2, lane);
+
+    constexpr int BAD_A = 1 << 30, BAD_B = 1 << 29, UNIT_MASK = BAD_B - 1;
+    auto tile_valid = [&](int tile) { return max(0, min(TILE, N - tile * TILE)); };
+    auto load_tile = [&](uint32_t dst, int tile) -> bool {
+        const uint8_t* src;
+        bool ok = true;
+        if (p.paged) {
+            const int page = __ldg(p.page_table + tile);
+            ok = (unsigned)page < (unsigned)p.num_pages;
+            if (!ok && lane == 0) atomicOr(p.status, STATUS_BAD_PAGE);
+            src = vbase + (ok ? (long long)page * p.stride_page : 0);
+        } else {
+            src = vbase + tile * tile_step;
+        }
+        const int nvalid = ok ? tile_valid(tile) : 0;
+        if (nvalid == TILE) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                cp_async16_full_hint(dst + vdst8[i & 1] + (i >> 1) * 1024, ROWC ? src + i * (8 * HEAD_DIM) : src + i * four_rows, kv_policy);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const bool rv = row8 + 4 * i < nvalid;
+                cp_async16_hint(dst + vdst8[i & 1] + (i >> 1) * 1024, rv ? src + i * four_rows : reinterpret_cast<const uint8_t*>(p.v), rv ? 16 : 0, kv_policy);
+            }
+        }
+        return ok;
+    };
+    auto issue = [&](uint32_t vs, int& u) {
+        const int ta = UNIT8_TILES * u;
+        int flags = load_tile(vs, ta) ? 0 : BAD_A;
+        if (ta + 1 < tiles && !load_tile(vs + TILE_BYTES8, ta + 1)) flags |= BAD_B;
+        // (logits past the end of the sequence are never used: their rows are masked)
+        if (score_lane) {
+            cp_async16(vs + score_dst, score_src + ta * TILE, 16);
+            if (ta + 1 < tiles) cp_async16(vs + score_dst + 64, score_src + ta * TILE + TILE, 16);
+        }
+        u |= flags;
+    };
+
+    float M0 = -INFINITY, M1 = -INFINITY;
+    {
+        const uint32_t k0 = (2 * tig < ncols) ? __ldcg(p.split_max + head0 + 2 * tig) : 0u;
+        const uint32_t k1 = (2 * tig + 1 < ncols) ? __ldcg(p.split_max + head0 + 2 * tig + 1) : 0u;
+        if (k0) M0 = __uint_as_float((k0 & 0x80000000u) ? (k0 & 0x7fffffffu) : ~k0) * LOG2E;
+        if (k1) M1 = __uint_as_float((k1 & 0x80000000u) ? (k1 & 0x7fffffffu) : ~k1) * LOG2E;
+    }
+    const bool h0 = 2 * tig < ncols && M0 != -INFINITY, h1 = 2 * tig + 1 < ncols && M1 != -INFINITY;
+    float l0 = 0.f, l1 = 0.f;
+    float o[8][4];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) { o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f; }
+    // logits of (position gid | gid + 8 of a tile, heads 2tig | 2tig + 1): head h's 32 floats start at 128 * h
+    const uint32_t slane = UNIT8_BYTES + (2 * tig) * 128 + gid * 4;
+    const int rr = lane & 7, mi = lane >> 3;
+    const uint32_t vlane = (rr + ((mi >> 1) << 3)) * ROW_BYTES8;
+    const uint32_t vswz = rr;
+
+    auto value_part = [&](uint32_t vs, uint32_t sl, int nvalid) {
+        float f0, f1, f2, f3;
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f0) : "r"(sl));
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f2) : "r"(sl + 32));
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f1) : "r"(sl + 128));
+        asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(f3) : "r"(sl + 160));
+        const bool v0 = gid < nvalid, v1 = gid + 8 < nvalid;
+        const float p0 = (v0 && h0) ? fast_exp2(f0 * LOG2E - M0) : 0.f, p1 = (v0 && h1) ? fast_exp2(f1 * LOG2E - M1) : 0.f;
+        const float p2 = (v1 && h0) ? fast_exp2(f2 * LOG2E - M0) : 0.f, p3 = (v1 && h1) ? fast_exp2(f3 * LOG2E - M1) : 0.f;
+        l0 += p0 + p2;
+        l1 += p1 + p3;
+        const uint32_t pb0 = movmatrix_trans(pack_f16(p0, p1));
+        const uint32_t pb1 = movmatrix_trans(pack_f16(p2, p3));
+        const uint32_t vb = vs + vlane;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            uint32_t m[4];
+            ldmatrix_x4_trans(vb + ((uint32_t)((2 * u + (mi & 1)) ^ vswz) << 4), m);
+            uint32_t x0, y0, x2, y2, x1, y1, x3, y3;
+            e4m3x4_to_f16x2x2(__byte_perm(m[0], 0, 0x3120), x0, y0);
+            e4m3x4_to_f16x2x2(__byte_perm(m[2], 0, 0x3120), x2, y2);
+            mma_f16_16816(o[2 * u], x0, y0, x2, y2, pb0, pb1);
+            e4m3x4_to_f16x2x2(__byte_perm(m[1], 0, 0x3120), x1, y1);
+            e4m3x4_to_f16x2x2(__byte_perm(m[3], 0, 0x3120), x3, y3);
+            mma_f16_16816(o[2 * u + 1], x1, y1, x3, y3, pb0, pb1);
+        }
+    };
+    auto consume = [&](uint32_t vs, int uf) {
+        const int ta = UNIT8_TILES * (uf & UNIT_MASK);
+        value_part(vs, vs + slane, (uf & BAD_A) ? 0 : tile_valid(ta));
+        if (ta + 1 < tiles) value_part(vs + TILE_BYTES8, vs + slane + 64, (uf & BAD_B) ? 0 : tile_valid(ta + 1));
+    };
+
+    int tl[STAGES];
+#pragma unroll
+    for (int s = 0; s < STAGES; ++s) tl[s] = -1;
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) {
+        int t = walk.template next<GRAB>();
+        if (t >= 0) issue(wbase + s * SLOT, t);
+        tl[s] = t;
+        cp_async_commit();
+    }
+    for (bool live = true; live;) {
+#pragma unroll
+        for (int s = 0; s < STAGES; ++s) {
+            if (tl[s] < 0) { live = false; break; }
+            cp_async_wait<STAGES - 2>();
+            __syncwarp();
+            const int sn = (s + STAGES - 1) % STAGES;
+            int t = walk.template next<GRAB>();
+            if (t >= 0) issue(wbase + sn * SLOT, t);
+            tl[sn] = t;
+            cp_async_commit();
+            consume(wbase + s * SLOT, tl[s]);
+        }
+    }
+    cp_async_wait<0>();
+#pragma unroll
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+        l0 += __shfl_xor_sync(0xffffffffu, l0, sh);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, sh);
+    }
+    __syncthreads();                                   // all rings drained; reuse the shared memory
+    const float vscale = p.v_scale ? __ldg(p.v_scale + g) : 1.f;
+    float* mo = reinterpret_cast<float*>(smem);       // [NW][8][128]
+    float* ml = mo + NW * 8 * HEAD_DIM;               // [NW][8]
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {                     // rows of the O^T fragments are d = 16t + 2gid and + 1 here
+        float* w0 = mo + ((warp * 8 + 2 * tig) * HEAD_DIM);
+        float* w1 = w0 + HEAD_DIM;
+        w0[16 * t + 2 * gid] = o[t][0] * vscale;
+        w1[16 * t + 2 * gid] = o[t][1] * vscale;
+        w0[16 * t + 2 * gid + 1] = o[t][2] * vscale;
+        w1[16 * t + 2 * gid + 1] = o[t][3] * vscale;
+    }
+    if (gid == 0) { ml[warp * 8 + 2 * tig] = l0; ml[warp * 8 + 2 * tig + 1] = l1; }
+    __syncthreads();
+    for (int e = threadIdx.x; e < ncols * (HEAD_DIM / 4); e += NW * 32) {
+        const int col = e >> 5, c = (e & 31) * 4;
+        float4 O = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int w = 0; w < NW; ++w) {
+            const float4 t = *reinterpret_cast<const float4*>(mo + (w * 8 + col) * HEAD_DIM + c);
+            O.x += t.x; O.y += t.y; O.z += t.z; O.w += t.w;
+        }
+        if (O.x != 0.f || O.y != 0.f || O.z != 0.f || O.w != 0.f)
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};\n" ::"l"(p.out + (long long)(head0 + col) * HEAD_DIM + c),
+                         "f"(O.x), "f"(O.y), "f"(O.z), "f"(O.w) : "memory");
+    }
+    if (threadIdx.x < ncols) {
+        float L = 0.f;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) L += ml[w * 8 + threadIdx.x];
+        if (L != 0.f) atomicAdd(p.split_sum + head0 + threadIdx.x, L);
+    }
+    __shared__ int s_last;
+    __syncthreads();
+    int* ctr = p.counters + (long long)g * p.ctr_stride;
+    if (threadIdx.x == 0) {
+        int old;
+        asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;\n" : "=r"(old) : "l"(ctr) : "memory");
+        s_last = (old == item_ctas - 1);
+    }
+    __syncthreads();
+    if (s_last) {
+        float* const rows = p.out_final ? p.out_final : p.out;
+        for (int e = threadIdx.x; e < ncols * HEAD_DIM; e += NW * 32) {
+            const float L = __ldcg(p.split_sum + head0 + (e >> 7));
+            const float O = __ldcg(p.out + (long long)head0 * HEAD_DIM + e);
+            rows[(long long)head0 * HEAD_DIM + e] = (L > 0.f) ? O / L : 0.f;
+        }
+        __syncthreads();
+        if (threadIdx.x < ncols) { p.split_sum[head0 + threadIdx.x] = 0.f; p.split_max[head0 + threadIdx.x] = 0u; }
+        if (threadIdx.x == 0) { *ctr = 0; *pool = 0; }
+    }
+}
+
 }  // namespace tidal

@@ -325,6 +325,8 @@ constexpr int SCORE_NW = 16, SCORE_STAGES = 3;     // key rows only, 4 KB per ti
 constexpr int VALUE_NW = 8, VALUE_STAGES = 3;      // value rows + logits, 4.5 KB per tile: two CTAs per SM, also beside a sparse layer's CTA
 constexpr size_t SCORE_SMEM = (size_t)SCORE_NW * SCORE_STAGES * TILE_BYTES + HIST_SMEM + 1024;
 constexpr size_t VALUE_SMEM = (size_t)VALUE_NW * VALUE_STAGES * (TILE_BYTES + 512) + 1024;
+constexpr int VALUE_NW8 = 6;                        // 8-bit caches: 32 positions (4 KB of codes + 1 KB of logits) per slot
+constexpr size_t VALUE_SMEM8 = (size_t)VALUE_NW8 * VALUE_STAGES * (UNIT8_BYTES + 1024) + 1024;
 constexpr int COMPACT_LIST_SMEM = 12288;      // candidates the compacting top-k keeps in shared memory
 
 int dense_grid(const tidal_ctx* ctx, const tidal_kv_t* kv) {
@@ -346,9 +348,9 @@ SelectPlan select_plan(const tidal_ctx* ctx, const tidal_kv_t* kv, int Hi, int k
 }
 
 // Inside a step a selection layer can run as two passes (split_select_kernels.cuh) when it has one
-// sequence, per-head scores with the fused histogram, a bf16 cache and fp32 outputs.
+// sequence, per-head scores with the fused histogram and fp32 outputs.
 bool can_split(const tidal_ctx* ctx, const tidal_kv_t* kv, const SelectPlan& sp) {
-    return ctx->split_select && ctx->layer_overlap && !ctx->out_bf16 && kv->kv_dtype == TIDAL_KV_BF16 && kv->batch == 1 &&
+    return ctx->split_select && ctx->layer_overlap && !ctx->out_bf16 && kv->batch == 1 &&
            !sp.agg && sp.fuse && !sp.compact && pooled_splits(kv, kv->num_kv_heads, dense_grid(ctx, kv)) > 0;
 }
 
@@ -440,8 +442,14 @@ tidal_status_t run_score_pass(tidal_ctx* ctx, const tidal_kv_t* kv, const void* 
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     ctx->launches++;
-    const cudaError_t e = kv->stride_pos == 2 * HEAD_DIM ? cudaLaunchKernelEx(&cfg, score_pass_kernel<SCORE_NW, SCORE_STAGES, true>, a)
-                                                         : cudaLaunchKernelEx(&cfg, score_pass_kernel<SCORE_NW, SCORE_STAGES, false>, a);
+    const bool rowc = kv->stride_pos == 2 * HEAD_DIM;     // K and V rows interleaved: constant offsets between the rows of a tile
+    cudaError_t e;
+    if (kv->kv_dtype == TIDAL_KV_FP8_E4M3)
+        e = rowc ? cudaLaunchKernelEx(&cfg, score_pass8_kernel<SCORE_NW, SCORE_STAGES, true>, a)
+                 : cudaLaunchKernelEx(&cfg, score_pass8_kernel<SCORE_NW, SCORE_STAGES, false>, a);
+    else
+        e = rowc ? cudaLaunchKernelEx(&cfg, score_pass_kernel<SCORE_NW, SCORE_STAGES, true>, a)
+                 : cudaLaunchKernelEx(&cfg, score_pass_kernel<SCORE_NW, SCORE_STAGES, false>, a);
     return e == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
 }
 
@@ -466,7 +474,11 @@ tidal_status_t run_value_pass(tidal_ctx* ctx, const tidal_kv_t* kv, float* out, 
     a.splits_per_item = per_item;
     if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
         return TIDAL_ERR_CUDA;
-    if (kv->stride_pos == 2 * HEAD_DIM) value_pass_kernel<VALUE_NW, VALUE_STAGES, true><<<grid, VALUE_NW * 32, VALUE_SMEM, ctx->side>>>(a);
+    const bool rowc = kv->stride_pos == 2 * HEAD_DIM;
+    if (kv->kv_dtype == TIDAL_KV_FP8_E4M3) {
+        if (rowc) value_pass8_kernel<VALUE_NW8, VALUE_STAGES, true><<<grid, VALUE_NW8 * 32, VALUE_SMEM8, ctx->side>>>(a);
+        else value_pass8_kernel<VALUE_NW8, VALUE_STAGES, false><<<grid, VALUE_NW8 * 32, VALUE_SMEM8, ctx->side>>>(a);
+    } else if (rowc) value_pass_kernel<VALUE_NW, VALUE_STAGES, true><<<grid, VALUE_NW * 32, VALUE_SMEM, ctx->side>>>(a);
     else value_pass_kernel<VALUE_NW, VALUE_STAGES, false><<<grid, VALUE_NW * 32, VALUE_SMEM, ctx->side>>>(a);
     ctx->launches++;
     if (cudaGetLastError() != cudaSuccess) return TIDAL_ERR_CUDA;
@@ -713,6 +725,10 @@ tidal_status_t tidal_create(tidal_ctx_t** out, int device, size_t workspace_byte
     const bool split_ok =
         cudaFuncSetAttribute(score_pass_kernel<SCORE_NW, SCORE_STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCORE_SMEM) == cudaSuccess &&
         cudaFuncSetAttribute(score_pass_kernel<SCORE_NW, SCORE_STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCORE_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(score_pass8_kernel<SCORE_NW, SCORE_STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCORE_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(score_pass8_kernel<SCORE_NW, SCORE_STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCORE_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(value_pass8_kernel<VALUE_NW8, VALUE_STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VALUE_SMEM8) == cudaSuccess &&
+        cudaFuncSetAttribute(value_pass8_kernel<VALUE_NW8, VALUE_STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VALUE_SMEM8) == cudaSuccess &&
         cudaFuncSetAttribute(value_pass_kernel<VALUE_NW, VALUE_STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VALUE_SMEM) == cudaSuccess &&
         cudaFuncSetAttribute(value_pass_kernel<VALUE_NW, VALUE_STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VALUE_SMEM) == cudaSuccess;
     const size_t topk_smem = 2 * (size_t)(MAX_CTX / 32) * sizeof(unsigned) + 8192 * sizeof(uint2);

@@ -539,6 +539,7 @@ def test_decode_step_replays_from_a_cuda_graph(td):
     eager = [o.clone() for o in outs]
     eager_idx = step.idx.clone()
     side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())      # the inputs were built on the current stream
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.stream(side):
         with torch.cuda.graph(graph, stream=side):
@@ -577,6 +578,7 @@ def test_library_records_and_replays_step_graphs(td):
         return [o.clone() for o in outs], step.idx.clone()
 
     side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())      # the inputs were built on the current stream
     for new_lens in (lens0, (lens0 // 2).clamp(min=70), lens0):
         layers[0].ctx_lens.copy_(new_lens)
         ref_outs, ref_idx = run_direct()
@@ -655,6 +657,8 @@ def test_two_contexts_on_two_streams_do_not_interfere(td):
     other = binding.Tidal(0)
     try:
         sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+        sa.wait_stream(torch.cuda.current_stream())        # the inputs were built on the current stream
+        sb.wait_stream(torch.cuda.current_stream())
         outs_a = [torch.zeros_like(o) for o in ref_outs]
         outs_b = [torch.zeros_like(o) for o in ref_outs]
         step_a = td.make_step(sched, layers, qs, outs_a, w.k)
@@ -853,6 +857,7 @@ def test_reserve_then_capture_the_first_call(td):
         outs = [torch.zeros_like(o) for o in ref_outs]
         step = fresh.make_step(sched, layers, qs, outs, w.k)
         side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())      # the inputs were built on the current stream
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.stream(side):
             with torch.cuda.graph(graph, stream=side):
@@ -1095,6 +1100,7 @@ def test_overlapping_layers_repeatably_equal_the_non_overlapped_step(td, shape):
         lays = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(L)]
     outs = [torch.zeros(w.batch, w.num_q_heads, 128, device=DEV) for _ in range(L)]
     side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())      # the inputs were built on the current stream
     with torch.cuda.stream(side):
         td.set_layer_overlap(False)
         try:
@@ -1121,14 +1127,24 @@ def test_overlapping_layers_repeatably_equal_the_non_overlapped_step(td, shape):
     assert td.device_status() == binding.OK
 
 
-@pytest.mark.parametrize("layout", ["hnd_interleaved", "nhd_separate", "paged"])
-@pytest.mark.parametrize("Hq,Hkv,N,k", [(32, 8, 20011, 1024), (16, 16, 24000, 900), (16, 2, 40001, 3000), (8, 4, 70000, 2048)])
-def test_two_pass_selection_layers_match_the_oracle(td, layout, Hq, Hkv, N, k):
+def _two_pass_cases():
+    shapes = [(32, 8, 20011, 1024), (16, 16, 24000, 900), (16, 2, 40001, 3000), (8, 4, 70000, 2048)]
+    cases = [(layout, *shape, False) for layout in ("hnd_interleaved", "nhd_separate", "paged") for shape in shapes]
+    # the same over caches of E4M3 codes (units of 32 positions: lengths that end in the first and in the second
+    # tile of a unit, a single tile, three tiles)
+    cases += [(layout, *shape, True) for layout in ("hnd_interleaved", "paged") for shape in shapes]
+    cases += [("paged", 32, 8, 20011 + 16, 1024, True), ("hnd_interleaved", 8, 1, 15, 8, True),
+              ("paged", 8, 2, 16 * 2 + 3, 16, True), ("hnd_interleaved", 16, 4, 16 * 64, 100, True)]
+    return cases
+
+
+@pytest.mark.parametrize("layout,Hq,Hkv,N,k,fp8", _two_pass_cases())
+def test_two_pass_selection_layers_match_the_oracle(td, layout, Hq, Hkv, N, k, fp8):
     """Inside a step (one sequence, per-head sets) a selection layer runs as a key pass and a value pass on
     two streams. Its output, its token sets and the sparse layers after it against the oracle, for groups of
-    1, 2, 4 and 8, context lengths with a ragged last tile, all layouts; and against the fused kernel that the
-    single-layer call uses. Two selection layers in a row share the score buffer: the second key pass must
-    wait for the first value pass."""
+    1, 2, 4 and 8, context lengths with a ragged last tile, all layouts, bf16 and FP8 caches; and against the
+    fused kernel that the single-layer call uses. Two selection layers in a row share the score buffer: the
+    second key pass must wait for the first value pass."""
     sched = [0, 1, 1, 2, 2]
     w = wl(1, Hq, Hkv, N, k, planted=8, seed=97, layers=len(sched))
     qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
@@ -1137,7 +1153,10 @@ def test_two_pass_selection_layers_match_the_oracle(td, layout, Hq, Hkv, N, k):
         lays = [synth.make_layer(w, i, DEV, layout="paged", q=qs[i], page_table=pt, num_pages=total) for i in range(len(sched))]
     else:
         lays = [synth.make_layer(w, i, DEV, layout=layout, q=qs[i]) for i in range(len(sched))]
+    if fp8:
+        lays = [synth.to_fp8(lay) for lay in lays]
     side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())      # the inputs were built on the current stream
     with torch.cuda.stream(side):
         outs, idx, cnt = td.decode_step(sched, lays, qs, w.k)
         side.synchronize()
