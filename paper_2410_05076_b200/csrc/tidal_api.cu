@@ -325,7 +325,7 @@ constexpr int SCORE_NW = 16, SCORE_STAGES = 3;     // key rows only, 4 KB per ti
 constexpr int VALUE_NW = 8, VALUE_STAGES = 3;      // value rows + logits, 4.5 KB per tile: two CTAs per SM, also beside a sparse layer's CTA
 constexpr size_t SCORE_SMEM = (size_t)SCORE_NW * SCORE_STAGES * TILE_BYTES + HIST_SMEM + 1024;
 constexpr size_t VALUE_SMEM = (size_t)VALUE_NW * VALUE_STAGES * (TILE_BYTES + 512) + 1024;
-constexpr int VALUE_NW8 = 6;                        // 8-bit caches: 32 positions (4 KB of codes + 1 KB of logits) per slot
+constexpr int VALUE_NW8 = 7;                        // 8-bit caches: 32 positions (4 KB of codes + 1 KB of logits) per slot
 constexpr size_t VALUE_SMEM8 = (size_t)VALUE_NW8 * VALUE_STAGES * (UNIT8_BYTES + 1024) + 1024;
 constexpr int COMPACT_LIST_SMEM = 12288;      // candidates the compacting top-k keeps in shared memory
 
