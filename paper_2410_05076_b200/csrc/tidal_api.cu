@@ -76,6 +76,16 @@ struct tidal_ctx {
     std::vector<StepGraph> graphs;
     uint64_t graph_clock = 0;
     bool graphs_enabled = true;
+    // The call before this one, byte for byte (arguments, the arrays they point to, the settings and the
+    // workspace addresses): a step loop repeats it, and then validation, layout and key building are skipped.
+    struct LastCall {
+        std::vector<unsigned char> raw;
+        cudaGraphExec_t exec = nullptr;
+        int launches = 0;
+    } last;
+    std::vector<unsigned char> raw_scratch;
+    cudaGraphExec_t ran_exec = nullptr;         // set by run_graphed: the graph it launched, if any
+    int ran_launches = 0;
 };
 
 namespace {
@@ -183,6 +193,7 @@ size_t ws_bytes_for(const tidal_kv_t* kv, int k, int num_layers_host) {
 }
 
 void drop_graphs(tidal_ctx* ctx) {
+    ctx->last.exec = nullptr;
     if (ctx->graphs.empty()) return;
     cudaDeviceSynchronize();
     for (auto& g : ctx->graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
@@ -653,6 +664,7 @@ bool graphable(const tidal_ctx* ctx, cudaStream_t st) {
 template <typename F>
 tidal_status_t run_graphed(tidal_ctx* ctx, KeyBuilder& kb, cudaStream_t st, F&& enqueue) {
     constexpr size_t MAX_GRAPHS = 16;
+    ctx->ran_exec = nullptr;
     if (!graphable(ctx, st)) return enqueue();
     ++ctx->graph_clock;
     for (auto& g : ctx->graphs) {
@@ -660,6 +672,7 @@ tidal_status_t run_graphed(tidal_ctx* ctx, KeyBuilder& kb, cudaStream_t st, F&& 
             g.last_use = ctx->graph_clock;
             if (cudaGraphLaunch(g.exec, st) != cudaSuccess) return TIDAL_ERR_CUDA;
             ctx->launches += g.launches;
+            ctx->ran_exec = g.exec; ctx->ran_launches = g.launches;
             return TIDAL_OK;
         }
     }
@@ -683,6 +696,7 @@ tidal_status_t run_graphed(tidal_ctx* ctx, KeyBuilder& kb, cudaStream_t st, F&& 
         size_t victim = 0;
         for (size_t i = 1; i < ctx->graphs.size(); ++i)
             if (ctx->graphs[i].last_use < ctx->graphs[victim].last_use) victim = i;
+        if (ctx->last.exec == ctx->graphs[victim].exec) ctx->last.exec = nullptr;
         cudaGraphExecDestroy(ctx->graphs[victim].exec);   // deferred by the runtime while a launch is in flight
         ctx->graphs.erase(ctx->graphs.begin() + victim);
     }
@@ -694,7 +708,46 @@ tidal_status_t run_graphed(tidal_ctx* ctx, KeyBuilder& kb, cudaStream_t st, F&& 
     ctx->graphs.push_back(std::move(g));
     if (cudaGraphLaunch(exec, st) != cudaSuccess) return TIDAL_ERR_CUDA;
     ctx->launches += recorded;
+    ctx->ran_exec = exec; ctx->ran_launches = recorded;
     return TIDAL_OK;
+}
+
+// The bytes that decide what a step call does: compared with the previous call's before anything else.
+void raw_call_key(std::vector<unsigned char>& r, const tidal_ctx* ctx, int tag, int32_t num_layers, const uint8_t* schedule,
+                  const tidal_kv_t* kvs, const void* const* qs, float* const* outs, const void* p0, const void* p1,
+                  int32_t k, int32_t granularity, cudaStream_t st) {
+    struct Head {
+        int tag; int32_t num_layers, k, granularity; cudaStream_t st; const void *p0, *p1, *ws, *state;
+        int out_bf16, attend_newest, layer_overlap, split_select; float select_margin;
+    } h;
+    std::memset(&h, 0, sizeof h);
+    h.tag = tag; h.num_layers = num_layers; h.k = k; h.granularity = granularity; h.st = st; h.p0 = p0; h.p1 = p1;
+    h.ws = ctx->ws; h.state = ctx->state; h.out_bf16 = ctx->out_bf16; h.attend_newest = ctx->attend_newest;
+    h.layer_overlap = ctx->layer_overlap; h.split_select = ctx->split_select; h.select_margin = ctx->select_margin;
+    const size_t L = (size_t)num_layers;
+    const size_t n_q = qs ? L * sizeof(void*) : 0, n_o = outs ? L * sizeof(void*) : 0;
+    r.resize(sizeof h + L + L * sizeof(tidal_kv_t) + n_q + n_o);
+    unsigned char* d = r.data();
+    std::memcpy(d, &h, sizeof h); d += sizeof h;
+    std::memcpy(d, schedule, L); d += L;
+    std::memcpy(d, kvs, L * sizeof(tidal_kv_t)); d += L * sizeof(tidal_kv_t);
+    if (n_q) { std::memcpy(d, qs, n_q); d += n_q; }
+    if (n_o) std::memcpy(d, outs, n_o);
+}
+
+// Same call as the last one, which ran as a graph: launch that graph again.
+bool replay_last(tidal_ctx* ctx, cudaStream_t st, tidal_status_t& rc) {
+    if (!ctx->last.exec || ctx->raw_scratch != ctx->last.raw || !graphable(ctx, st)) return false;
+    rc = cudaGraphLaunch(ctx->last.exec, st) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+    if (rc == TIDAL_OK) ctx->launches += ctx->last.launches;
+    return true;
+}
+
+void remember_last(tidal_ctx* ctx) {
+    if (!ctx->ran_exec) { ctx->last.exec = nullptr; return; }
+    ctx->last.raw = ctx->raw_scratch;
+    ctx->last.exec = ctx->ran_exec;
+    ctx->last.launches = ctx->ran_launches;
 }
 
 }  // namespace
@@ -983,20 +1036,27 @@ tidal_status_t tidal_decode_step(tidal_ctx_t* ctx, int32_t num_layers, const uin
                                  int32_t* idx_count, void* stream) {
     if (!ctx || num_layers <= 0 || !schedule || !kv_per_layer || !q_per_layer || !out_per_layer || !idx || k <= 0)
         return TIDAL_ERR_INVALID;
+    if (num_layers > 1024) return TIDAL_ERR_INVALID;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
-    tidal_status_t rc = decode_step_prepare(ctx, num_layers, schedule, kv_per_layer, q_per_layer, out_per_layer, k,
-                                            granularity, 0);
+    tidal_status_t rc;
+    raw_call_key(ctx->raw_scratch, ctx, 0, num_layers, schedule, kv_per_layer, q_per_layer, out_per_layer, idx, idx_count, k, granularity, st);
+    if (replay_last(ctx, st, rc)) return rc;
+    rc = decode_step_prepare(ctx, num_layers, schedule, kv_per_layer, q_per_layer, out_per_layer, k, granularity, 0);
     if (rc != TIDAL_OK) return rc;
+    // (the workspace may just have moved: the remembered bytes must name the addresses the graph was built with)
+    raw_call_key(ctx->raw_scratch, ctx, 0, num_layers, schedule, kv_per_layer, q_per_layer, out_per_layer, idx, idx_count, k, granularity, st);
     KeyBuilder kb;
     step_key(kb, ctx, 0, num_layers, schedule, kv_per_layer, k, granularity, 0);
     kb.add_raw(q_per_layer, sizeof(void*) * (size_t)num_layers);
     kb.add_raw(out_per_layer, sizeof(void*) * (size_t)num_layers);
     kb.add(idx); kb.add(idx_count);
-    return run_graphed(ctx, kb, st, [&]() {
+    rc = run_graphed(ctx, kb, st, [&]() {
         return decode_step_enqueue(ctx, num_layers, schedule, kv_per_layer, q_per_layer, out_per_layer, k, granularity,
                                    idx, idx_count, 0, st);
     });
+    if (rc == TIDAL_OK) remember_last(ctx); else ctx->last.exec = nullptr;
+    return rc;
 }
 
 tidal_status_t tidal_set_attend_newest(tidal_ctx_t* ctx, int32_t enabled) {
@@ -1037,9 +1097,15 @@ tidal_status_t tidal_decode_step_host(tidal_ctx_t* ctx, int32_t num_layers, cons
     if (!ctx || num_layers <= 0 || num_layers > 1024 || !schedule || !kv_per_layer || !q_host || !out_host || k <= 0)
         return TIDAL_ERR_INVALID;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return TIDAL_ERR_CUDA;
-    tidal_status_t rc = check_kv(&kv_per_layer[0]);
-    if (rc != TIDAL_OK) return rc;
     cudaStream_t st = (cudaStream_t)stream;
+    tidal_status_t rc;
+    raw_call_key(ctx->raw_scratch, ctx, 1, num_layers, schedule, kv_per_layer, nullptr, nullptr, q_host, out_host, k, granularity, st);
+    if (replay_last(ctx, st, rc)) {
+        if (rc != TIDAL_OK) return rc;
+        return cudaStreamSynchronize(st) == cudaSuccess ? TIDAL_OK : TIDAL_ERR_CUDA;
+    }
+    rc = check_kv(&kv_per_layer[0]);
+    if (rc != TIDAL_OK) return rc;
     // Size the workspace for every layer first so that the staging pointers stay put.
     size_t need = 0;
     for (int i = 0; i < num_layers; ++i) {
@@ -1105,7 +1171,14 @@ tidal_status_t tidal_decode_step_host(tidal_ctx_t* ctx, int32_t num_layers, cons
         step_key(kb, ctx, 1, num_layers, schedule, kv_per_layer, k, granularity, num_layers);
         kb.add(q_host); kb.add(out_host);
         rc = run_graphed(ctx, kb, st, enqueue);
+        if (rc == TIDAL_OK) {
+            raw_call_key(ctx->raw_scratch, ctx, 1, num_layers, schedule, kv_per_layer, nullptr, nullptr, q_host, out_host, k, granularity, st);
+            remember_last(ctx);
+        } else {
+            ctx->last.exec = nullptr;
+        }
     } else {
+        ctx->last.exec = nullptr;
         rc = enqueue();
     }
     if (rc != TIDAL_OK) return rc;
