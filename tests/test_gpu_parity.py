@@ -609,6 +609,60 @@ def test_library_records_and_replays_step_graphs(td):
     assert td.device_status() == binding.OK
 
 
+def test_a_repeated_call_is_replayed_only_while_nothing_changes(td):
+    """A step call that repeats the previous one byte for byte skips validation and launches the same graph
+    again; any change (another budget, other output buffers, other queries, a setting) must take the long
+    way. Two steps over the same caches are interleaved and every result is compared with the same step
+    enqueued kernel by kernel."""
+    sched = [0, 1, 2, 2]
+    w = wl(1, 8, 2, 3000, 64, seed=37, layers=len(sched))
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    qs_b = [synth.make_q(w, i + 10, DEV) for i in range(len(sched))]
+    layers = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(len(sched))]
+    outs_a = [torch.zeros(1, 8, 128, device=DEV) for _ in sched]
+    outs_b = [torch.zeros(1, 8, 128, device=DEV) for _ in sched]
+    step_a = td.make_step(sched, layers, qs, outs_a, 64)
+    step_b = td.make_step(sched, layers, qs_b, outs_b, 32)
+
+    def reference(step, outs):
+        step()                                            # default stream: kernel by kernel
+        torch.cuda.synchronize()
+        ref = ([o.clone() for o in outs], step.idx.clone())
+        for o in outs:
+            o.zero_()
+        step.idx.fill_(-7)
+        torch.cuda.synchronize()
+        return ref
+
+    ref_a, ref_b = reference(step_a, outs_a), reference(step_b, outs_b)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())      # the inputs were built on the current stream
+    with torch.cuda.stream(side):
+        for which in "aabaabbbab":
+            step, outs, ref = (step_a, outs_a, ref_a) if which == "a" else (step_b, outs_b, ref_b)
+            for o in outs:
+                o.zero_()
+            step.idx.fill_(-7)
+            step()
+            side.synchronize()
+            assert torch.equal(step.idx, ref[1]), which
+            for o, r in zip(outs, ref[0]):
+                assert torch.allclose(o, r, rtol=0, atol=5e-4), which
+        # a setting changes between two otherwise identical calls
+        step_a()
+        td.set_layer_overlap(False)
+        try:
+            for o in outs_a:
+                o.zero_()
+            step_a()
+            side.synchronize()
+        finally:
+            td.set_layer_overlap(True)
+        for o, r in zip(outs_a, ref_a[0]):
+            assert torch.allclose(o, r, rtol=0, atol=5e-4)
+    assert td.device_status() == binding.OK
+
+
 def test_bf16_outputs_are_the_fp32_results_rounded(td):
     """With the bf16 output type every call writes the rounded fp32 result; everything else is unchanged."""
     sched = [0, 1, 2]
