@@ -1,4 +1,5 @@
-// A token selection layer in two passes over the cache (one sequence, bf16, one set per query head).
+// A token selection layer in two passes over the cache (one sequence, one set per query head; bf16 caches,
+// and at the end of this file caches of E4M3 codes).
 //
 // Algorithm 1's selection layer needs the scaled logits of every cached token twice: for the softmax
 // of its own output and for argTopK. The fused kernel (attn_kernel<MODE_SELECT>) streams K and V
@@ -11,11 +12,10 @@
 //   value_pass_kernel  streams the VALUE rows only: softmax weights exp(s - M) come from the stored logits
 //                      and the final M, so every partial result has the same scale and CTAs simply add
 //                      their part of sum_j p_j v_j and of sum_j p_j to the output row and to the head's sum
-//                      with atomics; the last CTA of a KV head to finish divides the rows by the sums.
+//                      with reductions; the last CTA of a KV head to finish divides the rows by the sums.
 //
-// The step driver launches the value pass on a second stream, so that it runs beside the top-k and the
-// first sparse layers that follow: the top-k's latency chain and the ramp of the sparse chain are filled
-// with value rows streaming. Key and value rows interleave in memory at 256-byte granularity; reading every
+// The step driver launches the value pass on a second stream, so that it runs beside the top-k: the layer
+// then costs what its two streaming passes cost, the top-k's latency chain hides behind the second. Key and value rows interleave in memory at 256-byte granularity; reading every
 // other 256-byte row costs HBM nothing (measured: the same useful bandwidth as the dense stream).
 #pragma once
 
