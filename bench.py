@@ -500,7 +500,7 @@ def main():
                                 "head, written once and read back from L2) are not in the denominator")
     if select_entry:
         # inside a step the selection layer runs as key pass + value pass where that applies, else fused
-        two_pass = args.granularity == "qhead" and w.batch == 1 and args.kv_dtype == "bf16" and traffic.get("score") is not None
+        two_pass = args.granularity == "qhead" and w.batch == 1 and traffic.get("score") is not None
         parts = ("score", "value", "topk") if two_pass else ("select", "topk")
         select_entry["traffic"] = sum(traffic[k] for k in parts) if all(traffic.get(k) is not None for k in parts) else None
         select_entry["kernel"] = ("score_pass_kernel + value_pass_kernel + top-k (selection layers, two passes)" if two_pass

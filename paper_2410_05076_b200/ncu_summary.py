@@ -23,9 +23,9 @@ def kernel_key(name: str):
         return "select"
     if "attn_kernel<2" in name or "attn_kernel<(int)2" in name:
         return "sparse"
-    if "score_pass_kernel" in name:
+    if "score_pass" in name:
         return "score"
-    if "value_pass_kernel" in name:
+    if "value_pass" in name:
         return "value"
     if "topk" in name:
         return "topk"
