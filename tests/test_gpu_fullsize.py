@@ -147,27 +147,3 @@ def test_whole_step_of_config3_runs_and_matches_on_sampled_layers(td):
             ref = oracle.full_attn(okv, qb)
         util.check_out(outs[i].cpu().numpy(), ref, f"cfg3.step.layer{i}")
     assert td.device_status() == binding.OK
-
-
-def test_launch_plan_uses_the_whole_gpu(td):
-    """Loose guard against a broken launch plan (a single CTA would still be correct, only 100x slower):
-    at 128K the full layer must stream faster than 1 TB/s and the sparse layer gather faster than 0.5 TB/s."""
-    w = synth.workload("cfg3")
-    q = synth.make_q(w, 5, DEV)
-    lay = synth.make_layer(w, 5, DEV, q=q)
-    _, idx, cnt = td.select_attn(lay, q, w.k)
-
-    def timed(fn):
-        fn()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for _ in range(5):
-            fn()
-        b.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) / 5 * 1e-3
-
-    t_full = timed(lambda: td.full_attn(lay, q))
-    t_sparse = timed(lambda: td.sparse_attn(lay, q, idx, cnt))
-    assert lay.kv_bytes() / t_full > 1e12, t_full
-    assert 32 * 4096 * 512 / t_sparse > 0.5e12, t_sparse
