@@ -596,8 +596,10 @@ tidal_status_t run_sparse(tidal_ctx* ctx, const tidal_kv_t* kv, const void* q, c
     // more than a third (measured at cfg3: step 658 -> 645 us against a third everywhere).
     const int items = kv->batch * per_batch;
     if (chain != CHAIN_NONE) {
-        // (an 8-bit cache halves a layer's bytes but not its start-up and merge phases: four layers in flight)
-        const int depth = kv->kv_dtype == TIDAL_KV_FP8_E4M3 ? 4 : 3;
+        // (a layer that gathers fewer bytes, an 8-bit cache or a small budget, still has the same start-up and
+        // merge phases: four layers in flight below 48 MB per layer)
+        const long long row_bytes = kv->kv_dtype == TIDAL_KV_FP8_E4M3 ? 2 * ROW_BYTES8 : 4 * HEAD_DIM;
+        const int depth = (long long)items * k * row_bytes < (48ll << 20) ? 4 : 3;
         const int third = std::max(1, (full + depth * items / 2) / (depth * items));
         const int S = chain == CHAIN_FIRST ? std::max(third, (full + items) / (2 * items))
                       : chain == CHAIN_LAST ? third + 1 : third;
