@@ -220,7 +220,8 @@ tidal_status_t tidal_set_select_margin(tidal_ctx_t *ctx, float margin);
  * and its output (a sparse layer right after a selection layer always waits first: the top-k writes its
  * index list). With enabled = 0 a layer only prefetches cache rows ahead of the previous layer's end and
  * reads its query afterwards, as a caller would need whose queries are produced between the layers.
- * With the overlap on, a selection layer over one sequence (per-head sets, fp32 outputs)
+ * With the overlap on, a selection layer with per-head sets and fp32 outputs (one sequence, or a batch over a
+ * 16-bit cache)
  * also runs as two passes: keys first (logits, their histogram, the largest logit per head), then the
  * top-k on `stream` while the values are streamed on the context's second stream beside it and beside
  * the sparse layers that follow.

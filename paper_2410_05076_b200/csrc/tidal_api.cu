@@ -359,10 +359,11 @@ SelectPlan select_plan(const tidal_ctx* ctx, const tidal_kv_t* kv, int Hi, int k
 }
 
 // Inside a step a selection layer can run as two passes (split_select_kernels.cuh) when it has one
-// sequence, per-head scores with the fused histogram and fp32 outputs.
+// sequence (or a batch over a 16-bit cache), per-head scores with the fused histogram and fp32 outputs.
 bool can_split(const tidal_ctx* ctx, const tidal_kv_t* kv, const SelectPlan& sp) {
-    return ctx->split_select && ctx->layer_overlap && !ctx->out_bf16 && kv->batch == 1 &&
-           !sp.agg && sp.fuse && !sp.compact && pooled_splits(kv, kv->num_kv_heads, dense_grid(ctx, kv)) > 0;
+    if (!(ctx->split_select && ctx->layer_overlap && !ctx->out_bf16 && !sp.agg && sp.fuse && !sp.compact)) return false;
+    if (kv->batch == 1) return pooled_splits(kv, kv->num_kv_heads, dense_grid(ctx, kv)) > 0;
+    return kv->kv_dtype == TIDAL_KV_BF16;       // batches: the flat-split passes (16-bit caches)
 }
 
 // hist != nullptr: the kernel also accumulates the per-head histogram the top-k needs.
@@ -428,7 +429,7 @@ tidal_status_t run_score_pass(tidal_ctx* ctx, const tidal_kv_t* kv, const void* 
     AttnParams a;
     fill_common(a, ctx, kv, q, out, w);
     const int grid = dense_grid(ctx, kv);
-    a.splits_per_item = pooled_splits(kv, kv->num_kv_heads, grid);
+    a.splits_per_item = kv->batch == 1 ? pooled_splits(kv, kv->num_kv_heads, grid) : 0;
     a.scores = scores;
     a.score_stride = score_stride;
     a.hist = state_hist(ctx);
@@ -455,7 +456,10 @@ tidal_status_t run_score_pass(tidal_ctx* ctx, const tidal_kv_t* kv, const void* 
     ctx->launches++;
     const bool rowc = kv->stride_pos == 2 * HEAD_DIM;     // K and V rows interleaved: constant offsets between the rows of a tile
     cudaError_t e;
-    if (kv->kv_dtype == TIDAL_KV_FP8_E4M3)
+    if (kv->batch > 1)
+        e = rowc ? cudaLaunchKernelEx(&cfg, score_pass_flat_kernel<SCORE_NW, SCORE_STAGES, true>, a)
+                 : cudaLaunchKernelEx(&cfg, score_pass_flat_kernel<SCORE_NW, SCORE_STAGES, false>, a);
+    else if (kv->kv_dtype == TIDAL_KV_FP8_E4M3)
         e = rowc ? cudaLaunchKernelEx(&cfg, score_pass8_kernel<SCORE_NW, SCORE_STAGES, true>, a)
                  : cudaLaunchKernelEx(&cfg, score_pass8_kernel<SCORE_NW, SCORE_STAGES, false>, a);
     else
@@ -481,12 +485,15 @@ tidal_status_t run_value_pass(tidal_ctx* ctx, const tidal_kv_t* kv, float* out, 
     // most of the slots (its CTAs are the size of the sparse layers'): it shares the GPU with the top-k and the
     // first sparse layers; between 25 % and 100 % of the slots the step time moved by less than 2 %
     const int per_item = std::max(2, 85 * std::min(ctx->sparse_slots, GRID_MAX) / (100 * kv->num_kv_heads));
-    const int grid = per_item * kv->num_kv_heads;
-    a.splits_per_item = per_item;
+    const int grid = kv->batch == 1 ? per_item * kv->num_kv_heads : std::max(1, 85 * std::min(ctx->sparse_slots, GRID_MAX) / 100);
+    a.splits_per_item = kv->batch == 1 ? per_item : 0;
     if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
         return TIDAL_ERR_CUDA;
     const bool rowc = kv->stride_pos == 2 * HEAD_DIM;
-    if (kv->kv_dtype == TIDAL_KV_FP8_E4M3) {
+    if (kv->batch > 1) {
+        if (rowc) value_pass_flat_kernel<VALUE_NW, VALUE_STAGES, true><<<grid, VALUE_NW * 32, VALUE_SMEM, ctx->side>>>(a);
+        else value_pass_flat_kernel<VALUE_NW, VALUE_STAGES, false><<<grid, VALUE_NW * 32, VALUE_SMEM, ctx->side>>>(a);
+    } else if (kv->kv_dtype == TIDAL_KV_FP8_E4M3) {
         if (rowc) value_pass8_kernel<VALUE_NW8, VALUE_STAGES, true><<<grid, VALUE_NW8 * 32, VALUE_SMEM8, ctx->side>>>(a);
         else value_pass8_kernel<VALUE_NW8, VALUE_STAGES, false><<<grid, VALUE_NW8 * 32, VALUE_SMEM8, ctx->side>>>(a);
     } else if (rowc) value_pass_kernel<VALUE_NW, VALUE_STAGES, true><<<grid, VALUE_NW * 32, VALUE_SMEM, ctx->side>>>(a);
@@ -780,6 +787,10 @@ tidal_status_t tidal_create(tidal_ctx_t** out, int device, size_t workspace_byte
     const bool split_ok =
         cudaFuncSetAttribute(score_pass_kernel<SCORE_NW, SCORE_STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCORE_SMEM) == cudaSuccess &&
         cudaFuncSetAttribute(score_pass_kernel<SCORE_NW, SCORE_STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCORE_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(score_pass_flat_kernel<SCORE_NW, SCORE_STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCORE_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(score_pass_flat_kernel<SCORE_NW, SCORE_STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCORE_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(value_pass_flat_kernel<VALUE_NW, VALUE_STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VALUE_SMEM) == cudaSuccess &&
+        cudaFuncSetAttribute(value_pass_flat_kernel<VALUE_NW, VALUE_STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VALUE_SMEM) == cudaSuccess &&
         cudaFuncSetAttribute(score_pass8_kernel<SCORE_NW, SCORE_STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCORE_SMEM) == cudaSuccess &&
         cudaFuncSetAttribute(score_pass8_kernel<SCORE_NW, SCORE_STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCORE_SMEM) == cudaSuccess &&
         cudaFuncSetAttribute(value_pass8_kernel<VALUE_NW8, VALUE_STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VALUE_SMEM8) == cudaSuccess &&

@@ -591,7 +591,7 @@ def test_library_records_and_replays_step_graphs(td):
             step()                                        # a replay at the latest
             n2 = td.launch_count()
             side.synchronize()
-            assert n1 - n0 == n2 - n1 == 5                # 4 attention kernels + 1 top-k
+            assert n1 - n0 == n2 - n1 == 6                # full, key pass, value pass, top-k, two sparse layers
             assert torch.equal(step.idx, ref_idx)
             for o, r in zip(outs, ref_outs):
                 assert torch.allclose(o, r, rtol=0, atol=5e-4)
@@ -669,7 +669,12 @@ def test_bf16_outputs_are_the_fp32_results_rounded(td):
     w = wl(2, 8, 2, 700, 64, ragged=True, ctx_min=300, seed=31, layers=len(sched))
     qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
     layers = [synth.make_layer(w, i, DEV, q=qs[i]) for i in range(len(sched))]
-    ref_outs, ref_idx, _ = td.decode_step(sched, layers, qs, w.k)
+    # (bf16 outputs always come from the fused selection kernel; without the overlap so do the fp32 ones)
+    td.set_layer_overlap(False)
+    try:
+        ref_outs, ref_idx, _ = td.decode_step(sched, layers, qs, w.k)
+    finally:
+        td.set_layer_overlap(True)
     ref_full = td.full_attn(layers[0], qs[0])
     torch.cuda.synchronize()
     td.set_output_bf16(True)
@@ -1227,4 +1232,42 @@ def test_two_pass_selection_layers_match_the_oracle(td, layout, Hq, Hkv, N, k, f
     for i in (3, 4):
         ref = oracle.sparse_attn(util.oracle_kv(lays[i]), synth.bits(qs[i]), idx.cpu().numpy(), cnt.cpu().numpy())
         util.check_out(outs[i].cpu().numpy(), ref, f"sparse layer {i} after a two-pass selection")
+    assert td.device_status() == binding.OK
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,N,k,ragged,layout", [
+    (3, 16, 4, 9000, 500, True, "hnd_interleaved"), (8, 8, 2, 5000, 256, True, "paged"),
+    (2, 32, 8, 20000, 1024, False, "nhd_separate"), (5, 8, 8, 700, 64, True, "paged"),
+    (4, 8, 1, 90, 16, True, "hnd_interleaved"), (6, 16, 2, 33000, 2048, True, "paged")])
+def test_two_pass_selection_layers_of_a_batch_match_the_oracle(td, B, Hq, Hkv, N, k, ragged, layout):
+    """Batches run the two passes over a flat split of the (sequence, KV head, tile) space: CTAs cross item
+    and sequence boundaries. Outputs, token sets and the sparse layers after two consecutive selection
+    layers against the oracle, ragged lengths, all layouts."""
+    sched = [0, 1, 1, 2, 2]
+    w = wl(B, Hq, Hkv, N, k, planted=min(8, N), seed=131, ragged=ragged, ctx_min=max(1, N // 5), layers=len(sched))
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    if layout == "paged":
+        pt, total = synth.make_page_table(w, extra_pages=3)
+        lays = [synth.make_layer(w, i, DEV, layout="paged", q=qs[i], page_table=pt, num_pages=total) for i in range(len(sched))]
+    else:
+        lays = [synth.make_layer(w, i, DEV, layout=layout, q=qs[i]) for i in range(len(sched))]
+    lens = lays[0].ctx_lens.cpu().numpy()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())      # the inputs were built on the current stream
+    with torch.cuda.stream(side):
+        outs, idx, cnt = td.decode_step(sched, lays, qs, w.k)
+        side.synchronize()
+    assert cnt.cpu().numpy().tolist() == [min(k, int(n)) for n in lens]
+    for i in (1, 2):
+        okv, qb = util.oracle_kv(lays[i]), synth.bits(qs[i])
+        ref, sc = oracle.full_attn(okv, qb, want_scores=True)
+        util.check_out(outs[i].cpu().numpy(), ref, f"batch two-pass layer {i}")
+        if i == 2:
+            idx_h = idx.cpu().numpy()
+            for b in range(B):
+                for h in range(0, Hq, max(1, Hq // 4)):
+                    util.check_idx_row(idx_h[b, h], sc[b, h], w.k, int(lens[b]), f"batch two-pass idx[{b},{h}]")
+    for i in (3, 4):
+        ref = oracle.sparse_attn(util.oracle_kv(lays[i]), synth.bits(qs[i]), idx.cpu().numpy(), cnt.cpu().numpy())
+        util.check_out(outs[i].cpu().numpy(), ref, f"sparse layer {i} after a batch's two-pass selection")
     assert td.device_status() == binding.OK
