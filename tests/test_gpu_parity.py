@@ -1271,3 +1271,62 @@ def test_two_pass_selection_layers_of_a_batch_match_the_oracle(td, B, Hq, Hkv, N
         ref = oracle.sparse_attn(util.oracle_kv(lays[i]), synth.bits(qs[i]), idx.cpu().numpy(), cnt.cpu().numpy())
         util.check_out(outs[i].cpu().numpy(), ref, f"sparse layer {i} after a batch's two-pass selection")
     assert td.device_status() == binding.OK
+
+
+def _step_fuzz_cases(n, seed):
+    import random
+    rng = random.Random(seed)
+    cases = []
+    for _ in range(n):
+        B = rng.choice([1, 1, 1, 2, 3, 5])
+        Hkv = rng.choice([1, 2, 4, 8])
+        G = min(rng.choice([1, 2, 4, 8]), 32 // Hkv)
+        N = rng.choice([17, 100, 1000, 4096, 9001, 20000, 33333])
+        k = min(rng.choice([8, 64, 300, 1024]), N)
+        ragged = B > 1 and rng.random() < 0.7
+        layout = rng.choice(["hnd_interleaved", "paged", "nhd_separate"])
+        fp8 = layout != "nhd_separate" and rng.random() < 0.35
+        sched = rng.choice(["12", "0112", "12122", "00122212"])
+        cases.append((B, Hkv * G, Hkv, N, k, ragged, layout, fp8, sched))
+    return cases
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,N,k,ragged,layout,fp8,sched", _step_fuzz_cases(24, 20241006))
+def test_random_decode_steps_match_the_oracle(td, B, Hq, Hkv, N, k, ragged, layout, fp8, sched):
+    """Whole steps over random shapes, layouts, cache types and schedules (two calls in a row, the second a
+    replay): every full and selection layer, the last token sets and the sparse layers that use them against
+    the oracle. Covers the pooled, the flat-split and the FP8 variants of the two selection passes."""
+    sched = [int(c) for c in sched]
+    w = wl(B, Hq, Hkv, N, k, planted=min(8, N), seed=500 + N % 97 + B, ragged=ragged, ctx_min=max(1, N // 4), layers=len(sched))
+    qs = [synth.make_q(w, i, DEV) for i in range(len(sched))]
+    if layout == "paged":
+        pt, total = synth.make_page_table(w, extra_pages=3)
+        lays = [synth.make_layer(w, i, DEV, layout="paged", q=qs[i], page_table=pt, num_pages=total) for i in range(len(sched))]
+    else:
+        lays = [synth.make_layer(w, i, DEV, layout=layout, q=qs[i]) for i in range(len(sched))]
+    if fp8:
+        lays = [synth.to_fp8(lay) for lay in lays]
+    lens = lays[0].ctx_lens.cpu().numpy()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())      # the inputs were built on the current stream
+    with torch.cuda.stream(side):
+        outs, idx, cnt = td.decode_step(sched, lays, qs, w.k)
+        outs2, idx2, _ = td.decode_step(sched, lays, qs, w.k)
+        side.synchronize()
+    assert torch.equal(idx, idx2)
+    last_sel = max(i for i, t in enumerate(sched) if t == 1)
+    for i, t in enumerate(sched):
+        okv, qb = util.oracle_kv(lays[i]), synth.bits(qs[i])
+        if t != 2:
+            ref = oracle.full_attn(okv, qb)
+            util.check_out(outs[i].cpu().numpy(), ref, f"layer {i}")
+            util.check_out(outs2[i].cpu().numpy(), ref, f"layer {i}, second call")
+        elif i > last_sel:
+            ref = oracle.sparse_attn(okv, qb, idx.cpu().numpy(), cnt.cpu().numpy())
+            util.check_out(outs[i].cpu().numpy(), ref, f"sparse layer {i}")
+    _, sc = oracle.full_attn(util.oracle_kv(lays[last_sel]), synth.bits(qs[last_sel]), want_scores=True)
+    idx_h = idx.cpu().numpy()
+    for b in range(B):
+        for h in range(0, Hq, max(1, Hq // 3)):
+            util.check_idx_row(idx_h[b, h], sc[b, h], w.k, int(lens[b]), f"idx[{b},{h}]")
+    assert td.device_status() == binding.OK
