@@ -485,7 +485,7 @@ tidal_status_t run_value_pass(tidal_ctx* ctx, const tidal_kv_t* kv, float* out, 
     // most of the slots (its CTAs are the size of the sparse layers'): it shares the GPU with the top-k and the
     // first sparse layers; between 25 % and 100 % of the slots the step time moved by less than 2 %
     const int per_item = std::max(2, 85 * std::min(ctx->sparse_slots, GRID_MAX) / (100 * kv->num_kv_heads));
-    const int grid = kv->batch == 1 ? per_item * kv->num_kv_heads : std::max(1, 85 * std::min(ctx->sparse_slots, GRID_MAX) / 100);
+    const int grid = kv->batch == 1 ? per_item * kv->num_kv_heads : std::min(ctx->sparse_slots, GRID_MAX);
     a.splits_per_item = kv->batch == 1 ? per_item : 0;
     if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
         return TIDAL_ERR_CUDA;
